@@ -1,0 +1,139 @@
+/*
+ * fastrack.h -- C ABI of the GPU side of Fastrack's CPU<->GPU secure channel on NVIDIA B200.
+ *
+ * The library implements the one data-parallel path of the paper "Fastrack: Fast IO for Secure ML
+ * using GPU TEEs" (arXiv 2410.15240): authenticated decryption of a buffer that arrived over PCIe,
+ * its mirror (encryption + tagging of a buffer that is about to leave the GPU), and the chunked
+ * overlap of the PCIe copies with those kernels.
+ *
+ * Scheme (paper Section 2.3 "AES-GCM", Section 4.2 "Multi-chaining authentication"): AES-256 in
+ * counter mode plus the GMAC tag over GF(2^128), i.e. AES-256-GCM with 96-bit IVs and 128-bit tags.
+ * A buffer of `len` bytes is split into K = ceil(len / chunk_bytes) chunks; chunk k covers bytes
+ * [k*chunk_bytes, min(len, (k+1)*chunk_bytes)), is an independent GCM message with empty AAD under
+ *
+ *     IV_k = iv_base[0..7] || BE32( (BE32(iv_base[8..11]) + k) mod 2^32 ),
+ *
+ * and has its own 16-byte tag at byte 16*k of the tag array.  Chunk order is bound by the index
+ * inside IV_k: a chunk moved to another slot is decrypted under the wrong IV and rejected.
+ * Within a chunk, keystream block j is E_K(IV_k || BE32(2 + j)); the tag is
+ * GHASH_H(ciphertext zero-padded to 16 bytes || BE64(0) || BE64(8*len_k)) xor E_K(IV_k || BE32(1)).
+ *
+ * Conventions
+ *   - Every function returns FASTRACK_OK (0) or a negative FASTRACK_ERR_* code.  Nothing throws,
+ *     aborts or prints.  After FASTRACK_ERR_CUDA, fastrack_last_cuda_error(ctx) gives the CUDA code.
+ *   - Pointers named d_* are DEVICE pointers on the context's device, 16-byte aligned.  Pointers named
+ *     h_* are HOST pointers.  `key` and `iv_base` are always HOST pointers.  The caller owns every
+ *     data buffer; the context owns only key-derived tables, per-chunk scratch and internal streams.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - A context is bound to the device that was current at creation and must not be used from two
+ *     host threads, or on two streams, at the same time (calls share per-chunk scratch memory).
+ *   - IV discipline is the caller's: one call consumes the IV values iv_base .. iv_base + K - 1;
+ *     reusing an IV under the same key voids GCM's guarantees.  The library does not track this.
+ *   - K is derived from `len`; dropping trailing chunks is invisible to this layer, so `len` must
+ *     come from a trusted source.
+ *   - There is no CPU implementation behind these calls: without a usable CUDA device they fail.
+ */
+#ifndef FASTRACK_H
+#define FASTRACK_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(_WIN32)
+#define FASTRACK_API
+#else
+#define FASTRACK_API __attribute__((visibility("default")))
+#endif
+
+#define FASTRACK_OK               0
+#define FASTRACK_ERR_ARG         -1   /* null pointer, misaligned or partially overlapping buffers, bad n_streams */
+#define FASTRACK_ERR_CHUNK       -2   /* chunk_bytes is 0, not a multiple of 16, or above FASTRACK_MAX_CHUNK_BYTES */
+#define FASTRACK_ERR_NOT_PINNED  -3   /* h_cipher_pinned is not page-locked host memory */
+#define FASTRACK_ERR_CUDA        -4   /* a CUDA call failed; see fastrack_last_cuda_error */
+#define FASTRACK_ERR_NOMEM       -5   /* host or device allocation failed */
+#define FASTRACK_ERR_TOO_MANY    -6   /* more than 2^32 chunks in one call (the IV index is 32 bits) */
+
+/* Largest chunk: 1 GiB.  (GCM itself allows 2^36 - 32 bytes per message; the limit here keeps the
+ * per-context table of powers of H, 16 bytes per 16-byte block of a chunk, at most 1 GiB.) */
+#define FASTRACK_MAX_CHUNK_BYTES ((size_t)1 << 30)
+
+typedef struct fastrack_ctx fastrack_ctx;
+
+/* Context set-up (paper Section 2.3: the hash subkey H = E_K(0^128) "is used throughout the
+ * authentication process"; Section 4.2: every chain uses the same H).
+ * Copies the 32-byte AES-256 key (host pointer), expands it into the 15 round keys, derives H, and
+ * builds on the current device the tables the kernels need, sized for `chunk_bytes`: the byte tables
+ * of the fixed multiplier H^32 and the powers H^0 .. H^(chunk_bytes/16 + 64).  Allocates device
+ * memory and synchronises the device once.  chunk_bytes: multiple of 16, 16 .. FASTRACK_MAX_CHUNK_BYTES.
+ * On success *out is a new context; on failure *out is NULL. */
+FASTRACK_API int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fastrack_ctx** out);
+
+/* Zeroises the key material on host and device, frees tables, scratch and streams.  NULL is allowed.
+ * Synchronises the device. */
+FASTRACK_API void fastrack_ctx_destroy(fastrack_ctx* ctx);
+
+/* K = ceil(len / chunk_bytes); 0 for len == 0 or ctx == NULL (Section 4.2: one tag per chunk). */
+FASTRACK_API size_t fastrack_num_chunks(const fastrack_ctx* ctx, size_t len);
+
+/* Pre-sizes the per-chunk scratch (20 bytes per chunk) for buffers up to max_len bytes so that later
+ * calls allocate nothing.  Without it the first call that needs more chunks than any call before
+ * grows the scratch (cudaMalloc + a device synchronisation) before launching. */
+FASTRACK_API int fastrack_ctx_reserve(fastrack_ctx* ctx, size_t max_len);
+
+/* CUDA error code (cudaError_t as int) of the last failing CUDA call made through ctx, else 0. */
+FASTRACK_API int fastrack_last_cuda_error(const fastrack_ctx* ctx);
+
+/* GPU-side authenticated decryption (paper Section 4.2: "decrypt and authenticate the received
+ * data"; decryption kernel = AES-CTR, authentication = GMAC per chunk; here one fused pass).
+ *   iv_base  host, 12 bytes.
+ *   d_cipher device, len bytes of ciphertext, chunks back to back.
+ *   d_tags   device, 16*K bytes, tag of chunk k at byte 16*k.
+ *   d_plain  device, len bytes out.  d_plain == d_cipher (exactly) is allowed: in-place.  Any other
+ *            overlap with d_cipher is FASTRACK_ERR_ARG.
+ *   d_ok     device, K uint32 out: 1 = all 128 tag bits match, 0 = rejected.
+ * The plaintext of a rejected chunk is still written (Section 4.3 "eager evaluation" releases the
+ * plaintext before the verdict; Section 3: results are discarded on failure) -- consult d_ok.
+ * Asynchronous on `stream`: no host synchronisation; outputs are valid once the stream has been
+ * synchronised.  len == 0 succeeds and writes nothing. */
+FASTRACK_API int fastrack_decrypt_verify(fastrack_ctx* ctx, const uint8_t iv_base[12],
+                                         const void* d_cipher, size_t len, const void* d_tags,
+                                         void* d_plain, uint32_t* d_ok, void* stream);
+
+/* GPU-side encryption with one tag per chunk, for GPU->CPU copies (paper Section 2.3: encryption is
+ * the same keystream XOR; Section 4.2: one tag per chunk).
+ *   d_plain  device, len bytes in.   d_cipher device, len bytes out (d_cipher == d_plain allowed).
+ *   d_tags   device, 16*K bytes out.
+ * Asynchronous on `stream`, same rules as fastrack_decrypt_verify. */
+FASTRACK_API int fastrack_encrypt_tag(fastrack_ctx* ctx, const uint8_t iv_base[12],
+                                      const void* d_plain, size_t len, void* d_cipher, void* d_tags,
+                                      void* stream);
+
+/* Pipelined host->device transfer with decryption and verification (paper Section 4.3 "Decryption
+ * pipeline": the PCIe transfer is overlapped with the decryption and authentication kernels, so the
+ * transfer costs max(copy, kernels) instead of their sum).
+ * The buffer is cut into stages of whole chunks (one chunk per stage when chunk_bytes >= 1 MiB,
+ * otherwise as many chunks as fit in 1 MiB); stage i is copied pinned->device into its final place in
+ * d_plain with cudaMemcpyAsync on internal stream i mod n_streams and decrypted and verified in place
+ * by the same kernels on that stream, so the copy of stage i+1 overlaps the kernels of stage i.
+ *   h_cipher_pinned host, page-locked (cudaHostAlloc / cudaHostRegister), len bytes.
+ *   h_tags          host, 16*K bytes, pinned or pageable (copied once, up front).
+ *   d_plain, d_ok   device outputs as in fastrack_decrypt_verify.
+ *   n_streams       1..8.
+ * BLOCKING: returns after every internal stream has completed, so wall-clock time around the call is
+ * the effective transfer time.  Work already queued by the caller on other streams is not waited for. */
+FASTRACK_API int fastrack_pipelined_h2d(fastrack_ctx* ctx, const uint8_t iv_base[12],
+                                        const void* h_cipher_pinned, size_t len, const void* h_tags,
+                                        void* d_plain, uint32_t* d_ok, int n_streams);
+
+/* Number of kernels the library launched through ctx since creation (data-path launches only;
+ * cudaMemcpyAsync calls are not counted).  For benchmarks' bookkeeping. */
+FASTRACK_API uint64_t fastrack_launch_count(const fastrack_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FASTRACK_H */

@@ -1,0 +1,424 @@
+// fastrack.cu -- kernels, context and C ABI of the B200 (sm_100a) Fastrack channel library.
+// The entry points are documented in include/fastrack.h; the per-lane device code is in
+// fastrack_device.cuh.  There is no CPU data path here: host code only derives key material
+// (round keys, H, the byte tables of H^32) once per context and launches kernels.
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#include <new>
+
+#include "../../include/fastrack.h"
+#include "fastrack_device.cuh"
+#include "fastrack_keysetup.h"
+
+using namespace fr_host;
+
+#define FR_THREADS 512
+#define FR_WARPS (FR_THREADS / 32)
+
+// ------------------------------------------------------------------------------------ kernels ----
+
+// Fused pass: keystream, XOR, per-segment GHASH partial, per-chunk tag.  Segments are dealt to warps
+// round-robin; a warp XORs its segment's partial into the chunk's accumulator and takes a ticket; the
+// warp that takes the chunk's last ticket finishes the tag (no warp ever waits for another).
+template <bool ENCRYPT>
+__global__ void __launch_bounds__(FR_THREADS, 1) fr_crypt_kernel(const __grid_constant__ FrParams P)
+{
+    extern __shared__ __align__(256) char sm[];
+    fr_build_smem(sm, threadIdx.x, blockDim.x, P.te0, P.gh_tab);
+    __syncthreads();
+
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const FrLane L = fr_make_lane(lane);
+    const uint32_t total_warps = gridDim.x * (blockDim.x >> 5);
+
+    for (uint32_t item = warp * gridDim.x + blockIdx.x; item < P.n_items; item += total_warps) {
+        const uint32_t kk = item / P.segs_per_chunk, s = item - kk * P.segs_per_chunk;
+        const uint32_t nseg = fr_chunk_segs(P, kk);
+        if (s >= nseg) continue;                       // only the short last chunk has fewer segments
+
+        uint4 z = fr_process_segment_lane<ENCRYPT>(P, sm, L, lane, kk, s);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            z.x ^= __shfl_xor_sync(0xFFFFFFFFu, z.x, off);
+            z.y ^= __shfl_xor_sync(0xFFFFFFFFu, z.y, off);
+            z.z ^= __shfl_xor_sync(0xFFFFFFFFu, z.z, off);
+            z.w ^= __shfl_xor_sync(0xFFFFFFFFu, z.w, off);
+        }
+        bool finisher = true;
+        if (nseg > 1) {
+            uint32_t ticket = 0;
+            if (lane == 0) {
+                atomicXor(&P.acc[4 * kk + 0], z.x);
+                atomicXor(&P.acc[4 * kk + 1], z.y);
+                atomicXor(&P.acc[4 * kk + 2], z.z);
+                atomicXor(&P.acc[4 * kk + 3], z.w);
+                __threadfence();
+                ticket = atomicAdd(&P.cnt[kk], 1u);
+            }
+            ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
+            finisher = (ticket == nseg - 1);
+            if (finisher) {
+                __threadfence();
+                if (lane == 0) {                       // read the sum and leave the scratch zeroed
+                    z.x = atomicExch(&P.acc[4 * kk + 0], 0u);
+                    z.y = atomicExch(&P.acc[4 * kk + 1], 0u);
+                    z.z = atomicExch(&P.acc[4 * kk + 2], 0u);
+                    z.w = atomicExch(&P.acc[4 * kk + 3], 0u);
+                    atomicExch(&P.cnt[kk], 0u);
+                }
+                z.x = __shfl_sync(0xFFFFFFFFu, z.x, 0);
+                z.y = __shfl_sync(0xFFFFFFFFu, z.y, 0);
+                z.z = __shfl_sync(0xFFFFFFFFu, z.z, 0);
+                z.w = __shfl_sync(0xFFFFFFFFu, z.w, 0);
+            }
+        }
+        if (finisher) {
+            const uint4 tag = fr_chunk_tag(P, sm, L.lane4, kk, z);
+            if (lane == 0) {
+                if (ENCRYPT) {
+                    P.tags_out[kk] = tag;
+                } else {
+                    const uint4 t = P.tags_in[kk];
+                    const uint32_t diff = (tag.x ^ t.x) | (tag.y ^ t.y) | (tag.z ^ t.z) | (tag.w ^ t.w);
+                    P.ok[kk] = diff == 0u ? 1u : 0u;
+                }
+            }
+        }
+    }
+}
+
+// pow[i] = pow[i - half] * pow[half] for i in (half, min(2*half, n - 1)]: one doubling pass of the table
+// of powers (pow[half] itself was the last entry of the previous pass; pow[0] = 1 and pow[1] = H are given).
+__global__ void fr_pow_double_kernel(uint4* pow, uint32_t half, uint32_t n)
+{
+    const uint32_t i = half + 1u + blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t last = (2u * half < n - 1u) ? 2u * half : n - 1u;
+    if (i <= last) pow[i] = fr_gf128_mul(pow[i - half], pow[half]);
+}
+
+// ------------------------------------------------------------------------------------ context ----
+
+struct fastrack_ctx {
+    int device;
+    int num_sms;
+    size_t chunk_bytes;
+    uint32_t rk[60];
+    uint8_t h[16];
+    uint32_t* d_te0;
+    uint4* d_gh_tab;
+    uint4* d_pow;
+    size_t pow_entries;
+    uint32_t* d_scratch;       // acc[4*cap] then cnt[cap]
+    size_t scratch_chunks;
+    uint4* d_tags_stage;       // pipelined_h2d: device copy of the tags
+    size_t tags_stage_chunks;
+    cudaStream_t streams[8];
+    cudaEvent_t tags_ready;
+    int last_cuda_error;
+    uint64_t launches;
+    uint32_t seg_rows_override;   // 0 = automatic (FASTRACK_SEG_ROWS, for experiments)
+};
+
+#define FR_CUDA(ctx, call)                                              \
+    do {                                                                \
+        cudaError_t e_ = (call);                                        \
+        if (e_ != cudaSuccess) {                                        \
+            (ctx)->last_cuda_error = (int)e_;                           \
+            (void)cudaGetLastError();                                   \
+            return FASTRACK_ERR_CUDA;                                   \
+        }                                                               \
+    } while (0)
+
+static int ensure_scratch(fastrack_ctx* ctx, size_t chunks)
+{
+    if (chunks <= ctx->scratch_chunks) return FASTRACK_OK;
+    size_t cap = ctx->scratch_chunks ? ctx->scratch_chunks : 1024;
+    while (cap < chunks) cap *= 2;
+    FR_CUDA(ctx, cudaDeviceSynchronize());       // nothing may still be using the old scratch
+    uint32_t* fresh = nullptr;
+    cudaError_t e = cudaMalloc(&fresh, cap * 5 * sizeof(uint32_t));
+    if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); return FASTRACK_ERR_NOMEM; }
+    FR_CUDA(ctx, cudaMemset(fresh, 0, cap * 5 * sizeof(uint32_t)));
+    if (ctx->d_scratch) cudaFree(ctx->d_scratch);
+    ctx->d_scratch = fresh;
+    ctx->scratch_chunks = cap;
+    return FASTRACK_OK;
+}
+
+extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fastrack_ctx** out)
+{
+    if (out) *out = nullptr;
+    if (!key || !out) return FASTRACK_ERR_ARG;
+    if (chunk_bytes == 0 || (chunk_bytes & 15) || chunk_bytes > FASTRACK_MAX_CHUNK_BYTES) return FASTRACK_ERR_CHUNK;
+    fastrack_ctx* ctx = new (std::nothrow) fastrack_ctx();
+    if (!ctx) return FASTRACK_ERR_NOMEM;
+    memset(ctx, 0, sizeof *ctx);
+    ctx->chunk_bytes = chunk_bytes;
+    int rc = FASTRACK_OK;
+    auto fail = [&](int code) { fastrack_ctx_destroy(ctx); return code; };
+
+    cudaError_t e = cudaGetDevice(&ctx->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, ctx->device);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return fail(FASTRACK_ERR_CUDA); }
+    if (const char* env = getenv("FASTRACK_SEG_ROWS")) ctx->seg_rows_override = (uint32_t)strtoul(env, nullptr, 10);
+
+    // key material on the host: S-box, Te0, round keys, H, byte tables of H^32
+    uint8_t sbox[256];
+    uint32_t te0[256];
+    make_sbox(sbox);
+    for (int v = 0; v < 256; v++) {
+        uint8_t s1 = sbox[v], s2 = xtime(s1), s3 = (uint8_t)(s2 ^ s1);
+        te0[v] = (uint32_t)s2 | ((uint32_t)s1 << 8) | ((uint32_t)s1 << 16) | ((uint32_t)s3 << 24);
+    }
+    expand_key(key, sbox, ctx->rk);
+    uint8_t zero[16] = {0};
+    encrypt_block_host(ctx->rk, te0, sbox, zero, ctx->h);
+
+    Gf128 H = gf_load(ctx->h), G = H;
+    for (int i = 0; i < 5; i++) G = gf_mul(G, G);           // H^32
+    uint8_t* tab = (uint8_t*)malloc(65536);
+    if (!tab) return fail(FASTRACK_ERR_NOMEM);
+    for (int p = 0; p < 16; p++) {
+        Gf128 basis[8];
+        for (int b = 0; b < 8; b++) {
+            uint8_t blk[16] = {0};
+            blk[p] = (uint8_t)(1u << b);
+            basis[b] = gf_mul(gf_load(blk), G);
+        }
+        for (int v = 0; v < 256; v++) {
+            Gf128 acc = {0, 0};
+            for (int b = 0; b < 8; b++)
+                if (v & (1 << b)) { acc.hi ^= basis[b].hi; acc.lo ^= basis[b].lo; }
+            gf_store(acc, tab + (size_t)v * 256 + (size_t)p * 16);
+        }
+    }
+
+    ctx->pow_entries = chunk_bytes / 16 + 64 + 2;
+    do {
+        if ((e = cudaMalloc(&ctx->d_te0, sizeof te0)) != cudaSuccess) break;
+        if ((e = cudaMalloc(&ctx->d_gh_tab, 65536)) != cudaSuccess) break;
+        if ((e = cudaMalloc(&ctx->d_pow, ctx->pow_entries * 16)) != cudaSuccess) break;
+        if ((e = cudaMemcpy(ctx->d_te0, te0, sizeof te0, cudaMemcpyHostToDevice)) != cudaSuccess) break;
+        if ((e = cudaMemcpy(ctx->d_gh_tab, tab, 65536, cudaMemcpyHostToDevice)) != cudaSuccess) break;
+        uint8_t seed[32] = {0};
+        seed[0] = 0x80;                                     // H^0 = the field's one
+        memcpy(seed + 16, ctx->h, 16);                      // H^1
+        if ((e = cudaMemcpy(ctx->d_pow, seed, 32, cudaMemcpyHostToDevice)) != cudaSuccess) break;
+        for (size_t half = 1; half + 1 < ctx->pow_entries; half *= 2) {
+            size_t last = 2 * half < ctx->pow_entries - 1 ? 2 * half : ctx->pow_entries - 1;
+            size_t todo = last - half;
+            fr_pow_double_kernel<<<(unsigned)((todo + 255) / 256), 256>>>(ctx->d_pow, (uint32_t)half, (uint32_t)ctx->pow_entries);
+        }
+        if ((e = cudaGetLastError()) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        for (int i = 0; i < 8 && e == cudaSuccess; i++) e = cudaStreamCreateWithFlags(&ctx->streams[i], cudaStreamNonBlocking);
+        if (e != cudaSuccess) break;
+        if ((e = cudaEventCreateWithFlags(&ctx->tags_ready, cudaEventDisableTiming)) != cudaSuccess) break;
+        e = cudaDeviceSynchronize();
+    } while (0);
+    memset(tab, 0, 65536);
+    free(tab);
+    if (e != cudaSuccess) {
+        ctx->last_cuda_error = (int)e;
+        (void)cudaGetLastError();
+        return fail(e == cudaErrorMemoryAllocation ? FASTRACK_ERR_NOMEM : FASTRACK_ERR_CUDA);
+    }
+    rc = ensure_scratch(ctx, 1024);
+    if (rc != FASTRACK_OK) return fail(rc);
+    *out = ctx;
+    return FASTRACK_OK;
+}
+
+extern "C" void fastrack_ctx_destroy(fastrack_ctx* ctx)
+{
+    if (!ctx) return;
+    cudaDeviceSynchronize();
+    if (ctx->d_gh_tab) { cudaMemset(ctx->d_gh_tab, 0, 65536); }
+    if (ctx->d_pow) { cudaMemset(ctx->d_pow, 0, ctx->pow_entries * 16); }
+    cudaDeviceSynchronize();
+    cudaFree(ctx->d_te0);
+    cudaFree(ctx->d_gh_tab);
+    cudaFree(ctx->d_pow);
+    cudaFree(ctx->d_scratch);
+    cudaFree(ctx->d_tags_stage);
+    for (int i = 0; i < 8; i++)
+        if (ctx->streams[i]) cudaStreamDestroy(ctx->streams[i]);
+    if (ctx->tags_ready) cudaEventDestroy(ctx->tags_ready);
+    (void)cudaGetLastError();
+    volatile uint8_t* p = (volatile uint8_t*)ctx;
+    for (size_t i = 0; i < sizeof *ctx; i++) p[i] = 0;
+    delete ctx;
+}
+
+extern "C" size_t fastrack_num_chunks(const fastrack_ctx* ctx, size_t len)
+{
+    if (!ctx || len == 0) return 0;
+    return (len + ctx->chunk_bytes - 1) / ctx->chunk_bytes;
+}
+
+extern "C" int fastrack_ctx_reserve(fastrack_ctx* ctx, size_t max_len)
+{
+    if (!ctx) return FASTRACK_ERR_ARG;
+    return ensure_scratch(ctx, fastrack_num_chunks(ctx, max_len));
+}
+
+extern "C" int fastrack_last_cuda_error(const fastrack_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+extern "C" uint64_t fastrack_launch_count(const fastrack_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+// ------------------------------------------------------------------------------------ launches ----
+
+static uint32_t load_be32(const uint8_t* p) { return ((uint32_t)p[0] << 24) | ((uint32_t)p[1] << 16) | ((uint32_t)p[2] << 8) | p[3]; }
+static uint32_t load_le32(const uint8_t* p) { return ((uint32_t)p[3] << 24) | ((uint32_t)p[2] << 16) | ((uint32_t)p[1] << 8) | p[0]; }
+
+// Launch the fused pass over `len` bytes that start at chunk index `first_chunk` of the caller's buffer.
+static int launch_pass(fastrack_ctx* ctx, bool encrypt, const uint8_t iv_base[12], size_t first_chunk,
+                       const void* d_in, size_t len, void* d_out, const void* d_tags_in, void* d_tags_out,
+                       uint32_t* d_ok, cudaStream_t stream)
+{
+    FrParams P;
+    memset(&P, 0, sizeof P);
+    memcpy(P.rk, ctx->rk, sizeof P.rk);
+    P.iv_w0 = load_le32(iv_base);
+    P.iv_w1 = load_le32(iv_base + 4);
+    P.iv_ctr = load_be32(iv_base + 8) + (uint32_t)first_chunk;
+    P.len = len;
+    P.chunk_bytes = ctx->chunk_bytes;
+    const size_t n_chunks = (len + ctx->chunk_bytes - 1) / ctx->chunk_bytes;
+    P.n_chunks = (uint32_t)n_chunks;
+
+    // rows of the largest chunk in this launch, and the segment length that spreads the work
+    const size_t first_len = len < ctx->chunk_bytes ? len : ctx->chunk_bytes;
+    const size_t rows_ref = ((first_len + 15) / 16 + FR_ROW_BLOCKS - 1) / FR_ROW_BLOCKS;
+    const size_t total_rows = rows_ref * n_chunks;
+    const size_t warps = (size_t)ctx->num_sms * FR_WARPS;
+    size_t seg_rows = ctx->seg_rows_override ? ctx->seg_rows_override : (total_rows + 2 * warps - 1) / (2 * warps);
+    if (!ctx->seg_rows_override) {
+        if (seg_rows < 8) seg_rows = 8;
+        if (seg_rows > 128) seg_rows = 128;
+    }
+    size_t spc = (rows_ref + seg_rows - 1) / seg_rows;
+    while (spc * n_chunks >= ((size_t)1 << 31)) { seg_rows *= 2; spc = (rows_ref + seg_rows - 1) / seg_rows; }
+    seg_rows = (rows_ref + spc - 1) / spc;                 // equalise the segments of a chunk
+    P.seg_rows = (uint32_t)seg_rows;
+    P.segs_per_chunk = (uint32_t)spc;
+    P.n_items = (uint32_t)(spc * n_chunks);
+
+    P.in = (const uint8_t*)d_in;
+    P.out = (uint8_t*)d_out;
+    P.tags_in = (const uint4*)d_tags_in;
+    P.tags_out = (uint4*)d_tags_out;
+    P.ok = d_ok;
+    P.te0 = ctx->d_te0;
+    P.gh_tab = ctx->d_gh_tab;
+    P.pow = ctx->d_pow;
+    P.acc = ctx->d_scratch + 4 * first_chunk;
+    P.cnt = ctx->d_scratch + 4 * ctx->scratch_chunks + first_chunk;
+
+    unsigned grid = (unsigned)ctx->num_sms;
+    if (P.n_items < grid) grid = P.n_items;
+    if (encrypt) fr_crypt_kernel<true><<<grid, FR_THREADS, FR_SMEM_BYTES, stream>>>(P);
+    else         fr_crypt_kernel<false><<<grid, FR_THREADS, FR_SMEM_BYTES, stream>>>(P);
+    ctx->launches++;
+    FR_CUDA(ctx, cudaGetLastError());
+    return FASTRACK_OK;
+}
+
+static bool misaligned(const void* p, size_t a) { return ((uintptr_t)p & (a - 1)) != 0; }
+
+static bool bad_overlap(const void* a, const void* b, size_t len)
+{
+    if (a == b) return false;
+    uintptr_t x = (uintptr_t)a, y = (uintptr_t)b;
+    return x < y + len && y < x + len;
+}
+
+extern "C" int fastrack_decrypt_verify(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_cipher, size_t len,
+                                       const void* d_tags, void* d_plain, uint32_t* d_ok, void* stream)
+{
+    if (!ctx || !iv_base) return FASTRACK_ERR_ARG;
+    if (len == 0) return FASTRACK_OK;
+    if (!d_cipher || !d_tags || !d_plain || !d_ok) return FASTRACK_ERR_ARG;
+    if (misaligned(d_cipher, 16) || misaligned(d_plain, 16) || misaligned(d_tags, 16) || misaligned(d_ok, 4)) return FASTRACK_ERR_ARG;
+    if (bad_overlap(d_cipher, d_plain, len)) return FASTRACK_ERR_ARG;
+    const size_t K = fastrack_num_chunks(ctx, len);
+    if (K > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
+    int rc = ensure_scratch(ctx, K);
+    if (rc != FASTRACK_OK) return rc;
+    return launch_pass(ctx, false, iv_base, 0, d_cipher, len, d_plain, d_tags, nullptr, d_ok, (cudaStream_t)stream);
+}
+
+extern "C" int fastrack_encrypt_tag(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_plain, size_t len,
+                                    void* d_cipher, void* d_tags, void* stream)
+{
+    if (!ctx || !iv_base) return FASTRACK_ERR_ARG;
+    if (len == 0) return FASTRACK_OK;
+    if (!d_plain || !d_cipher || !d_tags) return FASTRACK_ERR_ARG;
+    if (misaligned(d_cipher, 16) || misaligned(d_plain, 16) || misaligned(d_tags, 16)) return FASTRACK_ERR_ARG;
+    if (bad_overlap(d_cipher, d_plain, len)) return FASTRACK_ERR_ARG;
+    const size_t K = fastrack_num_chunks(ctx, len);
+    if (K > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
+    int rc = ensure_scratch(ctx, K);
+    if (rc != FASTRACK_OK) return rc;
+    return launch_pass(ctx, true, iv_base, 0, d_plain, len, d_cipher, nullptr, d_tags, nullptr, (cudaStream_t)stream);
+}
+
+extern "C" int fastrack_pipelined_h2d(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* h_cipher_pinned, size_t len,
+                                      const void* h_tags, void* d_plain, uint32_t* d_ok, int n_streams)
+{
+    if (!ctx || !iv_base) return FASTRACK_ERR_ARG;
+    if (n_streams < 1 || n_streams > 8) return FASTRACK_ERR_ARG;
+    if (len == 0) return FASTRACK_OK;
+    if (!h_cipher_pinned || !h_tags || !d_plain || !d_ok) return FASTRACK_ERR_ARG;
+    if (misaligned(d_plain, 16) || misaligned(d_ok, 4)) return FASTRACK_ERR_ARG;
+    cudaPointerAttributes attr;
+    cudaError_t e = cudaPointerGetAttributes(&attr, h_cipher_pinned);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return FASTRACK_ERR_NOT_PINNED; }
+    if (attr.type != cudaMemoryTypeHost) return FASTRACK_ERR_NOT_PINNED;
+    const size_t K = fastrack_num_chunks(ctx, len);
+    if (K > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
+    int rc = ensure_scratch(ctx, K);
+    if (rc != FASTRACK_OK) return rc;
+    if (K > ctx->tags_stage_chunks) {
+        size_t cap = ctx->tags_stage_chunks ? ctx->tags_stage_chunks : 1024;
+        while (cap < K) cap *= 2;
+        FR_CUDA(ctx, cudaDeviceSynchronize());
+        cudaFree(ctx->d_tags_stage);
+        ctx->d_tags_stage = nullptr;
+        ctx->tags_stage_chunks = 0;
+        e = cudaMalloc(&ctx->d_tags_stage, cap * 16);
+        if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); return FASTRACK_ERR_NOMEM; }
+        ctx->tags_stage_chunks = cap;
+    }
+
+    // tags first, once; every other stream waits for that copy before its first kernel
+    FR_CUDA(ctx, cudaMemcpyAsync(ctx->d_tags_stage, h_tags, K * 16, cudaMemcpyHostToDevice, ctx->streams[0]));
+    FR_CUDA(ctx, cudaEventRecord(ctx->tags_ready, ctx->streams[0]));
+    for (int i = 1; i < n_streams; i++) FR_CUDA(ctx, cudaStreamWaitEvent(ctx->streams[i], ctx->tags_ready, 0));
+
+    const size_t cb = ctx->chunk_bytes;
+    const size_t min_stage = (size_t)1 << 20;
+    const size_t chunks_per_stage = cb >= min_stage ? 1 : min_stage / cb;
+    const size_t stage_bytes = chunks_per_stage * cb;
+    size_t stage = 0;
+    for (size_t off = 0; off < len; off += stage_bytes, stage++) {
+        const size_t n = len - off < stage_bytes ? len - off : stage_bytes;
+        const size_t k0 = off / cb;
+        cudaStream_t st = ctx->streams[stage % (size_t)n_streams];
+        uint8_t* dst = (uint8_t*)d_plain + off;
+        rc = FASTRACK_OK;
+        e = cudaMemcpyAsync(dst, (const uint8_t*)h_cipher_pinned + off, n, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); rc = FASTRACK_ERR_CUDA; }
+        if (rc == FASTRACK_OK) rc = launch_pass(ctx, false, iv_base, k0, dst, n, dst, ctx->d_tags_stage + k0, nullptr, d_ok + k0, st);
+        if (rc != FASTRACK_OK) {
+            for (int i = 0; i < n_streams; i++) cudaStreamSynchronize(ctx->streams[i]);
+            (void)cudaGetLastError();
+            return rc;
+        }
+    }
+    for (int i = 0; i < n_streams; i++) FR_CUDA(ctx, cudaStreamSynchronize(ctx->streams[i]));
+    return FASTRACK_OK;
+}

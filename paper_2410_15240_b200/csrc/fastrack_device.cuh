@@ -1,0 +1,293 @@
+// fastrack_device.cuh -- per-lane device code of the fused AES-256-CTR + GHASH pass (sm_100a).
+//
+// One warp works on one "segment": a run of consecutive rows of one chunk, a row being 32 consecutive
+// 16-byte blocks (512 B, one block per lane, so global loads and stores are 128-bit and coalesced).
+//
+// AES (paper Section 2.3, "The AES block cipher": AES in counter mode, every block independent):
+//   four round tables Te0..Te3 live in shared memory, each entry replicated 32 times so that lane l
+//   only ever touches bank l -- a table lookup is one conflict-free wavefront whatever the index.
+//   Row v of array T01 is [Te0[v] x32 | Te1[v] x32] (256 B), array T23 likewise; the byte address
+//   v*256 + 4*lane is produced by ONE byte-permute from the state word and the lane register.
+//
+// GHASH (paper Section 2.3, "Authentication with Galois Field"; Section 4.2 shortens the chain by
+// chunking, here every chain is additionally evaluated as a power sum):
+//   lane l of the warp folds blocks l, l+32, l+64, ... with Horner's rule and the FIXED multiplier
+//   H^32, Y <- (Y xor X) * H^32, using byte tables of H^32 in shared memory (entry for byte position p
+//   and byte value v at v*256 + p*16).  Lanes walk the 16 byte positions in a lane-dependent order
+//   (position = step xor (lane & 7)) so that the eight lanes of a quarter-warp always hit eight
+//   different 16-byte bank groups: every 128-bit lookup is conflict-free.  The lane's last block is
+//   not multiplied by H^32 but by the power of H that its distance from the end of the chunk calls
+//   for, with a general (bit-serial) product; the 32 lane values are then XOR-reduced.
+#pragma once
+#include <stdint.h>
+
+#define FR_SM_T01 0u          // AES rows [Te0 x32 | Te1 x32]
+#define FR_SM_T23 65536u      // AES rows [Te2 x32 | Te3 x32]
+#define FR_SM_GH 131072u      // byte tables of H^32
+#define FR_SMEM_BYTES 196608u
+
+#define FR_ROW_BLOCKS 32u     // blocks per row (one per lane)
+#define FR_HORNER_STRIDE 32u  // the fixed multiplier is H^32
+
+struct FrParams {
+    uint32_t rk[60];           // AES-256 round keys, word i = little-endian load of key-schedule bytes 4i..4i+3
+    uint32_t iv_w0, iv_w1;     // little-endian loads of iv_base[0..3], iv_base[4..7]
+    uint32_t iv_ctr;           // BE32(iv_base[8..11]) + index of this launch's first chunk
+    uint32_t seg_rows;         // rows per segment
+    uint32_t segs_per_chunk;   // segments of a full-size chunk
+    uint32_t n_chunks;         // chunks in this launch
+    uint32_t n_items;          // n_chunks * segs_per_chunk
+    uint32_t pad0;
+    uint64_t len;              // bytes in this launch
+    uint64_t chunk_bytes;
+    const uint8_t* in;
+    uint8_t* out;
+    const uint4* tags_in;      // decrypt
+    uint4* tags_out;           // encrypt
+    uint32_t* ok;              // decrypt
+    const uint32_t* te0;       // 256 words
+    const uint4* gh_tab;       // 4096 entries, same layout as shared memory
+    const uint4* pow;          // pow[e] = H^e
+    uint32_t* acc;             // per chunk 4 words, zero between launches
+    uint32_t* cnt;             // per chunk arrival counter, zero between launches
+};
+
+// Byte permute, PTX prmt.b32 in generic mode: result byte i = byte (sel nibble i & 7) of {a (0..3), b (4..7)};
+// nibble bit 3 replicates that byte's sign bit instead.
+#ifndef FR_PRMT
+__device__ __forceinline__ uint32_t fr_prmt_ptx(uint32_t a, uint32_t b, uint32_t s)
+{
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(s));
+    return r;
+}
+#define FR_PRMT(a, b, s) fr_prmt_ptx((a), (b), (s))
+#endif
+
+__device__ __forceinline__ uint32_t fr_bswap(uint32_t x) { return FR_PRMT(x, 0u, 0x0123u); }
+
+__device__ __forceinline__ uint4 fr_xor4(uint4 a, uint4 b)
+{
+    return make_uint4(a.x ^ b.x, a.y ^ b.y, a.z ^ b.z, a.w ^ b.w);
+}
+
+// Lane-constant registers.
+struct FrLane {
+    uint32_t lane4;      // 4 * lane: byte offset of this lane's bank inside a table row
+    uint32_t sel[4];     // GHASH selectors for byte step rho = 0..3
+    uint32_t qe, qo;     // GHASH slot bytes for even / odd word steps
+    uint32_t h;          // (lane >> 2) & 1
+};
+
+__device__ __forceinline__ FrLane fr_make_lane(uint32_t lane)
+{
+    FrLane L;
+    L.lane4 = lane * 4u;
+    uint32_t c = lane & 3u, h = (lane >> 2) & 1u;
+    L.h = h;
+    L.qe = 0; L.qo = 0;
+    for (uint32_t rho = 0; rho < 4; rho++) {
+        uint32_t cc = rho ^ c;
+        L.qe |= (((0u ^ h) << 6) | (cc << 4)) << (8 * rho);
+        L.qo |= (((1u ^ h) << 6) | (cc << 4)) << (8 * rho);
+        // result = [q.byte rho, v.byte cc, 0, 0]; the zeros are q.byte0's sign bit (always clear) replicated
+        L.sel[rho] = (4u + rho) | (cc << 4) | (0xCu << 8) | (0xCu << 12);
+    }
+    return L;
+}
+
+// Fill shared memory: replicate Te0 and its three byte rotations per lane, copy the H^32 byte tables.
+__device__ __forceinline__ void fr_build_smem(char* sm, uint32_t tid, uint32_t nthreads,
+                                              const uint32_t* __restrict__ te0, const uint4* __restrict__ gh_tab)
+{
+    // 256 rows x 2 arrays x 2 tables x 8 uint4 (32 words) each
+    for (uint32_t i = tid; i < 256u * 4u * 8u; i += nthreads) {
+        uint32_t q = i & 7u, t = (i >> 3) & 3u, v = i >> 5;
+        uint32_t e = te0[v];
+        uint32_t w = (t == 0) ? e : (t == 1) ? ((e << 8) | (e >> 24)) : (t == 2) ? ((e << 16) | (e >> 16)) : ((e << 24) | (e >> 8));
+        uint32_t off = ((t >> 1) ? FR_SM_T23 : FR_SM_T01) + v * 256u + (t & 1u) * 128u + q * 16u;
+        *(uint4*)(sm + off) = make_uint4(w, w, w, w);
+    }
+    for (uint32_t i = tid; i < 4096u; i += nthreads) *(uint4*)(sm + FR_SM_GH + i * 16u) = gh_tab[i];
+}
+
+// AES-256 forward cipher on the state (s0..s3), which already holds counter-block xor round key 0.
+#define FR_TA(w, k) FR_PRMT((w), lane4, 0x5504u | ((k) << 4))
+#define FR_LD32(off, addr) (*(const uint32_t*)(sm + (off) + (addr)))
+__device__ __forceinline__ uint4 fr_aes256_rounds(const char* sm, uint32_t lane4, const FrParams& P,
+                                                  uint32_t s0, uint32_t s1, uint32_t s2, uint32_t s3)
+{
+#pragma unroll
+    for (int r = 1; r < 14; r++) {
+        uint32_t t0 = FR_LD32(FR_SM_T01, FR_TA(s0, 0)) ^ FR_LD32(FR_SM_T01 + 128u, FR_TA(s1, 1)) ^
+                      FR_LD32(FR_SM_T23, FR_TA(s2, 2)) ^ FR_LD32(FR_SM_T23 + 128u, FR_TA(s3, 3)) ^ P.rk[4 * r + 0];
+        uint32_t t1 = FR_LD32(FR_SM_T01, FR_TA(s1, 0)) ^ FR_LD32(FR_SM_T01 + 128u, FR_TA(s2, 1)) ^
+                      FR_LD32(FR_SM_T23, FR_TA(s3, 2)) ^ FR_LD32(FR_SM_T23 + 128u, FR_TA(s0, 3)) ^ P.rk[4 * r + 1];
+        uint32_t t2 = FR_LD32(FR_SM_T01, FR_TA(s2, 0)) ^ FR_LD32(FR_SM_T01 + 128u, FR_TA(s3, 1)) ^
+                      FR_LD32(FR_SM_T23, FR_TA(s0, 2)) ^ FR_LD32(FR_SM_T23 + 128u, FR_TA(s1, 3)) ^ P.rk[4 * r + 2];
+        uint32_t t3 = FR_LD32(FR_SM_T01, FR_TA(s3, 0)) ^ FR_LD32(FR_SM_T01 + 128u, FR_TA(s0, 1)) ^
+                      FR_LD32(FR_SM_T23, FR_TA(s1, 2)) ^ FR_LD32(FR_SM_T23 + 128u, FR_TA(s2, 3)) ^ P.rk[4 * r + 3];
+        s0 = t0; s1 = t1; s2 = t2; s3 = t3;
+    }
+    // Last round: SubBytes + ShiftRows only.  Te2 has S in byte 0, Te3 in byte 1, Te0 in byte 2, Te1 in byte 3.
+    uint32_t o[4];
+    const uint32_t in[4] = {s0, s1, s2, s3};
+#pragma unroll
+    for (int c = 0; c < 4; c++) {
+        uint32_t a = FR_LD32(FR_SM_T23, FR_TA(in[c], 0));
+        uint32_t b = FR_LD32(FR_SM_T23 + 128u, FR_TA(in[(c + 1) & 3], 1));
+        uint32_t cc = FR_LD32(FR_SM_T01, FR_TA(in[(c + 2) & 3], 2));
+        uint32_t d = FR_LD32(FR_SM_T01 + 128u, FR_TA(in[(c + 3) & 3], 3));
+        uint32_t lo = FR_PRMT(a, b, 0x0050u);    // [a.0, b.1, -, -]
+        uint32_t hi = FR_PRMT(cc, d, 0x7200u);   // [-, -, c.2, d.3]
+        o[c] = FR_PRMT(lo, hi, 0x7610u) ^ P.rk[56 + c];
+    }
+    return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+// E_K(IV_k || BE32(ctr)) for chunk-relative IV word `ivw2` (little-endian load of IV_k[8..11]).
+__device__ __forceinline__ uint4 fr_aes256_ctr_block(const char* sm, uint32_t lane4, const FrParams& P,
+                                                     uint32_t ivw2, uint32_t ctr)
+{
+    return fr_aes256_rounds(sm, lane4, P, P.iv_w0 ^ P.rk[0], P.iv_w1 ^ P.rk[1], ivw2 ^ P.rk[2],
+                            fr_bswap(ctr) ^ P.rk[3]);
+}
+
+// v * H^32 through the byte tables (v, result: little-endian words of the block's 16 bytes).
+__device__ __forceinline__ uint4 fr_ghash_tabmul(const char* sm, const FrLane& L, uint4 v)
+{
+    // lanes with h = 1 walk the words in swapped pairs, so static word w holds actual word w ^ h
+    uint32_t s[4];
+    s[0] = L.h ? v.y : v.x; s[1] = L.h ? v.x : v.y; s[2] = L.h ? v.w : v.z; s[3] = L.h ? v.z : v.w;
+    uint4 acc = make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (int w = 0; w < 4; w++) {
+#pragma unroll
+        for (int rho = 0; rho < 4; rho++) {
+            uint32_t addr = FR_PRMT(s[w], (w & 1) ? L.qo : L.qe, L.sel[rho]);
+            uint4 t = *(const uint4*)(sm + FR_SM_GH + ((uint32_t)(w >> 1) << 7) + addr);
+            acc = fr_xor4(acc, t);
+        }
+    }
+    return acc;
+}
+
+// General product in GF(2^128) (GCM bit order: bit 0 of a block is the MSB of byte 0 and the
+// coefficient of x^0; "times x" is a right shift with 0xE1 folded into byte 0 on carry-out).
+__device__ __forceinline__ uint4 fr_gf128_mul(uint4 x, uint4 y)
+{
+    uint32_t xw[4] = {fr_bswap(x.x), fr_bswap(x.y), fr_bswap(x.z), fr_bswap(x.w)};
+    uint32_t v0 = fr_bswap(y.x), v1 = fr_bswap(y.y), v2 = fr_bswap(y.z), v3 = fr_bswap(y.w);
+    uint32_t z0 = 0, z1 = 0, z2 = 0, z3 = 0;
+#pragma unroll 1
+    for (int w = 0; w < 4; w++) {
+        uint32_t xb = xw[w];
+#pragma unroll 8
+        for (int b = 0; b < 32; b++) {
+            uint32_t m = (uint32_t)((int32_t)xb >> 31);
+            xb <<= 1;
+            z0 ^= v0 & m; z1 ^= v1 & m; z2 ^= v2 & m; z3 ^= v3 & m;
+            uint32_t carry = (0u - (v3 & 1u)) & 0xE1000000u;
+            v3 = (v3 >> 1) | (v2 << 31);
+            v2 = (v2 >> 1) | (v1 << 31);
+            v1 = (v1 >> 1) | (v0 << 31);
+            v0 = (v0 >> 1) ^ carry;
+        }
+    }
+    return make_uint4(fr_bswap(z0), fr_bswap(z1), fr_bswap(z2), fr_bswap(z3));
+}
+
+__device__ __forceinline__ uint64_t fr_chunk_len(const FrParams& P, uint32_t kk)
+{
+    uint64_t off = (uint64_t)kk * P.chunk_bytes;
+    uint64_t rem = P.len - off;
+    return rem < P.chunk_bytes ? rem : P.chunk_bytes;
+}
+
+__device__ __forceinline__ uint32_t fr_chunk_segs(const FrParams& P, uint32_t kk)
+{
+    uint32_t nblk = (uint32_t)((fr_chunk_len(P, kk) + 15) >> 4);
+    uint32_t rows = (nblk + FR_ROW_BLOCKS - 1) / FR_ROW_BLOCKS;
+    return (rows + P.seg_rows - 1) / P.seg_rows;
+}
+
+// Load / store the last, partial block of the buffer byte by byte (zero-padded in registers).
+__device__ __forceinline__ uint4 fr_load_partial(const uint8_t* p, uint32_t n)
+{
+    uint32_t w[4] = {0, 0, 0, 0};
+    for (uint32_t i = 0; i < n; i++) w[i >> 2] |= (uint32_t)p[i] << (8 * (i & 3));
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+__device__ __forceinline__ void fr_store_partial(uint8_t* p, uint4 v, uint32_t n)
+{
+    uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    for (uint32_t i = 0; i < n; i++) p[i] = (uint8_t)(w[i >> 2] >> (8 * (i & 3)));
+}
+
+__device__ __forceinline__ uint4 fr_mask_bytes(uint4 v, uint32_t n)
+{
+    uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    for (uint32_t i = 0; i < 4; i++) {
+        uint32_t lo = 4 * i;
+        if (n <= lo) w[i] = 0;
+        else if (n < lo + 4) w[i] &= (1u << (8 * (n - lo))) - 1u;
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// One lane's share of segment s of chunk kk: decrypt (or encrypt) its blocks, fold them into the
+// lane's Horner value, and return that value multiplied by the power of H that aligns it to the end
+// of the chunk.  XOR of the 32 lanes' results = the segment's contribution to the chunk's GHASH
+// (before the length block).
+template <bool ENCRYPT>
+__device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, const char* sm, const FrLane& L,
+                                                         uint32_t lane, uint32_t kk, uint32_t s)
+{
+    const uint64_t chunk_off = (uint64_t)kk * P.chunk_bytes;
+    const uint64_t len_k = fr_chunk_len(P, kk);
+    const uint32_t nblk = (uint32_t)((len_k + 15) >> 4);
+    const uint32_t rows = (nblk + FR_ROW_BLOCKS - 1) / FR_ROW_BLOCKS;
+    const uint32_t row0 = s * P.seg_rows;
+    uint32_t row1 = row0 + P.seg_rows;
+    if (row1 > rows) row1 = rows;
+    uint32_t seg_end = row1 * FR_ROW_BLOCKS;       // first block index after this segment
+    if (seg_end > nblk) seg_end = nblk;
+    const uint8_t* in = P.in + chunk_off;
+    uint8_t* out = P.out + chunk_off;
+    const uint32_t ivw2 = fr_bswap(P.iv_ctr + kk);
+
+    uint4 y = make_uint4(0, 0, 0, 0), pend = make_uint4(0, 0, 0, 0);
+    uint32_t j_last = 0xFFFFFFFFu;
+    for (uint32_t r = row0; r < row1; r++) {
+        const uint32_t j = r * FR_ROW_BLOCKS + lane;
+        if (j < seg_end) {
+            const uint64_t boff = (uint64_t)j << 4;
+            const bool full = len_k - boff >= 16;
+            const uint32_t nvalid = full ? 16u : (uint32_t)(len_k - boff);
+            uint4 x = full ? *(const uint4*)(in + boff) : fr_load_partial(in + boff, nvalid);
+            uint4 ks = fr_aes256_ctr_block(sm, L.lane4, P, ivw2, j + 2u);
+            uint4 o = fr_xor4(x, ks);
+            if (full) *(uint4*)(out + boff) = o; else fr_store_partial(out + boff, o, nvalid);
+            uint4 g = ENCRYPT ? (full ? o : fr_mask_bytes(o, nvalid)) : x;
+            uint4 v = fr_xor4(y, g);
+            if (j + FR_HORNER_STRIDE < seg_end) y = fr_ghash_tabmul(sm, L, v);
+            else { pend = v; j_last = j; }
+        }
+    }
+    if (j_last == 0xFFFFFFFFu) return make_uint4(0, 0, 0, 0);
+    // block j is multiplied by H^(nblk - j + 1): one for each later block, one for the length block
+    const uint32_t e = (nblk - 1u - j_last) + 2u;
+    return fr_gf128_mul(pend, P.pow[e]);
+}
+
+// Tag of chunk kk from its data sum: T = S xor LEN*H xor E_K(IV_k || 1)  (paper Section 2.3: the final
+// product is combined with the encrypted nonce block; Section 4.2: one such block per chain).
+__device__ __forceinline__ uint4 fr_chunk_tag(const FrParams& P, const char* sm, uint32_t lane4, uint32_t kk, uint4 S)
+{
+    const uint64_t bits = fr_chunk_len(P, kk) << 3;
+    uint4 lenblk = make_uint4(0, 0, fr_bswap((uint32_t)(bits >> 32)), fr_bswap((uint32_t)bits));
+    uint4 t = fr_gf128_mul(lenblk, P.pow[1]);
+    uint4 ekj0 = fr_aes256_ctr_block(sm, lane4, P, fr_bswap(P.iv_ctr + kk), 1u);
+    return fr_xor4(fr_xor4(S, t), ekj0);
+}

@@ -1,0 +1,148 @@
+"""ctypes binding of the C-ABI CUDA library (see include/fastrack.h for the contract).
+
+Argument marshalling only: every step of the path runs in the library's kernels.  Device and
+pinned-host buffers are passed as integer addresses (``tensor.data_ptr()``), streams as the integer
+``cudaStream_t`` (``torch.cuda.current_stream().cuda_stream``); ``key`` and ``iv_base`` are bytes.
+Importing this module raises if ``libfastrack.so`` has not been built -- there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libfastrack.so")
+
+OK = 0
+ERR_ARG, ERR_CHUNK, ERR_NOT_PINNED, ERR_CUDA, ERR_NOMEM, ERR_TOO_MANY = -1, -2, -3, -4, -5, -6
+MAX_CHUNK_BYTES = 1 << 30
+
+EXPORTS = ("fastrack_ctx_create", "fastrack_ctx_destroy", "fastrack_num_chunks", "fastrack_ctx_reserve",
+           "fastrack_last_cuda_error", "fastrack_decrypt_verify", "fastrack_encrypt_tag",
+           "fastrack_pipelined_h2d", "fastrack_launch_count")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2410_15240_b200.build` "
+                      "(there is no CPU fallback)")
+
+_lib = ctypes.CDLL(LIB_PATH)
+_vp, _sz, _int = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int
+_lib.fastrack_ctx_create.restype = _int
+_lib.fastrack_ctx_create.argtypes = [ctypes.c_char_p, _sz, ctypes.POINTER(_vp)]
+_lib.fastrack_ctx_destroy.restype = None
+_lib.fastrack_ctx_destroy.argtypes = [_vp]
+_lib.fastrack_num_chunks.restype = _sz
+_lib.fastrack_num_chunks.argtypes = [_vp, _sz]
+_lib.fastrack_ctx_reserve.restype = _int
+_lib.fastrack_ctx_reserve.argtypes = [_vp, _sz]
+_lib.fastrack_last_cuda_error.restype = _int
+_lib.fastrack_last_cuda_error.argtypes = [_vp]
+_lib.fastrack_launch_count.restype = ctypes.c_uint64
+_lib.fastrack_launch_count.argtypes = [_vp]
+_lib.fastrack_decrypt_verify.restype = _int
+_lib.fastrack_decrypt_verify.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp, _vp]
+_lib.fastrack_encrypt_tag.restype = _int
+_lib.fastrack_encrypt_tag.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp]
+_lib.fastrack_pipelined_h2d.restype = _int
+_lib.fastrack_pipelined_h2d.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp, _int]
+
+
+class FastrackError(RuntimeError):
+    def __init__(self, code: int, cuda_error: int = 0):
+        self.code, self.cuda_error = code, cuda_error
+        super().__init__(f"fastrack error {code}" + (f" (CUDA error {cuda_error})" if cuda_error else ""))
+
+
+def fastrack_ctx_create(key: bytes, chunk_bytes: int):
+    """-> (return code, context handle or None)."""
+    handle = _vp()
+    key_arg = bytes(key) if key is not None else None
+    rc = _lib.fastrack_ctx_create(key_arg, chunk_bytes, ctypes.byref(handle))
+    return rc, (handle.value if rc == OK else None)
+
+
+def fastrack_ctx_destroy(ctx) -> None:
+    _lib.fastrack_ctx_destroy(ctx)
+
+
+def fastrack_num_chunks(ctx, length: int) -> int:
+    return int(_lib.fastrack_num_chunks(ctx, length))
+
+
+def fastrack_ctx_reserve(ctx, max_len: int) -> int:
+    return _lib.fastrack_ctx_reserve(ctx, max_len)
+
+
+def fastrack_last_cuda_error(ctx) -> int:
+    return _lib.fastrack_last_cuda_error(ctx)
+
+
+def fastrack_launch_count(ctx) -> int:
+    return int(_lib.fastrack_launch_count(ctx))
+
+
+def fastrack_decrypt_verify(ctx, iv_base: bytes, d_cipher: int, length: int, d_tags: int, d_plain: int,
+                            d_ok: int, stream: int = 0) -> int:
+    return _lib.fastrack_decrypt_verify(ctx, iv_base, d_cipher, length, d_tags, d_plain, d_ok, stream)
+
+
+def fastrack_encrypt_tag(ctx, iv_base: bytes, d_plain: int, length: int, d_cipher: int, d_tags: int,
+                         stream: int = 0) -> int:
+    return _lib.fastrack_encrypt_tag(ctx, iv_base, d_plain, length, d_cipher, d_tags, stream)
+
+
+def fastrack_pipelined_h2d(ctx, iv_base: bytes, h_cipher_pinned: int, length: int, h_tags: int, d_plain: int,
+                           d_ok: int, n_streams: int) -> int:
+    return _lib.fastrack_pipelined_h2d(ctx, iv_base, h_cipher_pinned, length, h_tags, d_plain, d_ok, n_streams)
+
+
+class Context:
+    """RAII wrapper: ``with Context(key, chunk_bytes) as ctx: ctx.decrypt_verify(...)``; raises FastrackError."""
+
+    def __init__(self, key: bytes, chunk_bytes: int):
+        rc, handle = fastrack_ctx_create(key, chunk_bytes)
+        if rc != OK:
+            raise FastrackError(rc)
+        self.handle = handle
+        self.chunk_bytes = chunk_bytes
+
+    def _check(self, rc: int) -> None:
+        if rc != OK:
+            raise FastrackError(rc, fastrack_last_cuda_error(self.handle))
+
+    def num_chunks(self, length: int) -> int:
+        return fastrack_num_chunks(self.handle, length)
+
+    def reserve(self, max_len: int) -> None:
+        self._check(fastrack_ctx_reserve(self.handle, max_len))
+
+    def decrypt_verify(self, iv_base, d_cipher, length, d_tags, d_plain, d_ok, stream=0) -> None:
+        self._check(fastrack_decrypt_verify(self.handle, iv_base, d_cipher, length, d_tags, d_plain, d_ok, stream))
+
+    def encrypt_tag(self, iv_base, d_plain, length, d_cipher, d_tags, stream=0) -> None:
+        self._check(fastrack_encrypt_tag(self.handle, iv_base, d_plain, length, d_cipher, d_tags, stream))
+
+    def pipelined_h2d(self, iv_base, h_cipher_pinned, length, h_tags, d_plain, d_ok, n_streams=4) -> None:
+        self._check(fastrack_pipelined_h2d(self.handle, iv_base, h_cipher_pinned, length, h_tags, d_plain, d_ok,
+                                           n_streams))
+
+    @property
+    def launches(self) -> int:
+        return fastrack_launch_count(self.handle)
+
+    def close(self) -> None:
+        if self.handle is not None:
+            fastrack_ctx_destroy(self.handle)
+            self.handle = None
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

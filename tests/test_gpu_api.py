@@ -1,0 +1,87 @@
+"""GPU-side API and error-path checks of the C ABI."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2410_15240_b200 import fastrack, synth
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+if not torch.cuda.is_available():
+    pytest.skip("no CUDA device", allow_module_level=True)
+
+
+def test_context_lifecycle_and_chunk_count():
+    rc, ctx = fastrack.fastrack_ctx_create(bytes(32), 65536)
+    assert rc == fastrack.OK and ctx
+    assert fastrack.fastrack_num_chunks(ctx, 0) == 0
+    assert fastrack.fastrack_num_chunks(ctx, 1) == 1
+    assert fastrack.fastrack_num_chunks(ctx, 65536) == 1
+    assert fastrack.fastrack_num_chunks(ctx, 65537) == 2
+    assert fastrack.fastrack_ctx_reserve(ctx, 1 << 30) == fastrack.OK
+    assert fastrack.fastrack_last_cuda_error(ctx) == 0
+    assert fastrack.fastrack_launch_count(ctx) == 0
+    fastrack.fastrack_ctx_destroy(ctx)
+
+
+def test_argument_errors():
+    rc, ctx = fastrack.fastrack_ctx_create(bytes(32), 1024)
+    assert rc == fastrack.OK
+    buf = torch.zeros(8192, dtype=torch.uint8, device="cuda")
+    tags = torch.zeros(16 * 8, dtype=torch.uint8, device="cuda")
+    ok = torch.zeros(8, dtype=torch.int32, device="cuda")
+    b, t, o = buf.data_ptr(), tags.data_ptr(), ok.data_ptr()
+    iv = bytes(12)
+    D, E = fastrack.fastrack_decrypt_verify, fastrack.fastrack_encrypt_tag
+    assert D(ctx, iv, b, 0, t, b, o, 0) == fastrack.OK                       # len 0: nothing to do
+    assert D(ctx, None, b, 1024, t, b, o, 0) == fastrack.ERR_ARG
+    assert D(ctx, iv, 0, 1024, t, b, o, 0) == fastrack.ERR_ARG
+    assert D(ctx, iv, b, 1024, 0, b, o, 0) == fastrack.ERR_ARG
+    assert D(ctx, iv, b, 1024, t, 0, o, 0) == fastrack.ERR_ARG
+    assert D(ctx, iv, b, 1024, t, b, 0, 0) == fastrack.ERR_ARG
+    assert D(ctx, iv, b + 8, 1024, t, b + 4096, o, 0) == fastrack.ERR_ARG    # misaligned input
+    assert D(ctx, iv, b, 1024, t, b + 4096 + 4, o, 0) == fastrack.ERR_ARG    # misaligned output
+    assert D(ctx, iv, b, 1024, t + 8, b + 4096, o, 0) == fastrack.ERR_ARG    # misaligned tags
+    assert D(ctx, iv, b, 2048, t, b + 1024, o, 0) == fastrack.ERR_ARG        # partial overlap
+    assert D(ctx, iv, b + 1024, 2048, t, b, o, 0) == fastrack.ERR_ARG
+    assert E(ctx, iv, b, 2048, b + 16, t, 0) == fastrack.ERR_ARG
+    assert E(ctx, iv, b, 2048, b, 0, 0) == fastrack.ERR_ARG
+    assert D(ctx, iv, b, 2048, t, b + 2048, o, 0) == fastrack.OK             # adjacent, no overlap
+    assert D(ctx, iv, b, 2048, t, b, o, 0) == fastrack.OK                    # exact alias = in place
+    torch.cuda.synchronize()
+    # pipelined: pageable source is refused, stream count is bounded
+    pageable = np.zeros(4096, np.uint8)
+    h_tags = np.zeros(64, np.uint8)
+    P = fastrack.fastrack_pipelined_h2d
+    assert P(ctx, iv, pageable.ctypes.data, 4096, h_tags.ctypes.data, b, o, 2) == fastrack.ERR_NOT_PINNED
+    pinned = torch.zeros(4096, dtype=torch.uint8).pin_memory()
+    assert P(ctx, iv, pinned.data_ptr(), 4096, h_tags.ctypes.data, b, o, 0) == fastrack.ERR_ARG
+    assert P(ctx, iv, pinned.data_ptr(), 4096, h_tags.ctypes.data, b, o, 9) == fastrack.ERR_ARG
+    assert P(ctx, iv, pinned.data_ptr(), 0, h_tags.ctypes.data, b, o, 2) == fastrack.OK
+    assert P(ctx, iv, pinned.data_ptr(), 4096, h_tags.ctypes.data, b, o, 2) == fastrack.OK
+    assert fastrack.fastrack_launch_count(ctx) >= 3
+    fastrack.fastrack_ctx_destroy(ctx)
+
+
+def test_calls_are_asynchronous_and_ordered_on_the_stream():
+    """encrypt then decrypt queued back to back on one stream without host synchronisation in between."""
+    key, iv = synth.key_and_iv(0)
+    cb, n = 65536, 4 << 20
+    plain = synth.random_bytes(n, 0, salt=21)
+    K = n // cb
+    with fastrack.Context(key, cb) as ctx:
+        d_p = torch.from_numpy(plain).cuda()
+        d_c = torch.empty_like(d_p)
+        d_back = torch.empty_like(d_p)
+        d_t = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
+        d_ok = torch.zeros(K, dtype=torch.int32, device="cuda")
+        st = torch.cuda.Stream()
+        with torch.cuda.stream(st):
+            ctx.encrypt_tag(iv, d_p.data_ptr(), n, d_c.data_ptr(), d_t.data_ptr(), st.cuda_stream)
+            ctx.decrypt_verify(iv, d_c.data_ptr(), n, d_t.data_ptr(), d_back.data_ptr(), d_ok.data_ptr(), st.cuda_stream)
+        st.synchronize()
+        assert ctx.launches == 2
+        assert bool((d_back == d_p).all()) and bool((d_ok == 1).all())
+        c_ref, t_ref = oracle.mc_encrypt(key, iv, cb, plain, oracle.host_threads())
+        assert np.array_equal(d_c.cpu().numpy(), c_ref) and np.array_equal(d_t.cpu().numpy().reshape(K, 16), t_ref)

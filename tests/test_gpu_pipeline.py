@@ -1,0 +1,49 @@
+"""GPU parity of the pipelined H2D path (paper Section 4.3) against the CPU oracle."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2410_15240_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+if not torch.cuda.is_available():
+    pytest.skip("no CUDA device", allow_module_level=True)
+
+from gpu_harness import Gpu  # noqa: E402
+
+NT = oracle.host_threads()
+
+
+@pytest.mark.parametrize("n,cb", [(1, 16), (100, 1024), (1 << 20, 65536), ((1 << 20) + 17, 65536),
+                                  (3 * (1 << 20) + 5, 1 << 20), (9 * (1 << 20) + 12345, 256 * 1024),
+                                  ((5 << 20) - 16, 48 * 1024), (2 * (1 << 22) + 999, 1 << 22)])
+@pytest.mark.parametrize("n_streams", [1, 3])
+def test_pipelined_matches_oracle_small(n, cb, n_streams):
+    key, iv = synth.key_and_iv(2)
+    plain = synth.random_bytes(n, 2, salt=n)
+    c, t = oracle.mc_encrypt(key, iv, cb, plain, NT)
+    plan = synth.tamper_plan(n, cb, 2, fraction=0.1, salt=n)
+    synth.apply_tamper(c, t, cb, plan)
+    p_ref, ok_ref = oracle.mc_decrypt(key, iv, cb, c, t, NT)
+    with Gpu(key, cb) as g:
+        p, ok = g.pipelined(iv, c, t, n_streams)
+        assert np.array_equal(ok, ok_ref)
+        assert np.array_equal(p, p_ref)
+        p2, ok2 = g.pipelined(iv, c, t, n_streams, pinned_tags=True)      # context reuse
+        assert np.array_equal(ok2, ok_ref) and np.array_equal(p2, p_ref)
+    assert sorted(k for k, _, _ in plan) == [int(k) for k in np.flatnonzero(ok_ref == 0)]
+
+
+@pytest.mark.parametrize("cb,n_streams", [(256 * 1024, 2), (1 << 20, 3), (4 << 20, 4), (8 << 20, 2)])
+def test_config2_fp16_image_batch(cb, n_streams):
+    """fp16 256x3x224x224 ~ N(0,1) (77 070 336 B), oracle-encrypted, pipelined H2D + decrypt/verify."""
+    key, iv = synth.key_and_iv(2)
+    plain = synth.fp16_image_batch()
+    assert plain.size == 77_070_336
+    c, t = oracle.mc_encrypt(key, iv, cb, plain, NT)
+    with Gpu(key, cb) as g:
+        p, ok = g.pipelined(iv, c, t, n_streams)
+    assert (ok == 1).all() and ok.size == oracle.num_chunks(plain.size, cb)
+    assert np.array_equal(p, plain)
