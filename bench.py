@@ -1,0 +1,348 @@
+#!/usr/bin/env python
+"""Benchmark of the Fastrack GPU hot path on B200.
+
+One step = one pass of the whole hot path over one batch: GPU authenticated decryption
+(AES-256-CTR keystream + XOR + per-chunk GHASH + tag compare) of a 256 MiB buffer cut into 4 MiB
+chunks (K = 64).  `value` is payload GB/s with the ciphertext already resident in HBM; `e2e` is the
+same metric through fastrack_pipelined_h2d with the ciphertext in pinned HOST memory (PCIe copies
+inside the timed region) plus the device->host read of the K verdict words.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+N > 1: launched under torch.distributed.run, one rank per GPU; the path has no exchange step, so every
+rank runs an independent replica on its own buffer (weak scaling) and value = total bytes / max time.
+`--impl reference` times the CPU oracle (oracle/) on the host cores instead.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+LEN = 256 << 20
+CHUNK = 4 << 20
+METRIC = "decrypt_verify_throughput"
+UNIT = "GB/s"
+WORKLOAD = "AES-256-GCM multi-chain decrypt+verify, 256 MiB uniform random bytes, chunk 4 MiB (K=64)"
+
+# Roofline of the fused kernel: it is bound by shared-memory lookups (one 128-byte wavefront per clock
+# per SM), not by HBM.  Per 512-byte row (32 blocks, one warp): AES-256 needs at least 197 table
+# lookups per block when the first two rounds are shared between the 256 blocks that differ only in
+# the last counter byte (224 without that sharing), each one conflict-free wavefront per warp; GHASH
+# with 8-bit tables needs 16 128-bit lookups per block = 64 wavefronts per warp.
+SMS = 148
+WAVEFRONTS_PER_ROW_BEST = 197 + 64
+ROW_BYTES = 512
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "sm_max_mhz": float(p.get("sm_max_mhz", 1965.0)), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi samples (SM clock, throttle reasons) taken while the timed regions run."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.samples, self.proc, self.thread = [], None, None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) >= 7:
+                self.samples.append((time.time(), parts))
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+
+    def summary(self, windows):
+        inside = [p for t, p in self.samples if any(a <= t <= b for a, b in windows)]
+        use = inside if inside else [p for _, p in self.samples]
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": len(inside)}
+        if not use:
+            return out
+        try:
+            out["sm_mhz"] = statistics.median(float(p[0]) for p in use)
+            out["sm_max_mhz"] = max(float(p[1]) for p in use)
+            out["power_w_max"] = max(float(p[2]) for p in use)
+        except ValueError:
+            pass
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        out["reasons"] = [n for i, n in enumerate(names) if any(p[3 + i].lower().startswith("active") for p in use)]
+        return out
+
+
+class OracleSample:
+    """A bounded sample of the workload for the CPU oracle: `n_chunks` chunks of `chunk` bytes each
+    (chunk <= 4 MiB; the oracle's cost is linear in bytes), encrypted once, decrypted+verified per step."""
+
+    def __init__(self, n_chunks: int, chunk: int, threads: int):
+        import oracle
+        from paper_2410_15240_b200 import synth
+        self.oracle, self.threads, self.chunk = oracle, threads, chunk
+        self.key, self.iv = synth.key_and_iv(4)
+        self.n = n_chunks * chunk
+        self.plain = synth.random_bytes(self.n, 4)
+        self.cipher, self.tags = oracle.mc_encrypt(self.key, self.iv, chunk, self.plain, threads)
+
+    def step(self) -> float:
+        t0 = time.perf_counter()
+        back, ok = self.oracle.mc_decrypt(self.key, self.iv, self.chunk, self.cipher, self.tags, self.threads)
+        dt = time.perf_counter() - t0
+        assert ok.all() and (back == self.plain).all()
+        return dt
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle, as it stands, on the host cores (rank 0 only).
+
+    Each step decrypts+verifies one chunk per host thread; the chunk is the workload's 4 MiB when the
+    requested number of steps allows it, otherwise shortened so that the timed region stays near a minute."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+    threads = oracle.host_threads()
+    calib = OracleSample(threads, 64 << 10, threads)
+    rate = calib.n / min(calib.step() for _ in range(2))           # bytes/s over all threads
+    budget_s = 60.0
+    chunk = int(budget_s * rate / max(1, args.steps) / threads) // 16 * 16
+    chunk = max(64 << 10, min(CHUNK, chunk))
+    sample = OracleSample(threads, chunk, threads)
+    for _ in range(args.warmup):
+        calib.step()
+    times = [sample.step() for _ in range(args.steps)]
+    total = sum(times)
+    value = sample.n * len(times) / total / 1e9
+    what = f"{threads} chunks of {chunk} bytes per step (workload chunk: {CHUNK}), {threads} threads over chunks"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": total / len(times) * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "bytes_per_step": sample.n},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": what},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def run_gpu(args):
+    import numpy as np
+    import torch
+    from paper_2410_15240_b200 import fastrack, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback (use --impl reference for the oracle)")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    key, iv = synth.key_and_iv(4)
+    K = LEN // CHUNK
+    ctx = fastrack.Context(key, CHUNK)
+    ctx.reserve(LEN)
+    stream = torch.cuda.current_stream()
+    st = stream.cuda_stream
+
+    # inputs: random payload, encrypted once on the GPU (bench input, not a parity claim)
+    plain_h = torch.from_numpy(synth.random_bytes(LEN, 4, salt=rank)).pin_memory()
+    d_plain_src = plain_h.cuda()
+    d_cipher = torch.empty_like(d_plain_src)
+    d_tags = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
+    ctx.encrypt_tag(iv, d_plain_src.data_ptr(), LEN, d_cipher.data_ptr(), d_tags.data_ptr(), st)
+    d_out = torch.empty_like(d_cipher)
+    d_ok = torch.zeros(K, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    h_cipher = d_cipher.cpu().pin_memory()
+    h_tags = d_tags.cpu().pin_memory()
+    h_ok = torch.zeros(K, dtype=torch.int32).pin_memory()
+
+    def step():
+        ctx.decrypt_verify(iv, d_cipher.data_ptr(), LEN, d_tags.data_ptr(), d_out.data_ptr(), d_ok.data_ptr(), st)
+
+    def e2e_step():
+        ctx.pipelined_h2d(iv, h_cipher.data_ptr(), LEN, h_tags.data_ptr(), d_out.data_ptr(), d_ok.data_ptr(), args.streams)
+        h_ok.copy_(d_ok, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    windows = []
+
+    # ---- device-resident metric: exactly K steps, CUDA events on the launching stream, max over ranks
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    launches0 = ctx.launches
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    w0 = time.time()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    windows.append((w0, time.time()))
+    gpu_launches = ctx.launches - launches0
+    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    ms_per_step = ms_total / args.steps
+    assert bool((d_ok == 1).all()), "verification failed inside the benchmark"
+    assert bool((d_out == d_plain_src).all()), "decryption mismatch inside the benchmark"
+    value = world * LEN / (ms_per_step * 1e-3) / 1e9
+
+    if args.kernel_only:
+        if sampler is not None:
+            sampler.stop()
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                              "warmup": args.warmup, "ms_per_step": ms_per_step, "gpu_launches": gpu_launches,
+                              "config": {"workload": WORKLOAD}, "kernel_only": True}))
+        ctx.close()
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- encrypt+tag (mirror path), same size, for the record
+    enc_steps = max(3, min(args.steps, 50))
+    for _ in range(3):
+        ctx.encrypt_tag(iv, d_plain_src.data_ptr(), LEN, d_out.data_ptr(), d_tags.data_ptr(), st)
+    barrier()
+    e0.record(stream)
+    for _ in range(enc_steps):
+        ctx.encrypt_tag(iv, d_plain_src.data_ptr(), LEN, d_out.data_ptr(), d_tags.data_ptr(), st)
+    e1.record(stream)
+    barrier()
+    enc_gbs = world * LEN / (max_over_ranks(e0.elapsed_time(e1)) / enc_steps * 1e-3) / 1e9
+
+    # ---- end to end: pinned host ciphertext -> pipelined H2D + decrypt/verify -> verdicts back on the host
+    e2e_steps = max(3, min(args.steps, 30))
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    w0 = time.time()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    torch.cuda.synchronize()
+    e2e_s = max_over_ranks(time.perf_counter() - t0)
+    windows.append((w0, time.time()))
+    assert bool((h_ok == 1).all())
+    e2e_gbs = world * LEN / (e2e_s / e2e_steps) / 1e9
+
+    # ---- raw pinned cudaMemcpyAsync of the same bytes, same run (what the pipeline is compared with)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        d_out.copy_(h_cipher, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+    raw_s = max_over_ranks(time.perf_counter() - t0)
+    raw_gbs = world * LEN / (raw_s / e2e_steps) / 1e9
+
+    if sampler is not None:
+        sampler.stop()
+    if rank == 0:
+        pk = peaks()
+        clocks = sampler.summary(windows)
+        per_gpu = value / world
+        alu_peak = SMS * ROW_BYTES * pk["sm_max_mhz"] * 1e6 / WAVEFRONTS_PER_ROW_BEST / 1e9
+        hbm_payload_peak = pk["hbm_gbs"] / 2.0
+        traffic = None
+        tpath = os.path.join(ROOT, "profiles", "traffic_bytes_per_launch.json")
+        if os.path.exists(tpath):
+            with open(tpath) as f:
+                traffic = json.load(f).get("decrypt_verify_256MiB_cb4MiB")
+        import oracle
+        threads = oracle.host_threads()
+        n_sample = max(1, min(64, threads))
+        cpu_s = OracleSample(n_sample, CHUNK, threads).step()
+        cpu_gbs = n_sample * CHUNK / cpu_s / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "u8", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "len_bytes": LEN, "chunk_bytes": CHUNK, "chains": K,
+                       "l2": "inputs larger than L2 (256 MiB in + 256 MiB out per step)",
+                       "parallelism": "replicas only" if world > 1 else "single GPU", "pipeline_streams": args.streams},
+            "clocks": clocks,
+            "e2e": {"value": e2e_gbs, "unit": UNIT, "h2d_bytes_per_step": LEN + 16 * K, "d2h_bytes_per_step": 4 * K,
+                    "steps": e2e_steps, "raw_pinned_h2d_gbs": raw_gbs, "fraction_of_raw_pcie": e2e_gbs / raw_gbs},
+            "gpu_launches": gpu_launches,
+            "roofline": {"bound": "alu", "achieved": per_gpu, "peak": alu_peak, "unit": "GB/s", "frac": per_gpu / alu_peak,
+                         "traffic": traffic,
+                         "peak_source": f"shared-memory lookup rate: {SMS} SMs x 1 wavefront/clk x {pk['sm_max_mhz']:.0f} MHz x "
+                                        f"{ROW_BYTES} B per {WAVEFRONTS_PER_ROW_BEST} wavefronts (payload GB/s)",
+                         "hbm": {"achieved": 2 * per_gpu, "peak": pk["hbm_gbs"], "frac": 2 * per_gpu / pk["hbm_gbs"],
+                                 "unit": "GB/s", "peak_source": f"{pk['source']} copy bandwidth",
+                                 "payload_peak": hbm_payload_peak}},
+            "cpu_baseline": {"value": cpu_gbs, "unit": UNIT, "cores": threads, "kind": "oracle",
+                             "sample": f"{n_sample} of the 64 chunks (4 MiB each), {threads} threads over chunks, {cpu_s:.1f} s"},
+            "extra": {"encrypt_tag_gbs": enc_gbs},
+        }
+        print(json.dumps(line))
+    ctx.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--streams", type=int, default=4)
+    ap.add_argument("--impl", default="fastrack", choices=["fastrack", "reference"])
+    ap.add_argument("--kernel-only", action="store_true",
+                    help="time only the device-resident decrypt+verify loop (short run for profilers)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()
