@@ -43,6 +43,9 @@ WORKLOAD = "AES-256-GCM multi-chain decrypt+verify, 256 MiB uniform random bytes
 SMS = 148
 WAVEFRONTS_PER_ROW_BEST = 197 + 64
 ROW_BYTES = 512
+# dram__bytes_read.sum + dram__bytes_write.sum of one decrypt+verify launch on this exact workload, from the
+# ncu capture summarised in profiles/fr_crypt_kernel_decrypt_verify_256MiB_chunk4MiB.md (algorithmic: 2 x 256 MiB).
+DRAM_TRAFFIC_BYTES_PER_LAUNCH = 496.7e6
 
 
 def peaks():
@@ -290,11 +293,7 @@ def run_gpu(args):
         per_gpu = value / world
         alu_peak = SMS * ROW_BYTES * pk["sm_max_mhz"] * 1e6 / WAVEFRONTS_PER_ROW_BEST / 1e9
         hbm_payload_peak = pk["hbm_gbs"] / 2.0
-        traffic = None
-        tpath = os.path.join(ROOT, "profiles", "traffic_bytes_per_launch.json")
-        if os.path.exists(tpath):
-            with open(tpath) as f:
-                traffic = json.load(f).get("decrypt_verify_256MiB_cb4MiB")
+        traffic = DRAM_TRAFFIC_BYTES_PER_LAUNCH
         import oracle
         threads = oracle.host_threads()
         n_sample = max(1, min(64, threads))
