@@ -56,10 +56,14 @@ extern "C" {
 #define FASTRACK_ERR_CUDA        -4   /* a CUDA call failed; see fastrack_last_cuda_error */
 #define FASTRACK_ERR_NOMEM       -5   /* host or device allocation failed */
 #define FASTRACK_ERR_TOO_MANY    -6   /* more than 2^32 chunks in one call (the IV index is 32 bits) */
+#define FASTRACK_ERR_LIMIT       -7   /* more chunks than fastrack_decrypt_verify_noalloc's fixed scratch holds */
 
 /* Largest chunk: 1 GiB.  (GCM itself allows 2^36 - 32 bytes per message; the limit here keeps the
  * per-context table of powers of H, 16 bytes per 16-byte block of a chunk, at most 1 GiB.) */
 #define FASTRACK_MAX_CHUNK_BYTES ((size_t)1 << 30)
+
+/* Most chunks one fastrack_decrypt_verify_noalloc call may cover (its scratch is a fixed 320 KiB array). */
+#define FASTRACK_NOALLOC_MAX_CHUNKS 16384
 
 typedef struct fastrack_ctx fastrack_ctx;
 
@@ -128,6 +132,28 @@ FASTRACK_API int fastrack_encrypt_tag(fastrack_ctx* ctx, const uint8_t iv_base[1
 FASTRACK_API int fastrack_pipelined_h2d(fastrack_ctx* ctx, const uint8_t iv_base[12],
                                         const void* h_cipher_pinned, size_t len, const void* h_tags,
                                         void* d_plain, uint32_t* d_ok, int n_streams);
+
+/* fastrack_decrypt_verify for callers that must not allocate.  (The paper has no counterpart; this is a
+ * deployment variant of the same operation.)
+ * Who needs it: code that runs after start-up in a process whose device memory is fully owned by another
+ * allocator or a fixed budget, or inside a serving loop where the device-wide synchronisation that comes with
+ * a device allocation would stall every other stream.  fastrack_decrypt_verify grows its per-chunk scratch
+ * with cudaMalloc the first time a call covers more chunks than any call before; this variant never does:
+ * its per-chunk scratch is a fixed array inside the library image (320 KiB, held by every GPU that loads
+ * the library until the process exits), and it calls no cudaMalloc, cudaFree or other allocating routine.
+ * Arguments, outputs, alignment and overlap rules, and asynchrony on `stream` are exactly those of
+ * fastrack_decrypt_verify, and the results are bit-identical to it.  Differences:
+ *   - at most FASTRACK_NOALLOC_MAX_CHUNKS chunks per call; more returns FASTRACK_ERR_LIMIT and does nothing;
+ *   - the context's device must be the current device (else FASTRACK_ERR_ARG);
+ *   - the first call on each device looks up the array's device address (cudaGetSymbolAddress); make that
+ *     first call during start-up, before any stream capture begins;
+ *   - all calls on a device share the one array, which still holds what the previous call left: each call
+ *     first zeroes the part it will use, on `stream`.  Two calls whose GPU work overlaps (different streams,
+ *     different contexts or different host threads) race on it and produce wrong verdicts -- keep every
+ *     call of this entry point on one stream, or order them with events. */
+FASTRACK_API int fastrack_decrypt_verify_noalloc(fastrack_ctx* ctx, const uint8_t iv_base[12],
+                                                 const void* d_cipher, size_t len, const void* d_tags,
+                                                 void* d_plain, uint32_t* d_ok, void* stream);
 
 /* Number of kernels the library launched through ctx since creation (data-path launches only;
  * cudaMemcpyAsync calls are not counted).  For benchmarks' bookkeeping. */

@@ -422,3 +422,82 @@ extern "C" int fastrack_pipelined_h2d(fastrack_ctx* ctx, const uint8_t iv_base[1
     for (int i = 0; i < n_streams; i++) FR_CUDA(ctx, cudaStreamSynchronize(ctx->streams[i]));
     return FASTRACK_OK;
 }
+
+// ------------------------------------------------------------- entry point that allocates nothing ----
+//
+// Per-chunk scratch for fastrack_decrypt_verify_noalloc: FASTRACK_NOALLOC_MAX_CHUNKS accumulators of four
+// words, then as many arrival counters.  It is part of the library image, so every GPU that loads the
+// library holds these 320 KiB until the process exits, and every call on a device shares them.
+static __device__ __align__(256) uint32_t fr_static_scratch[5 * FASTRACK_NOALLOC_MAX_CHUNKS];
+
+// In host code the array's name above is only a handle for the runtime, not a device address; the real
+// address differs per device and is looked up once per device with that device current.
+#define FR_MAX_DEVICES 64
+static uint32_t* fr_static_scratch_addr[FR_MAX_DEVICES];
+
+extern "C" int fastrack_decrypt_verify_noalloc(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_cipher,
+                                               size_t len, const void* d_tags, void* d_plain, uint32_t* d_ok,
+                                               void* stream)
+{
+    if (!ctx || !iv_base) return FASTRACK_ERR_ARG;
+    if (len == 0) return FASTRACK_OK;
+    if (!d_cipher || !d_tags || !d_plain || !d_ok) return FASTRACK_ERR_ARG;
+    if (misaligned(d_cipher, 16) || misaligned(d_plain, 16) || misaligned(d_tags, 16) || misaligned(d_ok, 4)) return FASTRACK_ERR_ARG;
+    if (bad_overlap(d_cipher, d_plain, len)) return FASTRACK_ERR_ARG;
+    const size_t K = fastrack_num_chunks(ctx, len);
+    if (K > FASTRACK_NOALLOC_MAX_CHUNKS) return FASTRACK_ERR_LIMIT;
+
+    int dev = -1;
+    FR_CUDA(ctx, cudaGetDevice(&dev));
+    if (dev != ctx->device || dev < 0 || dev >= FR_MAX_DEVICES) return FASTRACK_ERR_ARG;
+    if (!fr_static_scratch_addr[dev]) {                 // first call on this device: resolve the symbol
+        uint32_t* ptr = nullptr;
+        FR_CUDA(ctx, cudaGetSymbolAddress((void**)&ptr, fr_static_scratch));
+        if (!ptr) return FASTRACK_ERR_CUDA;
+        fr_static_scratch_addr[dev] = ptr;
+    }
+    uint32_t* acc = fr_static_scratch_addr[dev];
+    uint32_t* cnt = acc + 4 * (size_t)FASTRACK_NOALLOC_MAX_CHUNKS;
+    cudaStream_t st = (cudaStream_t)stream;
+    // the array keeps whatever the previous call (possibly a failed one) left: zero what this call will use
+    FR_CUDA(ctx, cudaMemsetAsync(acc, 0, K * 4 * sizeof(uint32_t), st));
+    FR_CUDA(ctx, cudaMemsetAsync(cnt, 0, K * sizeof(uint32_t), st));
+
+    // same launch geometry as the allocating entry point, scratch pointers aside
+    FrParams P;
+    memset(&P, 0, sizeof P);
+    memcpy(P.rk, ctx->rk, sizeof P.rk);
+    P.iv_w0 = load_le32(iv_base);
+    P.iv_w1 = load_le32(iv_base + 4);
+    P.iv_ctr = load_be32(iv_base + 8);
+    P.len = len;
+    P.chunk_bytes = ctx->chunk_bytes;
+    P.n_chunks = (uint32_t)K;
+    const size_t first_len = len < ctx->chunk_bytes ? len : ctx->chunk_bytes;
+    const size_t rows_ref = ((first_len + 15) / 16 + FR_ROW_BLOCKS - 1) / FR_ROW_BLOCKS;
+    const size_t total_rows = rows_ref * K;
+    const size_t warps = (size_t)ctx->num_sms * FR_WARPS;
+    size_t seg_rows = (total_rows + 2 * warps - 1) / (2 * warps);
+    if (seg_rows < 8) seg_rows = 8;
+    if (seg_rows > 128) seg_rows = 128;
+    size_t spc = (rows_ref + seg_rows - 1) / seg_rows;
+    seg_rows = (rows_ref + spc - 1) / spc;
+    P.seg_rows = (uint32_t)seg_rows;
+    P.segs_per_chunk = (uint32_t)spc;
+    P.n_items = (uint32_t)(spc * K);
+    P.in = (const uint8_t*)d_cipher;
+    P.out = (uint8_t*)d_plain;
+    P.tags_in = (const uint4*)d_tags;
+    P.ok = d_ok;
+    P.te0 = ctx->d_te0;
+    P.gh_tab = ctx->d_gh_tab;
+    P.pow = ctx->d_pow;
+    P.acc = acc;
+    P.cnt = cnt;
+    unsigned grid = (unsigned)ctx->num_sms;
+    if (P.n_items < grid) grid = P.n_items;
+    fr_crypt_kernel<false><<<grid, FR_THREADS, FR_SMEM_BYTES, st>>>(P);
+    ctx->launches++;
+    FR_CUDA(ctx, cudaGetLastError());
+    return FASTRACK_OK;
+}

@@ -14,12 +14,13 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libfastrack.so")
 
 OK = 0
-ERR_ARG, ERR_CHUNK, ERR_NOT_PINNED, ERR_CUDA, ERR_NOMEM, ERR_TOO_MANY = -1, -2, -3, -4, -5, -6
+ERR_ARG, ERR_CHUNK, ERR_NOT_PINNED, ERR_CUDA, ERR_NOMEM, ERR_TOO_MANY, ERR_LIMIT = -1, -2, -3, -4, -5, -6, -7
+NOALLOC_MAX_CHUNKS = 16384
 MAX_CHUNK_BYTES = 1 << 30
 
 EXPORTS = ("fastrack_ctx_create", "fastrack_ctx_destroy", "fastrack_num_chunks", "fastrack_ctx_reserve",
            "fastrack_last_cuda_error", "fastrack_decrypt_verify", "fastrack_encrypt_tag",
-           "fastrack_pipelined_h2d", "fastrack_launch_count")
+           "fastrack_pipelined_h2d", "fastrack_launch_count", "fastrack_decrypt_verify_noalloc")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2410_15240_b200.build` "
@@ -41,6 +42,8 @@ _lib.fastrack_launch_count.restype = ctypes.c_uint64
 _lib.fastrack_launch_count.argtypes = [_vp]
 _lib.fastrack_decrypt_verify.restype = _int
 _lib.fastrack_decrypt_verify.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp, _vp]
+_lib.fastrack_decrypt_verify_noalloc.restype = _int
+_lib.fastrack_decrypt_verify_noalloc.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp, _vp]
 _lib.fastrack_encrypt_tag.restype = _int
 _lib.fastrack_encrypt_tag.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp]
 _lib.fastrack_pipelined_h2d.restype = _int
@@ -86,6 +89,13 @@ def fastrack_decrypt_verify(ctx, iv_base: bytes, d_cipher: int, length: int, d_t
     return _lib.fastrack_decrypt_verify(ctx, iv_base, d_cipher, length, d_tags, d_plain, d_ok, stream)
 
 
+def fastrack_decrypt_verify_noalloc(ctx, iv_base: bytes, d_cipher: int, length: int, d_tags: int, d_plain: int,
+                                    d_ok: int, stream: int = 0) -> int:
+    """fastrack_decrypt_verify for callers that must not allocate: fixed scratch inside the library,
+    at most NOALLOC_MAX_CHUNKS chunks per call, one call in flight per device at a time."""
+    return _lib.fastrack_decrypt_verify_noalloc(ctx, iv_base, d_cipher, length, d_tags, d_plain, d_ok, stream)
+
+
 def fastrack_encrypt_tag(ctx, iv_base: bytes, d_plain: int, length: int, d_cipher: int, d_tags: int,
                          stream: int = 0) -> int:
     return _lib.fastrack_encrypt_tag(ctx, iv_base, d_plain, length, d_cipher, d_tags, stream)
@@ -118,6 +128,10 @@ class Context:
 
     def decrypt_verify(self, iv_base, d_cipher, length, d_tags, d_plain, d_ok, stream=0) -> None:
         self._check(fastrack_decrypt_verify(self.handle, iv_base, d_cipher, length, d_tags, d_plain, d_ok, stream))
+
+    def decrypt_verify_noalloc(self, iv_base, d_cipher, length, d_tags, d_plain, d_ok, stream=0) -> None:
+        self._check(fastrack_decrypt_verify_noalloc(self.handle, iv_base, d_cipher, length, d_tags, d_plain, d_ok,
+                                                    stream))
 
     def encrypt_tag(self, iv_base, d_plain, length, d_cipher, d_tags, stream=0) -> None:
         self._check(fastrack_encrypt_tag(self.handle, iv_base, d_plain, length, d_cipher, d_tags, stream))

@@ -36,6 +36,8 @@ def test_error_codes_match_header():
     assert int(codes["FASTRACK_ERR_CUDA"]) == fastrack.ERR_CUDA
     assert int(codes["FASTRACK_ERR_NOMEM"]) == fastrack.ERR_NOMEM
     assert int(codes["FASTRACK_ERR_TOO_MANY"]) == fastrack.ERR_TOO_MANY
+    assert int(codes["FASTRACK_ERR_LIMIT"]) == fastrack.ERR_LIMIT
+    assert int(re.search(r"#define\s+FASTRACK_NOALLOC_MAX_CHUNKS\s+(\d+)", text).group(1)) == fastrack.NOALLOC_MAX_CHUNKS
 
 
 def test_argument_checks_that_need_no_device():
@@ -48,6 +50,7 @@ def test_argument_checks_that_need_no_device():
     assert fastrack.fastrack_ctx_reserve(None, 1) == fastrack.ERR_ARG
     assert fastrack.fastrack_decrypt_verify(None, bytes(12), 0, 16, 0, 0, 0, 0) == fastrack.ERR_ARG
     assert fastrack.fastrack_encrypt_tag(None, bytes(12), 0, 16, 0, 0, 0) == fastrack.ERR_ARG
+    assert fastrack.fastrack_decrypt_verify_noalloc(None, bytes(12), 0, 16, 0, 0, 0, 0) == fastrack.ERR_ARG
     assert fastrack.fastrack_pipelined_h2d(None, bytes(12), 0, 16, 0, 0, 0, 2) == fastrack.ERR_ARG
     fastrack.fastrack_ctx_destroy(None)          # allowed
 
