@@ -74,9 +74,10 @@ __global__ void __launch_bounds__(FR_THREADS, 1) fr_crypt_kernel(const __grid_co
                 z.w = __shfl_sync(0xFFFFFFFFu, z.w, 0);
             }
         }
-        if (finisher) {
-            const uint4 tag = fr_chunk_tag(P, sm, L.lane4, kk, z);
-            if (lane == 0) {
+        if (finisher && lane == 0) {
+            const uint4 lenh = (kk + 1u == P.n_chunks) ? P.lenh_last : P.lenh_full;
+            const uint4 tag = fr_xor4(z, lenh);           // z already holds GHASH of the data xor E_K(J0)
+            {
                 if (ENCRYPT) {
                     P.tags_out[kk] = tag;
                 } else {
@@ -274,6 +275,44 @@ extern "C" uint64_t fastrack_launch_count(const fastrack_ctx* ctx) { return ctx 
 static uint32_t load_be32(const uint8_t* p) { return ((uint32_t)p[0] << 24) | ((uint32_t)p[1] << 16) | ((uint32_t)p[2] << 8) | p[3]; }
 static uint32_t load_le32(const uint8_t* p) { return ((uint32_t)p[3] << 24) | ((uint32_t)p[2] << 16) | ((uint32_t)p[1] << 8) | p[0]; }
 
+
+// (BE64(0) || BE64(8 * bytes)) * H: the length block's term of a chunk of `bytes` bytes.
+static uint4 length_term(const fastrack_ctx* ctx, uint64_t bytes)
+{
+    uint8_t blk[16] = {0}, out[16];
+    const uint64_t bits = bytes * 8;
+    for (int i = 0; i < 8; i++) blk[8 + i] = (uint8_t)(bits >> (56 - 8 * i));
+    gf_store(gf_mul(gf_load(blk), gf_load(ctx->h)), out);
+    uint4 r;
+    memcpy(&r, out, 16);
+    return r;
+}
+
+// Segment geometry of a launch over `len` bytes: rows are aligned to the counter (block j sits at counter
+// j + 2), segments are whole multiples of 8 rows so that they start on a 256-counter group.
+static void plan_segments(const fastrack_ctx* ctx, size_t len, size_t n_chunks, FrParams& P)
+{
+    const size_t first_len = len < ctx->chunk_bytes ? len : ctx->chunk_bytes;
+    const size_t rows_ref = ((first_len + 15) / 16 + 2 + FR_ROW_BLOCKS - 1) / FR_ROW_BLOCKS;
+    const size_t total_rows = rows_ref * n_chunks;
+    const size_t warps = (size_t)ctx->num_sms * FR_WARPS;
+    size_t seg_rows = ctx->seg_rows_override ? ctx->seg_rows_override : (total_rows + 2 * warps - 1) / (2 * warps);
+    if (!ctx->seg_rows_override) {
+        if (seg_rows < 8) seg_rows = 8;
+        if (seg_rows > 128) seg_rows = 128;
+    }
+    size_t spc = (rows_ref + seg_rows - 1) / seg_rows;
+    while (spc * n_chunks >= ((size_t)1 << 31)) { seg_rows *= 2; spc = (rows_ref + seg_rows - 1) / seg_rows; }
+    seg_rows = ((rows_ref + spc - 1) / spc + 7) / 8 * 8;   // equalise the segments of a chunk, whole groups
+    spc = (rows_ref + seg_rows - 1) / seg_rows;
+    P.seg_rows = (uint32_t)seg_rows;
+    P.segs_per_chunk = (uint32_t)spc;
+    P.n_items = (uint32_t)(spc * n_chunks);
+    const size_t last_len = len - (n_chunks - 1) * ctx->chunk_bytes;
+    P.lenh_full = length_term(ctx, first_len);
+    P.lenh_last = length_term(ctx, last_len);
+}
+
 // Launch the fused pass over `len` bytes that start at chunk index `first_chunk` of the caller's buffer.
 static int launch_pass(fastrack_ctx* ctx, bool encrypt, const uint8_t iv_base[12], size_t first_chunk,
                        const void* d_in, size_t len, void* d_out, const void* d_tags_in, void* d_tags_out,
@@ -290,22 +329,7 @@ static int launch_pass(fastrack_ctx* ctx, bool encrypt, const uint8_t iv_base[12
     const size_t n_chunks = (len + ctx->chunk_bytes - 1) / ctx->chunk_bytes;
     P.n_chunks = (uint32_t)n_chunks;
 
-    // rows of the largest chunk in this launch, and the segment length that spreads the work
-    const size_t first_len = len < ctx->chunk_bytes ? len : ctx->chunk_bytes;
-    const size_t rows_ref = ((first_len + 15) / 16 + FR_ROW_BLOCKS - 1) / FR_ROW_BLOCKS;
-    const size_t total_rows = rows_ref * n_chunks;
-    const size_t warps = (size_t)ctx->num_sms * FR_WARPS;
-    size_t seg_rows = ctx->seg_rows_override ? ctx->seg_rows_override : (total_rows + 2 * warps - 1) / (2 * warps);
-    if (!ctx->seg_rows_override) {
-        if (seg_rows < 8) seg_rows = 8;
-        if (seg_rows > 128) seg_rows = 128;
-    }
-    size_t spc = (rows_ref + seg_rows - 1) / seg_rows;
-    while (spc * n_chunks >= ((size_t)1 << 31)) { seg_rows *= 2; spc = (rows_ref + seg_rows - 1) / seg_rows; }
-    seg_rows = (rows_ref + spc - 1) / spc;                 // equalise the segments of a chunk
-    P.seg_rows = (uint32_t)seg_rows;
-    P.segs_per_chunk = (uint32_t)spc;
-    P.n_items = (uint32_t)(spc * n_chunks);
+    plan_segments(ctx, len, n_chunks, P);
 
     P.in = (const uint8_t*)d_in;
     P.out = (uint8_t*)d_out;
@@ -473,18 +497,7 @@ extern "C" int fastrack_decrypt_verify_noalloc(fastrack_ctx* ctx, const uint8_t 
     P.len = len;
     P.chunk_bytes = ctx->chunk_bytes;
     P.n_chunks = (uint32_t)K;
-    const size_t first_len = len < ctx->chunk_bytes ? len : ctx->chunk_bytes;
-    const size_t rows_ref = ((first_len + 15) / 16 + FR_ROW_BLOCKS - 1) / FR_ROW_BLOCKS;
-    const size_t total_rows = rows_ref * K;
-    const size_t warps = (size_t)ctx->num_sms * FR_WARPS;
-    size_t seg_rows = (total_rows + 2 * warps - 1) / (2 * warps);
-    if (seg_rows < 8) seg_rows = 8;
-    if (seg_rows > 128) seg_rows = 128;
-    size_t spc = (rows_ref + seg_rows - 1) / seg_rows;
-    seg_rows = (rows_ref + spc - 1) / spc;
-    P.seg_rows = (uint32_t)seg_rows;
-    P.segs_per_chunk = (uint32_t)spc;
-    P.n_items = (uint32_t)(spc * K);
+    plan_segments(ctx, len, K, P);
     P.in = (const uint8_t*)d_cipher;
     P.out = (uint8_t*)d_plain;
     P.tags_in = (const uint4*)d_tags;

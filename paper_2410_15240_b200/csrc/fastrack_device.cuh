@@ -50,6 +50,8 @@ struct FrParams {
     const uint4* pow;          // pow[e] = H^e
     uint32_t* acc;             // per chunk 4 words, zero between launches
     uint32_t* cnt;             // per chunk arrival counter, zero between launches
+    uint4 lenh_full;           // (BE64(0) || BE64(8 * chunk_bytes)) * H: the length block's term of a full chunk
+    uint4 lenh_last;           // the same for the launch's last chunk (differs when that chunk is short)
 };
 
 // Byte permute, PTX prmt.b32 in generic mode: result byte i = byte (sel nibble i & 7) of {a (0..3), b (4..7)};
@@ -111,22 +113,25 @@ __device__ __forceinline__ void fr_build_smem(char* sm, uint32_t tid, uint32_t n
     for (uint32_t i = tid; i < 4096u; i += nthreads) *(uint4*)(sm + FR_SM_GH + i * 16u) = gh_tab[i];
 }
 
-// AES-256 forward cipher on the state (s0..s3), which already holds counter-block xor round key 0.
+// Table lookups: byte k of state word w, table t (address = one byte permute; see the header comment).
 #define FR_TA(w, k) FR_PRMT((w), lane4, 0x5504u | ((k) << 4))
 #define FR_LD32(off, addr) (*(const uint32_t*)(sm + (off) + (addr)))
+#define FR_TE0(w, k) FR_LD32(FR_SM_T01, FR_TA(w, k))
+#define FR_TE1(w, k) FR_LD32(FR_SM_T01 + 128u, FR_TA(w, k))
+#define FR_TE2(w, k) FR_LD32(FR_SM_T23, FR_TA(w, k))
+#define FR_TE3(w, k) FR_LD32(FR_SM_T23 + 128u, FR_TA(w, k))
+
+// Rounds FIRST..14 of the AES-256 forward cipher on a state that has been through rounds 0..FIRST-1.
+template <int FIRST>
 __device__ __forceinline__ uint4 fr_aes256_rounds(const char* sm, uint32_t lane4, const FrParams& P,
                                                   uint32_t s0, uint32_t s1, uint32_t s2, uint32_t s3)
 {
 #pragma unroll
-    for (int r = 1; r < 14; r++) {
-        uint32_t t0 = FR_LD32(FR_SM_T01, FR_TA(s0, 0)) ^ FR_LD32(FR_SM_T01 + 128u, FR_TA(s1, 1)) ^
-                      FR_LD32(FR_SM_T23, FR_TA(s2, 2)) ^ FR_LD32(FR_SM_T23 + 128u, FR_TA(s3, 3)) ^ P.rk[4 * r + 0];
-        uint32_t t1 = FR_LD32(FR_SM_T01, FR_TA(s1, 0)) ^ FR_LD32(FR_SM_T01 + 128u, FR_TA(s2, 1)) ^
-                      FR_LD32(FR_SM_T23, FR_TA(s3, 2)) ^ FR_LD32(FR_SM_T23 + 128u, FR_TA(s0, 3)) ^ P.rk[4 * r + 1];
-        uint32_t t2 = FR_LD32(FR_SM_T01, FR_TA(s2, 0)) ^ FR_LD32(FR_SM_T01 + 128u, FR_TA(s3, 1)) ^
-                      FR_LD32(FR_SM_T23, FR_TA(s0, 2)) ^ FR_LD32(FR_SM_T23 + 128u, FR_TA(s1, 3)) ^ P.rk[4 * r + 2];
-        uint32_t t3 = FR_LD32(FR_SM_T01, FR_TA(s3, 0)) ^ FR_LD32(FR_SM_T01 + 128u, FR_TA(s0, 1)) ^
-                      FR_LD32(FR_SM_T23, FR_TA(s1, 2)) ^ FR_LD32(FR_SM_T23 + 128u, FR_TA(s2, 3)) ^ P.rk[4 * r + 3];
+    for (int r = FIRST; r < 14; r++) {
+        uint32_t t0 = FR_TE0(s0, 0) ^ FR_TE1(s1, 1) ^ FR_TE2(s2, 2) ^ FR_TE3(s3, 3) ^ P.rk[4 * r + 0];
+        uint32_t t1 = FR_TE0(s1, 0) ^ FR_TE1(s2, 1) ^ FR_TE2(s3, 2) ^ FR_TE3(s0, 3) ^ P.rk[4 * r + 1];
+        uint32_t t2 = FR_TE0(s2, 0) ^ FR_TE1(s3, 1) ^ FR_TE2(s0, 2) ^ FR_TE3(s1, 3) ^ P.rk[4 * r + 2];
+        uint32_t t3 = FR_TE0(s3, 0) ^ FR_TE1(s0, 1) ^ FR_TE2(s1, 2) ^ FR_TE3(s2, 3) ^ P.rk[4 * r + 3];
         s0 = t0; s1 = t1; s2 = t2; s3 = t3;
     }
     // Last round: SubBytes + ShiftRows only.  Te2 has S in byte 0, Te3 in byte 1, Te0 in byte 2, Te1 in byte 3.
@@ -134,10 +139,10 @@ __device__ __forceinline__ uint4 fr_aes256_rounds(const char* sm, uint32_t lane4
     const uint32_t in[4] = {s0, s1, s2, s3};
 #pragma unroll
     for (int c = 0; c < 4; c++) {
-        uint32_t a = FR_LD32(FR_SM_T23, FR_TA(in[c], 0));
-        uint32_t b = FR_LD32(FR_SM_T23 + 128u, FR_TA(in[(c + 1) & 3], 1));
-        uint32_t cc = FR_LD32(FR_SM_T01, FR_TA(in[(c + 2) & 3], 2));
-        uint32_t d = FR_LD32(FR_SM_T01 + 128u, FR_TA(in[(c + 3) & 3], 3));
+        uint32_t a = FR_TE2(in[c], 0);
+        uint32_t b = FR_TE3(in[(c + 1) & 3], 1);
+        uint32_t cc = FR_TE0(in[(c + 2) & 3], 2);
+        uint32_t d = FR_TE1(in[(c + 3) & 3], 3);
         uint32_t lo = FR_PRMT(a, b, 0x0050u);    // [a.0, b.1, -, -]
         uint32_t hi = FR_PRMT(cc, d, 0x7200u);   // [-, -, c.2, d.3]
         o[c] = FR_PRMT(lo, hi, 0x7610u) ^ P.rk[56 + c];
@@ -145,12 +150,50 @@ __device__ __forceinline__ uint4 fr_aes256_rounds(const char* sm, uint32_t lane4
     return make_uint4(o[0], o[1], o[2], o[3]);
 }
 
-// E_K(IV_k || BE32(ctr)) for chunk-relative IV word `ivw2` (little-endian load of IV_k[8..11]).
-__device__ __forceinline__ uint4 fr_aes256_ctr_block(const char* sm, uint32_t lane4, const FrParams& P,
-                                                     uint32_t ivw2, uint32_t ctr)
+// Counter-mode sharing of the first two rounds.  In the counter block IV_k || BE32(ctr) only byte 15
+// changes from block to block, byte 14 every 256 blocks, bytes 12-13 hardly ever.  After round 1 three
+// of the four columns depend only on ctr >> 8, and in round 2 every output column takes exactly one
+// byte from the fast-changing column.  So per 256-counter group a lane keeps (t1, t2, t3) folded into
+// four words D0..D3, and per block rounds 1 and 2 cost 1 + 4 lookups instead of 32.
+struct FrCtrChunk {        // per chunk: the parts of round 1 that depend on the IV only
+    uint32_t a0, b1, b2, b3;
+};
+struct FrCtrGroup {        // per 256-counter group
+    uint32_t d0, d1, d2, d3;
+};
+
+__device__ __forceinline__ FrCtrChunk fr_ctr_chunk(const char* sm, uint32_t lane4, const FrParams& P, uint32_t ivw2)
 {
-    return fr_aes256_rounds(sm, lane4, P, P.iv_w0 ^ P.rk[0], P.iv_w1 ^ P.rk[1], ivw2 ^ P.rk[2],
-                            fr_bswap(ctr) ^ P.rk[3]);
+    const uint32_t s0 = P.iv_w0 ^ P.rk[0], s1 = P.iv_w1 ^ P.rk[1], s2 = ivw2 ^ P.rk[2];
+    FrCtrChunk c;
+    c.a0 = FR_TE0(s0, 0) ^ FR_TE1(s1, 1) ^ FR_TE2(s2, 2) ^ P.rk[4];
+    c.b1 = FR_TE0(s1, 0) ^ FR_TE1(s2, 1) ^ FR_TE3(s0, 3) ^ P.rk[5];
+    c.b2 = FR_TE0(s2, 0) ^ FR_TE2(s0, 2) ^ FR_TE3(s1, 3) ^ P.rk[6];
+    c.b3 = FR_TE1(s0, 1) ^ FR_TE2(s1, 2) ^ FR_TE3(s2, 3) ^ P.rk[7];
+    return c;
+}
+
+__device__ __forceinline__ FrCtrGroup fr_ctr_group(const char* sm, uint32_t lane4, const FrParams& P,
+                                                   const FrCtrChunk& c, uint32_t ctr)
+{
+    const uint32_t s3 = fr_bswap(ctr) ^ P.rk[3];          // bytes 0..2 = counter bytes 12..14 (byte 3 unused here)
+    const uint32_t t1 = c.b1 ^ FR_TE2(s3, 2), t2 = c.b2 ^ FR_TE1(s3, 1), t3 = c.b3 ^ FR_TE0(s3, 0);
+    FrCtrGroup g;
+    g.d0 = FR_TE1(t1, 1) ^ FR_TE2(t2, 2) ^ FR_TE3(t3, 3) ^ P.rk[8];
+    g.d1 = FR_TE0(t1, 0) ^ FR_TE1(t2, 1) ^ FR_TE2(t3, 2) ^ P.rk[9];
+    g.d2 = FR_TE0(t2, 0) ^ FR_TE1(t3, 1) ^ FR_TE3(t1, 3) ^ P.rk[10];
+    g.d3 = FR_TE0(t3, 0) ^ FR_TE2(t1, 2) ^ FR_TE3(t2, 3) ^ P.rk[11];
+    return g;
+}
+
+// E_K(IV_k || BE32(ctr)) given the chunk and group constants that belong to ctr.
+__device__ __forceinline__ uint4 fr_aes256_ctr_block(const char* sm, uint32_t lane4, const FrParams& P,
+                                                     const FrCtrChunk& c, const FrCtrGroup& g, uint32_t ctr)
+{
+    const uint32_t s3 = fr_bswap(ctr) ^ P.rk[3];
+    const uint32_t t0 = c.a0 ^ FR_TE3(s3, 3);
+    return fr_aes256_rounds<3>(sm, lane4, P, g.d0 ^ FR_TE0(t0, 0), g.d1 ^ FR_TE3(t0, 3), g.d2 ^ FR_TE2(t0, 2),
+                               g.d3 ^ FR_TE1(t0, 1));
 }
 
 // v * H^32 through the byte tables (v, result: little-endian words of the block's 16 bytes).
@@ -204,11 +247,15 @@ __device__ __forceinline__ uint64_t fr_chunk_len(const FrParams& P, uint32_t kk)
     return rem < P.chunk_bytes ? rem : P.chunk_bytes;
 }
 
+// Rows are aligned to the COUNTER, not to the block index: row r of a chunk holds counters 32r .. 32r+31,
+// lane = counter mod 32.  Data block j uses counter j + 2, so row 0 carries 30 data blocks; its lane 1
+// (counter 1) produces E_K(J0), the tag mask, as a by-product and lane 0 idles.
+__device__ __forceinline__ uint32_t fr_chunk_rows(uint32_t nblk) { return (nblk + 2u + FR_ROW_BLOCKS - 1) / FR_ROW_BLOCKS; }
+
 __device__ __forceinline__ uint32_t fr_chunk_segs(const FrParams& P, uint32_t kk)
 {
     uint32_t nblk = (uint32_t)((fr_chunk_len(P, kk) + 15) >> 4);
-    uint32_t rows = (nblk + FR_ROW_BLOCKS - 1) / FR_ROW_BLOCKS;
-    return (rows + P.seg_rows - 1) / P.seg_rows;
+    return (fr_chunk_rows(nblk) + P.seg_rows - 1) / P.seg_rows;
 }
 
 // Load / store the last, partial block of the buffer byte by byte (zero-padded in registers).
@@ -238,8 +285,8 @@ __device__ __forceinline__ uint4 fr_mask_bytes(uint4 v, uint32_t n)
 
 // One lane's share of segment s of chunk kk: decrypt (or encrypt) its blocks, fold them into the
 // lane's Horner value, and return that value multiplied by the power of H that aligns it to the end
-// of the chunk.  XOR of the 32 lanes' results = the segment's contribution to the chunk's GHASH
-// (before the length block).
+// of the chunk (lane 1 of the chunk's first segment adds E_K(J0)).  XOR of the 32 lanes' results over all
+// segments of the chunk = GHASH of the data blocks (before the length block) xor E_K(J0).
 template <bool ENCRYPT>
 __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, const char* sm, const FrLane& L,
                                                          uint32_t lane, uint32_t kk, uint32_t s)
@@ -247,47 +294,41 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
     const uint64_t chunk_off = (uint64_t)kk * P.chunk_bytes;
     const uint64_t len_k = fr_chunk_len(P, kk);
     const uint32_t nblk = (uint32_t)((len_k + 15) >> 4);
-    const uint32_t rows = (nblk + FR_ROW_BLOCKS - 1) / FR_ROW_BLOCKS;
+    const uint32_t rows = fr_chunk_rows(nblk);
     const uint32_t row0 = s * P.seg_rows;
     uint32_t row1 = row0 + P.seg_rows;
     if (row1 > rows) row1 = rows;
-    uint32_t seg_end = row1 * FR_ROW_BLOCKS;       // first block index after this segment
+    uint32_t seg_end = row1 * FR_ROW_BLOCKS - 2u;   // first block index after this segment
     if (seg_end > nblk) seg_end = nblk;
     const uint8_t* in = P.in + chunk_off;
     uint8_t* out = P.out + chunk_off;
-    const uint32_t ivw2 = fr_bswap(P.iv_ctr + kk);
+    const FrCtrChunk cc = fr_ctr_chunk(sm, L.lane4, P, fr_bswap(P.iv_ctr + kk));
+    FrCtrGroup cg = {0, 0, 0, 0};
 
-    uint4 y = make_uint4(0, 0, 0, 0), pend = make_uint4(0, 0, 0, 0);
+    uint4 y = make_uint4(0, 0, 0, 0), pend = make_uint4(0, 0, 0, 0), extra = make_uint4(0, 0, 0, 0);
     uint32_t j_last = 0xFFFFFFFFu;
     for (uint32_t r = row0; r < row1; r++) {
-        const uint32_t j = r * FR_ROW_BLOCKS + lane;
+        const uint32_t ctr = r * FR_ROW_BLOCKS + lane;
+        if (r == row0 || (r & 7u) == 0u) cg = fr_ctr_group(sm, L.lane4, P, cc, ctr);   // ctr >> 8 is the same for the whole row
+        const uint32_t j = ctr - 2u;                                                  // wraps for ctr < 2: then j >= seg_end
         if (j < seg_end) {
             const uint64_t boff = (uint64_t)j << 4;
             const bool full = len_k - boff >= 16;
             const uint32_t nvalid = full ? 16u : (uint32_t)(len_k - boff);
             uint4 x = full ? *(const uint4*)(in + boff) : fr_load_partial(in + boff, nvalid);
-            uint4 ks = fr_aes256_ctr_block(sm, L.lane4, P, ivw2, j + 2u);
+            uint4 ks = fr_aes256_ctr_block(sm, L.lane4, P, cc, cg, ctr);
             uint4 o = fr_xor4(x, ks);
             if (full) *(uint4*)(out + boff) = o; else fr_store_partial(out + boff, o, nvalid);
             uint4 g = ENCRYPT ? (full ? o : fr_mask_bytes(o, nvalid)) : x;
             uint4 v = fr_xor4(y, g);
             if (j + FR_HORNER_STRIDE < seg_end) y = fr_ghash_tabmul(sm, L, v);
             else { pend = v; j_last = j; }
+        } else if (ctr == 1u) {
+            extra = fr_aes256_ctr_block(sm, L.lane4, P, cc, cg, 1u);                   // E_K(J0)
         }
     }
-    if (j_last == 0xFFFFFFFFu) return make_uint4(0, 0, 0, 0);
+    if (j_last == 0xFFFFFFFFu) return extra;
     // block j is multiplied by H^(nblk - j + 1): one for each later block, one for the length block
     const uint32_t e = (nblk - 1u - j_last) + 2u;
-    return fr_gf128_mul(pend, P.pow[e]);
-}
-
-// Tag of chunk kk from its data sum: T = S xor LEN*H xor E_K(IV_k || 1)  (paper Section 2.3: the final
-// product is combined with the encrypted nonce block; Section 4.2: one such block per chain).
-__device__ __forceinline__ uint4 fr_chunk_tag(const FrParams& P, const char* sm, uint32_t lane4, uint32_t kk, uint4 S)
-{
-    const uint64_t bits = fr_chunk_len(P, kk) << 3;
-    uint4 lenblk = make_uint4(0, 0, fr_bswap((uint32_t)(bits >> 32)), fr_bswap((uint32_t)bits));
-    uint4 t = fr_gf128_mul(lenblk, P.pow[1]);
-    uint4 ekj0 = fr_aes256_ctr_block(sm, lane4, P, fr_bswap(P.iv_ctr + kk), 1u);
-    return fr_xor4(fr_xor4(S, t), ekj0);
+    return fr_xor4(fr_gf128_mul(pend, P.pow[e]), extra);
 }
