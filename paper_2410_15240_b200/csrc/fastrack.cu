@@ -14,7 +14,7 @@
 
 using namespace fr_host;
 
-#define FR_THREADS 512
+#define FR_THREADS 1024
 #define FR_WARPS (FR_THREADS / 32)
 
 // ------------------------------------------------------------------------------------ kernels ----
@@ -120,6 +120,7 @@ struct fastrack_ctx {
     int last_cuda_error;
     uint64_t launches;
     uint32_t seg_rows_override;   // 0 = automatic (FASTRACK_SEG_ROWS, for experiments)
+    size_t stage_bytes_override;  // 0 = automatic (FASTRACK_STAGE_BYTES, for experiments)
 };
 
 #define FR_CUDA(ctx, call)                                              \
@@ -164,6 +165,7 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, ctx->device);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return fail(FASTRACK_ERR_CUDA); }
     if (const char* env = getenv("FASTRACK_SEG_ROWS")) ctx->seg_rows_override = (uint32_t)strtoul(env, nullptr, 10);
+    if (const char* env = getenv("FASTRACK_STAGE_BYTES")) ctx->stage_bytes_override = (size_t)strtoull(env, nullptr, 10);
 
     // key material on the host: S-box, Te0, round keys, H, byte tables of H^32
     uint8_t sbox[256];
@@ -294,17 +296,29 @@ static void plan_segments(const fastrack_ctx* ctx, size_t len, size_t n_chunks, 
 {
     const size_t first_len = len < ctx->chunk_bytes ? len : ctx->chunk_bytes;
     const size_t rows_ref = ((first_len + 15) / 16 + 2 + FR_ROW_BLOCKS - 1) / FR_ROW_BLOCKS;
-    const size_t total_rows = rows_ref * n_chunks;
     const size_t warps = (size_t)ctx->num_sms * FR_WARPS;
-    size_t seg_rows = ctx->seg_rows_override ? ctx->seg_rows_override : (total_rows + 2 * warps - 1) / (2 * warps);
-    if (!ctx->seg_rows_override) {
-        if (seg_rows < 8) seg_rows = 8;
-        if (seg_rows > 128) seg_rows = 128;
+    // Every segment costs its rows plus one general GF(2^128) product per lane (about 4 rows' worth of
+    // integer work), and segments are dealt round-robin to the resident warps.  Try 1..8 segments per warp
+    // and keep the split with the least work on the busiest warp: large buffers get one long segment per
+    // warp with every warp busy, small ones get the shortest segments (lowest latency).
+    size_t seg_rows = 8, spc = (rows_ref + 7) / 8;
+    if (ctx->seg_rows_override) {
+        seg_rows = ctx->seg_rows_override;
+        spc = (rows_ref + seg_rows - 1) / seg_rows;
+    } else {
+        size_t best_cost = ~(size_t)0;
+        for (size_t m = 1; m <= 8; m++) {
+            size_t want = m * warps / n_chunks;
+            if (want < 1) want = 1;
+            size_t rows = ((rows_ref + want - 1) / want + 7) / 8 * 8;
+            if (rows > 1024) rows = 1024;
+            const size_t per_chunk = (rows_ref + rows - 1) / rows;
+            const size_t waves = (per_chunk * n_chunks + warps - 1) / warps;
+            const size_t cost = waves * (rows + 4);
+            if (cost < best_cost) { best_cost = cost; seg_rows = rows; spc = per_chunk; }
+        }
     }
-    size_t spc = (rows_ref + seg_rows - 1) / seg_rows;
     while (spc * n_chunks >= ((size_t)1 << 31)) { seg_rows *= 2; spc = (rows_ref + seg_rows - 1) / seg_rows; }
-    seg_rows = ((rows_ref + spc - 1) / spc + 7) / 8 * 8;   // equalise the segments of a chunk, whole groups
-    spc = (rows_ref + seg_rows - 1) / seg_rows;
     P.seg_rows = (uint32_t)seg_rows;
     P.segs_per_chunk = (uint32_t)spc;
     P.n_items = (uint32_t)(spc * n_chunks);
@@ -423,9 +437,16 @@ extern "C" int fastrack_pipelined_h2d(fastrack_ctx* ctx, const uint8_t iv_base[1
     FR_CUDA(ctx, cudaEventRecord(ctx->tags_ready, ctx->streams[0]));
     for (int i = 1; i < n_streams; i++) FR_CUDA(ctx, cudaStreamWaitEvent(ctx->streams[i], ctx->tags_ready, 0));
 
+    // Stage = the unit that is copied and then decrypted: whole chunks, about an eighth of the buffer but
+    // between 1 MiB (below that the per-copy and per-launch overheads dominate) and 16 MiB (so that the
+    // kernel of the last stage, the only one no copy hides, stays a small part of the whole).
     const size_t cb = ctx->chunk_bytes;
-    const size_t min_stage = (size_t)1 << 20;
-    const size_t chunks_per_stage = cb >= min_stage ? 1 : min_stage / cb;
+    size_t target = ctx->stage_bytes_override ? ctx->stage_bytes_override : len / 8;
+    if (!ctx->stage_bytes_override) {
+        if (target < ((size_t)1 << 20)) target = (size_t)1 << 20;
+        if (target > ((size_t)16 << 20)) target = (size_t)16 << 20;
+    }
+    const size_t chunks_per_stage = target <= cb ? 1 : (target + cb - 1) / cb;
     const size_t stage_bytes = chunks_per_stage * cb;
     size_t stage = 0;
     for (size_t off = 0; off < len; off += stage_bytes, stage++) {

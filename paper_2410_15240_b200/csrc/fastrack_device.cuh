@@ -215,29 +215,64 @@ __device__ __forceinline__ uint4 fr_ghash_tabmul(const char* sm, const FrLane& L
     return acc;
 }
 
-// General product in GF(2^128) (GCM bit order: bit 0 of a block is the MSB of byte 0 and the
-// coefficient of x^0; "times x" is a right shift with 0xE1 folded into byte 0 on carry-out).
+// General product in GF(2^128), GCM bit order (bit 0 of a block is the MSB of byte 0 and the coefficient
+// of x^0; the field polynomial is x^128 + x^7 + x^2 + x + 1).
+//
+// There is no carry-less multiply instruction, so the 128 x 128 polynomial product is built from
+// ordinary 32 x 32 -> 64 integer multiplies (they run on the FMA pipe, which this kernel otherwise
+// leaves idle): an operand word masked to every fourth bit has 8 live bits, so in the integer product
+// of two such words every 4-bit field holds a count of at most 8 and never carries into its
+// neighbour; the low bit of the field is the GF(2) sum.  A word is split into four such phases, the 16
+// phase products of a word pair are XORed by (phase sum mod 4), and each class keeps only its own bits.
+__device__ __forceinline__ uint32_t fr_to_natural(uint32_t le_word)     // bit i of the result = coefficient of x^(32w + i)
+{
+    return __brev(fr_bswap(le_word));
+}
+
 __device__ __forceinline__ uint4 fr_gf128_mul(uint4 x, uint4 y)
 {
-    uint32_t xw[4] = {fr_bswap(x.x), fr_bswap(x.y), fr_bswap(x.z), fr_bswap(x.w)};
-    uint32_t v0 = fr_bswap(y.x), v1 = fr_bswap(y.y), v2 = fr_bswap(y.z), v3 = fr_bswap(y.w);
-    uint32_t z0 = 0, z1 = 0, z2 = 0, z3 = 0;
-#pragma unroll 1
-    for (int w = 0; w < 4; w++) {
-        uint32_t xb = xw[w];
-#pragma unroll 8
-        for (int b = 0; b < 32; b++) {
-            uint32_t m = (uint32_t)((int32_t)xb >> 31);
-            xb <<= 1;
-            z0 ^= v0 & m; z1 ^= v1 & m; z2 ^= v2 & m; z3 ^= v3 & m;
-            uint32_t carry = (0u - (v3 & 1u)) & 0xE1000000u;
-            v3 = (v3 >> 1) | (v2 << 31);
-            v2 = (v2 >> 1) | (v1 << 31);
-            v1 = (v1 >> 1) | (v0 << 31);
-            v0 = (v0 >> 1) ^ carry;
+    const uint32_t a[4] = {fr_to_natural(x.x), fr_to_natural(x.y), fr_to_natural(x.z), fr_to_natural(x.w)};
+    const uint32_t b[4] = {fr_to_natural(y.x), fr_to_natural(y.y), fr_to_natural(y.z), fr_to_natural(y.w)};
+    uint32_t bs[4][4];
+#pragma unroll
+    for (int j = 0; j < 4; j++)
+#pragma unroll
+        for (int ps = 0; ps < 4; ps++) bs[j][ps] = b[j] & (0x11111111u << ps);
+
+    uint32_t p[8] = {0, 0, 0, 0, 0, 0, 0, 0};       // 256-bit carry-less product, natural order
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+        uint32_t r[4][5];                            // per class k: words i .. i+4 of this limb's partial product
+#pragma unroll
+        for (int k = 0; k < 4; k++)
+#pragma unroll
+            for (int w = 0; w < 5; w++) r[k][w] = 0;
+#pragma unroll
+        for (int ph = 0; ph < 4; ph++) {
+            const uint32_t av = a[i] & (0x11111111u << ph);
+#pragma unroll
+            for (int j = 0; j < 4; j++)
+#pragma unroll
+                for (int ps = 0; ps < 4; ps++) {
+                    const uint64_t m = (uint64_t)av * (uint64_t)bs[j][ps];
+                    r[(ph + ps) & 3][j] ^= (uint32_t)m;
+                    r[(ph + ps) & 3][j + 1] ^= (uint32_t)(m >> 32);
+                }
         }
+#pragma unroll
+        for (int w = 0; w < 5; w++)
+            p[i + w] ^= (r[0][w] & 0x11111111u) | (r[1][w] & 0x22222222u) | (r[2][w] & 0x44444444u) | (r[3][w] & 0x88888888u);
     }
-    return make_uint4(fr_bswap(z0), fr_bswap(z1), fr_bswap(z2), fr_bswap(z3));
+    // reduce: x^128 = x^7 + x^2 + x + 1.  Fold the high half t = p[4..7] as t ^ t<<1 ^ t<<2 ^ t<<7 (a 135-bit value).
+    uint32_t f[5];
+    f[0] = p[4] ^ (p[4] << 1) ^ (p[4] << 2) ^ (p[4] << 7);
+#pragma unroll
+    for (int w = 1; w < 4; w++)
+        f[w] = p[4 + w] ^ ((p[4 + w] << 1) | (p[3 + w] >> 31)) ^ ((p[4 + w] << 2) | (p[3 + w] >> 30)) ^ ((p[4 + w] << 7) | (p[3 + w] >> 25));
+    f[4] = (p[7] >> 31) ^ (p[7] >> 30) ^ (p[7] >> 25);      // bits 128..134: fold once more (at most 7 bits)
+    const uint32_t z0 = p[0] ^ f[0] ^ f[4] ^ (f[4] << 1) ^ (f[4] << 2) ^ (f[4] << 7);
+    const uint32_t z1 = p[1] ^ f[1], z2 = p[2] ^ f[2], z3 = p[3] ^ f[3];
+    return make_uint4(fr_bswap(__brev(z0)), fr_bswap(__brev(z1)), fr_bswap(__brev(z2)), fr_bswap(__brev(z3)));
 }
 
 __device__ __forceinline__ uint64_t fr_chunk_len(const FrParams& P, uint32_t kk)
