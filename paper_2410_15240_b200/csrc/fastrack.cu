@@ -19,18 +19,10 @@ using namespace fr_host;
 
 // ------------------------------------------------------------------------------------ kernels ----
 
-// Fused pass: keystream, XOR, per-segment GHASH partial, per-chunk tag.  Segments are dealt to warps
-// round-robin; a warp XORs its segment's partial into the chunk's accumulator and takes a ticket; the
-// warp that takes the chunk's last ticket finishes the tag (no warp ever waits for another).
-template <bool ENCRYPT>
-__global__ void __launch_bounds__(FR_THREADS, 1) fr_crypt_kernel(const __grid_constant__ FrParams P)
+template <bool ENCRYPT, bool ABS>
+__device__ __forceinline__ void fr_crypt_body(const FrParams& P, const char* sm, FrLane L)
 {
-    extern __shared__ __align__(256) char sm[];
-    fr_build_smem(sm, threadIdx.x, blockDim.x, P.te0, P.gh_tab);
-    __syncthreads();
-
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    const FrLane L = fr_make_lane(lane);
     const uint32_t total_warps = gridDim.x * (blockDim.x >> 5);
 
     for (uint32_t item = warp * gridDim.x + blockIdx.x; item < P.n_items; item += total_warps) {
@@ -38,7 +30,7 @@ __global__ void __launch_bounds__(FR_THREADS, 1) fr_crypt_kernel(const __grid_co
         const uint32_t nseg = fr_chunk_segs(P, kk);
         if (s >= nseg) continue;                       // only the short last chunk has fewer segments
 
-        uint4 z = fr_process_segment_lane<ENCRYPT>(P, sm, L, lane, kk, s);
+        uint4 z = fr_process_segment_lane<ENCRYPT, ABS>(P, sm, L, lane, kk, s);
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) {
             z.x ^= __shfl_xor_sync(0xFFFFFFFFu, z.x, off);
@@ -68,26 +60,41 @@ __global__ void __launch_bounds__(FR_THREADS, 1) fr_crypt_kernel(const __grid_co
                     z.w = atomicExch(&P.acc[4 * kk + 3], 0u);
                     atomicExch(&P.cnt[kk], 0u);
                 }
-                z.x = __shfl_sync(0xFFFFFFFFu, z.x, 0);
-                z.y = __shfl_sync(0xFFFFFFFFu, z.y, 0);
-                z.z = __shfl_sync(0xFFFFFFFFu, z.z, 0);
-                z.w = __shfl_sync(0xFFFFFFFFu, z.w, 0);
             }
         }
         if (finisher && lane == 0) {
             const uint4 lenh = (kk + 1u == P.n_chunks) ? P.lenh_last : P.lenh_full;
             const uint4 tag = fr_xor4(z, lenh);           // z already holds GHASH of the data xor E_K(J0)
-            {
-                if (ENCRYPT) {
-                    P.tags_out[kk] = tag;
-                } else {
-                    const uint4 t = P.tags_in[kk];
-                    const uint32_t diff = (tag.x ^ t.x) | (tag.y ^ t.y) | (tag.z ^ t.z) | (tag.w ^ t.w);
-                    P.ok[kk] = diff == 0u ? 1u : 0u;
-                }
+            if (ENCRYPT) {
+                P.tags_out[kk] = tag;
+            } else {
+                const uint4 t = P.tags_in[kk];
+                const uint32_t diff = (tag.x ^ t.x) | (tag.y ^ t.y) | (tag.z ^ t.z) | (tag.w ^ t.w);
+                P.ok[kk] = diff == 0u ? 1u : 0u;
             }
         }
     }
+}
+
+// Fused pass: keystream, XOR, per-segment GHASH partial, per-chunk tag.  Segments are dealt to warps
+// round-robin; a warp XORs its segment's partial into the chunk's accumulator and takes a ticket; the
+// warp that takes the chunk's last ticket finishes the tag (no warp ever waits for another).
+template <bool ENCRYPT>
+__global__ void __launch_bounds__(FR_THREADS, 1) fr_crypt_kernel(const __grid_constant__ FrParams P)
+{
+    extern __shared__ __align__(256) char sm[];
+    fr_build_smem(sm, threadIdx.x, blockDim.x, P.te0, P.gh_tab);
+    __syncthreads();
+    // Lane constants are made to depend on a value the compiler cannot see through and that is produced
+    // after the barrier, so that no table load can be scheduled above the barrier.
+    uint32_t after_barrier;
+    asm volatile("mov.u32 %0, 0;" : "=r"(after_barrier)::"memory");
+    FrLane L = fr_make_lane(threadIdx.x & 31u);
+    L.lane4 |= after_barrier;
+    L.qe |= after_barrier;
+    L.qo |= after_barrier;
+    if ((uint32_t)__cvta_generic_to_shared(sm) == FR_SMEM_ABS_BASE) fr_crypt_body<ENCRYPT, true>(P, sm, L);
+    else fr_crypt_body<ENCRYPT, false>(P, sm, L);
 }
 
 // pow[i] = pow[i - half] * pow[half] for i in (half, min(2*half, n - 1)]: one doubling pass of the table

@@ -113,16 +113,51 @@ __device__ __forceinline__ void fr_build_smem(char* sm, uint32_t tid, uint32_t n
     for (uint32_t i = tid; i < 4096u; i += nthreads) *(uint4*)(sm + FR_SM_GH + i * 16u) = gh_tab[i];
 }
 
-// Table lookups: byte k of state word w, table t (address = one byte permute; see the header comment).
+// Shared-memory loads.  The dynamic shared window of a kernel without static shared memory starts at shared
+// address FR_SMEM_ABS_BASE on this architecture (the first KiB is reserved by the system).  When the kernel has
+// checked that at run time (ABS = true), a lookup address is "constant + permuted bytes", and the constant goes
+// into the load's immediate field: no add instruction per lookup.  ABS = false is the portable form.
+#define FR_SMEM_ABS_BASE 0x400u
+
+template <bool ABS, uint32_t OFF>
+__device__ __forceinline__ uint32_t fr_lds32(const char* sm, uint32_t addr)
+{
+    if (ABS) {
+#ifdef __CUDA_ARCH__
+        uint32_t v;
+        asm("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(addr), "n"(FR_SMEM_ABS_BASE + OFF));
+        return v;
+#else
+        return 0;
+#endif
+    }
+    return *(const uint32_t*)(sm + OFF + addr);
+}
+
+template <bool ABS, uint32_t OFF>
+__device__ __forceinline__ uint4 fr_lds128(const char* sm, uint32_t addr)
+{
+    if (ABS) {
+#ifdef __CUDA_ARCH__
+        uint4 v;
+        asm("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4+%5];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr), "n"(FR_SMEM_ABS_BASE + OFF));
+        return v;
+#else
+        return make_uint4(0, 0, 0, 0);
+#endif
+    }
+    return *(const uint4*)(sm + OFF + addr);
+}
+
+// Table lookups: byte k of state word w (address = one byte permute; see the header comment).
 #define FR_TA(w, k) FR_PRMT((w), lane4, 0x5504u | ((k) << 4))
-#define FR_LD32(off, addr) (*(const uint32_t*)(sm + (off) + (addr)))
-#define FR_TE0(w, k) FR_LD32(FR_SM_T01, FR_TA(w, k))
-#define FR_TE1(w, k) FR_LD32(FR_SM_T01 + 128u, FR_TA(w, k))
-#define FR_TE2(w, k) FR_LD32(FR_SM_T23, FR_TA(w, k))
-#define FR_TE3(w, k) FR_LD32(FR_SM_T23 + 128u, FR_TA(w, k))
+#define FR_TE0(w, k) fr_lds32<ABS, FR_SM_T01>(sm, FR_TA(w, k))
+#define FR_TE1(w, k) fr_lds32<ABS, FR_SM_T01 + 128u>(sm, FR_TA(w, k))
+#define FR_TE2(w, k) fr_lds32<ABS, FR_SM_T23>(sm, FR_TA(w, k))
+#define FR_TE3(w, k) fr_lds32<ABS, FR_SM_T23 + 128u>(sm, FR_TA(w, k))
 
 // Rounds FIRST..14 of the AES-256 forward cipher on a state that has been through rounds 0..FIRST-1.
-template <int FIRST>
+template <bool ABS, int FIRST>
 __device__ __forceinline__ uint4 fr_aes256_rounds(const char* sm, uint32_t lane4, const FrParams& P,
                                                   uint32_t s0, uint32_t s1, uint32_t s2, uint32_t s3)
 {
@@ -162,6 +197,7 @@ struct FrCtrGroup {        // per 256-counter group
     uint32_t d0, d1, d2, d3;
 };
 
+template <bool ABS>
 __device__ __forceinline__ FrCtrChunk fr_ctr_chunk(const char* sm, uint32_t lane4, const FrParams& P, uint32_t ivw2)
 {
     const uint32_t s0 = P.iv_w0 ^ P.rk[0], s1 = P.iv_w1 ^ P.rk[1], s2 = ivw2 ^ P.rk[2];
@@ -173,6 +209,7 @@ __device__ __forceinline__ FrCtrChunk fr_ctr_chunk(const char* sm, uint32_t lane
     return c;
 }
 
+template <bool ABS>
 __device__ __forceinline__ FrCtrGroup fr_ctr_group(const char* sm, uint32_t lane4, const FrParams& P,
                                                    const FrCtrChunk& c, uint32_t ctr)
 {
@@ -187,16 +224,18 @@ __device__ __forceinline__ FrCtrGroup fr_ctr_group(const char* sm, uint32_t lane
 }
 
 // E_K(IV_k || BE32(ctr)) given the chunk and group constants that belong to ctr.
+template <bool ABS>
 __device__ __forceinline__ uint4 fr_aes256_ctr_block(const char* sm, uint32_t lane4, const FrParams& P,
                                                      const FrCtrChunk& c, const FrCtrGroup& g, uint32_t ctr)
 {
     const uint32_t s3 = fr_bswap(ctr) ^ P.rk[3];
     const uint32_t t0 = c.a0 ^ FR_TE3(s3, 3);
-    return fr_aes256_rounds<3>(sm, lane4, P, g.d0 ^ FR_TE0(t0, 0), g.d1 ^ FR_TE3(t0, 3), g.d2 ^ FR_TE2(t0, 2),
+    return fr_aes256_rounds<ABS, 3>(sm, lane4, P, g.d0 ^ FR_TE0(t0, 0), g.d1 ^ FR_TE3(t0, 3), g.d2 ^ FR_TE2(t0, 2),
                                g.d3 ^ FR_TE1(t0, 1));
 }
 
 // v * H^32 through the byte tables (v, result: little-endian words of the block's 16 bytes).
+template <bool ABS>
 __device__ __forceinline__ uint4 fr_ghash_tabmul(const char* sm, const FrLane& L, uint4 v)
 {
     // lanes with h = 1 walk the words in swapped pairs, so static word w holds actual word w ^ h
@@ -208,7 +247,7 @@ __device__ __forceinline__ uint4 fr_ghash_tabmul(const char* sm, const FrLane& L
 #pragma unroll
         for (int rho = 0; rho < 4; rho++) {
             uint32_t addr = FR_PRMT(s[w], (w & 1) ? L.qo : L.qe, L.sel[rho]);
-            uint4 t = *(const uint4*)(sm + FR_SM_GH + ((uint32_t)(w >> 1) << 7) + addr);
+            uint4 t = (w >> 1) ? fr_lds128<ABS, FR_SM_GH + 128u>(sm, addr) : fr_lds128<ABS, FR_SM_GH>(sm, addr);
             acc = fr_xor4(acc, t);
         }
     }
@@ -322,7 +361,7 @@ __device__ __forceinline__ uint4 fr_mask_bytes(uint4 v, uint32_t n)
 // lane's Horner value, and return that value multiplied by the power of H that aligns it to the end
 // of the chunk (lane 1 of the chunk's first segment adds E_K(J0)).  XOR of the 32 lanes' results over all
 // segments of the chunk = GHASH of the data blocks (before the length block) xor E_K(J0).
-template <bool ENCRYPT>
+template <bool ENCRYPT, bool ABS>
 __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, const char* sm, const FrLane& L,
                                                          uint32_t lane, uint32_t kk, uint32_t s)
 {
@@ -337,29 +376,29 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
     if (seg_end > nblk) seg_end = nblk;
     const uint8_t* in = P.in + chunk_off;
     uint8_t* out = P.out + chunk_off;
-    const FrCtrChunk cc = fr_ctr_chunk(sm, L.lane4, P, fr_bswap(P.iv_ctr + kk));
+    const FrCtrChunk cc = fr_ctr_chunk<ABS>(sm, L.lane4, P, fr_bswap(P.iv_ctr + kk));
     FrCtrGroup cg = {0, 0, 0, 0};
 
     uint4 y = make_uint4(0, 0, 0, 0), pend = make_uint4(0, 0, 0, 0), extra = make_uint4(0, 0, 0, 0);
     uint32_t j_last = 0xFFFFFFFFu;
     for (uint32_t r = row0; r < row1; r++) {
         const uint32_t ctr = r * FR_ROW_BLOCKS + lane;
-        if (r == row0 || (r & 7u) == 0u) cg = fr_ctr_group(sm, L.lane4, P, cc, ctr);   // ctr >> 8 is the same for the whole row
+        if (r == row0 || (r & 7u) == 0u) cg = fr_ctr_group<ABS>(sm, L.lane4, P, cc, ctr);   // ctr >> 8 is the same for the whole row
         const uint32_t j = ctr - 2u;                                                  // wraps for ctr < 2: then j >= seg_end
         if (j < seg_end) {
             const uint64_t boff = (uint64_t)j << 4;
             const bool full = len_k - boff >= 16;
             const uint32_t nvalid = full ? 16u : (uint32_t)(len_k - boff);
             uint4 x = full ? *(const uint4*)(in + boff) : fr_load_partial(in + boff, nvalid);
-            uint4 ks = fr_aes256_ctr_block(sm, L.lane4, P, cc, cg, ctr);
+            uint4 ks = fr_aes256_ctr_block<ABS>(sm, L.lane4, P, cc, cg, ctr);
             uint4 o = fr_xor4(x, ks);
             if (full) *(uint4*)(out + boff) = o; else fr_store_partial(out + boff, o, nvalid);
             uint4 g = ENCRYPT ? (full ? o : fr_mask_bytes(o, nvalid)) : x;
             uint4 v = fr_xor4(y, g);
-            if (j + FR_HORNER_STRIDE < seg_end) y = fr_ghash_tabmul(sm, L, v);
+            if (j + FR_HORNER_STRIDE < seg_end) y = fr_ghash_tabmul<ABS>(sm, L, v);
             else { pend = v; j_last = j; }
         } else if (ctr == 1u) {
-            extra = fr_aes256_ctr_block(sm, L.lane4, P, cc, cg, 1u);                   // E_K(J0)
+            extra = fr_aes256_ctr_block<ABS>(sm, L.lane4, P, cc, cg, 1u);                   // E_K(J0)
         }
     }
     if (j_last == 0xFFFFFFFFu) return extra;
