@@ -327,6 +327,88 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Device-resident and pipelined throughput over the benchmark configurations (one JSON line per cell)."""
+    import torch
+    from paper_2410_15240_b200 import fastrack, synth
+    torch.cuda.set_device(0)
+    key, iv = synth.key_and_iv(1)
+    stream = torch.cuda.current_stream()
+
+    def timed(fn, reps):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps * 1e-3
+
+    def device_cell(n, cb, label):
+        K = (n + cb - 1) // cb
+        with fastrack.Context(key, cb) as ctx:
+            d_p = torch.randint(0, 256, (n,), dtype=torch.uint8, device="cuda")
+            d_c, d_o = torch.empty_like(d_p), torch.empty_like(d_p)
+            d_t = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
+            d_ok = torch.zeros(K, dtype=torch.int32, device="cuda")
+            st = stream.cuda_stream
+            reps = max(5, min(200, int(2e9 // max(n, 1))))
+            t_enc = timed(lambda: ctx.encrypt_tag(iv, d_p.data_ptr(), n, d_c.data_ptr(), d_t.data_ptr(), st), reps)
+            t_dec = timed(lambda: ctx.decrypt_verify(iv, d_c.data_ptr(), n, d_t.data_ptr(), d_o.data_ptr(),
+                                                     d_ok.data_ptr(), st), reps)
+            assert bool((d_ok == 1).all()) and bool((d_o == d_p).all())
+        print(json.dumps({"cell": label, "len": n, "chunk": cb, "K": K, "decrypt_verify_gbs": n / t_dec / 1e9,
+                          "encrypt_tag_gbs": n / t_enc / 1e9, "decrypt_us": t_dec * 1e6}), flush=True)
+
+    def pipeline_cell(n, cb, n_streams, label):
+        K = (n + cb - 1) // cb
+        with fastrack.Context(key, cb) as ctx:
+            d_p = torch.randint(0, 256, (n,), dtype=torch.uint8, device="cuda")
+            d_c = torch.empty_like(d_p)
+            d_t = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
+            d_ok = torch.zeros(K, dtype=torch.int32, device="cuda")
+            ctx.encrypt_tag(iv, d_p.data_ptr(), n, d_c.data_ptr(), d_t.data_ptr(), stream.cuda_stream)
+            torch.cuda.synchronize()
+            h_c, h_t = d_c.cpu().pin_memory(), d_t.cpu().pin_memory()
+            d_o = torch.empty_like(d_p)
+            reps = 20
+
+            def wall(fn):
+                for _ in range(3):
+                    fn()
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                for _ in range(reps):
+                    fn()
+                torch.cuda.synchronize()
+                return (time.perf_counter() - t0) / reps
+
+            t_pipe = wall(lambda: ctx.pipelined_h2d(iv, h_c.data_ptr(), n, h_t.data_ptr(), d_o.data_ptr(),
+                                                    d_ok.data_ptr(), n_streams))
+            assert bool((d_ok == 1).all()) and bool((d_o == d_p).all())
+
+            def raw():
+                d_o.copy_(h_c, non_blocking=True)
+                torch.cuda.current_stream().synchronize()
+            t_raw = wall(raw)
+        print(json.dumps({"cell": label, "len": n, "chunk": cb, "K": K, "streams": n_streams,
+                          "pipelined_h2d_gbs": n / t_pipe / 1e9, "raw_pinned_h2d_gbs": n / t_raw / 1e9,
+                          "fraction_of_raw": t_raw / t_pipe}), flush=True)
+
+    for K in (1, 4, 16, 64, 256, 1024):                                   # config 1
+        device_cell(64 << 20, (64 << 20) // K, "config1")
+    for cb in (256 << 10, 1 << 20, 4 << 20, 8 << 20):                     # config 2
+        for ns in (2, 3, 4):
+            pipeline_cell(77_070_336, cb, ns, "config2")
+    device_cell(670_000_000, 4 << 20, "config3")
+    for e in range(6, 17):                                                # config 4 (device-resident throughput)
+        for cb in (16 << 10, 64 << 10, 256 << 10, 1 << 20, 4 << 20, 16 << 20):
+            device_cell(4 ** e, cb, "config4")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -336,8 +418,12 @@ def main():
     ap.add_argument("--impl", default="fastrack", choices=["fastrack", "reference"])
     ap.add_argument("--kernel-only", action="store_true",
                     help="time only the device-resident decrypt+verify loop (short run for profilers)")
+    ap.add_argument("--sweep", action="store_true",
+                    help="print throughput over the benchmark configurations instead of the one bench line")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_gpu(args)

@@ -119,10 +119,11 @@ FASTRACK_API int fastrack_encrypt_tag(fastrack_ctx* ctx, const uint8_t iv_base[1
 /* Pipelined host->device transfer with decryption and verification (paper Section 4.3 "Decryption
  * pipeline": the PCIe transfer is overlapped with the decryption and authentication kernels, so the
  * transfer costs max(copy, kernels) instead of their sum).
- * The buffer is cut into stages of whole chunks (about an eighth of the buffer, at least 1 MiB and at most
- * 16 MiB, never less than one chunk); stage i is copied pinned->device into its final place in d_plain with
- * cudaMemcpyAsync on internal stream i mod n_streams and decrypted and verified in place by the same
- * kernels on that stream, so the copy of stage i+1 overlaps the kernels of stage i.
+ * The buffer is cut into stages of whole chunks that shrink geometrically (half of the buffer, then half of
+ * the rest, ... down to about 2 MiB, never less than one chunk); stage i is copied pinned->device into its
+ * final place in d_plain with cudaMemcpyAsync on internal stream i mod n_streams and decrypted and verified
+ * in place by the same kernels on that stream, so the copy of stage i+1 overlaps the kernels of stage i and
+ * only the short last stage's kernel is exposed.
  *   h_cipher_pinned host, page-locked (cudaHostAlloc / cudaHostRegister), len bytes.
  *   h_tags          host, 16*K bytes, pinned or pageable (copied once, up front).
  *   d_plain, d_ok   device outputs as in fastrack_decrypt_verify.

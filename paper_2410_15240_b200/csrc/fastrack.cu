@@ -83,7 +83,7 @@ template <bool ENCRYPT>
 __global__ void __launch_bounds__(FR_THREADS, 1) fr_crypt_kernel(const __grid_constant__ FrParams P)
 {
     extern __shared__ __align__(256) char sm[];
-    fr_build_smem(sm, threadIdx.x, blockDim.x, P.te0, P.gh_tab);
+    fr_build_smem<FR_THREADS>(sm, threadIdx.x, P.te0, P.gh_tab);
     __syncthreads();
     // Lane constants are made to depend on a value the compiler cannot see through and that is produced
     // after the barrier, so that no table load can be scheduled above the barrier.
@@ -304,24 +304,34 @@ static void plan_segments(const fastrack_ctx* ctx, size_t len, size_t n_chunks, 
     const size_t first_len = len < ctx->chunk_bytes ? len : ctx->chunk_bytes;
     const size_t rows_ref = ((first_len + 15) / 16 + 2 + FR_ROW_BLOCKS - 1) / FR_ROW_BLOCKS;
     const size_t warps = (size_t)ctx->num_sms * FR_WARPS;
-    // Every segment costs its rows plus one general GF(2^128) product per lane (about 4 rows' worth of
-    // integer work), and segments are dealt round-robin to the resident warps.  Try 1..8 segments per warp
-    // and keep the split with the least work on the busiest warp: large buffers get one long segment per
-    // warp with every warp busy, small ones get the shortest segments (lowest latency).
+    // Segments are dealt round-robin to the resident warps.  Two things bound a launch: the latency of the
+    // busiest warp (about 1000 cycles per row when few warps run, plus about 4000 per segment for the closing
+    // GF(2^128) product, the atomics and the tag), and the shared-memory work of the busiest SM (about 270
+    // wavefront-cycles per row plus about 300 per segment).  Try short segments (2 or 4 rows, for small buffers)
+    // and 1..8 segments per warp in whole 8-row groups, and keep the split with the smaller bound.
     size_t seg_rows = 8, spc = (rows_ref + 7) / 8;
     if (ctx->seg_rows_override) {
         seg_rows = ctx->seg_rows_override;
         spc = (rows_ref + seg_rows - 1) / seg_rows;
     } else {
         size_t best_cost = ~(size_t)0;
-        for (size_t m = 1; m <= 8; m++) {
-            size_t want = m * warps / n_chunks;
-            if (want < 1) want = 1;
-            size_t rows = ((rows_ref + want - 1) / want + 7) / 8 * 8;
-            if (rows > 1024) rows = 1024;
+        for (int cand = 0; cand < 10; cand++) {
+            size_t rows;
+            if (cand < 2) {
+                rows = cand == 0 ? 2 : 4;
+            } else {
+                size_t want = (size_t)(cand - 1) * warps / n_chunks;
+                if (want < 1) want = 1;
+                rows = ((rows_ref + want - 1) / want + 7) / 8 * 8;
+                if (rows > 1024) rows = 1024;
+            }
             const size_t per_chunk = (rows_ref + rows - 1) / rows;
-            const size_t waves = (per_chunk * n_chunks + warps - 1) / warps;
-            const size_t cost = waves * (rows + 4);
+            const size_t items = per_chunk * n_chunks;
+            const size_t waves = (items + warps - 1) / warps;
+            const size_t per_sm = (items + (size_t)ctx->num_sms - 1) / (size_t)ctx->num_sms;
+            const size_t latency = waves * (rows * 1000 + 4000);
+            const size_t throughput = per_sm * (rows * 270 + 300);
+            const size_t cost = latency > throughput ? latency : throughput;
             if (cost < best_cost) { best_cost = cost; seg_rows = rows; spc = per_chunk; }
         }
     }
@@ -439,25 +449,33 @@ extern "C" int fastrack_pipelined_h2d(fastrack_ctx* ctx, const uint8_t iv_base[1
         ctx->tags_stage_chunks = cap;
     }
 
-    // tags first, once; every other stream waits for that copy before its first kernel
-    FR_CUDA(ctx, cudaMemcpyAsync(ctx->d_tags_stage, h_tags, K * 16, cudaMemcpyHostToDevice, ctx->streams[0]));
-    FR_CUDA(ctx, cudaEventRecord(ctx->tags_ready, ctx->streams[0]));
-    for (int i = 1; i < n_streams; i++) FR_CUDA(ctx, cudaStreamWaitEvent(ctx->streams[i], ctx->tags_ready, 0));
+    // tags: one small copy on a stream of its own; every working stream waits for it before its first kernel
+    cudaStream_t tag_stream = ctx->streams[7];
+    FR_CUDA(ctx, cudaMemcpyAsync(ctx->d_tags_stage, h_tags, K * 16, cudaMemcpyHostToDevice, tag_stream));
+    FR_CUDA(ctx, cudaEventRecord(ctx->tags_ready, tag_stream));
+    for (int i = 0; i < n_streams; i++)
+        if (ctx->streams[i] != tag_stream) FR_CUDA(ctx, cudaStreamWaitEvent(ctx->streams[i], ctx->tags_ready, 0));
 
-    // Stage = the unit that is copied and then decrypted: whole chunks, about an eighth of the buffer but
-    // between 1 MiB (below that the per-copy and per-launch overheads dominate) and 16 MiB (so that the
-    // kernel of the last stage, the only one no copy hides, stays a small part of the whole).
+    // Stage = the unit that is copied and then decrypted in place: whole chunks.  Only two things are not
+    // hidden behind a copy: a few microseconds per copy boundary and the kernel of the LAST stage.  So the
+    // stages shrink geometrically: the first takes half of the buffer, each next one half of what is left,
+    // down to about 2 MiB (never less than one chunk) -- few copies, and a short last kernel.  A stage's
+    // kernel is an order of magnitude faster than the next stage's copy, so it always finishes under it.
     const size_t cb = ctx->chunk_bytes;
-    size_t target = ctx->stage_bytes_override ? ctx->stage_bytes_override : len / 8;
-    if (!ctx->stage_bytes_override) {
-        if (target < ((size_t)1 << 20)) target = (size_t)1 << 20;
-        if (target > ((size_t)16 << 20)) target = (size_t)16 << 20;
-    }
-    const size_t chunks_per_stage = target <= cb ? 1 : (target + cb - 1) / cb;
-    const size_t stage_bytes = chunks_per_stage * cb;
-    size_t stage = 0;
-    for (size_t off = 0; off < len; off += stage_bytes, stage++) {
-        const size_t n = len - off < stage_bytes ? len - off : stage_bytes;
+    const size_t floor_bytes = (size_t)2 << 20;
+    const size_t min_stage = cb >= floor_bytes ? cb : (floor_bytes + cb - 1) / cb * cb;
+    size_t off = 0, stage = 0;
+    while (off < len) {
+        const size_t remaining = len - off;
+        size_t n;
+        if (ctx->stage_bytes_override) {
+            n = (ctx->stage_bytes_override + cb - 1) / cb * cb;
+        } else {
+            n = remaining / 2 / cb * cb;
+            if (n < min_stage) n = min_stage;
+            if (remaining < n + min_stage / 2) n = remaining;      // do not leave a sliver behind
+        }
+        if (n > remaining) n = remaining;
         const size_t k0 = off / cb;
         cudaStream_t st = ctx->streams[stage % (size_t)n_streams];
         uint8_t* dst = (uint8_t*)d_plain + off;
@@ -466,11 +484,14 @@ extern "C" int fastrack_pipelined_h2d(fastrack_ctx* ctx, const uint8_t iv_base[1
         if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); rc = FASTRACK_ERR_CUDA; }
         if (rc == FASTRACK_OK) rc = launch_pass(ctx, false, iv_base, k0, dst, n, dst, ctx->d_tags_stage + k0, nullptr, d_ok + k0, st);
         if (rc != FASTRACK_OK) {
-            for (int i = 0; i < n_streams; i++) cudaStreamSynchronize(ctx->streams[i]);
+            for (int i = 0; i < 8; i++) cudaStreamSynchronize(ctx->streams[i]);
             (void)cudaGetLastError();
             return rc;
         }
+        off += n;
+        stage++;
     }
+    FR_CUDA(ctx, cudaStreamSynchronize(tag_stream));
     for (int i = 0; i < n_streams; i++) FR_CUDA(ctx, cudaStreamSynchronize(ctx->streams[i]));
     return FASTRACK_OK;
 }

@@ -99,18 +99,29 @@ __device__ __forceinline__ FrLane fr_make_lane(uint32_t lane)
 }
 
 // Fill shared memory: replicate Te0 and its three byte rotations per lane, copy the H^32 byte tables.
-__device__ __forceinline__ void fr_build_smem(char* sm, uint32_t tid, uint32_t nthreads,
-                                              const uint32_t* __restrict__ te0, const uint4* __restrict__ gh_tab)
+// NTHREADS is a compile-time constant so that all of a thread's global loads are issued before the first store.
+template <uint32_t NTHREADS>
+__device__ __forceinline__ void fr_build_smem(char* sm, uint32_t tid, const uint32_t* __restrict__ te0,
+                                              const uint4* __restrict__ gh_tab)
 {
-    // 256 rows x 2 arrays x 2 tables x 8 uint4 (32 words) each
-    for (uint32_t i = tid; i < 256u * 4u * 8u; i += nthreads) {
-        uint32_t q = i & 7u, t = (i >> 3) & 3u, v = i >> 5;
-        uint32_t e = te0[v];
-        uint32_t w = (t == 0) ? e : (t == 1) ? ((e << 8) | (e >> 24)) : (t == 2) ? ((e << 16) | (e >> 16)) : ((e << 24) | (e >> 8));
-        uint32_t off = ((t >> 1) ? FR_SM_T23 : FR_SM_T01) + v * 256u + (t & 1u) * 128u + q * 16u;
+    constexpr uint32_t N_AES = 256u * 4u * 8u / NTHREADS;     // 256 rows x 2 arrays x 2 tables x 8 uint4 (32 words)
+    constexpr uint32_t N_GH = 4096u / NTHREADS;
+    static_assert(N_AES * NTHREADS == 8192u && N_GH * NTHREADS == 4096u, "thread count must divide the tables");
+    uint32_t e[N_AES];
+    uint4 g[N_GH];
+#pragma unroll
+    for (uint32_t n = 0; n < N_AES; n++) e[n] = te0[(tid + n * NTHREADS) >> 5];
+#pragma unroll
+    for (uint32_t n = 0; n < N_GH; n++) g[n] = gh_tab[tid + n * NTHREADS];
+#pragma unroll
+    for (uint32_t n = 0; n < N_AES; n++) {
+        const uint32_t i = tid + n * NTHREADS, q = i & 7u, t = (i >> 3) & 3u, v = i >> 5;
+        const uint32_t w = (t == 0) ? e[n] : (t == 1) ? ((e[n] << 8) | (e[n] >> 24)) : (t == 2) ? ((e[n] << 16) | (e[n] >> 16)) : ((e[n] << 24) | (e[n] >> 8));
+        const uint32_t off = ((t >> 1) ? FR_SM_T23 : FR_SM_T01) + v * 256u + (t & 1u) * 128u + q * 16u;
         *(uint4*)(sm + off) = make_uint4(w, w, w, w);
     }
-    for (uint32_t i = tid; i < 4096u; i += nthreads) *(uint4*)(sm + FR_SM_GH + i * 16u) = gh_tab[i];
+#pragma unroll
+    for (uint32_t n = 0; n < N_GH; n++) *(uint4*)(sm + FR_SM_GH + (tid + n * NTHREADS) * 16u) = g[n];
 }
 
 // Shared-memory loads.  The dynamic shared window of a kernel without static shared memory starts at shared
@@ -263,45 +274,54 @@ __device__ __forceinline__ uint4 fr_ghash_tabmul(const char* sm, const FrLane& L
 // of two such words every 4-bit field holds a count of at most 8 and never carries into its
 // neighbour; the low bit of the field is the GF(2) sum.  A word is split into four such phases, the 16
 // phase products of a word pair are XORed by (phase sum mod 4), and each class keeps only its own bits.
+// Karatsuba on top of that brings a 128 x 128 product down to nine word products.
 __device__ __forceinline__ uint32_t fr_to_natural(uint32_t le_word)     // bit i of the result = coefficient of x^(32w + i)
 {
     return __brev(fr_bswap(le_word));
+}
+
+// 32 x 32 -> 64 carry-less product from 16 integer multiplies (see above).
+__device__ __forceinline__ uint64_t fr_clmul32(uint32_t a, uint32_t b)
+{
+    uint32_t as[4], bs[4];
+#pragma unroll
+    for (int k = 0; k < 4; k++) { as[k] = a & (0x11111111u << k); bs[k] = b & (0x11111111u << k); }
+    uint64_t z[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int i = 0; i < 4; i++)
+#pragma unroll
+        for (int j = 0; j < 4; j++) z[(i + j) & 3] ^= (uint64_t)as[i] * (uint64_t)bs[j];
+    return (z[0] & 0x1111111111111111ull) | (z[1] & 0x2222222222222222ull) | (z[2] & 0x4444444444444444ull) |
+           (z[3] & 0x8888888888888888ull);
+}
+
+// 64 x 64 -> 128 by Karatsuba: three 32 x 32 products.
+__device__ __forceinline__ void fr_clmul64(uint32_t a0, uint32_t a1, uint32_t b0, uint32_t b1, uint32_t r[4])
+{
+    const uint64_t lo = fr_clmul32(a0, b0), hi = fr_clmul32(a1, b1);
+    const uint64_t mid = fr_clmul32(a0 ^ a1, b0 ^ b1) ^ lo ^ hi;
+    r[0] = (uint32_t)lo;
+    r[1] = (uint32_t)(lo >> 32) ^ (uint32_t)mid;
+    r[2] = (uint32_t)hi ^ (uint32_t)(mid >> 32);
+    r[3] = (uint32_t)(hi >> 32);
 }
 
 __device__ __forceinline__ uint4 fr_gf128_mul(uint4 x, uint4 y)
 {
     const uint32_t a[4] = {fr_to_natural(x.x), fr_to_natural(x.y), fr_to_natural(x.z), fr_to_natural(x.w)};
     const uint32_t b[4] = {fr_to_natural(y.x), fr_to_natural(y.y), fr_to_natural(y.z), fr_to_natural(y.w)};
-    uint32_t bs[4][4];
+    // 128 x 128 -> 256 by Karatsuba on the 64-bit halves: nine 32 x 32 products = 144 integer multiplies.
+    uint32_t lo[4], hi[4], mid[4];
+    fr_clmul64(a[0], a[1], b[0], b[1], lo);
+    fr_clmul64(a[2], a[3], b[2], b[3], hi);
+    fr_clmul64(a[0] ^ a[2], a[1] ^ a[3], b[0] ^ b[2], b[1] ^ b[3], mid);
+    uint32_t p[8];
 #pragma unroll
-    for (int j = 0; j < 4; j++)
-#pragma unroll
-        for (int ps = 0; ps < 4; ps++) bs[j][ps] = b[j] & (0x11111111u << ps);
-
-    uint32_t p[8] = {0, 0, 0, 0, 0, 0, 0, 0};       // 256-bit carry-less product, natural order
-#pragma unroll
-    for (int i = 0; i < 4; i++) {
-        uint32_t r[4][5];                            // per class k: words i .. i+4 of this limb's partial product
-#pragma unroll
-        for (int k = 0; k < 4; k++)
-#pragma unroll
-            for (int w = 0; w < 5; w++) r[k][w] = 0;
-#pragma unroll
-        for (int ph = 0; ph < 4; ph++) {
-            const uint32_t av = a[i] & (0x11111111u << ph);
-#pragma unroll
-            for (int j = 0; j < 4; j++)
-#pragma unroll
-                for (int ps = 0; ps < 4; ps++) {
-                    const uint64_t m = (uint64_t)av * (uint64_t)bs[j][ps];
-                    r[(ph + ps) & 3][j] ^= (uint32_t)m;
-                    r[(ph + ps) & 3][j + 1] ^= (uint32_t)(m >> 32);
-                }
-        }
-#pragma unroll
-        for (int w = 0; w < 5; w++)
-            p[i + w] ^= (r[0][w] & 0x11111111u) | (r[1][w] & 0x22222222u) | (r[2][w] & 0x44444444u) | (r[3][w] & 0x88888888u);
-    }
+    for (int w = 0; w < 4; w++) mid[w] ^= lo[w] ^ hi[w];
+    p[0] = lo[0]; p[1] = lo[1];
+    p[2] = lo[2] ^ mid[0]; p[3] = lo[3] ^ mid[1];
+    p[4] = hi[0] ^ mid[2]; p[5] = hi[1] ^ mid[3];
+    p[6] = hi[2]; p[7] = hi[3];
     // reduce: x^128 = x^7 + x^2 + x + 1.  Fold the high half t = p[4..7] as t ^ t<<1 ^ t<<2 ^ t<<7 (a 135-bit value).
     uint32_t f[5];
     f[0] = p[4] ^ (p[4] << 1) ^ (p[4] << 2) ^ (p[4] << 7);
@@ -376,11 +396,27 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
     if (seg_end > nblk) seg_end = nblk;
     const uint8_t* in = P.in + chunk_off;
     uint8_t* out = P.out + chunk_off;
+    // The lane's last block and its power of H follow from the geometry alone: fetch the power now, under the rows.
+    // Block j is multiplied by H^(nblk - j + 1): one for each later block, one for the length block.
+    uint32_t j_last = 0xFFFFFFFFu;
+    uint4 hpow = make_uint4(0, 0, 0, 0);
+    {
+        const uint32_t seg_begin = (row0 == 0) ? 0u : row0 * FR_ROW_BLOCKS - 2u;     // first block of this segment
+        if (seg_end > seg_begin) {
+            // largest j < seg_end with (j + 2) mod 32 == lane
+            const uint32_t top = seg_end + 1u;                                        // counter of block seg_end - 1
+            uint32_t c_last = (top & ~31u) | lane;
+            if (c_last > top) c_last -= 32u;
+            if (c_last >= 2u && c_last - 2u >= seg_begin && c_last <= top) {
+                j_last = c_last - 2u;
+                hpow = P.pow[(nblk - 1u - j_last) + 2u];
+            }
+        }
+    }
     const FrCtrChunk cc = fr_ctr_chunk<ABS>(sm, L.lane4, P, fr_bswap(P.iv_ctr + kk));
     FrCtrGroup cg = {0, 0, 0, 0};
 
     uint4 y = make_uint4(0, 0, 0, 0), pend = make_uint4(0, 0, 0, 0), extra = make_uint4(0, 0, 0, 0);
-    uint32_t j_last = 0xFFFFFFFFu;
     for (uint32_t r = row0; r < row1; r++) {
         const uint32_t ctr = r * FR_ROW_BLOCKS + lane;
         if (r == row0 || (r & 7u) == 0u) cg = fr_ctr_group<ABS>(sm, L.lane4, P, cc, ctr);   // ctr >> 8 is the same for the whole row
@@ -395,14 +431,12 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
             if (full) *(uint4*)(out + boff) = o; else fr_store_partial(out + boff, o, nvalid);
             uint4 g = ENCRYPT ? (full ? o : fr_mask_bytes(o, nvalid)) : x;
             uint4 v = fr_xor4(y, g);
-            if (j + FR_HORNER_STRIDE < seg_end) y = fr_ghash_tabmul<ABS>(sm, L, v);
-            else { pend = v; j_last = j; }
+            if (j != j_last) y = fr_ghash_tabmul<ABS>(sm, L, v);
+            else pend = v;
         } else if (ctr == 1u) {
             extra = fr_aes256_ctr_block<ABS>(sm, L.lane4, P, cc, cg, 1u);                   // E_K(J0)
         }
     }
     if (j_last == 0xFFFFFFFFu) return extra;
-    // block j is multiplied by H^(nblk - j + 1): one for each later block, one for the length block
-    const uint32_t e = (nblk - 1u - j_last) + 2u;
-    return fr_xor4(fr_gf128_mul(pend, P.pow[e]), extra);
+    return fr_xor4(fr_gf128_mul(pend, hpow), extra);
 }
