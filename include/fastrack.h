@@ -26,7 +26,8 @@
  *     data buffer; the context owns only key-derived tables, per-chunk scratch and internal streams.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *   - A context is bound to the device that was current at creation and must not be used from two
- *     host threads, or on two streams, at the same time (calls share per-chunk scratch memory).
+ *     host threads, or on two streams, at the same time (calls share per-chunk scratch memory); the one
+ *     exception is fastrack_verify, see there.
  *   - IV discipline is the caller's: one call consumes the IV values iv_base .. iv_base + K - 1;
  *     reusing an IV under the same key voids GCM's guarantees.  The library does not track this.
  *   - K is derived from `len`; dropping trailing chunks is invisible to this layer, so `len` must
@@ -133,6 +134,47 @@ FASTRACK_API int fastrack_encrypt_tag(fastrack_ctx* ctx, const uint8_t iv_base[1
 FASTRACK_API int fastrack_pipelined_h2d(fastrack_ctx* ctx, const uint8_t iv_base[12],
                                         const void* h_cipher_pinned, size_t len, const void* h_tags,
                                         void* d_plain, uint32_t* d_ok, int n_streams);
+
+/* ---- Split passes (paper Section 4.3, "Eager evaluation") -------------------------------------------------
+ * The paper lets the consumer start on the decrypted data before authentication has finished and runs the
+ * authentication kernel later, in parallel with the next batch's PCIe transfer; results are discarded if the
+ * verdict comes back negative (Section 3).  These two calls are the two halves of fastrack_decrypt_verify:
+ *
+ * fastrack_ctr_crypt: keystream + XOR only, d_out = d_in xor E_K(counter blocks).  It is its own inverse, so
+ *   it both decrypts and encrypts.  No tags are read or written.  d_out == d_in is allowed.
+ * fastrack_verify: GHASH of the CIPHERTEXT + tag compare only; d_cipher is not modified, d_ok as in
+ *   fastrack_decrypt_verify.  The ciphertext must therefore still exist when it runs (do not decrypt in place
+ *   if verification is deferred).  It uses a scratch bank of its own, so one fastrack_verify may run on
+ *   another stream concurrently with one call of any other kind on the same context.
+ * Both are asynchronous on `stream`; same pointer rules as fastrack_decrypt_verify.  For every input,
+ * ctr_crypt followed (or preceded) by verify gives exactly the plaintext and verdicts of the fused call. */
+FASTRACK_API int fastrack_ctr_crypt(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_in, size_t len,
+                                    void* d_out, void* stream);
+FASTRACK_API int fastrack_verify(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_cipher, size_t len,
+                                 const void* d_tags, uint32_t* d_ok, void* stream);
+
+/* ---- Keystream ahead of the data (paper Section 4.3, "Parallel AES evaluation") --------------------------
+ * AES(k, counter) does not depend on the ciphertext, so the one-time pad can be produced while the PCIe copy
+ * is still in flight; when the data arrives, decryption is one XOR.
+ *
+ * fastrack_keystream: writes the keystream of a len-byte buffer to d_pad (device, len bytes, same chunk
+ *   layout as the data) and E_K(IV_k || 1), the tag mask of every chunk, to d_mask (device, 16*K bytes).
+ * fastrack_xor_verify: d_plain = d_cipher xor d_pad, GHASH of the ciphertext, tag = GHASH xor d_mask[k],
+ *   compare -> d_ok.  No AES runs in this pass.  d_plain == d_cipher is allowed; d_pad must not overlap d_plain.
+ *   d_pad / d_mask must come from fastrack_keystream with the same context, iv_base and len.
+ * fastrack_pipelined_h2d_ahead: fastrack_pipelined_h2d with the keystream of the whole buffer produced first,
+ *   on an internal stream, under the first copy; the per-stage kernels then only XOR and authenticate, which
+ *   shortens the one kernel no copy hides (the last stage's).  d_pad: caller-provided device buffer of len
+ *   bytes, 16-byte aligned, not overlapping d_plain; its contents afterwards are the keystream (treat it as
+ *   secret and clear it).  Blocking, like fastrack_pipelined_h2d. */
+FASTRACK_API int fastrack_keystream(fastrack_ctx* ctx, const uint8_t iv_base[12], size_t len, void* d_pad,
+                                    void* d_mask, void* stream);
+FASTRACK_API int fastrack_xor_verify(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_cipher, size_t len,
+                                     const void* d_pad, const void* d_mask, const void* d_tags, void* d_plain,
+                                     uint32_t* d_ok, void* stream);
+FASTRACK_API int fastrack_pipelined_h2d_ahead(fastrack_ctx* ctx, const uint8_t iv_base[12],
+                                              const void* h_cipher_pinned, size_t len, const void* h_tags,
+                                              void* d_pad, void* d_plain, uint32_t* d_ok, int n_streams);
 
 /* fastrack_decrypt_verify for callers that must not allocate.  (The paper has no counterpart; this is a
  * deployment variant of the same operation.)

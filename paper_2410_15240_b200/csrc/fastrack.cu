@@ -19,7 +19,7 @@ using namespace fr_host;
 
 // ------------------------------------------------------------------------------------ kernels ----
 
-template <bool ENCRYPT, bool ABS>
+template <int MODE, bool ABS>
 __device__ __forceinline__ void fr_crypt_body(const FrParams& P, const char* sm, FrLane L)
 {
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
@@ -30,47 +30,49 @@ __device__ __forceinline__ void fr_crypt_body(const FrParams& P, const char* sm,
         const uint32_t nseg = fr_chunk_segs(P, kk);
         if (s >= nseg) continue;                       // only the short last chunk has fewer segments
 
-        uint4 z = fr_process_segment_lane<ENCRYPT, ABS>(P, sm, L, lane, kk, s);
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            z.x ^= __shfl_xor_sync(0xFFFFFFFFu, z.x, off);
-            z.y ^= __shfl_xor_sync(0xFFFFFFFFu, z.y, off);
-            z.z ^= __shfl_xor_sync(0xFFFFFFFFu, z.z, off);
-            z.w ^= __shfl_xor_sync(0xFFFFFFFFu, z.w, off);
-        }
-        bool finisher = true;
-        if (nseg > 1) {
-            uint32_t ticket = 0;
-            if (lane == 0) {
-                atomicXor(&P.acc[4 * kk + 0], z.x);
-                atomicXor(&P.acc[4 * kk + 1], z.y);
-                atomicXor(&P.acc[4 * kk + 2], z.z);
-                atomicXor(&P.acc[4 * kk + 3], z.w);
-                __threadfence();
-                ticket = atomicAdd(&P.cnt[kk], 1u);
+        uint4 z = fr_process_segment_lane<MODE, ABS>(P, sm, L, lane, kk, s);
+        if (MODE != FR_MODE_CTR && MODE != FR_MODE_PADGEN) {                // the other passes authenticate
+    #pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                z.x ^= __shfl_xor_sync(0xFFFFFFFFu, z.x, off);
+                z.y ^= __shfl_xor_sync(0xFFFFFFFFu, z.y, off);
+                z.z ^= __shfl_xor_sync(0xFFFFFFFFu, z.z, off);
+                z.w ^= __shfl_xor_sync(0xFFFFFFFFu, z.w, off);
             }
-            ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
-            finisher = (ticket == nseg - 1);
-            if (finisher) {
-                __threadfence();
-                if (lane == 0) {                       // read the sum and leave the scratch zeroed
-                    z.x = atomicExch(&P.acc[4 * kk + 0], 0u);
-                    z.y = atomicExch(&P.acc[4 * kk + 1], 0u);
-                    z.z = atomicExch(&P.acc[4 * kk + 2], 0u);
-                    z.w = atomicExch(&P.acc[4 * kk + 3], 0u);
-                    atomicExch(&P.cnt[kk], 0u);
+            bool finisher = true;
+            if (nseg > 1) {
+                uint32_t ticket = 0;
+                if (lane == 0) {
+                    atomicXor(&P.acc[4 * kk + 0], z.x);
+                    atomicXor(&P.acc[4 * kk + 1], z.y);
+                    atomicXor(&P.acc[4 * kk + 2], z.z);
+                    atomicXor(&P.acc[4 * kk + 3], z.w);
+                    __threadfence();
+                    ticket = atomicAdd(&P.cnt[kk], 1u);
+                }
+                ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
+                finisher = (ticket == nseg - 1);
+                if (finisher) {
+                    __threadfence();
+                    if (lane == 0) {                       // read the sum and leave the scratch zeroed
+                        z.x = atomicExch(&P.acc[4 * kk + 0], 0u);
+                        z.y = atomicExch(&P.acc[4 * kk + 1], 0u);
+                        z.z = atomicExch(&P.acc[4 * kk + 2], 0u);
+                        z.w = atomicExch(&P.acc[4 * kk + 3], 0u);
+                        atomicExch(&P.cnt[kk], 0u);
+                    }
                 }
             }
-        }
-        if (finisher && lane == 0) {
-            const uint4 lenh = (kk + 1u == P.n_chunks) ? P.lenh_last : P.lenh_full;
-            const uint4 tag = fr_xor4(z, lenh);           // z already holds GHASH of the data xor E_K(J0)
-            if (ENCRYPT) {
-                P.tags_out[kk] = tag;
-            } else {
-                const uint4 t = P.tags_in[kk];
-                const uint32_t diff = (tag.x ^ t.x) | (tag.y ^ t.y) | (tag.z ^ t.z) | (tag.w ^ t.w);
-                P.ok[kk] = diff == 0u ? 1u : 0u;
+            if (finisher && lane == 0) {
+                const uint4 lenh = (kk + 1u == P.n_chunks) ? P.lenh_last : P.lenh_full;
+                const uint4 tag = fr_xor4(z, lenh);           // z already holds GHASH of the data xor E_K(J0)
+                if (MODE == FR_MODE_ENC) {
+                    P.tags_out[kk] = tag;
+                } else {
+                    const uint4 t = P.tags_in[kk];
+                    const uint32_t diff = (tag.x ^ t.x) | (tag.y ^ t.y) | (tag.z ^ t.z) | (tag.w ^ t.w);
+                    P.ok[kk] = diff == 0u ? 1u : 0u;
+                }
             }
         }
     }
@@ -79,7 +81,7 @@ __device__ __forceinline__ void fr_crypt_body(const FrParams& P, const char* sm,
 // Fused pass: keystream, XOR, per-segment GHASH partial, per-chunk tag.  Segments are dealt to warps
 // round-robin; a warp XORs its segment's partial into the chunk's accumulator and takes a ticket; the
 // warp that takes the chunk's last ticket finishes the tag (no warp ever waits for another).
-template <bool ENCRYPT>
+template <int MODE>
 __global__ void __launch_bounds__(FR_THREADS, 1) fr_crypt_kernel(const __grid_constant__ FrParams P)
 {
     extern __shared__ __align__(256) char sm[];
@@ -93,8 +95,8 @@ __global__ void __launch_bounds__(FR_THREADS, 1) fr_crypt_kernel(const __grid_co
     L.lane4 |= after_barrier;
     L.qe |= after_barrier;
     L.qo |= after_barrier;
-    if ((uint32_t)__cvta_generic_to_shared(sm) == FR_SMEM_ABS_BASE) fr_crypt_body<ENCRYPT, true>(P, sm, L);
-    else fr_crypt_body<ENCRYPT, false>(P, sm, L);
+    if ((uint32_t)__cvta_generic_to_shared(sm) == FR_SMEM_ABS_BASE) fr_crypt_body<MODE, true>(P, sm, L);
+    else fr_crypt_body<MODE, false>(P, sm, L);
 }
 
 // pow[i] = pow[i - half] * pow[half] for i in (half, min(2*half, n - 1)]: one doubling pass of the table
@@ -118,12 +120,12 @@ struct fastrack_ctx {
     uint4* d_gh_tab;
     uint4* d_pow;
     size_t pow_entries;
-    uint32_t* d_scratch;       // acc[4*cap] then cnt[cap]
+    uint32_t* d_scratch;       // two banks, each acc[4*cap] then cnt[cap]; bank 1 serves fastrack_verify
     size_t scratch_chunks;
-    uint4* d_tags_stage;       // pipelined_h2d: device copy of the tags
+    uint4* d_tags_stage;       // pipelined calls: device copy of the tags, then (second half) the E_K(J0) masks
     size_t tags_stage_chunks;
     cudaStream_t streams[8];
-    cudaEvent_t tags_ready;
+    cudaEvent_t tags_ready, pad_ready;
     int last_cuda_error;
     uint64_t launches;
     uint32_t seg_rows_override;   // 0 = automatic (FASTRACK_SEG_ROWS, for experiments)
@@ -147,9 +149,9 @@ static int ensure_scratch(fastrack_ctx* ctx, size_t chunks)
     while (cap < chunks) cap *= 2;
     FR_CUDA(ctx, cudaDeviceSynchronize());       // nothing may still be using the old scratch
     uint32_t* fresh = nullptr;
-    cudaError_t e = cudaMalloc(&fresh, cap * 5 * sizeof(uint32_t));
+    cudaError_t e = cudaMalloc(&fresh, cap * 10 * sizeof(uint32_t));
     if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); return FASTRACK_ERR_NOMEM; }
-    FR_CUDA(ctx, cudaMemset(fresh, 0, cap * 5 * sizeof(uint32_t)));
+    FR_CUDA(ctx, cudaMemset(fresh, 0, cap * 10 * sizeof(uint32_t)));
     if (ctx->d_scratch) cudaFree(ctx->d_scratch);
     ctx->d_scratch = fresh;
     ctx->scratch_chunks = cap;
@@ -222,11 +224,16 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
             fr_pow_double_kernel<<<(unsigned)((todo + 255) / 256), 256>>>(ctx->d_pow, (uint32_t)half, (uint32_t)ctx->pow_entries);
         }
         if ((e = cudaGetLastError()) != cudaSuccess) break;
-        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
-        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_DEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_ENC>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_CTR>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_VERIFY>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_PADGEN>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_PADDEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
         for (int i = 0; i < 8 && e == cudaSuccess; i++) e = cudaStreamCreateWithFlags(&ctx->streams[i], cudaStreamNonBlocking);
         if (e != cudaSuccess) break;
         if ((e = cudaEventCreateWithFlags(&ctx->tags_ready, cudaEventDisableTiming)) != cudaSuccess) break;
+        if ((e = cudaEventCreateWithFlags(&ctx->pad_ready, cudaEventDisableTiming)) != cudaSuccess) break;
         e = cudaDeviceSynchronize();
     } while (0);
     memset(tab, 0, 65536);
@@ -257,6 +264,7 @@ extern "C" void fastrack_ctx_destroy(fastrack_ctx* ctx)
     for (int i = 0; i < 8; i++)
         if (ctx->streams[i]) cudaStreamDestroy(ctx->streams[i]);
     if (ctx->tags_ready) cudaEventDestroy(ctx->tags_ready);
+    if (ctx->pad_ready) cudaEventDestroy(ctx->pad_ready);
     (void)cudaGetLastError();
     volatile uint8_t* p = (volatile uint8_t*)ctx;
     for (size_t i = 0; i < sizeof *ctx; i++) p[i] = 0;
@@ -344,10 +352,21 @@ static void plan_segments(const fastrack_ctx* ctx, size_t len, size_t n_chunks, 
     P.lenh_last = length_term(ctx, last_len);
 }
 
-// Launch the fused pass over `len` bytes that start at chunk index `first_chunk` of the caller's buffer.
-static int launch_pass(fastrack_ctx* ctx, bool encrypt, const uint8_t iv_base[12], size_t first_chunk,
-                       const void* d_in, size_t len, void* d_out, const void* d_tags_in, void* d_tags_out,
-                       uint32_t* d_ok, cudaStream_t stream)
+// Buffers of one pass (which ones are used depends on the mode, see FrMode).
+struct PassBuffers {
+    const void* in = nullptr;
+    void* out = nullptr;
+    const void* pad = nullptr;
+    void* mask = nullptr;
+    const void* tags_in = nullptr;
+    void* tags_out = nullptr;
+    uint32_t* ok = nullptr;
+    int bank = 0;              // which half of the per-chunk scratch the pass uses
+};
+
+// Launch one pass over `len` bytes that start at chunk index `first_chunk` of the caller's buffer.
+static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], size_t first_chunk, size_t len,
+                       const PassBuffers& b, cudaStream_t stream)
 {
     FrParams P;
     memset(&P, 0, sizeof P);
@@ -362,21 +381,31 @@ static int launch_pass(fastrack_ctx* ctx, bool encrypt, const uint8_t iv_base[12
 
     plan_segments(ctx, len, n_chunks, P);
 
-    P.in = (const uint8_t*)d_in;
-    P.out = (uint8_t*)d_out;
-    P.tags_in = (const uint4*)d_tags_in;
-    P.tags_out = (uint4*)d_tags_out;
-    P.ok = d_ok;
+    P.in = (const uint8_t*)b.in;
+    P.out = (uint8_t*)b.out;
+    P.pad = (const uint8_t*)b.pad;
+    P.mask = (uint4*)b.mask;
+    P.tags_in = (const uint4*)b.tags_in;
+    P.tags_out = (uint4*)b.tags_out;
+    P.ok = b.ok;
     P.te0 = ctx->d_te0;
     P.gh_tab = ctx->d_gh_tab;
     P.pow = ctx->d_pow;
-    P.acc = ctx->d_scratch + 4 * first_chunk;
-    P.cnt = ctx->d_scratch + 4 * ctx->scratch_chunks + first_chunk;
+    uint32_t* bank = ctx->d_scratch + (size_t)b.bank * 5 * ctx->scratch_chunks;
+    P.acc = bank + 4 * first_chunk;
+    P.cnt = bank + 4 * ctx->scratch_chunks + first_chunk;
 
     unsigned grid = (unsigned)ctx->num_sms;
     if (P.n_items < grid) grid = P.n_items;
-    if (encrypt) fr_crypt_kernel<true><<<grid, FR_THREADS, FR_SMEM_BYTES, stream>>>(P);
-    else         fr_crypt_kernel<false><<<grid, FR_THREADS, FR_SMEM_BYTES, stream>>>(P);
+    switch (mode) {
+        case FR_MODE_DEC:    fr_crypt_kernel<FR_MODE_DEC><<<grid, FR_THREADS, FR_SMEM_BYTES, stream>>>(P); break;
+        case FR_MODE_ENC:    fr_crypt_kernel<FR_MODE_ENC><<<grid, FR_THREADS, FR_SMEM_BYTES, stream>>>(P); break;
+        case FR_MODE_CTR:    fr_crypt_kernel<FR_MODE_CTR><<<grid, FR_THREADS, FR_SMEM_BYTES, stream>>>(P); break;
+        case FR_MODE_VERIFY: fr_crypt_kernel<FR_MODE_VERIFY><<<grid, FR_THREADS, FR_SMEM_BYTES, stream>>>(P); break;
+        case FR_MODE_PADGEN: fr_crypt_kernel<FR_MODE_PADGEN><<<grid, FR_THREADS, FR_SMEM_BYTES, stream>>>(P); break;
+        case FR_MODE_PADDEC: fr_crypt_kernel<FR_MODE_PADDEC><<<grid, FR_THREADS, FR_SMEM_BYTES, stream>>>(P); break;
+        default: return FASTRACK_ERR_ARG;
+    }
     ctx->launches++;
     FR_CUDA(ctx, cudaGetLastError());
     return FASTRACK_OK;
@@ -403,7 +432,9 @@ extern "C" int fastrack_decrypt_verify(fastrack_ctx* ctx, const uint8_t iv_base[
     if (K > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
     int rc = ensure_scratch(ctx, K);
     if (rc != FASTRACK_OK) return rc;
-    return launch_pass(ctx, false, iv_base, 0, d_cipher, len, d_plain, d_tags, nullptr, d_ok, (cudaStream_t)stream);
+    PassBuffers b;
+    b.in = d_cipher; b.out = d_plain; b.tags_in = d_tags; b.ok = d_ok;
+    return launch_pass(ctx, FR_MODE_DEC, iv_base, 0, len, b, (cudaStream_t)stream);
 }
 
 extern "C" int fastrack_encrypt_tag(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_plain, size_t len,
@@ -418,17 +449,23 @@ extern "C" int fastrack_encrypt_tag(fastrack_ctx* ctx, const uint8_t iv_base[12]
     if (K > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
     int rc = ensure_scratch(ctx, K);
     if (rc != FASTRACK_OK) return rc;
-    return launch_pass(ctx, true, iv_base, 0, d_plain, len, d_cipher, nullptr, d_tags, nullptr, (cudaStream_t)stream);
+    PassBuffers b;
+    b.in = d_plain; b.out = d_cipher; b.tags_out = d_tags;
+    return launch_pass(ctx, FR_MODE_ENC, iv_base, 0, len, b, (cudaStream_t)stream);
 }
 
-extern "C" int fastrack_pipelined_h2d(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* h_cipher_pinned, size_t len,
-                                      const void* h_tags, void* d_plain, uint32_t* d_ok, int n_streams)
+// Common body of the two pipelined entry points.  d_pad == nullptr: fused decrypt+verify per stage.
+// d_pad != nullptr: the keystream for the whole buffer is produced first, on a stream of its own, while the
+// first copy is in flight; the stages then only XOR and authenticate.
+static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* h_cipher_pinned, size_t len,
+                          const void* h_tags, void* d_pad, void* d_plain, uint32_t* d_ok, int n_streams)
 {
     if (!ctx || !iv_base) return FASTRACK_ERR_ARG;
     if (n_streams < 1 || n_streams > 8) return FASTRACK_ERR_ARG;
     if (len == 0) return FASTRACK_OK;
     if (!h_cipher_pinned || !h_tags || !d_plain || !d_ok) return FASTRACK_ERR_ARG;
     if (misaligned(d_plain, 16) || misaligned(d_ok, 4)) return FASTRACK_ERR_ARG;
+    if (d_pad && (misaligned(d_pad, 16) || d_pad == d_plain || bad_overlap(d_pad, d_plain, len))) return FASTRACK_ERR_ARG;
     cudaPointerAttributes attr;
     cudaError_t e = cudaPointerGetAttributes(&attr, h_cipher_pinned);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return FASTRACK_ERR_NOT_PINNED; }
@@ -444,17 +481,27 @@ extern "C" int fastrack_pipelined_h2d(fastrack_ctx* ctx, const uint8_t iv_base[1
         cudaFree(ctx->d_tags_stage);
         ctx->d_tags_stage = nullptr;
         ctx->tags_stage_chunks = 0;
-        e = cudaMalloc(&ctx->d_tags_stage, cap * 16);
+        e = cudaMalloc(&ctx->d_tags_stage, cap * 32);       // tags, then the E_K(J0) masks of the keystream-ahead variant
         if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); return FASTRACK_ERR_NOMEM; }
         ctx->tags_stage_chunks = cap;
     }
+    uint4* d_mask = ctx->d_tags_stage + ctx->tags_stage_chunks;
 
     // tags: one small copy on a stream of its own; every working stream waits for it before its first kernel
-    cudaStream_t tag_stream = ctx->streams[7];
+    cudaStream_t tag_stream = ctx->streams[7], pad_stream = ctx->streams[6];
     FR_CUDA(ctx, cudaMemcpyAsync(ctx->d_tags_stage, h_tags, K * 16, cudaMemcpyHostToDevice, tag_stream));
     FR_CUDA(ctx, cudaEventRecord(ctx->tags_ready, tag_stream));
-    for (int i = 0; i < n_streams; i++)
+    if (d_pad) {
+        PassBuffers pb;
+        pb.out = d_pad; pb.mask = d_mask;
+        rc = launch_pass(ctx, FR_MODE_PADGEN, iv_base, 0, len, pb, pad_stream);
+        if (rc != FASTRACK_OK) { cudaStreamSynchronize(tag_stream); return rc; }
+        FR_CUDA(ctx, cudaEventRecord(ctx->pad_ready, pad_stream));
+    }
+    for (int i = 0; i < n_streams; i++) {
         if (ctx->streams[i] != tag_stream) FR_CUDA(ctx, cudaStreamWaitEvent(ctx->streams[i], ctx->tags_ready, 0));
+        if (d_pad && ctx->streams[i] != pad_stream) FR_CUDA(ctx, cudaStreamWaitEvent(ctx->streams[i], ctx->pad_ready, 0));
+    }
 
     // Stage = the unit that is copied and then decrypted in place: whole chunks.  Only two things are not
     // hidden behind a copy: a few microseconds per copy boundary and the kernel of the LAST stage.  So the
@@ -482,7 +529,12 @@ extern "C" int fastrack_pipelined_h2d(fastrack_ctx* ctx, const uint8_t iv_base[1
         rc = FASTRACK_OK;
         e = cudaMemcpyAsync(dst, (const uint8_t*)h_cipher_pinned + off, n, cudaMemcpyHostToDevice, st);
         if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); rc = FASTRACK_ERR_CUDA; }
-        if (rc == FASTRACK_OK) rc = launch_pass(ctx, false, iv_base, k0, dst, n, dst, ctx->d_tags_stage + k0, nullptr, d_ok + k0, st);
+        if (rc == FASTRACK_OK) {
+            PassBuffers b;
+            b.in = dst; b.out = dst; b.tags_in = ctx->d_tags_stage + k0; b.ok = d_ok + k0;
+            if (d_pad) { b.pad = (const uint8_t*)d_pad + off; b.mask = d_mask + k0; }
+            rc = launch_pass(ctx, d_pad ? FR_MODE_PADDEC : FR_MODE_DEC, iv_base, k0, n, b, st);
+        }
         if (rc != FASTRACK_OK) {
             for (int i = 0; i < 8; i++) cudaStreamSynchronize(ctx->streams[i]);
             (void)cudaGetLastError();
@@ -492,8 +544,84 @@ extern "C" int fastrack_pipelined_h2d(fastrack_ctx* ctx, const uint8_t iv_base[1
         stage++;
     }
     FR_CUDA(ctx, cudaStreamSynchronize(tag_stream));
+    if (d_pad) FR_CUDA(ctx, cudaStreamSynchronize(pad_stream));
     for (int i = 0; i < n_streams; i++) FR_CUDA(ctx, cudaStreamSynchronize(ctx->streams[i]));
     return FASTRACK_OK;
+}
+
+extern "C" int fastrack_pipelined_h2d(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* h_cipher_pinned, size_t len,
+                                      const void* h_tags, void* d_plain, uint32_t* d_ok, int n_streams)
+{
+    return pipelined_impl(ctx, iv_base, h_cipher_pinned, len, h_tags, nullptr, d_plain, d_ok, n_streams);
+}
+
+extern "C" int fastrack_pipelined_h2d_ahead(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* h_cipher_pinned,
+                                            size_t len, const void* h_tags, void* d_pad, void* d_plain, uint32_t* d_ok,
+                                            int n_streams)
+{
+    if (!d_pad) return FASTRACK_ERR_ARG;
+    return pipelined_impl(ctx, iv_base, h_cipher_pinned, len, h_tags, d_pad, d_plain, d_ok, n_streams);
+}
+
+extern "C" int fastrack_ctr_crypt(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_in, size_t len, void* d_out,
+                                  void* stream)
+{
+    if (!ctx || !iv_base) return FASTRACK_ERR_ARG;
+    if (len == 0) return FASTRACK_OK;
+    if (!d_in || !d_out) return FASTRACK_ERR_ARG;
+    if (misaligned(d_in, 16) || misaligned(d_out, 16) || bad_overlap(d_in, d_out, len)) return FASTRACK_ERR_ARG;
+    if (fastrack_num_chunks(ctx, len) > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
+    PassBuffers b;
+    b.in = d_in; b.out = d_out;
+    return launch_pass(ctx, FR_MODE_CTR, iv_base, 0, len, b, (cudaStream_t)stream);
+}
+
+extern "C" int fastrack_verify(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_cipher, size_t len,
+                               const void* d_tags, uint32_t* d_ok, void* stream)
+{
+    if (!ctx || !iv_base) return FASTRACK_ERR_ARG;
+    if (len == 0) return FASTRACK_OK;
+    if (!d_cipher || !d_tags || !d_ok) return FASTRACK_ERR_ARG;
+    if (misaligned(d_cipher, 16) || misaligned(d_tags, 16) || misaligned(d_ok, 4)) return FASTRACK_ERR_ARG;
+    const size_t K = fastrack_num_chunks(ctx, len);
+    if (K > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
+    int rc = ensure_scratch(ctx, K);
+    if (rc != FASTRACK_OK) return rc;
+    PassBuffers b;
+    b.in = d_cipher; b.out = const_cast<void*>(d_cipher); b.tags_in = d_tags; b.ok = d_ok; b.bank = 1;
+    return launch_pass(ctx, FR_MODE_VERIFY, iv_base, 0, len, b, (cudaStream_t)stream);
+}
+
+extern "C" int fastrack_keystream(fastrack_ctx* ctx, const uint8_t iv_base[12], size_t len, void* d_pad, void* d_mask,
+                                  void* stream)
+{
+    if (!ctx || !iv_base) return FASTRACK_ERR_ARG;
+    if (len == 0) return FASTRACK_OK;
+    if (!d_pad || !d_mask) return FASTRACK_ERR_ARG;
+    if (misaligned(d_pad, 16) || misaligned(d_mask, 16)) return FASTRACK_ERR_ARG;
+    if (fastrack_num_chunks(ctx, len) > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
+    PassBuffers b;
+    b.out = d_pad; b.mask = d_mask;
+    return launch_pass(ctx, FR_MODE_PADGEN, iv_base, 0, len, b, (cudaStream_t)stream);
+}
+
+extern "C" int fastrack_xor_verify(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_cipher, size_t len,
+                                   const void* d_pad, const void* d_mask, const void* d_tags, void* d_plain,
+                                   uint32_t* d_ok, void* stream)
+{
+    if (!ctx || !iv_base) return FASTRACK_ERR_ARG;
+    if (len == 0) return FASTRACK_OK;
+    if (!d_cipher || !d_pad || !d_mask || !d_tags || !d_plain || !d_ok) return FASTRACK_ERR_ARG;
+    if (misaligned(d_cipher, 16) || misaligned(d_plain, 16) || misaligned(d_pad, 16) || misaligned(d_mask, 16) ||
+        misaligned(d_tags, 16) || misaligned(d_ok, 4)) return FASTRACK_ERR_ARG;
+    if (bad_overlap(d_cipher, d_plain, len) || d_pad == d_plain || bad_overlap(d_pad, d_plain, len)) return FASTRACK_ERR_ARG;
+    const size_t K = fastrack_num_chunks(ctx, len);
+    if (K > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
+    int rc = ensure_scratch(ctx, K);
+    if (rc != FASTRACK_OK) return rc;
+    PassBuffers b;
+    b.in = d_cipher; b.out = d_plain; b.pad = d_pad; b.mask = const_cast<void*>(d_mask); b.tags_in = d_tags; b.ok = d_ok;
+    return launch_pass(ctx, FR_MODE_PADDEC, iv_base, 0, len, b, (cudaStream_t)stream);
 }
 
 // ------------------------------------------------------------- entry point that allocates nothing ----
@@ -558,7 +686,7 @@ extern "C" int fastrack_decrypt_verify_noalloc(fastrack_ctx* ctx, const uint8_t 
     P.cnt = cnt;
     unsigned grid = (unsigned)ctx->num_sms;
     if (P.n_items < grid) grid = P.n_items;
-    fr_crypt_kernel<false><<<grid, FR_THREADS, FR_SMEM_BYTES, st>>>(P);
+    fr_crypt_kernel<FR_MODE_DEC><<<grid, FR_THREADS, FR_SMEM_BYTES, st>>>(P);
     ctx->launches++;
     FR_CUDA(ctx, cudaGetLastError());
     return FASTRACK_OK;

@@ -26,6 +26,18 @@
 #define FR_SM_GH 131072u      // byte tables of H^32
 #define FR_SMEM_BYTES 196608u
 
+// What one pass does.  DEC / ENC are the fused passes.  CTR and VERIFY split them (paper Section 4.3, eager
+// evaluation: plaintext first, authentication later).  PADGEN / PADDEC split the keystream from the XOR
+// (Section 4.3, parallel AES evaluation: the one-time pad is produced while the copy is in flight).
+enum FrMode : int {
+    FR_MODE_DEC = 0,      // keystream, P = C xor KS, GHASH over C, compare tags
+    FR_MODE_ENC = 1,      // keystream, C = P xor KS, GHASH over C, store tags
+    FR_MODE_CTR = 2,      // keystream and XOR only
+    FR_MODE_VERIFY = 3,   // GHASH over C and tag compare only (C is not modified)
+    FR_MODE_PADGEN = 4,   // keystream only, written to a pad buffer, plus E_K(J0) per chunk
+    FR_MODE_PADDEC = 5    // P = C xor pad, GHASH over C, compare tags (no AES at all)
+};
+
 #define FR_ROW_BLOCKS 32u     // blocks per row (one per lane)
 #define FR_HORNER_STRIDE 32u  // the fixed multiplier is H^32
 
@@ -50,6 +62,8 @@ struct FrParams {
     const uint4* pow;          // pow[e] = H^e
     uint32_t* acc;             // per chunk 4 words, zero between launches
     uint32_t* cnt;             // per chunk arrival counter, zero between launches
+    const uint8_t* pad;        // FR_MODE_PADDEC: keystream made ahead of time, same layout as the data
+    uint4* mask;               // E_K(J0) per chunk: written by FR_MODE_PADGEN, read by FR_MODE_PADDEC
     uint4 lenh_full;           // (BE64(0) || BE64(8 * chunk_bytes)) * H: the length block's term of a full chunk
     uint4 lenh_last;           // the same for the launch's last chunk (differs when that chunk is short)
 };
@@ -381,10 +395,16 @@ __device__ __forceinline__ uint4 fr_mask_bytes(uint4 v, uint32_t n)
 // lane's Horner value, and return that value multiplied by the power of H that aligns it to the end
 // of the chunk (lane 1 of the chunk's first segment adds E_K(J0)).  XOR of the 32 lanes' results over all
 // segments of the chunk = GHASH of the data blocks (before the length block) xor E_K(J0).
-template <bool ENCRYPT, bool ABS>
+// Modes without GHASH (CTR, PADGEN) return zero.
+template <int MODE, bool ABS>
 __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, const char* sm, const FrLane& L,
                                                          uint32_t lane, uint32_t kk, uint32_t s)
 {
+    constexpr bool DO_AES = MODE == FR_MODE_DEC || MODE == FR_MODE_ENC || MODE == FR_MODE_CTR || MODE == FR_MODE_PADGEN;
+    constexpr bool DO_GHASH = MODE == FR_MODE_DEC || MODE == FR_MODE_ENC || MODE == FR_MODE_VERIFY || MODE == FR_MODE_PADDEC;
+    constexpr bool DO_LOAD = MODE != FR_MODE_PADGEN;
+    constexpr bool DO_STORE = MODE != FR_MODE_VERIFY;
+
     const uint64_t chunk_off = (uint64_t)kk * P.chunk_bytes;
     const uint64_t len_k = fr_chunk_len(P, kk);
     const uint32_t nblk = (uint32_t)((len_k + 15) >> 4);
@@ -396,11 +416,12 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
     if (seg_end > nblk) seg_end = nblk;
     const uint8_t* in = P.in + chunk_off;
     uint8_t* out = P.out + chunk_off;
+    const uint8_t* pad = P.pad + chunk_off;
     // The lane's last block and its power of H follow from the geometry alone: fetch the power now, under the rows.
     // Block j is multiplied by H^(nblk - j + 1): one for each later block, one for the length block.
     uint32_t j_last = 0xFFFFFFFFu;
     uint4 hpow = make_uint4(0, 0, 0, 0);
-    {
+    if (DO_GHASH) {
         const uint32_t seg_begin = (row0 == 0) ? 0u : row0 * FR_ROW_BLOCKS - 2u;     // first block of this segment
         if (seg_end > seg_begin) {
             // largest j < seg_end with (j + 2) mod 32 == lane
@@ -413,30 +434,44 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
             }
         }
     }
-    const FrCtrChunk cc = fr_ctr_chunk<ABS>(sm, L.lane4, P, fr_bswap(P.iv_ctr + kk));
+    FrCtrChunk cc = {0, 0, 0, 0};
+    if (DO_AES || row0 == 0) cc = fr_ctr_chunk<ABS>(sm, L.lane4, P, fr_bswap(P.iv_ctr + kk));   // VERIFY needs E_K(J0) only
     FrCtrGroup cg = {0, 0, 0, 0};
 
     uint4 y = make_uint4(0, 0, 0, 0), pend = make_uint4(0, 0, 0, 0), extra = make_uint4(0, 0, 0, 0);
     for (uint32_t r = row0; r < row1; r++) {
         const uint32_t ctr = r * FR_ROW_BLOCKS + lane;
-        if (r == row0 || (r & 7u) == 0u) cg = fr_ctr_group<ABS>(sm, L.lane4, P, cc, ctr);   // ctr >> 8 is the same for the whole row
+        if (DO_AES || r == 0) {
+            if (r == row0 || (r & 7u) == 0u) cg = fr_ctr_group<ABS>(sm, L.lane4, P, cc, ctr);   // ctr >> 8 is the same for the whole row
+        }
         const uint32_t j = ctr - 2u;                                                  // wraps for ctr < 2: then j >= seg_end
         if (j < seg_end) {
             const uint64_t boff = (uint64_t)j << 4;
             const bool full = len_k - boff >= 16;
             const uint32_t nvalid = full ? 16u : (uint32_t)(len_k - boff);
-            uint4 x = full ? *(const uint4*)(in + boff) : fr_load_partial(in + boff, nvalid);
-            uint4 ks = fr_aes256_ctr_block<ABS>(sm, L.lane4, P, cc, cg, ctr);
-            uint4 o = fr_xor4(x, ks);
-            if (full) *(uint4*)(out + boff) = o; else fr_store_partial(out + boff, o, nvalid);
-            uint4 g = ENCRYPT ? (full ? o : fr_mask_bytes(o, nvalid)) : x;
-            uint4 v = fr_xor4(y, g);
-            if (j != j_last) y = fr_ghash_tabmul<ABS>(sm, L, v);
-            else pend = v;
-        } else if (ctr == 1u) {
-            extra = fr_aes256_ctr_block<ABS>(sm, L.lane4, P, cc, cg, 1u);                   // E_K(J0)
+            uint4 x = make_uint4(0, 0, 0, 0);
+            if (DO_LOAD) x = full ? *(const uint4*)(in + boff) : fr_load_partial(in + boff, nvalid);
+            uint4 ks = make_uint4(0, 0, 0, 0);
+            if (DO_AES) ks = fr_aes256_ctr_block<ABS>(sm, L.lane4, P, cc, cg, ctr);
+            else if (MODE == FR_MODE_PADDEC) ks = full ? *(const uint4*)(pad + boff) : fr_load_partial(pad + boff, nvalid);
+            const uint4 o = fr_xor4(x, ks);
+            if (DO_STORE) { if (full) *(uint4*)(out + boff) = o; else fr_store_partial(out + boff, o, nvalid); }
+            if (DO_GHASH) {
+                const uint4 g = (MODE == FR_MODE_ENC) ? (full ? o : fr_mask_bytes(o, nvalid)) : x;
+                const uint4 v = fr_xor4(y, g);
+                if (j != j_last) y = fr_ghash_tabmul<ABS>(sm, L, v);
+                else pend = v;
+            }
+        } else if (ctr == 1u && MODE != FR_MODE_CTR) {
+            if (MODE == FR_MODE_PADDEC) {
+                extra = P.mask[kk];
+            } else {
+                extra = fr_aes256_ctr_block<ABS>(sm, L.lane4, P, cc, cg, 1u);         // E_K(J0)
+                if (MODE == FR_MODE_PADGEN) P.mask[kk] = extra;
+            }
         }
     }
+    if (!DO_GHASH) return make_uint4(0, 0, 0, 0);
     if (j_last == 0xFFFFFFFFu) return extra;
     return fr_xor4(fr_gf128_mul(pend, hpow), extra);
 }

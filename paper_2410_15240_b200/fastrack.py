@@ -20,7 +20,9 @@ MAX_CHUNK_BYTES = 1 << 30
 
 EXPORTS = ("fastrack_ctx_create", "fastrack_ctx_destroy", "fastrack_num_chunks", "fastrack_ctx_reserve",
            "fastrack_last_cuda_error", "fastrack_decrypt_verify", "fastrack_encrypt_tag",
-           "fastrack_pipelined_h2d", "fastrack_launch_count", "fastrack_decrypt_verify_noalloc")
+           "fastrack_pipelined_h2d", "fastrack_launch_count", "fastrack_decrypt_verify_noalloc",
+           "fastrack_ctr_crypt", "fastrack_verify", "fastrack_keystream", "fastrack_xor_verify",
+           "fastrack_pipelined_h2d_ahead")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2410_15240_b200.build` "
@@ -46,6 +48,16 @@ _lib.fastrack_decrypt_verify_noalloc.restype = _int
 _lib.fastrack_decrypt_verify_noalloc.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp, _vp]
 _lib.fastrack_encrypt_tag.restype = _int
 _lib.fastrack_encrypt_tag.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp]
+_lib.fastrack_ctr_crypt.restype = _int
+_lib.fastrack_ctr_crypt.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp]
+_lib.fastrack_verify.restype = _int
+_lib.fastrack_verify.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp]
+_lib.fastrack_keystream.restype = _int
+_lib.fastrack_keystream.argtypes = [_vp, ctypes.c_char_p, _sz, _vp, _vp, _vp]
+_lib.fastrack_xor_verify.restype = _int
+_lib.fastrack_xor_verify.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.fastrack_pipelined_h2d_ahead.restype = _int
+_lib.fastrack_pipelined_h2d_ahead.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp, _vp, _int]
 _lib.fastrack_pipelined_h2d.restype = _int
 _lib.fastrack_pipelined_h2d.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp, _int]
 
@@ -106,6 +118,29 @@ def fastrack_pipelined_h2d(ctx, iv_base: bytes, h_cipher_pinned: int, length: in
     return _lib.fastrack_pipelined_h2d(ctx, iv_base, h_cipher_pinned, length, h_tags, d_plain, d_ok, n_streams)
 
 
+def fastrack_ctr_crypt(ctx, iv_base: bytes, d_in: int, length: int, d_out: int, stream: int = 0) -> int:
+    return _lib.fastrack_ctr_crypt(ctx, iv_base, d_in, length, d_out, stream)
+
+
+def fastrack_verify(ctx, iv_base: bytes, d_cipher: int, length: int, d_tags: int, d_ok: int, stream: int = 0) -> int:
+    return _lib.fastrack_verify(ctx, iv_base, d_cipher, length, d_tags, d_ok, stream)
+
+
+def fastrack_keystream(ctx, iv_base: bytes, length: int, d_pad: int, d_mask: int, stream: int = 0) -> int:
+    return _lib.fastrack_keystream(ctx, iv_base, length, d_pad, d_mask, stream)
+
+
+def fastrack_xor_verify(ctx, iv_base: bytes, d_cipher: int, length: int, d_pad: int, d_mask: int, d_tags: int,
+                        d_plain: int, d_ok: int, stream: int = 0) -> int:
+    return _lib.fastrack_xor_verify(ctx, iv_base, d_cipher, length, d_pad, d_mask, d_tags, d_plain, d_ok, stream)
+
+
+def fastrack_pipelined_h2d_ahead(ctx, iv_base: bytes, h_cipher_pinned: int, length: int, h_tags: int, d_pad: int,
+                                 d_plain: int, d_ok: int, n_streams: int) -> int:
+    return _lib.fastrack_pipelined_h2d_ahead(ctx, iv_base, h_cipher_pinned, length, h_tags, d_pad, d_plain, d_ok,
+                                             n_streams)
+
+
 class Context:
     """RAII wrapper: ``with Context(key, chunk_bytes) as ctx: ctx.decrypt_verify(...)``; raises FastrackError."""
 
@@ -139,6 +174,23 @@ class Context:
     def pipelined_h2d(self, iv_base, h_cipher_pinned, length, h_tags, d_plain, d_ok, n_streams=4) -> None:
         self._check(fastrack_pipelined_h2d(self.handle, iv_base, h_cipher_pinned, length, h_tags, d_plain, d_ok,
                                            n_streams))
+
+    def ctr_crypt(self, iv_base, d_in, length, d_out, stream=0) -> None:
+        self._check(fastrack_ctr_crypt(self.handle, iv_base, d_in, length, d_out, stream))
+
+    def verify(self, iv_base, d_cipher, length, d_tags, d_ok, stream=0) -> None:
+        self._check(fastrack_verify(self.handle, iv_base, d_cipher, length, d_tags, d_ok, stream))
+
+    def keystream(self, iv_base, length, d_pad, d_mask, stream=0) -> None:
+        self._check(fastrack_keystream(self.handle, iv_base, length, d_pad, d_mask, stream))
+
+    def xor_verify(self, iv_base, d_cipher, length, d_pad, d_mask, d_tags, d_plain, d_ok, stream=0) -> None:
+        self._check(fastrack_xor_verify(self.handle, iv_base, d_cipher, length, d_pad, d_mask, d_tags, d_plain, d_ok,
+                                        stream))
+
+    def pipelined_h2d_ahead(self, iv_base, h_cipher_pinned, length, h_tags, d_pad, d_plain, d_ok, n_streams=4) -> None:
+        self._check(fastrack_pipelined_h2d_ahead(self.handle, iv_base, h_cipher_pinned, length, h_tags, d_pad, d_plain,
+                                                 d_ok, n_streams))
 
     @property
     def launches(self) -> int:

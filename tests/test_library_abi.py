@@ -16,7 +16,7 @@ def declared_functions():
 
 def test_header_and_binding_agree():
     names = declared_functions()
-    assert len(names) >= 9
+    assert len(names) >= 15
     assert sorted(fastrack.EXPORTS) == names
 
 
@@ -51,6 +51,11 @@ def test_argument_checks_that_need_no_device():
     assert fastrack.fastrack_decrypt_verify(None, bytes(12), 0, 16, 0, 0, 0, 0) == fastrack.ERR_ARG
     assert fastrack.fastrack_encrypt_tag(None, bytes(12), 0, 16, 0, 0, 0) == fastrack.ERR_ARG
     assert fastrack.fastrack_decrypt_verify_noalloc(None, bytes(12), 0, 16, 0, 0, 0, 0) == fastrack.ERR_ARG
+    assert fastrack.fastrack_ctr_crypt(None, bytes(12), 0, 16, 0, 0) == fastrack.ERR_ARG
+    assert fastrack.fastrack_verify(None, bytes(12), 0, 16, 0, 0, 0) == fastrack.ERR_ARG
+    assert fastrack.fastrack_keystream(None, bytes(12), 16, 0, 0, 0) == fastrack.ERR_ARG
+    assert fastrack.fastrack_xor_verify(None, bytes(12), 0, 16, 0, 0, 0, 0, 0, 0) == fastrack.ERR_ARG
+    assert fastrack.fastrack_pipelined_h2d_ahead(None, bytes(12), 0, 16, 0, 0, 0, 0, 2) == fastrack.ERR_ARG
     assert fastrack.fastrack_pipelined_h2d(None, bytes(12), 0, 16, 0, 0, 0, 2) == fastrack.ERR_ARG
     fastrack.fastrack_ctx_destroy(None)          # allowed
 
