@@ -498,10 +498,7 @@ static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const vo
         if (rc != FASTRACK_OK) { cudaStreamSynchronize(tag_stream); return rc; }
         FR_CUDA(ctx, cudaEventRecord(ctx->pad_ready, pad_stream));
     }
-    for (int i = 0; i < n_streams; i++) {
-        if (ctx->streams[i] != tag_stream) FR_CUDA(ctx, cudaStreamWaitEvent(ctx->streams[i], ctx->tags_ready, 0));
-        if (d_pad && ctx->streams[i] != pad_stream) FR_CUDA(ctx, cudaStreamWaitEvent(ctx->streams[i], ctx->pad_ready, 0));
-    }
+    bool waited[8] = {false, false, false, false, false, false, false, false};   // per working stream: events already awaited
 
     // Stage = the unit that is copied and then decrypted in place: whole chunks.  Only two things are not
     // hidden behind a copy: a few microseconds per copy boundary and the kernel of the LAST stage.  So the
@@ -529,6 +526,14 @@ static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const vo
         rc = FASTRACK_OK;
         e = cudaMemcpyAsync(dst, (const uint8_t*)h_cipher_pinned + off, n, cudaMemcpyHostToDevice, st);
         if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); rc = FASTRACK_ERR_CUDA; }
+        const size_t si = stage % (size_t)n_streams;
+        if (rc == FASTRACK_OK && !waited[si]) {
+            // the stream's first kernel (not its first copy) waits for the tags and, if used, the keystream
+            waited[si] = true;
+            if (st != tag_stream) e = cudaStreamWaitEvent(st, ctx->tags_ready, 0);
+            if (e == cudaSuccess && d_pad && st != pad_stream) e = cudaStreamWaitEvent(st, ctx->pad_ready, 0);
+            if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); rc = FASTRACK_ERR_CUDA; }
+        }
         if (rc == FASTRACK_OK) {
             PassBuffers b;
             b.in = dst; b.out = dst; b.tags_in = ctx->d_tags_stage + k0; b.ok = d_ok + k0;
