@@ -89,6 +89,15 @@ FASTRACK_API size_t fastrack_num_chunks(const fastrack_ctx* ctx, size_t len);
  * grows the scratch (cudaMalloc + a device synchronisation) before launching. */
 FASTRACK_API int fastrack_ctx_reserve(fastrack_ctx* ctx, size_t max_len);
 
+/* Paper-faithful framing (Section 4.2: every chunk is "attached to one byte of additional authentication data
+ * to indicate the chunk order"; Section 4.4: the serial number in the AAD defeats reordering).
+ * chains_per_sample = n in 1..256: the buffer is a sequence of samples of n chunks each, and chunk k
+ * authenticates the single byte (k mod n) as AAD (so the length block carries an AAD length of 8 bits).
+ * chains_per_sample = 0 (the default at creation): AAD empty, chunk order bound by the IV index only.
+ * The IV rule is unchanged in both cases.  Applies to every later call on the context, of every kind; both
+ * ends must use the same setting (a mismatch rejects every chunk).  Takes effect for calls issued afterwards. */
+FASTRACK_API int fastrack_ctx_set_framing(fastrack_ctx* ctx, unsigned chains_per_sample);
+
 /* CUDA error code (cudaError_t as int) of the last failing CUDA call made through ctx, else 0. */
 FASTRACK_API int fastrack_last_cuda_error(const fastrack_ctx* ctx);
 

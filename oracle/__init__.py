@@ -52,6 +52,8 @@ def _load():
         "fo_num_chunks": (sz, [sz, sz]),
         "fo_mc_encrypt": (None, [u8p, u8p, sz, u8p, sz, u8p, u8p, i32]),
         "fo_mc_decrypt": (None, [u8p, u8p, sz, u8p, sz, u8p, u8p, u8p, i32]),
+        "fo_mc_encrypt_framed": (None, [u8p, u8p, sz, ctypes.c_uint, u8p, sz, u8p, u8p, i32]),
+        "fo_mc_decrypt_framed": (None, [u8p, u8p, sz, ctypes.c_uint, u8p, sz, u8p, u8p, u8p, i32]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -184,4 +186,26 @@ def mc_decrypt(key, iv_base, chunk_bytes: int, c, tags, n_threads: int = 1):
     ok = np.zeros(K, np.uint32)
     _load().fo_mc_decrypt(_ptr(k), _ptr(v), int(chunk_bytes), _ptr(cc), cc.size, _ptr(t), _ptr(p),
                           _ptr(ok), int(n_threads))
+    return p, ok
+
+
+def mc_encrypt_framed(key, iv_base, chunk_bytes: int, chains_per_sample: int, p, n_threads: int = 1):
+    """Multi-chain encrypt with the paper's one-byte serial-number AAD per chunk (k mod chains_per_sample)."""
+    k, v, pp = _arr(key, 32), _arr(iv_base, 12), _arr(p)
+    K = num_chunks(pp.size, chunk_bytes)
+    c = np.zeros(pp.size, np.uint8)
+    tags = np.zeros((K, 16), np.uint8)
+    _load().fo_mc_encrypt_framed(_ptr(k), _ptr(v), int(chunk_bytes), int(chains_per_sample), _ptr(pp), pp.size,
+                                 _ptr(c), _ptr(tags), int(n_threads))
+    return c, tags
+
+
+def mc_decrypt_framed(key, iv_base, chunk_bytes: int, chains_per_sample: int, c, tags, n_threads: int = 1):
+    k, v, cc = _arr(key, 32), _arr(iv_base, 12), _arr(c)
+    K = num_chunks(cc.size, chunk_bytes)
+    t = _arr(tags, 16 * K)
+    p = np.zeros(cc.size, np.uint8)
+    ok = np.zeros(K, np.uint32)
+    _load().fo_mc_decrypt_framed(_ptr(k), _ptr(v), int(chunk_bytes), int(chains_per_sample), _ptr(cc), cc.size,
+                                 _ptr(t), _ptr(p), _ptr(ok), int(n_threads))
     return p, ok

@@ -313,6 +313,7 @@ typedef struct {
     const uint8_t* tags_in;     /* decrypt */
     uint32_t* ok;               /* decrypt */
     int encrypt;
+    unsigned chains_per_sample; /* 0: no AAD; n > 0: chunk k carries the one-byte AAD (k mod n) */
 } mc_job;
 
 static void* mc_worker(void* arg)
@@ -323,10 +324,14 @@ static void* mc_worker(void* arg)
         size_t n = j->len - off < j->chunk_bytes ? j->len - off : j->chunk_bytes;
         uint8_t iv[12];
         fo_chunk_iv(j->iv_base, k, iv);
+        /* paper Section 4.2 / 4.4: one byte of AAD per chunk holds its serial number inside the sample */
+        uint8_t serial = j->chains_per_sample ? (uint8_t)(k % j->chains_per_sample) : 0;
+        const uint8_t* aad = j->chains_per_sample ? &serial : NULL;
+        size_t aad_len = j->chains_per_sample ? 1 : 0;
         if (j->encrypt)
-            fo_gcm_encrypt(j->key, iv, NULL, 0, j->in + off, n, j->out + off, j->tags_out + 16 * k);
+            fo_gcm_encrypt(j->key, iv, aad, aad_len, j->in + off, n, j->out + off, j->tags_out + 16 * k);
         else
-            j->ok[k] = (uint32_t)fo_gcm_decrypt(j->key, iv, NULL, 0, j->in + off, n,
+            j->ok[k] = (uint32_t)fo_gcm_decrypt(j->key, iv, aad, aad_len, j->in + off, n,
                                                 j->tags_in + 16 * k, j->out + off);
     }
     return NULL;
@@ -376,5 +381,28 @@ FO_API void fo_mc_decrypt(const uint8_t key[32], const uint8_t iv_base[12], size
     mc_job j; memset(&j, 0, sizeof j);
     j.key = key; j.iv_base = iv_base; j.chunk_bytes = chunk_bytes; j.len = len;
     j.in = c; j.out = p; j.tags_in = tags; j.ok = ok; j.encrypt = 0;
+    mc_run(j, n_threads);
+}
+
+/* Paper-faithful framing (Sections 4.2 and 4.4): every sample is cut into chains_per_sample chunks and each
+ * chunk authenticates, as its one byte of AAD, its serial number inside the sample (k mod chains_per_sample).
+ * Everything else is as in fo_mc_encrypt / fo_mc_decrypt; chains_per_sample in 1..256. */
+FO_API void fo_mc_encrypt_framed(const uint8_t key[32], const uint8_t iv_base[12], size_t chunk_bytes,
+                                 unsigned chains_per_sample, const uint8_t* p, size_t len, uint8_t* c,
+                                 uint8_t* tags, int n_threads)
+{
+    mc_job j; memset(&j, 0, sizeof j);
+    j.key = key; j.iv_base = iv_base; j.chunk_bytes = chunk_bytes; j.len = len;
+    j.in = p; j.out = c; j.tags_out = tags; j.encrypt = 1; j.chains_per_sample = chains_per_sample;
+    mc_run(j, n_threads);
+}
+
+FO_API void fo_mc_decrypt_framed(const uint8_t key[32], const uint8_t iv_base[12], size_t chunk_bytes,
+                                 unsigned chains_per_sample, const uint8_t* c, size_t len, const uint8_t* tags,
+                                 uint8_t* p, uint32_t* ok, int n_threads)
+{
+    mc_job j; memset(&j, 0, sizeof j);
+    j.key = key; j.iv_base = iv_base; j.chunk_bytes = chunk_bytes; j.len = len;
+    j.in = c; j.out = p; j.tags_in = tags; j.ok = ok; j.encrypt = 0; j.chains_per_sample = chains_per_sample;
     mc_run(j, n_threads);
 }

@@ -128,6 +128,7 @@ struct fastrack_ctx {
     cudaEvent_t tags_ready, pad_ready;
     int last_cuda_error;
     uint64_t launches;
+    uint32_t aad_mod;             // 0 = no AAD, else chains per sample of the serial-number framing
     uint32_t seg_rows_override;   // 0 = automatic (FASTRACK_SEG_ROWS, for experiments)
     size_t stage_bytes_override;  // 0 = automatic (FASTRACK_STAGE_BYTES, for experiments)
 };
@@ -283,6 +284,13 @@ extern "C" int fastrack_ctx_reserve(fastrack_ctx* ctx, size_t max_len)
     return ensure_scratch(ctx, fastrack_num_chunks(ctx, max_len));
 }
 
+extern "C" int fastrack_ctx_set_framing(fastrack_ctx* ctx, unsigned chains_per_sample)
+{
+    if (!ctx || chains_per_sample > 256) return FASTRACK_ERR_ARG;
+    ctx->aad_mod = chains_per_sample;
+    return FASTRACK_OK;
+}
+
 extern "C" int fastrack_last_cuda_error(const fastrack_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
 
 extern "C" uint64_t fastrack_launch_count(const fastrack_ctx* ctx) { return ctx ? ctx->launches : 0; }
@@ -293,11 +301,12 @@ static uint32_t load_be32(const uint8_t* p) { return ((uint32_t)p[0] << 24) | ((
 static uint32_t load_le32(const uint8_t* p) { return ((uint32_t)p[3] << 24) | ((uint32_t)p[2] << 16) | ((uint32_t)p[1] << 8) | p[0]; }
 
 
-// (BE64(0) || BE64(8 * bytes)) * H: the length block's term of a chunk of `bytes` bytes.
+// (BE64(8 * aad bytes) || BE64(8 * bytes)) * H: the length block's term of a chunk of `bytes` bytes.
 static uint4 length_term(const fastrack_ctx* ctx, uint64_t bytes)
 {
     uint8_t blk[16] = {0}, out[16];
     const uint64_t bits = bytes * 8;
+    if (ctx->aad_mod) blk[7] = 8;                    // BE64(bit length of the AAD): one byte
     for (int i = 0; i < 8; i++) blk[8 + i] = (uint8_t)(bits >> (56 - 8 * i));
     gf_store(gf_mul(gf_load(blk), gf_load(ctx->h)), out);
     uint4 r;
@@ -374,6 +383,8 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
     P.iv_w0 = load_le32(iv_base);
     P.iv_w1 = load_le32(iv_base + 4);
     P.iv_ctr = load_be32(iv_base + 8) + (uint32_t)first_chunk;
+    P.first_chunk = (uint32_t)first_chunk;
+    P.aad_mod = ctx->aad_mod;
     P.len = len;
     P.chunk_bytes = ctx->chunk_bytes;
     const size_t n_chunks = (len + ctx->chunk_bytes - 1) / ctx->chunk_bytes;
@@ -676,6 +687,7 @@ extern "C" int fastrack_decrypt_verify_noalloc(fastrack_ctx* ctx, const uint8_t 
     P.iv_w0 = load_le32(iv_base);
     P.iv_w1 = load_le32(iv_base + 4);
     P.iv_ctr = load_be32(iv_base + 8);
+    P.aad_mod = ctx->aad_mod;
     P.len = len;
     P.chunk_bytes = ctx->chunk_bytes;
     P.n_chunks = (uint32_t)K;

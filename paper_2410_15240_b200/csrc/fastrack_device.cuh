@@ -45,11 +45,12 @@ struct FrParams {
     uint32_t rk[60];           // AES-256 round keys, word i = little-endian load of key-schedule bytes 4i..4i+3
     uint32_t iv_w0, iv_w1;     // little-endian loads of iv_base[0..3], iv_base[4..7]
     uint32_t iv_ctr;           // BE32(iv_base[8..11]) + index of this launch's first chunk
+    uint32_t first_chunk;      // index of this launch's first chunk in the caller's buffer
     uint32_t seg_rows;         // rows per segment
     uint32_t segs_per_chunk;   // segments of a full-size chunk
     uint32_t n_chunks;         // chunks in this launch
     uint32_t n_items;          // n_chunks * segs_per_chunk
-    uint32_t pad0;
+    uint32_t aad_mod;          // 0: no AAD; n: chunk k authenticates the one byte (first chunk index + k) mod n as AAD
     uint64_t len;              // bytes in this launch
     uint64_t chunk_bytes;
     const uint8_t* in;
@@ -418,19 +419,21 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
     uint8_t* out = P.out + chunk_off;
     const uint8_t* pad = P.pad + chunk_off;
     // The lane's last block and its power of H follow from the geometry alone: fetch the power now, under the rows.
-    // Block j is multiplied by H^(nblk - j + 1): one for each later block, one for the length block.
-    uint32_t j_last = 0xFFFFFFFFu;
+    // The block at counter c (block index c - 2) is multiplied by H^(nblk + 3 - c): one factor for each later
+    // block and one for the length block.  With the serial-number framing, counter 1 of the chunk carries the
+    // AAD block, which GHASH absorbs before the first ciphertext block: the same rule gives it H^(nblk + 2).
+    uint32_t c_last = 0;                              // counter of this lane's last GHASH block in the segment, 0 = none
     uint4 hpow = make_uint4(0, 0, 0, 0);
     if (DO_GHASH) {
-        const uint32_t seg_begin = (row0 == 0) ? 0u : row0 * FR_ROW_BLOCKS - 2u;     // first block of this segment
-        if (seg_end > seg_begin) {
-            // largest j < seg_end with (j + 2) mod 32 == lane
-            const uint32_t top = seg_end + 1u;                                        // counter of block seg_end - 1
-            uint32_t c_last = (top & ~31u) | lane;
-            if (c_last > top) c_last -= 32u;
-            if (c_last >= 2u && c_last - 2u >= seg_begin && c_last <= top) {
-                j_last = c_last - 2u;
-                hpow = P.pow[(nblk - 1u - j_last) + 2u];
+        const uint32_t c_begin = (row0 == 0) ? (P.aad_mod ? 1u : 2u) : row0 * FR_ROW_BLOCKS;
+        const uint32_t c_end = seg_end + 2u;          // counters of this segment's blocks are below c_end
+        if (c_end > c_begin) {
+            const uint32_t top = c_end - 1u;
+            uint32_t c = (top & ~31u) | lane;         // largest counter <= top that belongs to this lane
+            if (c > top) c -= 32u;                    // may wrap below zero: then c > top still
+            if (c >= c_begin && c <= top) {
+                c_last = c;
+                hpow = P.pow[nblk + 3u - c];
             }
         }
     }
@@ -459,7 +462,7 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
             if (DO_GHASH) {
                 const uint4 g = (MODE == FR_MODE_ENC) ? (full ? o : fr_mask_bytes(o, nvalid)) : x;
                 const uint4 v = fr_xor4(y, g);
-                if (j != j_last) y = fr_ghash_tabmul<ABS>(sm, L, v);
+                if (ctr != c_last) y = fr_ghash_tabmul<ABS>(sm, L, v);
                 else pend = v;
             }
         } else if (ctr == 1u && MODE != FR_MODE_CTR) {
@@ -469,9 +472,14 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
                 extra = fr_aes256_ctr_block<ABS>(sm, L.lane4, P, cc, cg, 1u);         // E_K(J0)
                 if (MODE == FR_MODE_PADGEN) P.mask[kk] = extra;
             }
+            if (DO_GHASH && P.aad_mod) {                                              // the one-byte AAD block
+                const uint4 v = make_uint4((P.first_chunk + kk) % P.aad_mod, 0, 0, 0);    // y is still zero here
+                if (ctr != c_last) y = fr_ghash_tabmul<ABS>(sm, L, v);
+                else pend = v;
+            }
         }
     }
     if (!DO_GHASH) return make_uint4(0, 0, 0, 0);
-    if (j_last == 0xFFFFFFFFu) return extra;
+    if (c_last == 0u) return extra;
     return fr_xor4(fr_gf128_mul(pend, hpow), extra);
 }

@@ -22,7 +22,7 @@ EXPORTS = ("fastrack_ctx_create", "fastrack_ctx_destroy", "fastrack_num_chunks",
            "fastrack_last_cuda_error", "fastrack_decrypt_verify", "fastrack_encrypt_tag",
            "fastrack_pipelined_h2d", "fastrack_launch_count", "fastrack_decrypt_verify_noalloc",
            "fastrack_ctr_crypt", "fastrack_verify", "fastrack_keystream", "fastrack_xor_verify",
-           "fastrack_pipelined_h2d_ahead")
+           "fastrack_pipelined_h2d_ahead", "fastrack_ctx_set_framing")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2410_15240_b200.build` "
@@ -38,6 +38,8 @@ _lib.fastrack_num_chunks.restype = _sz
 _lib.fastrack_num_chunks.argtypes = [_vp, _sz]
 _lib.fastrack_ctx_reserve.restype = _int
 _lib.fastrack_ctx_reserve.argtypes = [_vp, _sz]
+_lib.fastrack_ctx_set_framing.restype = _int
+_lib.fastrack_ctx_set_framing.argtypes = [_vp, ctypes.c_uint]
 _lib.fastrack_last_cuda_error.restype = _int
 _lib.fastrack_last_cuda_error.argtypes = [_vp]
 _lib.fastrack_launch_count.restype = ctypes.c_uint64
@@ -86,6 +88,10 @@ def fastrack_num_chunks(ctx, length: int) -> int:
 
 def fastrack_ctx_reserve(ctx, max_len: int) -> int:
     return _lib.fastrack_ctx_reserve(ctx, max_len)
+
+
+def fastrack_ctx_set_framing(ctx, chains_per_sample: int) -> int:
+    return _lib.fastrack_ctx_set_framing(ctx, chains_per_sample)
 
 
 def fastrack_last_cuda_error(ctx) -> int:
@@ -157,6 +163,9 @@ class Context:
 
     def num_chunks(self, length: int) -> int:
         return fastrack_num_chunks(self.handle, length)
+
+    def set_framing(self, chains_per_sample: int) -> None:
+        self._check(fastrack_ctx_set_framing(self.handle, chains_per_sample))
 
     def reserve(self, max_len: int) -> None:
         self._check(fastrack_ctx_reserve(self.handle, max_len))

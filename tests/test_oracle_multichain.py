@@ -104,3 +104,26 @@ def test_cost_accounting_of_n_chains():
         K = oracle.num_chunks(length, cb)
         assert 16 * K / length < 0.01
     assert abs(16 * 16 / (1 << 20) - 0.000244) < 1e-6
+
+
+@pytest.mark.parametrize("length,cb,n", [(64, 32, 16), (1000, 96, 4), (4097, 1024, 3), (5000, 16, 256), (40, 32, 1)])
+def test_framed_chunks_are_openssl_gcm_calls_with_a_serial_byte_as_aad(length, cb, n):
+    """Paper Sections 4.2 / 4.4: chunk k authenticates the byte (k mod n) as AAD; independent check by OpenSSL."""
+    from cryptography.hazmat.primitives.ciphers.aead import AESGCM
+    rng = np.random.default_rng(length + cb + n)
+    key, base, p = rng.bytes(32), rng.bytes(12), rng.bytes(length)
+    c, tags = oracle.mc_encrypt_framed(key, base, cb, n, p, n_threads=3)
+    K = (length + cb - 1) // cb
+    for k in range(K):
+        ref = AESGCM(key).encrypt(oracle.chunk_iv(base, k), p[k * cb:(k + 1) * cb], bytes([k % n]))
+        assert c[k * cb:(k + 1) * cb].tobytes() + tags[k].tobytes() == ref
+    back, ok = oracle.mc_decrypt_framed(key, base, cb, n, c, tags, n_threads=2)
+    assert ok.all() and back.tobytes() == p
+    # the ciphertext does not depend on the framing, every tag does
+    c0, t0 = oracle.mc_encrypt(key, base, cb, p)
+    assert np.array_equal(c0, c) and all(not np.array_equal(t0[k], tags[k]) for k in range(K))
+    # a verifier without the framing (or with another sample size) rejects every chunk
+    assert not oracle.mc_decrypt(key, base, cb, c, tags)[1].any()
+    if 1 < n < 256 and K > 1:
+        _, ok2 = oracle.mc_decrypt_framed(key, base, cb, n + 1, c, tags)
+        assert [bool(x) for x in ok2] == [(k % n) == (k % (n + 1)) for k in range(K)]
