@@ -162,6 +162,15 @@ FASTRACK_API int fastrack_ctr_crypt(fastrack_ctx* ctx, const uint8_t iv_base[12]
 FASTRACK_API int fastrack_verify(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_cipher, size_t len,
                                  const void* d_tags, uint32_t* d_ok, void* stream);
 
+/* ---- Sequential-chain comparator (paper Section 4.2, the baseline authentication kernel) ------------------
+ * Same inputs, outputs and verdicts as fastrack_verify, computed the way the paper's starting point does it:
+ * every chunk's GMAC chain is walked block by block by ONE thread ("the GMAC function will sequentially
+ * evaluate m block multiplications"), so the only parallelism is across chunks and the time falls as 1/K when
+ * a buffer is cut into K chunks (Section 5.3: 16 chains, up to 16x).  It exists to reproduce that curve next
+ * to the parallel kernels; do not use it for throughput.  Asynchronous on `stream`; needs no scratch. */
+FASTRACK_API int fastrack_verify_sequential(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_cipher,
+                                            size_t len, const void* d_tags, uint32_t* d_ok, void* stream);
+
 /* ---- Keystream ahead of the data (paper Section 4.3, "Parallel AES evaluation") --------------------------
  * AES(k, counter) does not depend on the ciphertext, so the one-time pad can be produced while the PCIe copy
  * is still in flight; when the data arrives, decryption is one XOR.

@@ -108,6 +108,49 @@ __global__ void fr_pow_double_kernel(uint4* pow, uint32_t half, uint32_t n)
     if (i <= last) pow[i] = fr_gf128_mul(pow[i - half], pow[half]);
 }
 
+// Comparator, not the fast path: the authentication kernel in the shape the paper starts from (Section 4.2:
+// "the GMAC function will sequentially evaluate m block multiplications"; parallel only across chains).
+// One THREAD walks one chunk's whole chain, Y <- (Y xor X_i) * H, with the byte tables of H itself in shared
+// memory, then the length block, then E_K(J0) and the tag compare.  Time grows with the chain length, so it
+// falls as 1/K when a buffer is cut into K chunks -- the effect the paper's multi-chaining exploits.
+__global__ void __launch_bounds__(32, 1) fr_verify_sequential_kernel(const __grid_constant__ FrParams P)
+{
+    extern __shared__ __align__(256) char sm[];
+    fr_build_smem_any(sm, threadIdx.x, blockDim.x, P.te0, P.gh_tab);      // gh_tab holds the tables of H^1 here
+    __syncthreads();
+    const uint32_t lane = threadIdx.x;
+    const FrLane L = fr_make_lane(lane);
+    const uint32_t kk = blockIdx.x * 32u + lane;
+    if (kk >= P.n_chunks) return;
+    const uint64_t len_k = fr_chunk_len(P, kk);
+    const uint32_t nblk = (uint32_t)((len_k + 15) >> 4);
+    const uint8_t* in = P.in + (uint64_t)kk * P.chunk_bytes;
+    uint4 y = make_uint4(0, 0, 0, 0);
+    if (P.aad_mod) y = fr_ghash_tabmul<false>(sm, L, make_uint4((P.first_chunk + kk) % P.aad_mod, 0, 0, 0));
+    uint32_t j = 0;
+    for (; j + 8 <= nblk && ((uint64_t)(j + 8) << 4) <= len_k; j += 8) {      // eight loads in flight per thread
+        uint4 x[8];
+#pragma unroll
+        for (int u = 0; u < 8; u++) x[u] = *(const uint4*)(in + ((uint64_t)(j + u) << 4));
+#pragma unroll
+        for (int u = 0; u < 8; u++) y = fr_ghash_tabmul<false>(sm, L, fr_xor4(y, x[u]));
+    }
+    for (; j < nblk; j++) {
+        const uint64_t boff = (uint64_t)j << 4;
+        const bool full = len_k - boff >= 16;
+        const uint4 x = full ? *(const uint4*)(in + boff) : fr_load_partial(in + boff, (uint32_t)(len_k - boff));
+        y = fr_ghash_tabmul<false>(sm, L, fr_xor4(y, x));
+    }
+    const uint64_t bits = len_k << 3;
+    const uint4 lenblk = make_uint4(0, P.aad_mod ? fr_bswap(8u) : 0u, fr_bswap((uint32_t)(bits >> 32)), fr_bswap((uint32_t)bits));
+    y = fr_ghash_tabmul<false>(sm, L, fr_xor4(y, lenblk));
+    const FrCtrChunk cc = fr_ctr_chunk<false>(sm, L.lane4, P, fr_bswap(P.iv_ctr + kk));
+    const FrCtrGroup cg = fr_ctr_group<false>(sm, L.lane4, P, cc, 1u);
+    const uint4 tag = fr_xor4(y, fr_aes256_ctr_block<false>(sm, L.lane4, P, cc, cg, 1u));
+    const uint4 t = P.tags_in[kk];
+    P.ok[kk] = ((tag.x ^ t.x) | (tag.y ^ t.y) | (tag.z ^ t.z) | (tag.w ^ t.w)) == 0u ? 1u : 0u;
+}
+
 // ------------------------------------------------------------------------------------ context ----
 
 struct fastrack_ctx {
@@ -117,7 +160,8 @@ struct fastrack_ctx {
     uint32_t rk[60];
     uint8_t h[16];
     uint32_t* d_te0;
-    uint4* d_gh_tab;
+    uint4* d_gh_tab;           // byte tables of H^32
+    uint4* d_gh1_tab;          // byte tables of H (sequential-chain comparator only)
     uint4* d_pow;
     size_t pow_entries;
     uint32_t* d_scratch;       // two banks, each acc[4*cap] then cnt[cap]; bank 1 serves fastrack_verify
@@ -191,20 +235,23 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
 
     Gf128 H = gf_load(ctx->h), G = H;
     for (int i = 0; i < 5; i++) G = gf_mul(G, G);           // H^32
-    uint8_t* tab = (uint8_t*)malloc(65536);
+    uint8_t* tab = (uint8_t*)malloc(2 * 65536);             // tables of H^32, then of H
     if (!tab) return fail(FASTRACK_ERR_NOMEM);
-    for (int p = 0; p < 16; p++) {
-        Gf128 basis[8];
-        for (int b = 0; b < 8; b++) {
-            uint8_t blk[16] = {0};
-            blk[p] = (uint8_t)(1u << b);
-            basis[b] = gf_mul(gf_load(blk), G);
-        }
-        for (int v = 0; v < 256; v++) {
-            Gf128 acc = {0, 0};
-            for (int b = 0; b < 8; b++)
-                if (v & (1 << b)) { acc.hi ^= basis[b].hi; acc.lo ^= basis[b].lo; }
-            gf_store(acc, tab + (size_t)v * 256 + (size_t)p * 16);
+    for (int which = 0; which < 2; which++) {
+        const Gf128 mult = which == 0 ? G : H;
+        for (int p = 0; p < 16; p++) {
+            Gf128 basis[8];
+            for (int b = 0; b < 8; b++) {
+                uint8_t blk[16] = {0};
+                blk[p] = (uint8_t)(1u << b);
+                basis[b] = gf_mul(gf_load(blk), mult);
+            }
+            for (int v = 0; v < 256; v++) {
+                Gf128 acc = {0, 0};
+                for (int b = 0; b < 8; b++)
+                    if (v & (1 << b)) { acc.hi ^= basis[b].hi; acc.lo ^= basis[b].lo; }
+                gf_store(acc, tab + (size_t)which * 65536 + (size_t)v * 256 + (size_t)p * 16);
+            }
         }
     }
 
@@ -212,9 +259,11 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
     do {
         if ((e = cudaMalloc(&ctx->d_te0, sizeof te0)) != cudaSuccess) break;
         if ((e = cudaMalloc(&ctx->d_gh_tab, 65536)) != cudaSuccess) break;
+        if ((e = cudaMalloc(&ctx->d_gh1_tab, 65536)) != cudaSuccess) break;
         if ((e = cudaMalloc(&ctx->d_pow, ctx->pow_entries * 16)) != cudaSuccess) break;
         if ((e = cudaMemcpy(ctx->d_te0, te0, sizeof te0, cudaMemcpyHostToDevice)) != cudaSuccess) break;
         if ((e = cudaMemcpy(ctx->d_gh_tab, tab, 65536, cudaMemcpyHostToDevice)) != cudaSuccess) break;
+        if ((e = cudaMemcpy(ctx->d_gh1_tab, tab + 65536, 65536, cudaMemcpyHostToDevice)) != cudaSuccess) break;
         uint8_t seed[32] = {0};
         seed[0] = 0x80;                                     // H^0 = the field's one
         memcpy(seed + 16, ctx->h, 16);                      // H^1
@@ -231,13 +280,14 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
         if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_VERIFY>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
         if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_PADGEN>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
         if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_PADDEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_verify_sequential_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
         for (int i = 0; i < 8 && e == cudaSuccess; i++) e = cudaStreamCreateWithFlags(&ctx->streams[i], cudaStreamNonBlocking);
         if (e != cudaSuccess) break;
         if ((e = cudaEventCreateWithFlags(&ctx->tags_ready, cudaEventDisableTiming)) != cudaSuccess) break;
         if ((e = cudaEventCreateWithFlags(&ctx->pad_ready, cudaEventDisableTiming)) != cudaSuccess) break;
         e = cudaDeviceSynchronize();
     } while (0);
-    memset(tab, 0, 65536);
+    memset(tab, 0, 2 * 65536);
     free(tab);
     if (e != cudaSuccess) {
         ctx->last_cuda_error = (int)e;
@@ -255,10 +305,12 @@ extern "C" void fastrack_ctx_destroy(fastrack_ctx* ctx)
     if (!ctx) return;
     cudaDeviceSynchronize();
     if (ctx->d_gh_tab) { cudaMemset(ctx->d_gh_tab, 0, 65536); }
+    if (ctx->d_gh1_tab) { cudaMemset(ctx->d_gh1_tab, 0, 65536); }
     if (ctx->d_pow) { cudaMemset(ctx->d_pow, 0, ctx->pow_entries * 16); }
     cudaDeviceSynchronize();
     cudaFree(ctx->d_te0);
     cudaFree(ctx->d_gh_tab);
+    cudaFree(ctx->d_gh1_tab);
     cudaFree(ctx->d_pow);
     cudaFree(ctx->d_scratch);
     cudaFree(ctx->d_tags_stage);
@@ -606,6 +658,36 @@ extern "C" int fastrack_verify(fastrack_ctx* ctx, const uint8_t iv_base[12], con
     PassBuffers b;
     b.in = d_cipher; b.out = const_cast<void*>(d_cipher); b.tags_in = d_tags; b.ok = d_ok; b.bank = 1;
     return launch_pass(ctx, FR_MODE_VERIFY, iv_base, 0, len, b, (cudaStream_t)stream);
+}
+
+extern "C" int fastrack_verify_sequential(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_cipher, size_t len,
+                                          const void* d_tags, uint32_t* d_ok, void* stream)
+{
+    if (!ctx || !iv_base) return FASTRACK_ERR_ARG;
+    if (len == 0) return FASTRACK_OK;
+    if (!d_cipher || !d_tags || !d_ok) return FASTRACK_ERR_ARG;
+    if (misaligned(d_cipher, 16) || misaligned(d_tags, 16) || misaligned(d_ok, 4)) return FASTRACK_ERR_ARG;
+    const size_t K = fastrack_num_chunks(ctx, len);
+    if (K > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
+    FrParams P;
+    memset(&P, 0, sizeof P);
+    memcpy(P.rk, ctx->rk, sizeof P.rk);
+    P.iv_w0 = load_le32(iv_base);
+    P.iv_w1 = load_le32(iv_base + 4);
+    P.iv_ctr = load_be32(iv_base + 8);
+    P.aad_mod = ctx->aad_mod;
+    P.len = len;
+    P.chunk_bytes = ctx->chunk_bytes;
+    P.n_chunks = (uint32_t)K;
+    P.in = (const uint8_t*)d_cipher;
+    P.tags_in = (const uint4*)d_tags;
+    P.ok = d_ok;
+    P.te0 = ctx->d_te0;
+    P.gh_tab = ctx->d_gh1_tab;
+    fr_verify_sequential_kernel<<<(unsigned)((K + 31) / 32), 32, FR_SMEM_BYTES, (cudaStream_t)stream>>>(P);
+    ctx->launches++;
+    FR_CUDA(ctx, cudaGetLastError());
+    return FASTRACK_OK;
 }
 
 extern "C" int fastrack_keystream(fastrack_ctx* ctx, const uint8_t iv_base[12], size_t len, void* d_pad, void* d_mask,

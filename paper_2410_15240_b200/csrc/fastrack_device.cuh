@@ -139,6 +139,18 @@ __device__ __forceinline__ void fr_build_smem(char* sm, uint32_t tid, const uint
     for (uint32_t n = 0; n < N_GH; n++) *(uint4*)(sm + FR_SM_GH + (tid + n * NTHREADS) * 16u) = g[n];
 }
 
+// The same fill with a run-time thread count (small launches where set-up time does not matter).
+__device__ __forceinline__ void fr_build_smem_any(char* sm, uint32_t tid, uint32_t nthreads,
+                                                  const uint32_t* __restrict__ te0, const uint4* __restrict__ gh_tab)
+{
+    for (uint32_t i = tid; i < 8192u; i += nthreads) {
+        const uint32_t q = i & 7u, t = (i >> 3) & 3u, v = i >> 5, e = te0[v];
+        const uint32_t w = (t == 0) ? e : (t == 1) ? ((e << 8) | (e >> 24)) : (t == 2) ? ((e << 16) | (e >> 16)) : ((e << 24) | (e >> 8));
+        *(uint4*)(sm + ((t >> 1) ? FR_SM_T23 : FR_SM_T01) + v * 256u + (t & 1u) * 128u + q * 16u) = make_uint4(w, w, w, w);
+    }
+    for (uint32_t i = tid; i < 4096u; i += nthreads) *(uint4*)(sm + FR_SM_GH + i * 16u) = gh_tab[i];
+}
+
 // Shared-memory loads.  The dynamic shared window of a kernel without static shared memory starts at shared
 // address FR_SMEM_ABS_BASE on this architecture (the first KiB is reserved by the system).  When the kernel has
 // checked that at run time (ABS = true), a lookup address is "constant + permuted bytes", and the constant goes

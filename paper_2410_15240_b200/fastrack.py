@@ -22,7 +22,7 @@ EXPORTS = ("fastrack_ctx_create", "fastrack_ctx_destroy", "fastrack_num_chunks",
            "fastrack_last_cuda_error", "fastrack_decrypt_verify", "fastrack_encrypt_tag",
            "fastrack_pipelined_h2d", "fastrack_launch_count", "fastrack_decrypt_verify_noalloc",
            "fastrack_ctr_crypt", "fastrack_verify", "fastrack_keystream", "fastrack_xor_verify",
-           "fastrack_pipelined_h2d_ahead", "fastrack_ctx_set_framing")
+           "fastrack_pipelined_h2d_ahead", "fastrack_ctx_set_framing", "fastrack_verify_sequential")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2410_15240_b200.build` "
@@ -54,6 +54,8 @@ _lib.fastrack_ctr_crypt.restype = _int
 _lib.fastrack_ctr_crypt.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp]
 _lib.fastrack_verify.restype = _int
 _lib.fastrack_verify.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp]
+_lib.fastrack_verify_sequential.restype = _int
+_lib.fastrack_verify_sequential.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp]
 _lib.fastrack_keystream.restype = _int
 _lib.fastrack_keystream.argtypes = [_vp, ctypes.c_char_p, _sz, _vp, _vp, _vp]
 _lib.fastrack_xor_verify.restype = _int
@@ -132,6 +134,11 @@ def fastrack_verify(ctx, iv_base: bytes, d_cipher: int, length: int, d_tags: int
     return _lib.fastrack_verify(ctx, iv_base, d_cipher, length, d_tags, d_ok, stream)
 
 
+def fastrack_verify_sequential(ctx, iv_base: bytes, d_cipher: int, length: int, d_tags: int, d_ok: int,
+                               stream: int = 0) -> int:
+    return _lib.fastrack_verify_sequential(ctx, iv_base, d_cipher, length, d_tags, d_ok, stream)
+
+
 def fastrack_keystream(ctx, iv_base: bytes, length: int, d_pad: int, d_mask: int, stream: int = 0) -> int:
     return _lib.fastrack_keystream(ctx, iv_base, length, d_pad, d_mask, stream)
 
@@ -189,6 +196,9 @@ class Context:
 
     def verify(self, iv_base, d_cipher, length, d_tags, d_ok, stream=0) -> None:
         self._check(fastrack_verify(self.handle, iv_base, d_cipher, length, d_tags, d_ok, stream))
+
+    def verify_sequential(self, iv_base, d_cipher, length, d_tags, d_ok, stream=0) -> None:
+        self._check(fastrack_verify_sequential(self.handle, iv_base, d_cipher, length, d_tags, d_ok, stream))
 
     def keystream(self, iv_base, length, d_pad, d_mask, stream=0) -> None:
         self._check(fastrack_keystream(self.handle, iv_base, length, d_pad, d_mask, stream))

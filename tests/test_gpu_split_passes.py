@@ -157,3 +157,30 @@ def test_split_pass_argument_errors():
     assert A(ctx, iv, pinned.data_ptr(), 4096, h_tags.ctypes.data, b + 4096, b, o, 2) == fastrack.OK
     torch.cuda.synchronize()
     fastrack.fastrack_ctx_destroy(ctx)
+
+
+@pytest.mark.parametrize("n,cb,chains", [(1, 16, 0), (1000, 64, 0), (70001, 4096, 0), ((1 << 20) + 5, 65536, 0),
+                                         (200 * 1024 + 9, 1024, 0), (70001, 4096, 16), (33 * 160 + 3, 160, 3)])
+def test_sequential_chain_comparator_gives_the_same_verdicts(n, cb, chains):
+    """The one-thread-per-chain kernel (the paper's starting point) must agree with the oracle as well."""
+    key, iv = synth.key_and_iv(1)
+    plain = synth.random_bytes(n, 1, salt=n + 7)
+    if chains:
+        c, t = oracle.mc_encrypt_framed(key, iv, cb, chains, plain, NT)
+    else:
+        c, t = oracle.mc_encrypt(key, iv, cb, plain, NT)
+    plan = synth.tamper_plan(n, cb, 1, fraction=0.2, salt=n + 7)
+    synth.apply_tamper(c, t, cb, plan)
+    if chains:
+        _, ok_ref = oracle.mc_decrypt_framed(key, iv, cb, chains, c, t, NT)
+    else:
+        _, ok_ref = oracle.mc_decrypt(key, iv, cb, c, t, NT)
+    K = ok_ref.size
+    with fastrack.Context(key, cb) as ctx:
+        ctx.set_framing(chains)
+        d_c, d_t = dev(c), dev(t)
+        d_ok = torch.full((K,), 7, dtype=torch.int32, device="cuda")
+        ctx.verify_sequential(iv, d_c.data_ptr(), n, d_t.data_ptr(), d_ok.data_ptr(), torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        assert np.array_equal(d_ok.cpu().numpy().view(np.uint32), ok_ref)
+        assert np.array_equal(d_c.cpu().numpy(), c)
