@@ -216,6 +216,22 @@ FASTRACK_API int fastrack_decrypt_verify_noalloc(fastrack_ctx* ctx, const uint8_
                                                  const void* d_cipher, size_t len, const void* d_tags,
                                                  void* d_plain, uint32_t* d_ok, void* stream);
 
+/* Pipelined device->host transfer with encryption and tagging: the mirror of fastrack_pipelined_h2d for
+ * GPU->CPU copies (paper Section 2.3: encryption is the same keystream XOR; Section 4.2: one tag per chunk;
+ * Section 4.3: the transfer is overlapped with the kernels).
+ * The buffer is cut into stages of whole chunks that GROW geometrically (about 2 MiB first, then twice as much,
+ * ... the last one about half of the buffer); stage i is encrypted and tagged from d_plain into d_cipher on
+ * internal stream i mod n_streams and then copied, with its tags, to the host on the same stream, so the copy
+ * of stage i overlaps the kernel of stage i+1 and only the short first stage's kernel is exposed.
+ *   d_plain         device, len bytes in (not modified unless d_cipher == d_plain).
+ *   d_cipher        device, len bytes of ciphertext staging; d_cipher == d_plain (exactly) encrypts in place.
+ *   h_cipher_pinned host, page-locked, len bytes out.
+ *   h_tags          host, 16*K bytes out, pinned or pageable.
+ *   n_streams       1..8.
+ * BLOCKING: returns when the ciphertext and the tags are complete in host memory. */
+FASTRACK_API int fastrack_pipelined_d2h(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_plain, size_t len,
+                                        void* d_cipher, void* h_cipher_pinned, void* h_tags, int n_streams);
+
 /* Number of kernels the library launched through ctx since creation (data-path launches only;
  * cudaMemcpyAsync calls are not counted).  For benchmarks' bookkeeping. */
 FASTRACK_API uint64_t fastrack_launch_count(const fastrack_ctx* ctx);

@@ -517,6 +517,36 @@ extern "C" int fastrack_encrypt_tag(fastrack_ctx* ctx, const uint8_t iv_base[12]
     return launch_pass(ctx, FR_MODE_ENC, iv_base, 0, len, b, (cudaStream_t)stream);
 }
 
+// Stage = the unit that is copied and processed in place: whole chunks.  In a pipelined transfer only two
+// things are not hidden behind a copy: a few microseconds per copy boundary and ONE kernel (the last stage's
+// on the way in, the first stage's on the way out).  So the stages shrink geometrically: half of the buffer,
+// then half of the rest, ... down to about 2 MiB (never less than one chunk) -- few copies, and a short
+// exposed kernel.  A stage's kernel is an order of magnitude faster than its neighbour's copy, so it always
+// finishes under it.  Returns the stage sizes in descending order (host->device order).
+#define FR_MAX_STAGES 96
+static size_t plan_stages(const fastrack_ctx* ctx, size_t len, size_t out[FR_MAX_STAGES])
+{
+    const size_t cb = ctx->chunk_bytes;
+    const size_t floor_bytes = (size_t)2 << 20;
+    const size_t min_stage = cb >= floor_bytes ? cb : (floor_bytes + cb - 1) / cb * cb;
+    size_t off = 0, count = 0;
+    while (off < len) {
+        const size_t remaining = len - off;
+        size_t n;
+        if (ctx->stage_bytes_override) {
+            n = (ctx->stage_bytes_override + cb - 1) / cb * cb;
+        } else {
+            n = remaining / 2 / cb * cb;
+            if (n < min_stage) n = min_stage;
+            if (remaining < n + min_stage / 2) n = remaining;      // do not leave a sliver behind
+        }
+        if (n > remaining || count == FR_MAX_STAGES - 1) n = remaining;
+        out[count++] = n;
+        off += n;
+    }
+    return count;
+}
+
 // Common body of the two pipelined entry points.  d_pad == nullptr: fused decrypt+verify per stage.
 // d_pad != nullptr: the keystream for the whole buffer is produced first, on a stream of its own, while the
 // first copy is in flight; the stages then only XOR and authenticate.
@@ -563,26 +593,12 @@ static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const vo
     }
     bool waited[8] = {false, false, false, false, false, false, false, false};   // per working stream: events already awaited
 
-    // Stage = the unit that is copied and then decrypted in place: whole chunks.  Only two things are not
-    // hidden behind a copy: a few microseconds per copy boundary and the kernel of the LAST stage.  So the
-    // stages shrink geometrically: the first takes half of the buffer, each next one half of what is left,
-    // down to about 2 MiB (never less than one chunk) -- few copies, and a short last kernel.  A stage's
-    // kernel is an order of magnitude faster than the next stage's copy, so it always finishes under it.
+    size_t stage_bytes[FR_MAX_STAGES];
+    const size_t n_stages = plan_stages(ctx, len, stage_bytes);
     const size_t cb = ctx->chunk_bytes;
-    const size_t floor_bytes = (size_t)2 << 20;
-    const size_t min_stage = cb >= floor_bytes ? cb : (floor_bytes + cb - 1) / cb * cb;
-    size_t off = 0, stage = 0;
-    while (off < len) {
-        const size_t remaining = len - off;
-        size_t n;
-        if (ctx->stage_bytes_override) {
-            n = (ctx->stage_bytes_override + cb - 1) / cb * cb;
-        } else {
-            n = remaining / 2 / cb * cb;
-            if (n < min_stage) n = min_stage;
-            if (remaining < n + min_stage / 2) n = remaining;      // do not leave a sliver behind
-        }
-        if (n > remaining) n = remaining;
+    size_t off = 0;
+    for (size_t stage = 0; stage < n_stages; stage++) {
+        const size_t n = stage_bytes[stage];
         const size_t k0 = off / cb;
         cudaStream_t st = ctx->streams[stage % (size_t)n_streams];
         uint8_t* dst = (uint8_t*)d_plain + off;
@@ -609,7 +625,6 @@ static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const vo
             return rc;
         }
         off += n;
-        stage++;
     }
     FR_CUDA(ctx, cudaStreamSynchronize(tag_stream));
     if (d_pad) FR_CUDA(ctx, cudaStreamSynchronize(pad_stream));
@@ -629,6 +644,65 @@ extern "C" int fastrack_pipelined_h2d_ahead(fastrack_ctx* ctx, const uint8_t iv_
 {
     if (!d_pad) return FASTRACK_ERR_ARG;
     return pipelined_impl(ctx, iv_base, h_cipher_pinned, len, h_tags, d_pad, d_plain, d_ok, n_streams);
+}
+
+extern "C" int fastrack_pipelined_d2h(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_plain, size_t len,
+                                      void* d_cipher, void* h_cipher_pinned, void* h_tags, int n_streams)
+{
+    if (!ctx || !iv_base) return FASTRACK_ERR_ARG;
+    if (n_streams < 1 || n_streams > 8) return FASTRACK_ERR_ARG;
+    if (len == 0) return FASTRACK_OK;
+    if (!d_plain || !d_cipher || !h_cipher_pinned || !h_tags) return FASTRACK_ERR_ARG;
+    if (misaligned(d_plain, 16) || misaligned(d_cipher, 16) || bad_overlap(d_plain, d_cipher, len)) return FASTRACK_ERR_ARG;
+    cudaPointerAttributes attr;
+    cudaError_t e = cudaPointerGetAttributes(&attr, h_cipher_pinned);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return FASTRACK_ERR_NOT_PINNED; }
+    if (attr.type != cudaMemoryTypeHost) return FASTRACK_ERR_NOT_PINNED;
+    const size_t K = fastrack_num_chunks(ctx, len);
+    if (K > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
+    int rc = ensure_scratch(ctx, K);
+    if (rc != FASTRACK_OK) return rc;
+    if (K > ctx->tags_stage_chunks) {
+        size_t cap = ctx->tags_stage_chunks ? ctx->tags_stage_chunks : 1024;
+        while (cap < K) cap *= 2;
+        FR_CUDA(ctx, cudaDeviceSynchronize());
+        cudaFree(ctx->d_tags_stage);
+        ctx->d_tags_stage = nullptr;
+        ctx->tags_stage_chunks = 0;
+        e = cudaMalloc(&ctx->d_tags_stage, cap * 32);
+        if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); return FASTRACK_ERR_NOMEM; }
+        ctx->tags_stage_chunks = cap;
+    }
+    // On the way out the FIRST stage's kernel is the exposed one: smallest stage first.  The plan is made on
+    // whole chunks (K * chunk_bytes) and walked backwards, so every stage starts on a chunk boundary and the
+    // short last chunk, if any, stays at the end of the last (largest) stage.
+    size_t stage_bytes[FR_MAX_STAGES];
+    const size_t cb = ctx->chunk_bytes;
+    const size_t n_stages = plan_stages(ctx, K * cb, stage_bytes);
+    size_t off = 0;
+    for (size_t i = 0; i < n_stages; i++) {
+        size_t n = stage_bytes[n_stages - 1 - i];
+        if (n > len - off) n = len - off;
+        const size_t k0 = off / cb;
+        cudaStream_t st = ctx->streams[i % (size_t)n_streams];
+        PassBuffers b;
+        b.in = (const uint8_t*)d_plain + off; b.out = (uint8_t*)d_cipher + off; b.tags_out = ctx->d_tags_stage + k0;
+        rc = launch_pass(ctx, FR_MODE_ENC, iv_base, k0, n, b, st);
+        if (rc == FASTRACK_OK) {
+            e = cudaMemcpyAsync((uint8_t*)h_cipher_pinned + off, (const uint8_t*)d_cipher + off, n, cudaMemcpyDeviceToHost, st);
+            if (e == cudaSuccess) e = cudaMemcpyAsync((uint8_t*)h_tags + 16 * k0, ctx->d_tags_stage + k0, 16 * ((n + cb - 1) / cb),
+                                                      cudaMemcpyDeviceToHost, st);
+            if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); rc = FASTRACK_ERR_CUDA; }
+        }
+        if (rc != FASTRACK_OK) {
+            for (int s2 = 0; s2 < 8; s2++) cudaStreamSynchronize(ctx->streams[s2]);
+            (void)cudaGetLastError();
+            return rc;
+        }
+        off += n;
+    }
+    for (int i = 0; i < n_streams; i++) FR_CUDA(ctx, cudaStreamSynchronize(ctx->streams[i]));
+    return FASTRACK_OK;
 }
 
 extern "C" int fastrack_ctr_crypt(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_in, size_t len, void* d_out,

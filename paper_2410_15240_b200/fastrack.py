@@ -22,7 +22,7 @@ EXPORTS = ("fastrack_ctx_create", "fastrack_ctx_destroy", "fastrack_num_chunks",
            "fastrack_last_cuda_error", "fastrack_decrypt_verify", "fastrack_encrypt_tag",
            "fastrack_pipelined_h2d", "fastrack_launch_count", "fastrack_decrypt_verify_noalloc",
            "fastrack_ctr_crypt", "fastrack_verify", "fastrack_keystream", "fastrack_xor_verify",
-           "fastrack_pipelined_h2d_ahead", "fastrack_ctx_set_framing", "fastrack_verify_sequential")
+           "fastrack_pipelined_h2d_ahead", "fastrack_ctx_set_framing", "fastrack_verify_sequential", "fastrack_pipelined_d2h")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2410_15240_b200.build` "
@@ -62,6 +62,8 @@ _lib.fastrack_xor_verify.restype = _int
 _lib.fastrack_xor_verify.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.fastrack_pipelined_h2d_ahead.restype = _int
 _lib.fastrack_pipelined_h2d_ahead.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp, _vp, _int]
+_lib.fastrack_pipelined_d2h.restype = _int
+_lib.fastrack_pipelined_d2h.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp, _int]
 _lib.fastrack_pipelined_h2d.restype = _int
 _lib.fastrack_pipelined_h2d.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp, _int]
 
@@ -154,6 +156,11 @@ def fastrack_pipelined_h2d_ahead(ctx, iv_base: bytes, h_cipher_pinned: int, leng
                                              n_streams)
 
 
+def fastrack_pipelined_d2h(ctx, iv_base: bytes, d_plain: int, length: int, d_cipher: int, h_cipher_pinned: int,
+                           h_tags: int, n_streams: int) -> int:
+    return _lib.fastrack_pipelined_d2h(ctx, iv_base, d_plain, length, d_cipher, h_cipher_pinned, h_tags, n_streams)
+
+
 class Context:
     """RAII wrapper: ``with Context(key, chunk_bytes) as ctx: ctx.decrypt_verify(...)``; raises FastrackError."""
 
@@ -210,6 +217,10 @@ class Context:
     def pipelined_h2d_ahead(self, iv_base, h_cipher_pinned, length, h_tags, d_pad, d_plain, d_ok, n_streams=4) -> None:
         self._check(fastrack_pipelined_h2d_ahead(self.handle, iv_base, h_cipher_pinned, length, h_tags, d_pad, d_plain,
                                                  d_ok, n_streams))
+
+    def pipelined_d2h(self, iv_base, d_plain, length, d_cipher, h_cipher_pinned, h_tags, n_streams=4) -> None:
+        self._check(fastrack_pipelined_d2h(self.handle, iv_base, d_plain, length, d_cipher, h_cipher_pinned, h_tags,
+                                           n_streams))
 
     @property
     def launches(self) -> int:

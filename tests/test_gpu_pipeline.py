@@ -47,3 +47,29 @@ def test_config2_fp16_image_batch(cb, n_streams):
         p, ok = g.pipelined(iv, c, t, n_streams)
     assert (ok == 1).all() and ok.size == oracle.num_chunks(plain.size, cb)
     assert np.array_equal(p, plain)
+
+
+@pytest.mark.parametrize("n,cb,n_streams,in_place", [(1, 16, 1, False), (100, 1024, 2, True), ((1 << 20) + 17, 65536, 2, False),
+                                                      ((9 << 20) + 12345, 256 * 1024, 3, True),
+                                                      (2 * (1 << 22) + 999, 1 << 22, 4, False), (77_070_336, 4 << 20, 4, False)])
+def test_pipelined_d2h_encrypt_matches_oracle(n, cb, n_streams, in_place):
+    """GPU encrypt+tag with overlapped device->host copies; the host side (oracle) verifies and decrypts."""
+    from paper_2410_15240_b200 import fastrack
+    key, iv = synth.key_and_iv(3)
+    plain = synth.fp16_image_batch() if n == 77_070_336 else synth.random_bytes(n, 3, salt=n)
+    c_ref, t_ref = oracle.mc_encrypt(key, iv, cb, plain, NT)
+    K = t_ref.shape[0]
+    with fastrack.Context(key, cb) as ctx:
+        d_p = torch.from_numpy(plain).cuda()
+        d_c = d_p if in_place else torch.empty_like(d_p)
+        h_c = torch.full((n,), 0xEE, dtype=torch.uint8).pin_memory()
+        h_t = torch.zeros(16 * K, dtype=torch.uint8)
+        torch.cuda.synchronize()
+        for _ in range(1 if in_place else 2):
+            ctx.pipelined_d2h(iv, d_p.data_ptr(), n, d_c.data_ptr(), h_c.data_ptr(), h_t.data_ptr(), n_streams)
+            assert np.array_equal(h_c.numpy(), c_ref)
+            assert np.array_equal(h_t.numpy().reshape(K, 16), t_ref)
+        if not in_place:
+            assert np.array_equal(d_p.cpu().numpy(), plain)
+    back, ok = oracle.mc_decrypt(key, iv, cb, h_c.numpy(), h_t.numpy(), NT)
+    assert ok.all() and np.array_equal(back, plain)

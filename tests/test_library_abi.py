@@ -16,7 +16,7 @@ def declared_functions():
 
 def test_header_and_binding_agree():
     names = declared_functions()
-    assert len(names) >= 17
+    assert len(names) >= 18
     assert sorted(fastrack.EXPORTS) == names
 
 
@@ -59,6 +59,7 @@ def test_argument_checks_that_need_no_device():
     assert fastrack.fastrack_xor_verify(None, bytes(12), 0, 16, 0, 0, 0, 0, 0, 0) == fastrack.ERR_ARG
     assert fastrack.fastrack_pipelined_h2d_ahead(None, bytes(12), 0, 16, 0, 0, 0, 0, 2) == fastrack.ERR_ARG
     assert fastrack.fastrack_pipelined_h2d(None, bytes(12), 0, 16, 0, 0, 0, 2) == fastrack.ERR_ARG
+    assert fastrack.fastrack_pipelined_d2h(None, bytes(12), 0, 16, 0, 0, 0, 2) == fastrack.ERR_ARG
     fastrack.fastrack_ctx_destroy(None)          # allowed
 
 
