@@ -398,12 +398,72 @@ def run_sweep(args):
                           "pipelined_h2d_gbs": n / t_pipe / 1e9, "raw_pinned_h2d_gbs": n / t_raw / 1e9,
                           "fraction_of_raw": t_raw / t_pipe}), flush=True)
 
+    def d2h_cell(n, cb, n_streams, label):
+        K = (n + cb - 1) // cb
+        with fastrack.Context(key, cb) as ctx:
+            d_p = torch.randint(0, 256, (n,), dtype=torch.uint8, device="cuda")
+            d_c = torch.empty_like(d_p)
+            h_c = torch.empty(n, dtype=torch.uint8).pin_memory()
+            h_t = torch.empty(16 * K, dtype=torch.uint8).pin_memory()
+            reps = 10
+
+            def wall(fn):
+                for _ in range(2):
+                    fn()
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                for _ in range(reps):
+                    fn()
+                torch.cuda.synchronize()
+                return (time.perf_counter() - t0) / reps
+
+            t_pipe = wall(lambda: ctx.pipelined_d2h(iv, d_p.data_ptr(), n, d_c.data_ptr(), h_c.data_ptr(), h_t.data_ptr(),
+                                                    n_streams))
+
+            def raw():
+                h_c.copy_(d_p, non_blocking=True)
+                torch.cuda.current_stream().synchronize()
+            t_raw = wall(raw)
+        print(json.dumps({"cell": label, "len": n, "chunk": cb, "K": K, "streams": n_streams,
+                          "pipelined_d2h_gbs": n / t_pipe / 1e9, "raw_pinned_d2h_gbs": n / t_raw / 1e9,
+                          "fraction_of_raw": t_raw / t_pipe}), flush=True)
+
+    def modes_cell(n, cb, label):
+        """Split passes and the sequential-chain comparator, device-resident."""
+        K = (n + cb - 1) // cb
+        with fastrack.Context(key, cb) as ctx:
+            st = stream.cuda_stream
+            d_p = torch.randint(0, 256, (n,), dtype=torch.uint8, device="cuda")
+            d_c, d_o, d_pad = torch.empty_like(d_p), torch.empty_like(d_p), torch.empty_like(d_p)
+            d_t = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
+            d_m = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
+            d_ok = torch.zeros(K, dtype=torch.int32, device="cuda")
+            ctx.encrypt_tag(iv, d_p.data_ptr(), n, d_c.data_ptr(), d_t.data_ptr(), st)
+            reps = 20
+            out = {"cell": label, "len": n, "chunk": cb, "K": K}
+            out["ctr_crypt_gbs"] = n / timed(lambda: ctx.ctr_crypt(iv, d_c.data_ptr(), n, d_o.data_ptr(), st), reps) / 1e9
+            out["verify_gbs"] = n / timed(lambda: ctx.verify(iv, d_c.data_ptr(), n, d_t.data_ptr(), d_ok.data_ptr(), st), reps) / 1e9
+            out["keystream_gbs"] = n / timed(lambda: ctx.keystream(iv, n, d_pad.data_ptr(), d_m.data_ptr(), st), reps) / 1e9
+            out["xor_verify_gbs"] = n / timed(lambda: ctx.xor_verify(iv, d_c.data_ptr(), n, d_pad.data_ptr(), d_m.data_ptr(),
+                                                                     d_t.data_ptr(), d_o.data_ptr(), d_ok.data_ptr(), st), reps) / 1e9
+            assert bool((d_ok == 1).all()) and bool((d_o == d_p).all())
+            out["verify_sequential_us"] = timed(lambda: ctx.verify_sequential(iv, d_c.data_ptr(), n, d_t.data_ptr(),
+                                                                                d_ok.data_ptr(), st), 1 if K < 64 else 5) * 1e6
+            out["verify_us"] = n / out["verify_gbs"] / 1e3
+            assert bool((d_ok == 1).all())
+        print(json.dumps(out), flush=True)
+
     for K in (1, 4, 16, 64, 256, 1024):                                   # config 1
         device_cell(64 << 20, (64 << 20) // K, "config1")
     for cb in (256 << 10, 1 << 20, 4 << 20, 8 << 20):                     # config 2
         for ns in (2, 3, 4):
             pipeline_cell(77_070_336, cb, ns, "config2")
     device_cell(670_000_000, 4 << 20, "config3")
+    for ns in (2, 4):
+        d2h_cell(670_000_000, 4 << 20, ns, "config3_d2h")
+    modes_cell(256 << 20, 4 << 20, "split_passes")
+    for K in (16, 64, 256, 1024, 4096):
+        modes_cell(64 << 20, (64 << 20) // K, "split_passes_vs_K")
     for e in range(6, 17):                                                # config 4 (device-resident throughput)
         for cb in (16 << 10, 64 << 10, 256 << 10, 1 << 20, 4 << 20, 16 << 20):
             device_cell(4 ** e, cb, "config4")
