@@ -157,34 +157,60 @@ def run_reference(args):
     }))
 
 
+class Ranks:
+    """One process per GPU; the path has no exchange step, so the ranks are independent replicas and the only
+    collectives are the barrier around the timed region and the MAX of the per-rank times."""
+
+    def __init__(self, backend: str, device: str):
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        self.device = device
+        self.dist = None
+        if self.world > 1:
+            import torch
+            import torch.distributed as dist
+            kwargs = {"device_id": torch.device("cuda", self.local)} if backend == "nccl" else {}
+            dist.init_process_group(backend, **kwargs)
+            self.dist = dist
+
+    def barrier(self):
+        import torch
+        if self.device == "cuda":
+            torch.cuda.synchronize()
+        if self.dist is not None:
+            self.dist.barrier()
+        if self.device == "cuda":
+            torch.cuda.synchronize()
+
+    def max_over_ranks(self, x: float) -> float:
+        if self.dist is None:
+            return x
+        import torch
+        t = torch.tensor([x], dtype=torch.float64, device=self.device)
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def aggregate_throughput(self, bytes_per_rank: int, seconds_this_rank: float) -> float:
+        """Whole-job bytes per second: every rank moved bytes_per_rank, the job took the slowest rank's time."""
+        return self.world * bytes_per_rank / self.max_over_ranks(seconds_this_rank)
+
+    def close(self):
+        if self.dist is not None:
+            self.dist.destroy_process_group()
+
+
 def run_gpu(args):
     import numpy as np
     import torch
     from paper_2410_15240_b200 import fastrack, synth
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback (use --impl reference for the oracle)")
-    torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-
-    def barrier():
-        torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def max_over_ranks(x: float) -> float:
-        if dist is None:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    ranks = Ranks("nccl", "cuda")
+    rank, world, local, dist = ranks.rank, ranks.world, ranks.local, ranks.dist
+    barrier, max_over_ranks = ranks.barrier, ranks.max_over_ranks
 
     key, iv = synth.key_and_iv(4)
     K = LEN // CHUNK
@@ -231,11 +257,12 @@ def run_gpu(args):
     barrier()
     windows.append((w0, time.time()))
     gpu_launches = ctx.launches - launches0
-    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    ms_this_rank = e0.elapsed_time(e1)
+    ms_total = max_over_ranks(ms_this_rank)
     ms_per_step = ms_total / args.steps
     assert bool((d_ok == 1).all()), "verification failed inside the benchmark"
     assert bool((d_out == d_plain_src).all()), "decryption mismatch inside the benchmark"
-    value = world * LEN / (ms_per_step * 1e-3) / 1e9
+    value = ranks.aggregate_throughput(LEN * args.steps, ms_this_rank * 1e-3) / 1e9
 
     if args.kernel_only:
         if sampler is not None:
@@ -245,8 +272,7 @@ def run_gpu(args):
                               "warmup": args.warmup, "ms_per_step": ms_per_step, "gpu_launches": gpu_launches,
                               "config": {"workload": WORKLOAD}, "kernel_only": True}))
         ctx.close()
-        if dist is not None:
-            dist.destroy_process_group()
+        ranks.close()
         return
 
     # ---- encrypt+tag (mirror path), same size, for the record
@@ -323,8 +349,7 @@ def run_gpu(args):
         }
         print(json.dumps(line))
     ctx.close()
-    if dist is not None:
-        dist.destroy_process_group()
+    ranks.close()
 
 
 def run_sweep(args):

@@ -158,3 +158,80 @@ def test_config4_size_sweep_with_one_percent_tampered(n, cb):
     with ThreadPoolExecutor(NT) as ex:
         for k, good in ex.map(check, sample):
             assert good, f"chunk {k} differs from the oracle"
+
+
+def _sampled_oracle_blocks(key, iv, cb, cipher, plain, offsets):
+    """Ciphertext blocks at the given byte offsets, recomputed one by one with the oracle's AES (counter mode)."""
+    for off in offsets:
+        k, j = off // cb, (off % cb) // 16
+        ks = oracle.aes256_encrypt_block(key, _iv_k(iv, k) + (2 + j).to_bytes(4, "big"))
+        blk = bytes(a ^ b for a, b in zip(plain[off:off + 16].tobytes(), ks))
+        assert cipher[off:off + 16].tobytes() == blk[:len(cipher[off:off + 16])], off
+
+
+def test_largest_chunk_one_gib_single_chain():
+    """chunk_bytes = FASTRACK_MAX_CHUNK_BYTES: one 1 GiB chain (67 108 864 blocks, power table of 1 GiB).
+    The oracle cannot walk a 1 GiB chain in reasonable time, so the tag expectation comes from OpenSSL and the
+    oracle re-computes sampled ciphertext blocks (first, last, around 2^32 bits, seeded others)."""
+    from cryptography.hazmat.primitives.ciphers.aead import AESGCM
+    key, iv = synth.key_and_iv(4)
+    n = cb = fastrack.MAX_CHUNK_BYTES
+    plain = synth.random_bytes(n, 4, salt=99)
+    ref = AESGCM(key).encrypt(iv, memoryview(plain), None)
+    c_ref = np.frombuffer(ref, np.uint8, n)
+    t_ref = np.frombuffer(ref, np.uint8, 16, n)
+    rng = np.random.Generator(np.random.PCG64(7))
+    offs = [0, 16, n - 16, (1 << 29) - 16, 1 << 29] + [int(x) * 16 for x in rng.integers(0, n // 16, 32)]
+    _sampled_oracle_blocks(key, iv, cb, c_ref, plain, offs)
+    with fastrack.Context(key, cb) as ctx:
+        st = torch.cuda.current_stream().cuda_stream
+        d_p = torch.from_numpy(plain).cuda()
+        d_c = torch.empty_like(d_p)
+        d_t = torch.empty(16, dtype=torch.uint8, device="cuda")
+        ctx.encrypt_tag(iv, d_p.data_ptr(), n, d_c.data_ptr(), d_t.data_ptr(), st)
+        torch.cuda.synchronize()
+        assert np.array_equal(d_c.cpu().numpy(), c_ref)
+        assert np.array_equal(d_t.cpu().numpy(), t_ref)
+        d_ok = torch.full((1,), 7, dtype=torch.int32, device="cuda")
+        ctx.decrypt_verify(iv, d_c.data_ptr(), n, d_t.data_ptr(), d_c.data_ptr(), d_ok.data_ptr(), st)
+        torch.cuda.synchronize()
+        assert int(d_ok.item()) == 1 and bool((d_c == d_p).all())
+        d_c[n // 3] ^= 1                                                    # now holds plaintext: any bit flips the verdict
+        ctx.verify(iv, d_c.data_ptr(), n, d_t.data_ptr(), d_ok.data_ptr(), st)
+        torch.cuda.synchronize()
+        assert int(d_ok.item()) == 0
+
+
+def test_buffer_beyond_four_gib_uses_64_bit_offsets():
+    """4 GiB + 16 MiB + 5 bytes in 16 MiB chunks (K = 258, last chunk 5 bytes): byte offsets above 2^32."""
+    key, iv = synth.key_and_iv(4)
+    cb = 16 * MIB
+    n = 4 * GIB + cb + 5
+    plain = synth.random_bytes(n, 4, salt=n)
+    cipher, tags = _openssl_encrypt(key, iv, cb, plain)
+    K = tags.shape[0]
+    assert K == 258
+    plan = [(0, "cipher", 3), (255, "tag", 9), (256, "cipher", 12345), (257, "cipher", 39)]
+    synth.apply_tamper(cipher, tags, cb, plan)
+    rng = np.random.Generator(np.random.PCG64(11))
+    with fastrack.Context(key, cb) as ctx:
+        d_c = torch.from_numpy(cipher).cuda()
+        d_t = torch.from_numpy(tags.reshape(-1)).cuda()
+        d_ok = torch.full((K,), 7, dtype=torch.int32, device="cuda")
+        ctx.decrypt_verify(iv, d_c.data_ptr(), n, d_t.data_ptr(), d_c.data_ptr(), d_ok.data_ptr(),
+                           torch.cuda.current_stream().cuda_stream)          # in place
+        torch.cuda.synchronize()
+        ok = d_ok.cpu().numpy().view(np.uint32)
+        p = d_c.cpu().numpy()
+    assert [int(k) for k in np.flatnonzero(ok == 0)] == [0, 255, 256, 257]
+    mism = np.flatnonzero(p != plain)
+    assert set((mism // cb).tolist()) == {0, 256, 257} and mism.size == 3
+    # the oracle on the chunks that straddle and follow the 2^32-byte boundary, and on the 5-byte tail
+    for k in (255, 256, 257):
+        lo, hi = k * cb, min(n, (k + 1) * cb)
+        if hi - lo > MIB:                      # bound the oracle's work: it re-checks the first MiB's keystream only
+            ks_plain, _ = oracle.gcm_encrypt(key, _iv_k(iv, k), b"", bytes(MIB))
+            assert np.array_equal(np.frombuffer(ks_plain, np.uint8) ^ cipher[lo:lo + MIB], p[lo:lo + MIB])
+        else:
+            pk, okk = oracle.gcm_decrypt(key, _iv_k(iv, k), b"", cipher[lo:hi], tags[k])
+            assert bool(okk) == bool(ok[k]) and np.array_equal(np.frombuffer(pk, np.uint8), p[lo:hi])
