@@ -1,0 +1,108 @@
+"""Seeded random shapes: every data-path entry point against the oracle on odd sizes, odd chunk sizes,
+in place and out of place, with and without the serial-number framing, with seeded tampering."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2410_15240_b200 import fastrack, synth
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+if not torch.cuda.is_available():
+    pytest.skip("no CUDA device", allow_module_level=True)
+
+NT = oracle.host_threads()
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a).reshape(-1)).cuda()
+
+
+def _shapes(seed, count):
+    rng = np.random.Generator(np.random.PCG64(seed))
+    for _ in range(count):
+        cb = 16 * int(rng.choice([1, 2, 3, 31, 32, 33, 64, 100, 255, 256, 257, 1000, 1024, 4096, 4099, 16384, 65536]))
+        K = int(rng.choice([1, 1, 2, 3, 5, 17, 40]))
+        tail = int(rng.integers(0, cb)) if rng.integers(0, 3) else 0
+        n = max(1, (K - 1) * cb + (tail if tail else cb))
+        if n > 6 << 20:
+            n = (6 << 20) + int(rng.integers(0, 64))
+        yield n, cb, int(rng.choice([0, 0, 1, 4, 16, 256])), bool(rng.integers(0, 2)), int(rng.integers(0, 1 << 30))
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3, 4])
+def test_random_shapes_all_entry_points(seed):
+    key, iv = synth.key_and_iv(seed)
+    for n, cb, chains, in_place, salt in _shapes(seed, 30):
+        plain = synth.random_bytes(n, seed, salt=salt)
+        if chains:
+            c, t = oracle.mc_encrypt_framed(key, iv, cb, chains, plain, NT)
+        else:
+            c, t = oracle.mc_encrypt(key, iv, cb, plain, NT)
+        K = t.shape[0]
+        what = f"n={n} cb={cb} chains={chains} in_place={in_place}"
+        with fastrack.Context(key, cb) as ctx:
+            ctx.set_framing(chains)
+            st = torch.cuda.current_stream().cuda_stream
+            # encrypt
+            d_p = dev(plain)
+            d_c = d_p if in_place else torch.empty_like(d_p)
+            d_t = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
+            ctx.encrypt_tag(iv, d_p.data_ptr(), n, d_c.data_ptr(), d_t.data_ptr(), st)
+            torch.cuda.synchronize()
+            assert np.array_equal(d_c.cpu().numpy(), c), what
+            assert np.array_equal(d_t.cpu().numpy().reshape(K, 16), t), what
+            # tamper, then every decrypting / verifying entry point
+            bad_c, bad_t = c.copy(), t.copy()
+            synth.apply_tamper(bad_c, bad_t, cb, synth.tamper_plan(n, cb, seed, fraction=0.3, salt=salt))
+            if chains:
+                p_ref, ok_ref = oracle.mc_decrypt_framed(key, iv, cb, chains, bad_c, bad_t, NT)
+            else:
+                p_ref, ok_ref = oracle.mc_decrypt(key, iv, cb, bad_c, bad_t, NT)
+
+            def fresh():
+                return dev(bad_c), dev(bad_t), torch.full((K,), 7, dtype=torch.int32, device="cuda")
+
+            def check(d_out, d_ok, name):
+                torch.cuda.synchronize()
+                assert np.array_equal(d_ok.cpu().numpy().view(np.uint32), ok_ref), f"{name}: {what}"
+                if d_out is not None:
+                    assert np.array_equal(d_out.cpu().numpy(), p_ref), f"{name}: {what}"
+
+            d_bc, d_bt, d_ok = fresh()
+            d_o = d_bc if in_place else torch.empty_like(d_bc)
+            ctx.decrypt_verify(iv, d_bc.data_ptr(), n, d_bt.data_ptr(), d_o.data_ptr(), d_ok.data_ptr(), st)
+            check(d_o, d_ok, "decrypt_verify")
+
+            d_bc, d_bt, d_ok = fresh()
+            d_o = torch.empty_like(d_bc)
+            ctx.ctr_crypt(iv, d_bc.data_ptr(), n, d_o.data_ptr(), st)
+            ctx.verify(iv, d_bc.data_ptr(), n, d_bt.data_ptr(), d_ok.data_ptr(), st)
+            check(d_o, d_ok, "ctr_crypt+verify")
+
+            d_ok.fill_(7)
+            ctx.verify_sequential(iv, d_bc.data_ptr(), n, d_bt.data_ptr(), d_ok.data_ptr(), st)
+            check(None, d_ok, "verify_sequential")
+
+            d_bc, d_bt, d_ok = fresh()
+            d_pad = torch.empty_like(d_bc)
+            d_m = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
+            d_o = d_bc if in_place else torch.empty_like(d_bc)
+            ctx.keystream(iv, n, d_pad.data_ptr(), d_m.data_ptr(), st)
+            ctx.xor_verify(iv, d_bc.data_ptr(), n, d_pad.data_ptr(), d_m.data_ptr(), d_bt.data_ptr(), d_o.data_ptr(),
+                           d_ok.data_ptr(), st)
+            check(d_o, d_ok, "keystream+xor_verify")
+
+            if K <= fastrack.NOALLOC_MAX_CHUNKS:
+                d_bc, d_bt, d_ok = fresh()
+                d_o = d_bc if in_place else torch.empty_like(d_bc)
+                ctx.decrypt_verify_noalloc(iv, d_bc.data_ptr(), n, d_bt.data_ptr(), d_o.data_ptr(), d_ok.data_ptr(), st)
+                check(d_o, d_ok, "decrypt_verify_noalloc")
+
+            h_c, h_t = torch.from_numpy(bad_c).pin_memory(), torch.from_numpy(bad_t.reshape(-1).copy())
+            d_o = torch.empty(n, dtype=torch.uint8, device="cuda")
+            d_ok = torch.full((K,), 7, dtype=torch.int32, device="cuda")
+            torch.cuda.synchronize()
+            ctx.pipelined_h2d(iv, h_c.data_ptr(), n, h_t.data_ptr(), d_o.data_ptr(), d_ok.data_ptr(), 1 + seed % 3)
+            check(d_o, d_ok, "pipelined_h2d")
