@@ -95,7 +95,7 @@ __global__ void __launch_bounds__(FR_THREADS, 1) fr_crypt_kernel(const __grid_co
     L.lane4 |= after_barrier;
     L.qe |= after_barrier;
     L.qo |= after_barrier;
-    if ((uint32_t)__cvta_generic_to_shared(sm) == FR_SMEM_ABS_BASE) fr_crypt_body<MODE, true>(P, sm, L);
+    if ((uint32_t)__cvta_generic_to_shared(sm) == FR_SMEM_ABS_BASE && !P.generic_smem) fr_crypt_body<MODE, true>(P, sm, L);
     else fr_crypt_body<MODE, false>(P, sm, L);
 }
 
@@ -175,6 +175,7 @@ struct fastrack_ctx {
     uint32_t aad_mod;             // 0 = no AAD, else chains per sample of the serial-number framing
     uint32_t seg_rows_override;   // 0 = automatic (FASTRACK_SEG_ROWS, for experiments)
     size_t stage_bytes_override;  // 0 = automatic (FASTRACK_STAGE_BYTES, for experiments)
+    uint32_t generic_smem;        // FASTRACK_GENERIC_SMEM=1: exercise the portable addressing path (tests)
 };
 
 #define FR_CUDA(ctx, call)                                              \
@@ -219,6 +220,7 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, ctx->device);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return fail(FASTRACK_ERR_CUDA); }
     if (const char* env = getenv("FASTRACK_SEG_ROWS")) ctx->seg_rows_override = (uint32_t)strtoul(env, nullptr, 10);
+    if (const char* env = getenv("FASTRACK_GENERIC_SMEM")) ctx->generic_smem = (uint32_t)(strtoul(env, nullptr, 10) != 0);
     if (const char* env = getenv("FASTRACK_STAGE_BYTES")) ctx->stage_bytes_override = (size_t)strtoull(env, nullptr, 10);
 
     // key material on the host: S-box, Te0, round keys, H, byte tables of H^32
@@ -437,6 +439,7 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
     P.iv_ctr = load_be32(iv_base + 8) + (uint32_t)first_chunk;
     P.first_chunk = (uint32_t)first_chunk;
     P.aad_mod = ctx->aad_mod;
+    P.generic_smem = ctx->generic_smem;
     P.len = len;
     P.chunk_bytes = ctx->chunk_bytes;
     const size_t n_chunks = (len + ctx->chunk_bytes - 1) / ctx->chunk_bytes;
@@ -844,6 +847,7 @@ extern "C" int fastrack_decrypt_verify_noalloc(fastrack_ctx* ctx, const uint8_t 
     P.iv_w1 = load_le32(iv_base + 4);
     P.iv_ctr = load_be32(iv_base + 8);
     P.aad_mod = ctx->aad_mod;
+    P.generic_smem = ctx->generic_smem;
     P.len = len;
     P.chunk_bytes = ctx->chunk_bytes;
     P.n_chunks = (uint32_t)K;

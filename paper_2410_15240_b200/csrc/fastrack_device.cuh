@@ -50,6 +50,7 @@ struct FrParams {
     uint32_t segs_per_chunk;   // segments of a full-size chunk
     uint32_t n_chunks;         // chunks in this launch
     uint32_t n_items;          // n_chunks * segs_per_chunk
+    uint32_t generic_smem;     // 1: use the portable shared-memory addressing even where the absolute form would do
     uint32_t aad_mod;          // 0: no AAD; n: chunk k authenticates the one byte (first chunk index + k) mod n as AAD
     uint64_t len;              // bytes in this launch
     uint64_t chunk_bytes;

@@ -106,3 +106,37 @@ def test_random_shapes_all_entry_points(seed):
             torch.cuda.synchronize()
             ctx.pipelined_h2d(iv, h_c.data_ptr(), n, h_t.data_ptr(), d_o.data_ptr(), d_ok.data_ptr(), 1 + seed % 3)
             check(d_o, d_ok, "pipelined_h2d")
+
+
+def test_portable_shared_addressing_path(monkeypatch):
+    """The kernel puts table base addresses into load immediates when the shared window starts where it
+    expects, and falls back to ordinary pointer arithmetic otherwise.  FASTRACK_GENERIC_SMEM=1 forces the
+    fallback so that it is exercised on hardware where the fast form applies."""
+    monkeypatch.setenv("FASTRACK_GENERIC_SMEM", "1")
+    key, iv = synth.key_and_iv(7)
+    for n, cb, chains in [(1, 16, 0), (70001, 4096, 0), ((1 << 20) + 33, 65536, 16), ((5 << 20) + 7, 1 << 20, 0)]:
+        plain = synth.random_bytes(n, 7, salt=n)
+        c, t = (oracle.mc_encrypt_framed(key, iv, cb, chains, plain, NT) if chains else oracle.mc_encrypt(key, iv, cb, plain, NT))
+        K = t.shape[0]
+        bad_c, bad_t = c.copy(), t.copy()
+        synth.apply_tamper(bad_c, bad_t, cb, synth.tamper_plan(n, cb, 7, fraction=0.3, salt=n))
+        p_ref, ok_ref = (oracle.mc_decrypt_framed(key, iv, cb, chains, bad_c, bad_t, NT) if chains
+                         else oracle.mc_decrypt(key, iv, cb, bad_c, bad_t, NT))
+        with fastrack.Context(key, cb) as ctx:                      # the variable is read at context creation
+            ctx.set_framing(chains)
+            st = torch.cuda.current_stream().cuda_stream
+            d_p = dev(plain)
+            d_c = torch.empty_like(d_p)
+            d_t = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
+            ctx.encrypt_tag(iv, d_p.data_ptr(), n, d_c.data_ptr(), d_t.data_ptr(), st)
+            d_bc, d_bt = dev(bad_c), dev(bad_t)
+            d_o = torch.empty_like(d_bc)
+            d_ok = torch.full((K,), 7, dtype=torch.int32, device="cuda")
+            d_ok2 = torch.full((K,), 7, dtype=torch.int32, device="cuda")
+            ctx.decrypt_verify(iv, d_bc.data_ptr(), n, d_bt.data_ptr(), d_o.data_ptr(), d_ok.data_ptr(), st)
+            ctx.verify(iv, d_bc.data_ptr(), n, d_bt.data_ptr(), d_ok2.data_ptr(), st)
+            torch.cuda.synchronize()
+            assert np.array_equal(d_c.cpu().numpy(), c) and np.array_equal(d_t.cpu().numpy().reshape(K, 16), t)
+            assert np.array_equal(d_o.cpu().numpy(), p_ref)
+            assert np.array_equal(d_ok.cpu().numpy().view(np.uint32), ok_ref)
+            assert np.array_equal(d_ok2.cpu().numpy().view(np.uint32), ok_ref)
