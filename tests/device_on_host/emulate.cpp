@@ -1,0 +1,202 @@
+// emulate.cpp -- TEST INFRASTRUCTURE ONLY: the per-lane device functions of the CUDA library
+// (paper_2410_15240_b200/csrc/fastrack_device.cuh) compiled as plain C++ and driven lane by lane on the host,
+// so that the CPU-only test run can compare the kernels' arithmetic (table layouts, lane rotations, counter
+// sharing, Horner exponents, ragged tails, framing, every pass mode) with the oracle before anything reaches
+// a GPU.  It stands in for the few lines of kernel code that are not in that header: shared memory is a host
+// array, the warp XOR tree and the per-chunk accumulator are plain loops.  It is built by
+// tests/test_device_code_on_host.py into a temporary directory, is never shipped, and nothing in the product
+// can reach it (the product has no CPU data path).
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <algorithm>
+#include <vector>
+
+// ---- what the device header needs from CUDA, as plain C++ ----
+#define __device__
+#define __forceinline__ inline
+struct uint4 { uint32_t x, y, z, w; };
+static inline uint4 make_uint4(uint32_t a, uint32_t b, uint32_t c, uint32_t d) { return uint4{a, b, c, d}; }
+
+// PTX prmt.b32, generic mode: nibble bits 0-2 pick a byte of {a, b}, bit 3 replicates that byte's sign bit.
+static inline uint32_t host_prmt(uint32_t a, uint32_t b, uint32_t s)
+{
+    uint8_t src[8];
+    for (int i = 0; i < 4; i++) { src[i] = (uint8_t)(a >> (8 * i)); src[4 + i] = (uint8_t)(b >> (8 * i)); }
+    uint32_t r = 0;
+    for (int i = 0; i < 4; i++) {
+        const uint32_t n = (s >> (4 * i)) & 0xf;
+        uint8_t v = src[n & 7];
+        if (n & 8) v = (v & 0x80) ? 0xff : 0x00;
+        r |= (uint32_t)v << (8 * i);
+    }
+    return r;
+}
+#define FR_PRMT(a, b, s) host_prmt((a), (b), (s))
+
+static inline uint32_t __brev(uint32_t x)
+{
+    uint32_t r = 0;
+    for (int i = 0; i < 32; i++) r |= ((x >> i) & 1u) << (31 - i);
+    return r;
+}
+
+#include "../../paper_2410_15240_b200/csrc/fastrack_device.cuh"
+#include "../../paper_2410_15240_b200/csrc/fastrack_keysetup.h"
+using namespace fr_host;
+
+namespace {
+
+struct Setup {
+    FrParams P;
+    uint32_t te0[256];
+    uint8_t h[16];
+    std::vector<uint8_t> gh_tab;     // byte tables of H^32
+    std::vector<uint4> pow;          // powers of H
+    std::vector<char> sm;            // the "shared memory" image
+};
+
+// The same derivation fastrack_ctx_create performs (host part) plus the power table and the shared-memory fill.
+void setup(Setup& S, const uint8_t key[32], size_t cb)
+{
+    memset(&S.P, 0, sizeof S.P);
+    uint8_t sbox[256];
+    make_sbox(sbox);
+    for (int v = 0; v < 256; v++) {
+        const uint8_t s1 = sbox[v], s2 = xtime(s1), s3 = (uint8_t)(s2 ^ s1);
+        S.te0[v] = (uint32_t)s2 | ((uint32_t)s1 << 8) | ((uint32_t)s1 << 16) | ((uint32_t)s3 << 24);
+    }
+    expand_key(key, sbox, S.P.rk);
+    const uint8_t zero[16] = {0};
+    encrypt_block_host(S.P.rk, S.te0, sbox, zero, S.h);
+    Gf128 G = gf_load(S.h);
+    for (int i = 0; i < 5; i++) G = gf_mul(G, G);
+    S.gh_tab.assign(65536, 0);
+    for (int p = 0; p < 16; p++) {
+        Gf128 basis[8];
+        for (int b = 0; b < 8; b++) {
+            uint8_t blk[16] = {0};
+            blk[p] = (uint8_t)(1u << b);
+            basis[b] = gf_mul(gf_load(blk), G);
+        }
+        for (int v = 0; v < 256; v++) {
+            Gf128 acc = {0, 0};
+            for (int b = 0; b < 8; b++)
+                if (v & (1 << b)) { acc.hi ^= basis[b].hi; acc.lo ^= basis[b].lo; }
+            gf_store(acc, &S.gh_tab[(size_t)v * 256 + (size_t)p * 16]);
+        }
+    }
+    const size_t npow = cb / 16 + 66;
+    S.pow.assign(npow, uint4{0, 0, 0, 0});
+    uint8_t seed[32] = {0};
+    seed[0] = 0x80;
+    memcpy(seed + 16, S.h, 16);
+    memcpy(S.pow.data(), seed, 32);
+    for (size_t half = 1; half + 1 < npow; half *= 2)                       // fr_pow_double_kernel, pass by pass
+        for (size_t i = half + 1; i <= std::min(2 * half, npow - 1); i++) S.pow[i] = fr_gf128_mul(S.pow[i - half], S.pow[half]);
+    S.sm.assign(FR_SMEM_BYTES, 0);
+    for (uint32_t tid = 0; tid < 1024; tid++) fr_build_smem<1024>(S.sm.data(), tid, S.te0, (const uint4*)S.gh_tab.data());
+    S.P.te0 = S.te0;
+    S.P.gh_tab = (const uint4*)S.gh_tab.data();
+    S.P.pow = S.pow.data();
+}
+
+uint4 length_term(const Setup& S, uint64_t bytes, uint32_t aad_mod)
+{
+    uint8_t blk[16] = {0}, o[16];
+    const uint64_t bits = bytes * 8;
+    if (aad_mod) blk[7] = 8;
+    for (int i = 0; i < 8; i++) blk[8 + i] = (uint8_t)(bits >> (56 - 8 * i));
+    gf_store(gf_mul(gf_load(blk), gf_load(S.h)), o);
+    uint4 r;
+    memcpy(&r, o, 16);
+    return r;
+}
+
+template <int MODE>
+void run_pass(Setup& S, uint32_t n_chunks, std::vector<uint4>& acc)
+{
+    for (uint32_t item = 0; item < S.P.n_items; item++) {
+        const uint32_t kk = item / S.P.segs_per_chunk, s = item - kk * S.P.segs_per_chunk;
+        if (s >= fr_chunk_segs(S.P, kk)) continue;
+        for (uint32_t lane = 0; lane < 32; lane++) {                        // the warp, one lane after the other
+            const FrLane L = fr_make_lane(lane);
+            acc[kk] = fr_xor4(acc[kk], fr_process_segment_lane<MODE, false>(S.P, S.sm.data(), L, lane, kk, s));
+        }
+    }
+    (void)n_chunks;
+}
+
+}  // namespace
+
+// One pass of mode `mode` (FrMode) over a buffer; seg_rows as the host planner would choose it (any value >= 1).
+extern "C" int emu_pass(int mode, const uint8_t* key, const uint8_t* iv_base, size_t cb, const uint8_t* in, size_t len,
+                        uint8_t* out, const uint8_t* pad, uint8_t* mask, const uint8_t* tags_in, uint8_t* tags_out,
+                        uint32_t* ok, uint32_t seg_rows, uint32_t first_chunk, uint32_t aad_mod)
+{
+    Setup S;
+    setup(S, key, cb);
+    FrParams& P = S.P;
+    auto be32 = [](const uint8_t* p) { return ((uint32_t)p[0] << 24) | ((uint32_t)p[1] << 16) | ((uint32_t)p[2] << 8) | p[3]; };
+    auto le32 = [](const uint8_t* p) { return ((uint32_t)p[3] << 24) | ((uint32_t)p[2] << 16) | ((uint32_t)p[1] << 8) | p[0]; };
+    P.iv_w0 = le32(iv_base);
+    P.iv_w1 = le32(iv_base + 4);
+    P.iv_ctr = be32(iv_base + 8) + first_chunk;
+    P.first_chunk = first_chunk;
+    P.aad_mod = aad_mod;
+    P.len = len;
+    P.chunk_bytes = cb;
+    const size_t n_chunks = (len + cb - 1) / cb;
+    const size_t first_len = std::min(len, cb);
+    const size_t rows_ref = ((first_len + 15) / 16 + 2 + 31) / 32;
+    P.seg_rows = seg_rows ? seg_rows : 8;
+    P.segs_per_chunk = (uint32_t)((rows_ref + P.seg_rows - 1) / P.seg_rows);
+    P.n_chunks = (uint32_t)n_chunks;
+    P.n_items = (uint32_t)(P.segs_per_chunk * n_chunks);
+    P.lenh_full = length_term(S, first_len, aad_mod);
+    P.lenh_last = length_term(S, len - (n_chunks - 1) * cb, aad_mod);
+    P.in = in;
+    P.out = out;
+    P.pad = pad;
+    P.mask = (uint4*)mask;
+    std::vector<uint4> acc(n_chunks, uint4{0, 0, 0, 0});
+    switch (mode) {
+        case FR_MODE_DEC: run_pass<FR_MODE_DEC>(S, P.n_chunks, acc); break;
+        case FR_MODE_ENC: run_pass<FR_MODE_ENC>(S, P.n_chunks, acc); break;
+        case FR_MODE_CTR: run_pass<FR_MODE_CTR>(S, P.n_chunks, acc); return 0;
+        case FR_MODE_VERIFY: run_pass<FR_MODE_VERIFY>(S, P.n_chunks, acc); break;
+        case FR_MODE_PADGEN: run_pass<FR_MODE_PADGEN>(S, P.n_chunks, acc); return 0;
+        case FR_MODE_PADDEC: run_pass<FR_MODE_PADDEC>(S, P.n_chunks, acc); break;
+        default: return -1;
+    }
+    for (uint32_t kk = 0; kk < n_chunks; kk++) {                            // the finishing warp's part
+        const uint4 tag = fr_xor4(acc[kk], (kk + 1 == n_chunks) ? P.lenh_last : P.lenh_full);
+        if (mode == FR_MODE_ENC) memcpy(tags_out + 16 * kk, &tag, 16);
+        else ok[kk] = memcmp(&tag, tags_in + 16 * kk, 16) == 0;
+    }
+    return 0;
+}
+
+extern "C" void emu_gf128_mul_device(const uint8_t* a, const uint8_t* b, uint8_t* o)
+{
+    uint4 x, y;
+    memcpy(&x, a, 16);
+    memcpy(&y, b, 16);
+    const uint4 z = fr_gf128_mul(x, y);
+    memcpy(o, &z, 16);
+}
+
+extern "C" void emu_gf128_mul_keysetup(const uint8_t* a, const uint8_t* b, uint8_t* o)
+{
+    gf_store(gf_mul(gf_load(a), gf_load(b)), o);
+}
+
+// Round keys (240 bytes, as the little-endian words the kernel receives) and H from the host-side key set-up.
+extern "C" void emu_keysetup(const uint8_t* key, uint8_t* round_keys, uint8_t* h)
+{
+    Setup S;
+    setup(S, key, 16);
+    memcpy(round_keys, S.P.rk, 240);
+    memcpy(h, S.h, 16);
+}

@@ -1,0 +1,128 @@
+"""The CUDA library's per-lane device code, compiled as plain C++ and run lane by lane on the host, against the
+oracle (tests/device_on_host/emulate.cpp explains what is and is not emulated).  This is test infrastructure:
+it lets the CPU-only run check the kernels' arithmetic; the GPU tests check the real thing."""
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+import pytest
+
+import oracle
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+DEC, ENC, CTR, VERIFY, PADGEN, PADDEC = range(6)
+
+
+@pytest.fixture(scope="module")
+def emu(tmp_path_factory):
+    so = tmp_path_factory.mktemp("device_on_host") / "libemulate.so"
+    subprocess.check_call(["g++", "-O2", "-std=c++17", "-shared", "-fPIC", "-o", str(so),
+                           os.path.join(ROOT, "tests", "device_on_host", "emulate.cpp")])
+    lib = ctypes.CDLL(str(so))
+    V, Z, U = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_uint32
+    lib.emu_pass.argtypes = [ctypes.c_int, V, V, Z, V, Z, V, V, V, V, V, V, U, U, U]
+    lib.emu_pass.restype = ctypes.c_int
+    for name in ("emu_gf128_mul_device", "emu_gf128_mul_keysetup"):
+        getattr(lib, name).argtypes = [ctypes.c_char_p] * 3
+    lib.emu_keysetup.argtypes = [ctypes.c_char_p, V, V]
+    return lib
+
+
+def run(lib, mode, key, iv, cb, data, n, pad=None, mask=None, tags=None, seg=8, first=0, aad=0):
+    K = (n + cb - 1) // cb
+    k = np.frombuffer(key, np.uint8).copy()
+    v = np.frombuffer(iv, np.uint8).copy()
+    src = np.ascontiguousarray(data, np.uint8) if data is not None else np.zeros(n, np.uint8)
+    out = np.full(n + 64, 0xA5, np.uint8)
+    tin = np.ascontiguousarray(tags, np.uint8) if tags is not None else np.zeros((K, 16), np.uint8)
+    tout = np.zeros((K, 16), np.uint8)
+    ok = np.full(K, 7, np.uint32)
+    pad_a = np.ascontiguousarray(pad, np.uint8) if pad is not None else np.zeros(n, np.uint8)
+    mask_a = np.ascontiguousarray(mask, np.uint8) if mask is not None else np.zeros((K, 16), np.uint8)
+    if mode == VERIFY:
+        out[:n] = src                                   # the pass does not store; keep the guard check meaningful
+    rc = lib.emu_pass(mode, k.ctypes.data, v.ctypes.data, cb, src.ctypes.data, n, out.ctypes.data, pad_a.ctypes.data,
+                      mask_a.ctypes.data, tin.ctypes.data, tout.ctypes.data, ok.ctypes.data, seg, first, aad)
+    assert rc == 0 and (out[n:] == 0xA5).all()
+    return out[:n], tout, ok, mask_a
+
+
+def test_key_setup_matches_oracle(emu):
+    rng = np.random.default_rng(1)
+    for _ in range(8):
+        key = rng.bytes(32)
+        rk = np.zeros(240, np.uint8)
+        h = np.zeros(16, np.uint8)
+        emu.emu_keysetup(key, rk.ctypes.data, h.ctypes.data)
+        assert rk.tobytes() == oracle.aes256_key_expand(key)
+        assert h.tobytes() == oracle.hash_subkey(key)
+
+
+def test_both_gf128_products_match_oracle(emu):
+    rng = np.random.default_rng(2)
+    cases = [(rng.bytes(16), rng.bytes(16)) for _ in range(2000)] + [(bytes([0xFF] * 16),) * 2]
+    for i in range(0, 128, 3):
+        for j in (0, 1, 31, 32, 33, 63, 64, 65, 96, 127):
+            x, y = bytearray(16), bytearray(16)
+            x[i // 8] |= 1 << (7 - i % 8)
+            y[j // 8] |= 1 << (7 - j % 8)
+            cases.append((bytes(x), bytes(y)))
+    for a, b in cases:
+        ref = oracle.gf128_mul(a, b)
+        for fn in (emu.emu_gf128_mul_device, emu.emu_gf128_mul_keysetup):
+            o = ctypes.create_string_buffer(16)
+            fn(a, b, o)
+            assert o.raw == ref
+
+
+SHAPES = [(1, 16, 8), (16, 16, 8), (15, 64, 2), (17, 64, 4), (33, 32, 8), (480, 480, 8), (512, 512, 1), (513, 1024, 8),
+          (1000, 256, 2), (4096, 1024, 8), (5000, 2048, 4), (70000, 16384, 8), (70001, 65536, 16), (200000, 65536, 24),
+          (100, 65536, 8), (300000, 100000 // 16 * 16, 3)]
+
+
+@pytest.mark.parametrize("n,cb,seg", SHAPES)
+@pytest.mark.parametrize("aad", [0, 16])
+def test_fused_and_split_passes_match_oracle(emu, n, cb, seg, aad):
+    rng = np.random.default_rng(n + cb + aad)
+    key, iv = rng.bytes(32), rng.bytes(8) + bytes([0xFF, 0xFF, 0xFF, 0xFE])
+    p = np.frombuffer(rng.bytes(n), np.uint8)
+    if aad:
+        c_ref, t_ref = oracle.mc_encrypt_framed(key, iv, cb, aad, p, 4)
+    else:
+        c_ref, t_ref = oracle.mc_encrypt(key, iv, cb, p, 4)
+    K = t_ref.shape[0]
+    c, t, _, _ = run(emu, ENC, key, iv, cb, p, n, seg=seg, aad=aad)
+    assert np.array_equal(c, c_ref) and np.array_equal(t, t_ref)
+
+    bad_c, bad_t = c_ref.copy(), t_ref.copy()
+    bad_c[n // 2] ^= 0x10
+    if K > 1:
+        bad_t[K - 1, 3] ^= 4
+    if aad:
+        p_ref, ok_ref = oracle.mc_decrypt_framed(key, iv, cb, aad, bad_c, bad_t, 4)
+    else:
+        p_ref, ok_ref = oracle.mc_decrypt(key, iv, cb, bad_c, bad_t, 4)
+    out, _, ok, _ = run(emu, DEC, key, iv, cb, bad_c, n, tags=bad_t, seg=seg, aad=aad)
+    assert np.array_equal(out, p_ref) and np.array_equal(ok, ok_ref)
+
+    out, _, _, _ = run(emu, CTR, key, iv, cb, bad_c, n, seg=seg, aad=aad)
+    assert np.array_equal(out, p_ref)
+    _, _, ok, _ = run(emu, VERIFY, key, iv, cb, bad_c, n, tags=bad_t, seg=seg, aad=aad)
+    assert np.array_equal(ok, ok_ref)
+
+    pad, _, _, mask = run(emu, PADGEN, key, iv, cb, None, n, seg=seg, aad=aad)
+    assert np.array_equal(pad, oracle.mc_encrypt(key, iv, cb, np.zeros(n, np.uint8), 4)[0])
+    out, _, ok, _ = run(emu, PADDEC, key, iv, cb, bad_c, n, pad=pad, mask=mask, tags=bad_t, seg=seg, aad=aad)
+    assert np.array_equal(out, p_ref) and np.array_equal(ok, ok_ref)
+
+
+def test_a_stage_that_starts_at_a_later_chunk(emu):
+    """Pipelined calls launch a pass per stage: IV index and serial number continue from the stage's first chunk."""
+    rng = np.random.default_rng(77)
+    key, iv = rng.bytes(32), rng.bytes(12)
+    cb, n, first, aad = 1024, 1024 * 7 + 100, 5, 3
+    p = np.frombuffer(rng.bytes(cb * first + n), np.uint8)
+    c_ref, t_ref = oracle.mc_encrypt_framed(key, iv, cb, aad, p, 4)
+    c, t, _, _ = run(emu, ENC, key, iv, cb, p[cb * first:], n, seg=8, first=first, aad=aad)
+    assert np.array_equal(c, c_ref[cb * first:]) and np.array_equal(t, t_ref[first:])
