@@ -188,6 +188,13 @@ struct fastrack_ctx {
         }                                                               \
     } while (0)
 
+// Zeroing that the compiler may not drop (key-derived data about to be freed).
+static void secure_zero(void* p, size_t n)
+{
+    volatile uint8_t* q = (volatile uint8_t*)p;
+    for (size_t i = 0; i < n; i++) q[i] = 0;
+}
+
 static int ensure_scratch(fastrack_ctx* ctx, size_t chunks)
 {
     if (chunks <= ctx->scratch_chunks) return FASTRACK_OK;
@@ -289,7 +296,7 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
         if ((e = cudaEventCreateWithFlags(&ctx->pad_ready, cudaEventDisableTiming)) != cudaSuccess) break;
         e = cudaDeviceSynchronize();
     } while (0);
-    memset(tab, 0, 2 * 65536);
+    secure_zero(tab, 2 * 65536);
     free(tab);
     if (e != cudaSuccess) {
         ctx->last_cuda_error = (int)e;
@@ -321,8 +328,7 @@ extern "C" void fastrack_ctx_destroy(fastrack_ctx* ctx)
     if (ctx->tags_ready) cudaEventDestroy(ctx->tags_ready);
     if (ctx->pad_ready) cudaEventDestroy(ctx->pad_ready);
     (void)cudaGetLastError();
-    volatile uint8_t* p = (volatile uint8_t*)ctx;
-    for (size_t i = 0; i < sizeof *ctx; i++) p[i] = 0;
+    secure_zero(ctx, sizeof *ctx);
     delete ctx;
 }
 
