@@ -55,3 +55,53 @@ def test_counter_wraps_inside_last_four_bytes_only():
     for j in (0, 1, 254, 255, 256, 299):
         ctr_block = iv + (2 + j).to_bytes(4, "big")
         assert c[16 * j:16 * j + 16] == oracle.aes256_encrypt_block(key, ctr_block)
+
+
+def test_ghash_is_linear_over_equal_shapes():
+    """GHASH_H(A, C) xor GHASH_H(A', C') xor GHASH_H(A xor A', C xor C') = GHASH_H(0, 0) for equal lengths:
+    the map is affine, the length block being the constant part."""
+    rng = np.random.default_rng(41)
+    h = rng.bytes(16)
+    for la, lc in [(0, 16), (0, 100), (13, 77), (32, 4096)]:
+        a1, a2, c1, c2 = rng.bytes(la), rng.bytes(la), rng.bytes(lc), rng.bytes(lc)
+        ax = bytes(x ^ y for x, y in zip(a1, a2))
+        cx = bytes(x ^ y for x, y in zip(c1, c2))
+        g = [oracle.ghash(h, a1, c1), oracle.ghash(h, a2, c2), oracle.ghash(h, ax, cx), oracle.ghash(h, bytes(la), bytes(lc))]
+        acc = bytes(16)
+        for t in g:
+            acc = bytes(x ^ y for x, y in zip(acc, t))
+        assert acc == bytes(16)
+
+
+def test_ctr_keystream_is_data_independent_and_xor_symmetric():
+    rng = np.random.default_rng(42)
+    key, iv = rng.bytes(32), rng.bytes(12)
+    for n in (1, 16, 33, 1000):
+        p1, p2 = rng.bytes(n), rng.bytes(n)
+        c1, _ = oracle.gcm_encrypt(key, iv, b"", p1)
+        c2, _ = oracle.gcm_encrypt(key, iv, b"", p2)
+        assert bytes(a ^ b for a, b in zip(c1, c2)) == bytes(a ^ b for a, b in zip(p1, p2))
+        ks, _ = oracle.gcm_encrypt(key, iv, b"", bytes(n))
+        assert bytes(a ^ b for a, b in zip(ks, p1)) == c1
+        # one flipped ciphertext bit flips exactly that plaintext bit (and the verdict)
+        bad = bytearray(c1)
+        bad[n // 2] ^= 0x20
+        _, t1 = oracle.gcm_encrypt(key, iv, b"", p1)
+        back, ok = oracle.gcm_decrypt(key, iv, b"", bytes(bad), t1)
+        assert not ok
+        diff = [i for i in range(n) if back[i] != p1[i]]
+        assert diff == [n // 2] and back[n // 2] ^ p1[n // 2] == 0x20
+
+
+def test_tag_of_empty_message_is_len_block_times_h_xor_mask():
+    """No data, no AAD: GHASH is 0 * H = 0 (the length block is all zero), so the tag is E_K(J0) itself."""
+    rng = np.random.default_rng(43)
+    key, iv = rng.bytes(32), rng.bytes(12)
+    _, t = oracle.gcm_encrypt(key, iv, b"", b"")
+    assert t == oracle.aes256_encrypt_block(key, iv + bytes([0, 0, 0, 1]))
+    # one block of zeros as AAD only: tag = (LEN * H) xor E_K(J0) with LEN = BE64(128) || BE64(0)
+    _, t = oracle.gcm_encrypt(key, iv, bytes(16), b"")
+    h = oracle.hash_subkey(key)
+    lenblk = (128).to_bytes(8, "big") + bytes(8)
+    expect = bytes(a ^ b for a, b in zip(oracle.gf128_mul(lenblk, h), oracle.aes256_encrypt_block(key, iv + bytes([0, 0, 0, 1]))))
+    assert t == expect
