@@ -140,3 +140,51 @@ def test_portable_shared_addressing_path(monkeypatch):
             assert np.array_equal(d_o.cpu().numpy(), p_ref)
             assert np.array_equal(d_ok.cpu().numpy().view(np.uint32), ok_ref)
             assert np.array_equal(d_ok2.cpu().numpy().view(np.uint32), ok_ref)
+
+
+def test_one_context_many_mixed_calls_leave_scratch_clean():
+    """200 calls of every kind, sizes going up and down, on ONE context: every call must still be exact,
+    i.e. each pass leaves the per-chunk accumulators and counters (both banks) zeroed for the next one."""
+    key, iv = synth.key_and_iv(9)
+    cb = 8192
+    rng = np.random.Generator(np.random.PCG64(9))
+    sizes = [cb * int(k) + int(t) for k, t in zip(rng.integers(1, 300, 12), rng.integers(0, cb, 12))]
+    cases = []
+    for n in sizes:
+        plain = synth.random_bytes(n, 9, salt=n)
+        c, t = oracle.mc_encrypt(key, iv, cb, plain, NT)
+        synth.apply_tamper(c, t, cb, synth.tamper_plan(n, cb, 9, fraction=0.05, salt=n))
+        p_ref, ok_ref = oracle.mc_decrypt(key, iv, cb, c, t, NT)
+        cases.append((n, dev(c), dev(t), p_ref, ok_ref, dev(plain)))
+    with fastrack.Context(key, cb) as ctx:
+        st = torch.cuda.current_stream().cuda_stream
+        for it in range(200):
+            n, d_c, d_t, p_ref, ok_ref, d_plain = cases[int(rng.integers(0, len(cases)))]
+            K = ok_ref.size
+            kind = int(rng.integers(0, 5))
+            d_o = torch.empty(n, dtype=torch.uint8, device="cuda")
+            d_ok = torch.full((K,), 7, dtype=torch.int32, device="cuda")
+            if kind == 0:
+                ctx.decrypt_verify(iv, d_c.data_ptr(), n, d_t.data_ptr(), d_o.data_ptr(), d_ok.data_ptr(), st)
+            elif kind == 1:
+                ctx.verify(iv, d_c.data_ptr(), n, d_t.data_ptr(), d_ok.data_ptr(), st)
+                d_o = None
+            elif kind == 2:
+                ctx.decrypt_verify_noalloc(iv, d_c.data_ptr(), n, d_t.data_ptr(), d_o.data_ptr(), d_ok.data_ptr(), st)
+            elif kind == 3:
+                d_pad = torch.empty(n, dtype=torch.uint8, device="cuda")
+                d_m = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
+                ctx.keystream(iv, n, d_pad.data_ptr(), d_m.data_ptr(), st)
+                ctx.xor_verify(iv, d_c.data_ptr(), n, d_pad.data_ptr(), d_m.data_ptr(), d_t.data_ptr(), d_o.data_ptr(),
+                               d_ok.data_ptr(), st)
+            else:
+                d_tt = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
+                ctx.encrypt_tag(iv, d_plain.data_ptr(), n, d_o.data_ptr(), d_tt.data_ptr(), st)   # tags unchecked here
+                ctx.decrypt_verify(iv, d_o.data_ptr(), n, d_tt.data_ptr(), d_o.data_ptr(), d_ok.data_ptr(), st)
+                torch.cuda.synchronize()
+                assert bool((d_ok == 1).all()) and bool((d_o == d_plain).all()), f"iteration {it}"
+                continue
+            torch.cuda.synchronize()
+            assert np.array_equal(d_ok.cpu().numpy().view(np.uint32), ok_ref), f"iteration {it} kind {kind}"
+            if d_o is not None:
+                assert np.array_equal(d_o.cpu().numpy(), p_ref), f"iteration {it} kind {kind}"
