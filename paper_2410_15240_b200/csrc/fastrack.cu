@@ -86,6 +86,12 @@ __global__ void __launch_bounds__(FR_THREADS, 1) fr_crypt_kernel(const __grid_co
 {
     extern __shared__ __align__(256) char sm[];
     fr_build_smem<FR_THREADS>(sm, threadIdx.x, P.te0, P.gh_tab);
+    // Programmatic dependent launch: the table build above touches only per-context constants, so it may run
+    // while the previous kernel in the stream is still finishing; everything below waits until that kernel has
+    // completed and its writes are visible (a no-op when the launch carries no such dependency).  Kernels queued
+    // behind this one may be scheduled as soon as SMs free up; they wait at the same point.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;");
     __syncthreads();
     // Lane constants are made to depend on a value the compiler cannot see through and that is produced
     // after the barrier, so that no table load can be scheduled above the barrier.
@@ -176,6 +182,7 @@ struct fastrack_ctx {
     uint32_t seg_rows_override;   // 0 = automatic (FASTRACK_SEG_ROWS, for experiments)
     size_t stage_bytes_override;  // 0 = automatic (FASTRACK_STAGE_BYTES, for experiments)
     uint32_t generic_smem;        // FASTRACK_GENERIC_SMEM=1: exercise the portable addressing path (tests)
+    uint32_t no_overlap_launch;   // FASTRACK_NO_OVERLAP_LAUNCH=1: plain stream-ordered launches (experiments)
 };
 
 #define FR_CUDA(ctx, call)                                              \
@@ -228,6 +235,7 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
     if (e != cudaSuccess) { (void)cudaGetLastError(); return fail(FASTRACK_ERR_CUDA); }
     if (const char* env = getenv("FASTRACK_SEG_ROWS")) ctx->seg_rows_override = (uint32_t)strtoul(env, nullptr, 10);
     if (const char* env = getenv("FASTRACK_GENERIC_SMEM")) ctx->generic_smem = (uint32_t)(strtoul(env, nullptr, 10) != 0);
+    if (const char* env = getenv("FASTRACK_NO_OVERLAP_LAUNCH")) ctx->no_overlap_launch = (uint32_t)(strtoul(env, nullptr, 10) != 0);
     if (const char* env = getenv("FASTRACK_STAGE_BYTES")) ctx->stage_bytes_override = (size_t)strtoull(env, nullptr, 10);
 
     // key material on the host: S-box, Te0, round keys, H, byte tables of H^32
@@ -469,15 +477,31 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
 
     unsigned grid = (unsigned)ctx->num_sms;
     if (P.n_items < grid) grid = P.n_items;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(FR_THREADS);
+    cfg.dynamicSmemBytes = FR_SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    if (!ctx->no_overlap_launch) {
+        // let this kernel's table build overlap the tail of the previous kernel in the stream (see the kernel)
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+    cudaError_t le;
     switch (mode) {
-        case FR_MODE_DEC:    fr_crypt_kernel<FR_MODE_DEC><<<grid, FR_THREADS, FR_SMEM_BYTES, stream>>>(P); break;
-        case FR_MODE_ENC:    fr_crypt_kernel<FR_MODE_ENC><<<grid, FR_THREADS, FR_SMEM_BYTES, stream>>>(P); break;
-        case FR_MODE_CTR:    fr_crypt_kernel<FR_MODE_CTR><<<grid, FR_THREADS, FR_SMEM_BYTES, stream>>>(P); break;
-        case FR_MODE_VERIFY: fr_crypt_kernel<FR_MODE_VERIFY><<<grid, FR_THREADS, FR_SMEM_BYTES, stream>>>(P); break;
-        case FR_MODE_PADGEN: fr_crypt_kernel<FR_MODE_PADGEN><<<grid, FR_THREADS, FR_SMEM_BYTES, stream>>>(P); break;
-        case FR_MODE_PADDEC: fr_crypt_kernel<FR_MODE_PADDEC><<<grid, FR_THREADS, FR_SMEM_BYTES, stream>>>(P); break;
+        case FR_MODE_DEC:    le = cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_DEC>, P); break;
+        case FR_MODE_ENC:    le = cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_ENC>, P); break;
+        case FR_MODE_CTR:    le = cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_CTR>, P); break;
+        case FR_MODE_VERIFY: le = cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_VERIFY>, P); break;
+        case FR_MODE_PADGEN: le = cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_PADGEN>, P); break;
+        case FR_MODE_PADDEC: le = cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_PADDEC>, P); break;
         default: return FASTRACK_ERR_ARG;
     }
+    if (le != cudaSuccess) { ctx->last_cuda_error = (int)le; (void)cudaGetLastError(); return FASTRACK_ERR_CUDA; }
     ctx->launches++;
     FR_CUDA(ctx, cudaGetLastError());
     return FASTRACK_OK;
