@@ -45,7 +45,7 @@ WAVEFRONTS_PER_ROW_BEST = 197 + 64
 ROW_BYTES = 512
 # dram__bytes_read.sum + dram__bytes_write.sum of one decrypt+verify launch on this exact workload, from the
 # ncu capture summarised in profiles/fr_crypt_kernel_decrypt_verify_256MiB_chunk4MiB.md (algorithmic: 2 x 256 MiB).
-DRAM_TRAFFIC_BYTES_PER_LAUNCH = 512.3e6
+DRAM_TRAFFIC_BYTES_PER_LAUNCH = 501.9e6
 
 
 def peaks():
