@@ -613,17 +613,10 @@ static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const vo
     }
     uint4* d_mask = ctx->d_tags_stage + ctx->tags_stage_chunks;
 
-    // tags: one small copy on a stream of its own; every working stream waits for it before its first kernel
+    // Tags: one small copy on a stream of its own.  It (and, if asked for, the keystream kernel) is issued right
+    // after the first payload copy has been queued, so that nothing delays that copy; every working stream waits
+    // for both before its first kernel.
     cudaStream_t tag_stream = ctx->streams[7], pad_stream = ctx->streams[6];
-    FR_CUDA(ctx, cudaMemcpyAsync(ctx->d_tags_stage, h_tags, K * 16, cudaMemcpyHostToDevice, tag_stream));
-    FR_CUDA(ctx, cudaEventRecord(ctx->tags_ready, tag_stream));
-    if (d_pad) {
-        PassBuffers pb;
-        pb.out = d_pad; pb.mask = d_mask;
-        rc = launch_pass(ctx, FR_MODE_PADGEN, iv_base, 0, len, pb, pad_stream);
-        if (rc != FASTRACK_OK) { cudaStreamSynchronize(tag_stream); return rc; }
-        FR_CUDA(ctx, cudaEventRecord(ctx->pad_ready, pad_stream));
-    }
     bool waited[8] = {false, false, false, false, false, false, false, false};   // per working stream: events already awaited
 
     size_t stage_bytes[FR_MAX_STAGES];
@@ -638,6 +631,19 @@ static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const vo
         rc = FASTRACK_OK;
         e = cudaMemcpyAsync(dst, (const uint8_t*)h_cipher_pinned + off, n, cudaMemcpyHostToDevice, st);
         if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); rc = FASTRACK_ERR_CUDA; }
+        if (rc == FASTRACK_OK && stage == 0) {
+            e = cudaMemcpyAsync(ctx->d_tags_stage, h_tags, K * 16, cudaMemcpyHostToDevice, tag_stream);
+            if (e == cudaSuccess) e = cudaEventRecord(ctx->tags_ready, tag_stream);
+            if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); rc = FASTRACK_ERR_CUDA; }
+            if (rc == FASTRACK_OK && d_pad) {
+                PassBuffers pb;
+                pb.out = d_pad; pb.mask = d_mask;
+                rc = launch_pass(ctx, FR_MODE_PADGEN, iv_base, 0, len, pb, pad_stream);
+                if (rc == FASTRACK_OK && (e = cudaEventRecord(ctx->pad_ready, pad_stream)) != cudaSuccess) {
+                    ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); rc = FASTRACK_ERR_CUDA;
+                }
+            }
+        }
         const size_t si = stage % (size_t)n_streams;
         if (rc == FASTRACK_OK && !waited[si]) {
             // the stream's first kernel (not its first copy) waits for the tags and, if used, the keystream
