@@ -72,7 +72,8 @@ typedef struct fastrack_ctx fastrack_ctx;
  * authentication process"; Section 4.2: every chain uses the same H).
  * Copies the 32-byte AES-256 key (host pointer), expands it into the 15 round keys, derives H, and
  * builds on the current device the tables the kernels need, sized for `chunk_bytes`: the byte tables
- * of the fixed multiplier H^32 and the powers H^0 .. H^(chunk_bytes/16 + 64).  Allocates device
+ * of the fixed multiplier H^32 (and of H, for the sequential comparator) and the powers
+ * H^0 .. H^(chunk_bytes/16 + 65), 16 bytes each, i.e. a table as large as one chunk.  Allocates device
  * memory and synchronises the device once.  chunk_bytes: multiple of 16, 16 .. FASTRACK_MAX_CHUNK_BYTES.
  * On success *out is a new context; on failure *out is NULL. */
 FASTRACK_API int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fastrack_ctx** out);
@@ -84,7 +85,7 @@ FASTRACK_API void fastrack_ctx_destroy(fastrack_ctx* ctx);
 /* K = ceil(len / chunk_bytes); 0 for len == 0 or ctx == NULL (Section 4.2: one tag per chunk). */
 FASTRACK_API size_t fastrack_num_chunks(const fastrack_ctx* ctx, size_t len);
 
-/* Pre-sizes the per-chunk scratch (20 bytes per chunk) for buffers up to max_len bytes so that later
+/* Pre-sizes the per-chunk scratch (40 bytes per chunk: two banks of a 16-byte accumulator and a counter) for buffers up to max_len bytes so that later
  * calls allocate nothing.  Without it the first call that needs more chunks than any call before
  * grows the scratch (cudaMalloc + a device synchronisation) before launching. */
 FASTRACK_API int fastrack_ctx_reserve(fastrack_ctx* ctx, size_t max_len);
