@@ -509,6 +509,34 @@ def run_sweep(args):
             device_cell(4 ** e, cb, "config4")
 
 
+def run_trace(args):
+    """Stage-level timelines of fastrack_pipelined_h2d (best of 20 traced calls), one JSON line per transfer."""
+    import torch
+    from paper_2410_15240_b200 import fastrack, synth
+    torch.cuda.set_device(0)
+    key, iv = synth.key_and_iv(2)
+    for n, cb, ns in ((77_070_336, 4 << 20, 2), (LEN, CHUNK, args.streams)):
+        with fastrack.Context(key, cb) as ctx:
+            K = ctx.num_chunks(n)
+            d_p = torch.randint(0, 256, (n,), dtype=torch.uint8, device="cuda")
+            d_c = torch.empty_like(d_p)
+            d_t = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
+            ctx.encrypt_tag(iv, d_p.data_ptr(), n, d_c.data_ptr(), d_t.data_ptr(), 0)
+            torch.cuda.synchronize()
+            h_c, h_t = d_c.cpu().pin_memory(), d_t.cpu().pin_memory()
+            d_o = torch.empty_like(d_p)
+            d_ok = torch.zeros(K, dtype=torch.int32, device="cuda")
+            ctx.set_trace(True)
+            best = None
+            for _ in range(20):
+                ctx.pipelined_h2d(iv, h_c.data_ptr(), n, h_t.data_ptr(), d_o.data_ptr(), d_ok.data_ptr(), ns)
+                tr = ctx.get_trace()
+                if best is None or tr[-1]["kernel_end_ms"] < best[-1]["kernel_end_ms"]:
+                    best = tr
+            assert bool((d_ok == 1).all()) and bool((d_o == d_p).all())
+        print(json.dumps({"len": n, "chunk": cb, "streams": ns, "stages": best}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -520,8 +548,11 @@ def main():
                     help="time only the device-resident decrypt+verify loop (short run for profilers)")
     ap.add_argument("--sweep", action="store_true",
                     help="print throughput over the benchmark configurations instead of the one bench line")
+    ap.add_argument("--trace", action="store_true", help="print stage-level timelines of the pipelined H2D call")
     args = ap.parse_args()
-    if args.sweep:
+    if args.trace:
+        run_trace(args)
+    elif args.sweep:
         run_sweep(args)
     elif args.impl == "reference":
         run_reference(args)

@@ -233,6 +233,21 @@ FASTRACK_API int fastrack_decrypt_verify_noalloc(fastrack_ctx* ctx, const uint8_
 FASTRACK_API int fastrack_pipelined_d2h(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_plain, size_t len,
                                         void* d_cipher, void* h_cipher_pinned, void* h_tags, int n_streams);
 
+/* Stage-level trace of pipelined host->device calls (paper Section 4.3 argues that the copy of one piece hides
+ * the kernels of the previous one; this shows it).  While enabled, every fastrack_pipelined_h2d /
+ * fastrack_pipelined_h2d_ahead call records three CUDA events per stage on the stage's stream -- before its copy,
+ * after its copy, after its kernel -- and fastrack_ctx_get_trace returns, for the most recent call, each stage's
+ * byte range, stream index and those three times in milliseconds since the first copy was started.
+ * Enabling creates the events (allocation; do it at start-up); tracing adds about a microsecond per event.
+ * fastrack_ctx_get_trace copies at most `cap` entries to `out` (may be NULL) and returns the number of stages. */
+typedef struct {
+    size_t offset, bytes;          /* byte range of the stage inside the buffer */
+    int stream;                    /* index of the internal stream it ran on */
+    float copy_start_ms, copy_end_ms, kernel_end_ms;
+} fastrack_stage_trace;
+FASTRACK_API int fastrack_ctx_set_trace(fastrack_ctx* ctx, int enable);
+FASTRACK_API size_t fastrack_ctx_get_trace(const fastrack_ctx* ctx, fastrack_stage_trace* out, size_t cap);
+
 /* Number of kernels the library launched through ctx since creation (data-path launches only;
  * cudaMemcpyAsync calls are not counted).  For benchmarks' bookkeeping. */
 FASTRACK_API uint64_t fastrack_launch_count(const fastrack_ctx* ctx);

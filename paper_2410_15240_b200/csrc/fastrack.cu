@@ -15,6 +15,7 @@
 using namespace fr_host;
 
 #define FR_THREADS 1024
+#define FR_MAX_STAGES 96      // most stages a pipelined call is cut into
 #define FR_WARPS (FR_THREADS / 32)
 
 // ------------------------------------------------------------------------------------ kernels ----
@@ -176,6 +177,10 @@ struct fastrack_ctx {
     size_t tags_stage_chunks;
     cudaStream_t streams[8];
     cudaEvent_t tags_ready, pad_ready;
+    int trace_on;                               // stage-level event trace of pipelined calls
+    cudaEvent_t trace_ev[3 * FR_MAX_STAGES];    // per stage: before the copy, after the copy, after the kernel
+    fastrack_stage_trace trace[FR_MAX_STAGES];
+    size_t trace_count;
     int last_cuda_error;
     uint64_t launches;
     uint32_t aad_mod;             // 0 = no AAD, else chains per sample of the serial-number framing
@@ -335,6 +340,8 @@ extern "C" void fastrack_ctx_destroy(fastrack_ctx* ctx)
         if (ctx->streams[i]) cudaStreamDestroy(ctx->streams[i]);
     if (ctx->tags_ready) cudaEventDestroy(ctx->tags_ready);
     if (ctx->pad_ready) cudaEventDestroy(ctx->pad_ready);
+    for (int i = 0; i < 3 * FR_MAX_STAGES; i++)
+        if (ctx->trace_ev[i]) cudaEventDestroy(ctx->trace_ev[i]);
     (void)cudaGetLastError();
     secure_zero(ctx, sizeof *ctx);
     delete ctx;
@@ -357,6 +364,25 @@ extern "C" int fastrack_ctx_set_framing(fastrack_ctx* ctx, unsigned chains_per_s
     if (!ctx || chains_per_sample > 256) return FASTRACK_ERR_ARG;
     ctx->aad_mod = chains_per_sample;
     return FASTRACK_OK;
+}
+
+extern "C" int fastrack_ctx_set_trace(fastrack_ctx* ctx, int enable)
+{
+    if (!ctx) return FASTRACK_ERR_ARG;
+    if (enable && !ctx->trace_ev[0]) {
+        for (int i = 0; i < 3 * FR_MAX_STAGES; i++) FR_CUDA(ctx, cudaEventCreate(&ctx->trace_ev[i]));
+    }
+    ctx->trace_on = enable ? 1 : 0;
+    ctx->trace_count = 0;
+    return FASTRACK_OK;
+}
+
+extern "C" size_t fastrack_ctx_get_trace(const fastrack_ctx* ctx, fastrack_stage_trace* out, size_t cap)
+{
+    if (!ctx) return 0;
+    if (out)
+        for (size_t i = 0; i < ctx->trace_count && i < cap; i++) out[i] = ctx->trace[i];
+    return ctx->trace_count;
 }
 
 extern "C" int fastrack_last_cuda_error(const fastrack_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
@@ -556,7 +582,6 @@ extern "C" int fastrack_encrypt_tag(fastrack_ctx* ctx, const uint8_t iv_base[12]
 // then half of the rest, ... down to about 2 MiB (never less than one chunk) -- few copies, and a short
 // exposed kernel.  A stage's kernel is an order of magnitude faster than its neighbour's copy, so it always
 // finishes under it.  Returns the stage sizes in descending order (host->device order).
-#define FR_MAX_STAGES 96
 static size_t plan_stages(const fastrack_ctx* ctx, size_t len, size_t out[FR_MAX_STAGES])
 {
     const size_t cb = ctx->chunk_bytes;
@@ -629,8 +654,11 @@ static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const vo
         cudaStream_t st = ctx->streams[stage % (size_t)n_streams];
         uint8_t* dst = (uint8_t*)d_plain + off;
         rc = FASTRACK_OK;
+        const bool tracing = ctx->trace_on && stage < FR_MAX_STAGES;
+        if (tracing) cudaEventRecord(ctx->trace_ev[3 * stage], st);
         e = cudaMemcpyAsync(dst, (const uint8_t*)h_cipher_pinned + off, n, cudaMemcpyHostToDevice, st);
         if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); rc = FASTRACK_ERR_CUDA; }
+        if (tracing) cudaEventRecord(ctx->trace_ev[3 * stage + 1], st);
         if (rc == FASTRACK_OK && stage == 0) {
             e = cudaMemcpyAsync(ctx->d_tags_stage, h_tags, K * 16, cudaMemcpyHostToDevice, tag_stream);
             if (e == cudaSuccess) e = cudaEventRecord(ctx->tags_ready, tag_stream);
@@ -658,6 +686,12 @@ static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const vo
             if (d_pad) { b.pad = (const uint8_t*)d_pad + off; b.mask = d_mask + k0; }
             rc = launch_pass(ctx, d_pad ? FR_MODE_PADDEC : FR_MODE_DEC, iv_base, k0, n, b, st);
         }
+        if (tracing) {
+            cudaEventRecord(ctx->trace_ev[3 * stage + 2], st);
+            ctx->trace[stage].offset = off;
+            ctx->trace[stage].bytes = n;
+            ctx->trace[stage].stream = (int)(stage % (size_t)n_streams);
+        }
         if (rc != FASTRACK_OK) {
             for (int i = 0; i < 8; i++) cudaStreamSynchronize(ctx->streams[i]);
             (void)cudaGetLastError();
@@ -668,6 +702,15 @@ static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const vo
     FR_CUDA(ctx, cudaStreamSynchronize(tag_stream));
     if (d_pad) FR_CUDA(ctx, cudaStreamSynchronize(pad_stream));
     for (int i = 0; i < n_streams; i++) FR_CUDA(ctx, cudaStreamSynchronize(ctx->streams[i]));
+    if (ctx->trace_on) {
+        ctx->trace_count = n_stages < FR_MAX_STAGES ? n_stages : FR_MAX_STAGES;
+        for (size_t i = 0; i < ctx->trace_count; i++) {
+            cudaEventElapsedTime(&ctx->trace[i].copy_start_ms, ctx->trace_ev[0], ctx->trace_ev[3 * i]);
+            cudaEventElapsedTime(&ctx->trace[i].copy_end_ms, ctx->trace_ev[0], ctx->trace_ev[3 * i + 1]);
+            cudaEventElapsedTime(&ctx->trace[i].kernel_end_ms, ctx->trace_ev[0], ctx->trace_ev[3 * i + 2]);
+        }
+        (void)cudaGetLastError();
+    }
     return FASTRACK_OK;
 }
 

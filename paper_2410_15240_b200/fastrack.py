@@ -22,7 +22,7 @@ EXPORTS = ("fastrack_ctx_create", "fastrack_ctx_destroy", "fastrack_num_chunks",
            "fastrack_last_cuda_error", "fastrack_decrypt_verify", "fastrack_encrypt_tag",
            "fastrack_pipelined_h2d", "fastrack_launch_count", "fastrack_decrypt_verify_noalloc",
            "fastrack_ctr_crypt", "fastrack_verify", "fastrack_keystream", "fastrack_xor_verify",
-           "fastrack_pipelined_h2d_ahead", "fastrack_ctx_set_framing", "fastrack_verify_sequential", "fastrack_pipelined_d2h")
+           "fastrack_pipelined_h2d_ahead", "fastrack_ctx_set_framing", "fastrack_verify_sequential", "fastrack_pipelined_d2h", "fastrack_ctx_set_trace", "fastrack_ctx_get_trace")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2410_15240_b200.build` "
@@ -40,6 +40,15 @@ _lib.fastrack_ctx_reserve.restype = _int
 _lib.fastrack_ctx_reserve.argtypes = [_vp, _sz]
 _lib.fastrack_ctx_set_framing.restype = _int
 _lib.fastrack_ctx_set_framing.argtypes = [_vp, ctypes.c_uint]
+class StageTrace(ctypes.Structure):
+    _fields_ = [("offset", ctypes.c_size_t), ("bytes", ctypes.c_size_t), ("stream", ctypes.c_int),
+                ("copy_start_ms", ctypes.c_float), ("copy_end_ms", ctypes.c_float), ("kernel_end_ms", ctypes.c_float)]
+
+
+_lib.fastrack_ctx_set_trace.restype = _int
+_lib.fastrack_ctx_set_trace.argtypes = [_vp, _int]
+_lib.fastrack_ctx_get_trace.restype = _sz
+_lib.fastrack_ctx_get_trace.argtypes = [_vp, ctypes.POINTER(StageTrace), _sz]
 _lib.fastrack_last_cuda_error.restype = _int
 _lib.fastrack_last_cuda_error.argtypes = [_vp]
 _lib.fastrack_launch_count.restype = ctypes.c_uint64
@@ -96,6 +105,20 @@ def fastrack_ctx_reserve(ctx, max_len: int) -> int:
 
 def fastrack_ctx_set_framing(ctx, chains_per_sample: int) -> int:
     return _lib.fastrack_ctx_set_framing(ctx, chains_per_sample)
+
+
+def fastrack_ctx_set_trace(ctx, enable: int) -> int:
+    return _lib.fastrack_ctx_set_trace(ctx, int(enable))
+
+
+def fastrack_ctx_get_trace(ctx):
+    """-> list of dicts, one per stage of the most recent pipelined host->device call."""
+    n = int(_lib.fastrack_ctx_get_trace(ctx, None, 0))
+    if n == 0:
+        return []
+    buf = (StageTrace * n)()
+    n = int(_lib.fastrack_ctx_get_trace(ctx, buf, n))
+    return [{f: getattr(buf[i], f) for f, _ in StageTrace._fields_} for i in range(n)]
 
 
 def fastrack_last_cuda_error(ctx) -> int:
@@ -180,6 +203,12 @@ class Context:
 
     def set_framing(self, chains_per_sample: int) -> None:
         self._check(fastrack_ctx_set_framing(self.handle, chains_per_sample))
+
+    def set_trace(self, enable: bool) -> None:
+        self._check(fastrack_ctx_set_trace(self.handle, int(enable)))
+
+    def get_trace(self):
+        return fastrack_ctx_get_trace(self.handle)
 
     def reserve(self, max_len: int) -> None:
         self._check(fastrack_ctx_reserve(self.handle, max_len))

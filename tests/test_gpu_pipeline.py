@@ -73,3 +73,39 @@ def test_pipelined_d2h_encrypt_matches_oracle(n, cb, n_streams, in_place):
             assert np.array_equal(d_p.cpu().numpy(), plain)
     back, ok = oracle.mc_decrypt(key, iv, cb, h_c.numpy(), h_t.numpy(), NT)
     assert ok.all() and np.array_equal(back, plain)
+
+
+def test_stage_trace_shows_copies_hiding_kernels():
+    """Section 4.3: the copy of stage i+1 runs while the kernel of stage i does, so a stage's kernel ends before
+    the next stage's copy does; only the last kernel sticks out."""
+    from paper_2410_15240_b200 import fastrack
+    key, iv = synth.key_and_iv(2)
+    cb, n = 1 << 20, 64 << 20
+    with fastrack.Context(key, cb) as ctx:
+        K = ctx.num_chunks(n)
+        d_p = torch.randint(0, 256, (n,), dtype=torch.uint8, device="cuda")
+        d_c = torch.empty_like(d_p)
+        d_t = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
+        ctx.encrypt_tag(iv, d_p.data_ptr(), n, d_c.data_ptr(), d_t.data_ptr(), 0)
+        torch.cuda.synchronize()
+        h_c, h_t = d_c.cpu().pin_memory(), d_t.cpu()
+        d_o = torch.empty_like(d_p)
+        d_ok = torch.zeros(K, dtype=torch.int32, device="cuda")
+        assert ctx.get_trace() == []
+        ctx.set_trace(True)
+        for _ in range(2):
+            ctx.pipelined_h2d(iv, h_c.data_ptr(), n, h_t.data_ptr(), d_o.data_ptr(), d_ok.data_ptr(), 2)
+        tr = ctx.get_trace()
+        assert bool((d_ok == 1).all()) and bool((d_o == d_p).all())
+        ctx.set_trace(False)
+        assert ctx.get_trace() == []
+    assert len(tr) >= 4
+    assert tr[0]["offset"] == 0 and sum(s["bytes"] for s in tr) == n
+    for a, b in zip(tr, tr[1:]):
+        assert b["offset"] == a["offset"] + a["bytes"] and b["bytes"] <= a["bytes"]          # shrinking stages
+        assert a["copy_start_ms"] <= a["copy_end_ms"] <= a["kernel_end_ms"]
+        assert b["copy_start_ms"] >= a["copy_start_ms"]
+        assert a["kernel_end_ms"] <= b["copy_end_ms"] + 0.02, "a stage's kernel should finish under the next copy"
+    total = tr[-1]["kernel_end_ms"]
+    copies = sum(s["copy_end_ms"] - s["copy_start_ms"] for s in tr)
+    assert total < 1.15 * copies                                                              # the kernels are hidden

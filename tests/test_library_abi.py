@@ -16,7 +16,7 @@ def declared_functions():
 
 def test_header_and_binding_agree():
     names = declared_functions()
-    assert len(names) >= 18
+    assert len(names) >= 20
     assert sorted(fastrack.EXPORTS) == names
 
 
@@ -49,6 +49,8 @@ def test_argument_checks_that_need_no_device():
     assert fastrack.fastrack_launch_count(None) == 0
     assert fastrack.fastrack_ctx_reserve(None, 1) == fastrack.ERR_ARG
     assert fastrack.fastrack_ctx_set_framing(None, 16) == fastrack.ERR_ARG
+    assert fastrack.fastrack_ctx_set_trace(None, 1) == fastrack.ERR_ARG
+    assert fastrack.fastrack_ctx_get_trace(None) == []
     assert fastrack.fastrack_decrypt_verify(None, bytes(12), 0, 16, 0, 0, 0, 0) == fastrack.ERR_ARG
     assert fastrack.fastrack_encrypt_tag(None, bytes(12), 0, 16, 0, 0, 0) == fastrack.ERR_ARG
     assert fastrack.fastrack_decrypt_verify_noalloc(None, bytes(12), 0, 16, 0, 0, 0, 0) == fastrack.ERR_ARG
