@@ -130,8 +130,8 @@ FASTRACK_API int fastrack_encrypt_tag(fastrack_ctx* ctx, const uint8_t iv_base[1
 /* Pipelined host->device transfer with decryption and verification (paper Section 4.3 "Decryption
  * pipeline": the PCIe transfer is overlapped with the decryption and authentication kernels, so the
  * transfer costs max(copy, kernels) instead of their sum).
- * The buffer is cut into stages of whole chunks that shrink geometrically (half of the buffer, then half of
- * the rest, ... down to about 2 MiB, never less than one chunk); stage i is copied pinned->device into its
+ * The buffer is cut into stages of whole chunks that shrink geometrically (three quarters of the buffer, then
+ * three quarters of the rest, ... down to about 2 MiB, never less than one chunk); stage i is copied pinned->device into its
  * final place in d_plain with cudaMemcpyAsync on internal stream i mod n_streams and decrypted and verified
  * in place by the same kernels on that stream, so the copy of stage i+1 overlaps the kernels of stage i and
  * only the short last stage's kernel is exposed.
@@ -220,8 +220,8 @@ FASTRACK_API int fastrack_decrypt_verify_noalloc(fastrack_ctx* ctx, const uint8_
 /* Pipelined device->host transfer with encryption and tagging: the mirror of fastrack_pipelined_h2d for
  * GPU->CPU copies (paper Section 2.3: encryption is the same keystream XOR; Section 4.2: one tag per chunk;
  * Section 4.3: the transfer is overlapped with the kernels).
- * The buffer is cut into stages of whole chunks that GROW geometrically (about 2 MiB first, then twice as much,
- * ... the last one about half of the buffer); stage i is encrypted and tagged from d_plain into d_cipher on
+ * The buffer is cut into stages of whole chunks that GROW geometrically (about 2 MiB first, then four times as much,
+ * ... the last one about three quarters of the buffer); stage i is encrypted and tagged from d_plain into d_cipher on
  * internal stream i mod n_streams and then copied, with its tags, to the host on the same stream, so the copy
  * of stage i overlaps the kernel of stage i+1 and only the short first stage's kernel is exposed.
  *   d_plain         device, len bytes in (not modified unless d_cipher == d_plain).

@@ -578,10 +578,10 @@ extern "C" int fastrack_encrypt_tag(fastrack_ctx* ctx, const uint8_t iv_base[12]
 
 // Stage = the unit that is copied and processed in place: whole chunks.  In a pipelined transfer only two
 // things are not hidden behind a copy: a few microseconds per copy boundary and ONE kernel (the last stage's
-// on the way in, the first stage's on the way out).  So the stages shrink geometrically: half of the buffer,
-// then half of the rest, ... down to about 2 MiB (never less than one chunk) -- few copies, and a short
-// exposed kernel.  A stage's kernel is an order of magnitude faster than its neighbour's copy, so it always
-// finishes under it.  Returns the stage sizes in descending order (host->device order).
+// on the way in, the first stage's on the way out).  So the stages shrink geometrically: three quarters of
+// the buffer, then three quarters of the rest, ... down to about 2 MiB (never less than one chunk) -- few copies,
+// and a short exposed kernel.  A stage's kernel is 6-9 times faster than a copy of the same size, so it still
+// finishes under the next stage's copy, which is a quarter as large.  Returns the stage sizes in descending order (host->device order).
 static size_t plan_stages(const fastrack_ctx* ctx, size_t len, size_t out[FR_MAX_STAGES])
 {
     const size_t cb = ctx->chunk_bytes;
@@ -594,7 +594,7 @@ static size_t plan_stages(const fastrack_ctx* ctx, size_t len, size_t out[FR_MAX
         if (ctx->stage_bytes_override) {
             n = (ctx->stage_bytes_override + cb - 1) / cb * cb;
         } else {
-            n = remaining / 2 / cb * cb;
+            n = (remaining / 4 * 3) / cb * cb;
             if (n < min_stage) n = min_stage;
             if (remaining < n + min_stage / 2) n = remaining;      // do not leave a sliver behind
         }
