@@ -145,6 +145,26 @@ FASTRACK_API int fastrack_pipelined_h2d(fastrack_ctx* ctx, const uint8_t iv_base
                                         const void* h_cipher_pinned, size_t len, const void* h_tags,
                                         void* d_plain, uint32_t* d_ok, int n_streams);
 
+/* ---- A batch of samples, each with its own IV (paper Section 4.2) -------------------------------------------
+ * The paper splits every input SAMPLE (an image, a sub-graph) into n chunks with n tags, and a batch holds many
+ * samples that their owner encrypted one by one.  These two calls take such a batch in one launch:
+ * n_samples samples of sample_bytes bytes each, back to back; sample s was (or is to be) encrypted as its own
+ * multi-chain message under the 12-byte IV base d_iv_bases[12*s .. 12*s+11], i.e. its chunk k uses
+ * IV = that base with k added to its last four bytes, and -- with fastrack_ctx_set_framing(ctx, n) -- the AAD
+ * byte (k mod n).  A sample has ceil(sample_bytes / chunk_bytes) chunks, only its last may be short; tags and
+ * verdicts are laid out sample after sample (sample s, chunk k at index s * chunks_per_sample + k).
+ *   d_iv_bases   DEVICE, 12 * n_samples bytes (they normally arrive with the batch); no alignment needed.
+ *   sample_bytes multiple of 16 (so that every sample stays 16-byte aligned).
+ * The result is exactly what n_samples separate calls of fastrack_decrypt_verify / fastrack_encrypt_tag with
+ * the respective IV bases would give, without their n_samples launches.  Asynchronous on `stream`; pointer and
+ * overlap rules as for the single-buffer calls. */
+FASTRACK_API int fastrack_decrypt_verify_samples(fastrack_ctx* ctx, const void* d_iv_bases, size_t sample_bytes,
+                                                 size_t n_samples, const void* d_cipher, const void* d_tags,
+                                                 void* d_plain, uint32_t* d_ok, void* stream);
+FASTRACK_API int fastrack_encrypt_tag_samples(fastrack_ctx* ctx, const void* d_iv_bases, size_t sample_bytes,
+                                              size_t n_samples, const void* d_plain, void* d_cipher, void* d_tags,
+                                              void* stream);
+
 /* ---- Split passes (paper Section 4.3, "Eager evaluation") -------------------------------------------------
  * The paper lets the consumer start on the decrypted data before authentication has finished and runs the
  * authentication kernel later, in parallel with the next batch's PCIe transfer; results are discarded if the

@@ -65,7 +65,7 @@ __device__ __forceinline__ void fr_crypt_body(const FrParams& P, const char* sm,
                 }
             }
             if (finisher && lane == 0) {
-                const uint4 lenh = (kk + 1u == P.n_chunks) ? P.lenh_last : P.lenh_full;
+                const uint4 lenh = ((kk + 1u) % P.chunks_per_sample == 0u) ? P.lenh_last : P.lenh_full;
                 const uint4 tag = fr_xor4(z, lenh);           // z already holds GHASH of the data xor E_K(J0)
                 if (MODE == FR_MODE_ENC) {
                     P.tags_out[kk] = tag;
@@ -129,11 +129,12 @@ __global__ void __launch_bounds__(32, 1) fr_verify_sequential_kernel(const __gri
     const FrLane L = fr_make_lane(lane);
     const uint32_t kk = blockIdx.x * 32u + lane;
     if (kk >= P.n_chunks) return;
-    const uint64_t len_k = fr_chunk_len(P, kk);
+    const FrChunk ck = fr_chunk_info(P, kk);
+    const uint64_t len_k = ck.len;
     const uint32_t nblk = (uint32_t)((len_k + 15) >> 4);
-    const uint8_t* in = P.in + (uint64_t)kk * P.chunk_bytes;
+    const uint8_t* in = P.in + ck.off;
     uint4 y = make_uint4(0, 0, 0, 0);
-    if (P.aad_mod) y = fr_ghash_tabmul<false>(sm, L, make_uint4((P.first_chunk + kk) % P.aad_mod, 0, 0, 0));
+    if (P.aad_mod) y = fr_ghash_tabmul<false>(sm, L, make_uint4(ck.serial % P.aad_mod, 0, 0, 0));
     uint32_t j = 0;
     for (; j + 8 <= nblk && ((uint64_t)(j + 8) << 4) <= len_k; j += 8) {      // eight loads in flight per thread
         uint4 x[8];
@@ -151,7 +152,7 @@ __global__ void __launch_bounds__(32, 1) fr_verify_sequential_kernel(const __gri
     const uint64_t bits = len_k << 3;
     const uint4 lenblk = make_uint4(0, P.aad_mod ? fr_bswap(8u) : 0u, fr_bswap((uint32_t)(bits >> 32)), fr_bswap((uint32_t)bits));
     y = fr_ghash_tabmul<false>(sm, L, fr_xor4(y, lenblk));
-    const FrCtrChunk cc = fr_ctr_chunk<false>(sm, L.lane4, P, fr_bswap(P.iv_ctr + kk));
+    const FrCtrChunk cc = fr_ctr_chunk<false>(sm, L.lane4, P, ck.iv_w0, ck.iv_w1, fr_bswap(ck.iv_ctr));
     const FrCtrGroup cg = fr_ctr_group<false>(sm, L.lane4, P, cc, 1u);
     const uint4 tag = fr_xor4(y, fr_aes256_ctr_block<false>(sm, L.lane4, P, cc, cg, 1u));
     const uint4 t = P.tags_in[kk];
@@ -408,11 +409,12 @@ static uint4 length_term(const fastrack_ctx* ctx, uint64_t bytes)
     return r;
 }
 
-// Segment geometry of a launch over `len` bytes: rows are aligned to the counter (block j sits at counter
+// Segment geometry of a launch over n_chunks chunks of samples of `sample_bytes` bytes (a plain buffer is one
+// sample): rows are aligned to the counter (block j sits at counter
 // j + 2), segments are whole multiples of 8 rows so that they start on a 256-counter group.
-static void plan_segments(const fastrack_ctx* ctx, size_t len, size_t n_chunks, FrParams& P)
+static void plan_segments(const fastrack_ctx* ctx, size_t sample_bytes, size_t n_chunks, FrParams& P)
 {
-    const size_t first_len = len < ctx->chunk_bytes ? len : ctx->chunk_bytes;
+    const size_t first_len = sample_bytes < ctx->chunk_bytes ? sample_bytes : ctx->chunk_bytes;
     const size_t rows_ref = ((first_len + 15) / 16 + 2 + FR_ROW_BLOCKS - 1) / FR_ROW_BLOCKS;
     const size_t warps = (size_t)ctx->num_sms * FR_WARPS;
     // Segments are dealt round-robin to the resident warps.  Two things bound a launch: the latency of the
@@ -450,7 +452,10 @@ static void plan_segments(const fastrack_ctx* ctx, size_t len, size_t n_chunks, 
     P.seg_rows = (uint32_t)seg_rows;
     P.segs_per_chunk = (uint32_t)spc;
     P.n_items = (uint32_t)(spc * n_chunks);
-    const size_t last_len = len - (n_chunks - 1) * ctx->chunk_bytes;
+    const size_t cps = (sample_bytes + ctx->chunk_bytes - 1) / ctx->chunk_bytes;
+    const size_t last_len = sample_bytes - (cps - 1) * ctx->chunk_bytes;     // a sample's last chunk may be short
+    P.sample_bytes = sample_bytes;
+    P.chunks_per_sample = (uint32_t)cps;
     P.lenh_full = length_term(ctx, first_len);
     P.lenh_last = length_term(ctx, last_len);
 }
@@ -465,6 +470,8 @@ struct PassBuffers {
     void* tags_out = nullptr;
     uint32_t* ok = nullptr;
     int bank = 0;              // which half of the per-chunk scratch the pass uses
+    const void* ivs = nullptr; // batch of samples: per-sample IV bases on the device (then iv_base is unused)
+    size_t sample_bytes = 0;   // batch of samples: bytes per sample (0: the launch is one plain buffer)
 };
 
 // Launch one pass over `len` bytes that start at chunk index `first_chunk` of the caller's buffer.
@@ -474,18 +481,23 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
     FrParams P;
     memset(&P, 0, sizeof P);
     memcpy(P.rk, ctx->rk, sizeof P.rk);
-    P.iv_w0 = load_le32(iv_base);
-    P.iv_w1 = load_le32(iv_base + 4);
-    P.iv_ctr = load_be32(iv_base + 8) + (uint32_t)first_chunk;
+    if (iv_base) {
+        P.iv_w0 = load_le32(iv_base);
+        P.iv_w1 = load_le32(iv_base + 4);
+        P.iv_ctr = load_be32(iv_base + 8) + (uint32_t)first_chunk;
+    }
+    P.ivs = (const uint8_t*)b.ivs;
     P.first_chunk = (uint32_t)first_chunk;
     P.aad_mod = ctx->aad_mod;
     P.generic_smem = ctx->generic_smem;
     P.len = len;
     P.chunk_bytes = ctx->chunk_bytes;
-    const size_t n_chunks = (len + ctx->chunk_bytes - 1) / ctx->chunk_bytes;
+    const size_t sample_bytes = b.sample_bytes ? b.sample_bytes : len;
+    const size_t cps = (sample_bytes + ctx->chunk_bytes - 1) / ctx->chunk_bytes;
+    const size_t n_chunks = (len / sample_bytes) * cps;            // len is a whole number of samples
     P.n_chunks = (uint32_t)n_chunks;
 
-    plan_segments(ctx, len, n_chunks, P);
+    plan_segments(ctx, sample_bytes, n_chunks, P);
 
     P.in = (const uint8_t*)b.in;
     P.out = (uint8_t*)b.out;
@@ -787,6 +799,55 @@ extern "C" int fastrack_pipelined_d2h(fastrack_ctx* ctx, const uint8_t iv_base[1
     return FASTRACK_OK;
 }
 
+// Argument checks shared by the two batch-of-samples entry points.
+static int check_samples(fastrack_ctx* ctx, const void* d_iv_bases, size_t sample_bytes, size_t n_samples, size_t* K_out)
+{
+    if (!ctx || !d_iv_bases) return FASTRACK_ERR_ARG;
+    if (sample_bytes == 0 || (sample_bytes & 15)) return FASTRACK_ERR_ARG;       // samples must stay 16-byte aligned
+    if (n_samples > ((size_t)1 << 40) / sample_bytes) return FASTRACK_ERR_TOO_MANY;
+    const size_t cps = (sample_bytes + ctx->chunk_bytes - 1) / ctx->chunk_bytes;
+    if (cps * n_samples > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
+    *K_out = cps * n_samples;
+    return FASTRACK_OK;
+}
+
+extern "C" int fastrack_decrypt_verify_samples(fastrack_ctx* ctx, const void* d_iv_bases, size_t sample_bytes,
+                                               size_t n_samples, const void* d_cipher, const void* d_tags, void* d_plain,
+                                               uint32_t* d_ok, void* stream)
+{
+    size_t K = 0;
+    int rc = check_samples(ctx, d_iv_bases, sample_bytes, n_samples, &K);
+    if (rc != FASTRACK_OK) return rc;
+    if (n_samples == 0) return FASTRACK_OK;
+    const size_t len = sample_bytes * n_samples;
+    if (!d_cipher || !d_tags || !d_plain || !d_ok) return FASTRACK_ERR_ARG;
+    if (misaligned(d_cipher, 16) || misaligned(d_plain, 16) || misaligned(d_tags, 16) || misaligned(d_ok, 4)) return FASTRACK_ERR_ARG;
+    if (bad_overlap(d_cipher, d_plain, len)) return FASTRACK_ERR_ARG;
+    rc = ensure_scratch(ctx, K);
+    if (rc != FASTRACK_OK) return rc;
+    PassBuffers b;
+    b.in = d_cipher; b.out = d_plain; b.tags_in = d_tags; b.ok = d_ok; b.ivs = d_iv_bases; b.sample_bytes = sample_bytes;
+    return launch_pass(ctx, FR_MODE_DEC, nullptr, 0, len, b, (cudaStream_t)stream);
+}
+
+extern "C" int fastrack_encrypt_tag_samples(fastrack_ctx* ctx, const void* d_iv_bases, size_t sample_bytes, size_t n_samples,
+                                            const void* d_plain, void* d_cipher, void* d_tags, void* stream)
+{
+    size_t K = 0;
+    int rc = check_samples(ctx, d_iv_bases, sample_bytes, n_samples, &K);
+    if (rc != FASTRACK_OK) return rc;
+    if (n_samples == 0) return FASTRACK_OK;
+    const size_t len = sample_bytes * n_samples;
+    if (!d_plain || !d_cipher || !d_tags) return FASTRACK_ERR_ARG;
+    if (misaligned(d_cipher, 16) || misaligned(d_plain, 16) || misaligned(d_tags, 16)) return FASTRACK_ERR_ARG;
+    if (bad_overlap(d_cipher, d_plain, len)) return FASTRACK_ERR_ARG;
+    rc = ensure_scratch(ctx, K);
+    if (rc != FASTRACK_OK) return rc;
+    PassBuffers b;
+    b.in = d_plain; b.out = d_cipher; b.tags_out = d_tags; b.ivs = d_iv_bases; b.sample_bytes = sample_bytes;
+    return launch_pass(ctx, FR_MODE_ENC, nullptr, 0, len, b, (cudaStream_t)stream);
+}
+
 extern "C" int fastrack_ctr_crypt(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_in, size_t len, void* d_out,
                                   void* stream)
 {
@@ -835,6 +896,8 @@ extern "C" int fastrack_verify_sequential(fastrack_ctx* ctx, const uint8_t iv_ba
     P.len = len;
     P.chunk_bytes = ctx->chunk_bytes;
     P.n_chunks = (uint32_t)K;
+    P.sample_bytes = len;
+    P.chunks_per_sample = (uint32_t)K;
     P.in = (const uint8_t*)d_cipher;
     P.tags_in = (const uint4*)d_tags;
     P.ok = d_ok;

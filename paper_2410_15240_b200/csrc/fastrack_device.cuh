@@ -51,9 +51,13 @@ struct FrParams {
     uint32_t n_chunks;         // chunks in this launch
     uint32_t n_items;          // n_chunks * segs_per_chunk
     uint32_t generic_smem;     // 1: use the portable shared-memory addressing even where the absolute form would do
-    uint32_t aad_mod;          // 0: no AAD; n: chunk k authenticates the one byte (first chunk index + k) mod n as AAD
+    uint32_t aad_mod;          // 0: no AAD; n: a chunk authenticates the one byte (its serial number mod n) as AAD
     uint64_t len;              // bytes in this launch
     uint64_t chunk_bytes;
+    uint64_t sample_bytes;     // the launch is a sequence of equal samples of this many bytes (one sample: = len)
+    uint32_t chunks_per_sample;  // ceil(sample_bytes / chunk_bytes); only a sample's last chunk may be short
+    uint32_t pad1;
+    const uint8_t* ivs;        // per-sample 12-byte IV bases (device), or null: one IV base for the whole launch
     const uint8_t* in;
     uint8_t* out;
     const uint4* tags_in;      // decrypt
@@ -237,9 +241,10 @@ struct FrCtrGroup {        // per 256-counter group
 };
 
 template <bool ABS>
-__device__ __forceinline__ FrCtrChunk fr_ctr_chunk(const char* sm, uint32_t lane4, const FrParams& P, uint32_t ivw2)
+__device__ __forceinline__ FrCtrChunk fr_ctr_chunk(const char* sm, uint32_t lane4, const FrParams& P, uint32_t ivw0,
+                                                   uint32_t ivw1, uint32_t ivw2)
 {
-    const uint32_t s0 = P.iv_w0 ^ P.rk[0], s1 = P.iv_w1 ^ P.rk[1], s2 = ivw2 ^ P.rk[2];
+    const uint32_t s0 = ivw0 ^ P.rk[0], s1 = ivw1 ^ P.rk[1], s2 = ivw2 ^ P.rk[2];
     FrCtrChunk c;
     c.a0 = FR_TE0(s0, 0) ^ FR_TE1(s1, 1) ^ FR_TE2(s2, 2) ^ P.rk[4];
     c.b1 = FR_TE0(s1, 0) ^ FR_TE1(s2, 1) ^ FR_TE3(s0, 3) ^ P.rk[5];
@@ -362,10 +367,43 @@ __device__ __forceinline__ uint4 fr_gf128_mul(uint4 x, uint4 y)
     return make_uint4(fr_bswap(__brev(z0)), fr_bswap(__brev(z1)), fr_bswap(__brev(z2)), fr_bswap(__brev(z3)));
 }
 
+// Where chunk kk of the launch lives and what it is keyed with.  The launch is a sequence of equal samples
+// (a plain buffer is one sample); inside a sample the chunks are chunk_bytes long except possibly the last.
+struct FrChunk {
+    uint64_t off, len;          // byte offset in the launch's buffers, byte length
+    uint32_t iv_w0, iv_w1;      // little-endian loads of the IV base's bytes 0..3 and 4..7
+    uint32_t iv_ctr;            // value of the IV's last four bytes for this chunk (big-endian integer)
+    uint32_t serial;            // index the IV and the serial-number AAD count with
+    bool last_of_sample;
+};
+
+__device__ __forceinline__ FrChunk fr_chunk_info(const FrParams& P, uint32_t kk)
+{
+    FrChunk c;
+    const uint32_t sample = kk / P.chunks_per_sample, k = kk - sample * P.chunks_per_sample;
+    const uint64_t in_sample = (uint64_t)k * P.chunk_bytes, rem = P.sample_bytes - in_sample;
+    c.off = (uint64_t)sample * P.sample_bytes + in_sample;
+    c.len = rem < P.chunk_bytes ? rem : P.chunk_bytes;
+    c.last_of_sample = (k + 1u == P.chunks_per_sample);
+    if (P.ivs) {                 // a batch of samples, each encrypted under its own IV base: chunk k of the sample
+        const uint8_t* iv = P.ivs + 12ull * sample;
+        c.iv_w0 = (uint32_t)iv[0] | ((uint32_t)iv[1] << 8) | ((uint32_t)iv[2] << 16) | ((uint32_t)iv[3] << 24);
+        c.iv_w1 = (uint32_t)iv[4] | ((uint32_t)iv[5] << 8) | ((uint32_t)iv[6] << 16) | ((uint32_t)iv[7] << 24);
+        c.serial = k;
+        c.iv_ctr = (((uint32_t)iv[8] << 24) | ((uint32_t)iv[9] << 16) | ((uint32_t)iv[10] << 8) | (uint32_t)iv[11]) + k;
+    } else {
+        c.iv_w0 = P.iv_w0;
+        c.iv_w1 = P.iv_w1;
+        c.serial = P.first_chunk + kk;
+        c.iv_ctr = P.iv_ctr + kk;
+    }
+    return c;
+}
+
 __device__ __forceinline__ uint64_t fr_chunk_len(const FrParams& P, uint32_t kk)
 {
-    uint64_t off = (uint64_t)kk * P.chunk_bytes;
-    uint64_t rem = P.len - off;
+    const uint32_t k = kk % P.chunks_per_sample;
+    const uint64_t rem = P.sample_bytes - (uint64_t)k * P.chunk_bytes;
     return rem < P.chunk_bytes ? rem : P.chunk_bytes;
 }
 
@@ -419,8 +457,9 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
     constexpr bool DO_LOAD = MODE != FR_MODE_PADGEN;
     constexpr bool DO_STORE = MODE != FR_MODE_VERIFY;
 
-    const uint64_t chunk_off = (uint64_t)kk * P.chunk_bytes;
-    const uint64_t len_k = fr_chunk_len(P, kk);
+    const FrChunk ck = fr_chunk_info(P, kk);
+    const uint64_t chunk_off = ck.off;
+    const uint64_t len_k = ck.len;
     const uint32_t nblk = (uint32_t)((len_k + 15) >> 4);
     const uint32_t rows = fr_chunk_rows(nblk);
     const uint32_t row0 = s * P.seg_rows;
@@ -451,7 +490,7 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
         }
     }
     FrCtrChunk cc = {0, 0, 0, 0};
-    if (DO_AES || row0 == 0) cc = fr_ctr_chunk<ABS>(sm, L.lane4, P, fr_bswap(P.iv_ctr + kk));   // VERIFY needs E_K(J0) only
+    if (DO_AES || row0 == 0) cc = fr_ctr_chunk<ABS>(sm, L.lane4, P, ck.iv_w0, ck.iv_w1, fr_bswap(ck.iv_ctr));   // VERIFY needs E_K(J0) only
     FrCtrGroup cg = {0, 0, 0, 0};
 
     uint4 y = make_uint4(0, 0, 0, 0), pend = make_uint4(0, 0, 0, 0), extra = make_uint4(0, 0, 0, 0);
@@ -486,7 +525,7 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
                 if (MODE == FR_MODE_PADGEN) P.mask[kk] = extra;
             }
             if (DO_GHASH && P.aad_mod) {                                              // the one-byte AAD block
-                const uint4 v = make_uint4((P.first_chunk + kk) % P.aad_mod, 0, 0, 0);    // y is still zero here
+                const uint4 v = make_uint4(ck.serial % P.aad_mod, 0, 0, 0);              // y is still zero here
                 if (ctr != c_last) y = fr_ghash_tabmul<ABS>(sm, L, v);
                 else pend = v;
             }

@@ -22,7 +22,8 @@ EXPORTS = ("fastrack_ctx_create", "fastrack_ctx_destroy", "fastrack_num_chunks",
            "fastrack_last_cuda_error", "fastrack_decrypt_verify", "fastrack_encrypt_tag",
            "fastrack_pipelined_h2d", "fastrack_launch_count", "fastrack_decrypt_verify_noalloc",
            "fastrack_ctr_crypt", "fastrack_verify", "fastrack_keystream", "fastrack_xor_verify",
-           "fastrack_pipelined_h2d_ahead", "fastrack_ctx_set_framing", "fastrack_verify_sequential", "fastrack_pipelined_d2h", "fastrack_ctx_set_trace", "fastrack_ctx_get_trace")
+           "fastrack_pipelined_h2d_ahead", "fastrack_ctx_set_framing", "fastrack_verify_sequential", "fastrack_pipelined_d2h", "fastrack_ctx_set_trace", "fastrack_ctx_get_trace",
+           "fastrack_decrypt_verify_samples", "fastrack_encrypt_tag_samples")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2410_15240_b200.build` "
@@ -59,6 +60,10 @@ _lib.fastrack_decrypt_verify_noalloc.restype = _int
 _lib.fastrack_decrypt_verify_noalloc.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp, _vp]
 _lib.fastrack_encrypt_tag.restype = _int
 _lib.fastrack_encrypt_tag.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp]
+_lib.fastrack_decrypt_verify_samples.restype = _int
+_lib.fastrack_decrypt_verify_samples.argtypes = [_vp, _vp, _sz, _sz, _vp, _vp, _vp, _vp, _vp]
+_lib.fastrack_encrypt_tag_samples.restype = _int
+_lib.fastrack_encrypt_tag_samples.argtypes = [_vp, _vp, _sz, _sz, _vp, _vp, _vp, _vp]
 _lib.fastrack_ctr_crypt.restype = _int
 _lib.fastrack_ctr_crypt.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp]
 _lib.fastrack_verify.restype = _int
@@ -151,6 +156,17 @@ def fastrack_pipelined_h2d(ctx, iv_base: bytes, h_cipher_pinned: int, length: in
     return _lib.fastrack_pipelined_h2d(ctx, iv_base, h_cipher_pinned, length, h_tags, d_plain, d_ok, n_streams)
 
 
+def fastrack_decrypt_verify_samples(ctx, d_iv_bases: int, sample_bytes: int, n_samples: int, d_cipher: int, d_tags: int,
+                                    d_plain: int, d_ok: int, stream: int = 0) -> int:
+    return _lib.fastrack_decrypt_verify_samples(ctx, d_iv_bases, sample_bytes, n_samples, d_cipher, d_tags, d_plain, d_ok,
+                                                stream)
+
+
+def fastrack_encrypt_tag_samples(ctx, d_iv_bases: int, sample_bytes: int, n_samples: int, d_plain: int, d_cipher: int,
+                                 d_tags: int, stream: int = 0) -> int:
+    return _lib.fastrack_encrypt_tag_samples(ctx, d_iv_bases, sample_bytes, n_samples, d_plain, d_cipher, d_tags, stream)
+
+
 def fastrack_ctr_crypt(ctx, iv_base: bytes, d_in: int, length: int, d_out: int, stream: int = 0) -> int:
     return _lib.fastrack_ctr_crypt(ctx, iv_base, d_in, length, d_out, stream)
 
@@ -226,6 +242,14 @@ class Context:
     def pipelined_h2d(self, iv_base, h_cipher_pinned, length, h_tags, d_plain, d_ok, n_streams=4) -> None:
         self._check(fastrack_pipelined_h2d(self.handle, iv_base, h_cipher_pinned, length, h_tags, d_plain, d_ok,
                                            n_streams))
+
+    def decrypt_verify_samples(self, d_iv_bases, sample_bytes, n_samples, d_cipher, d_tags, d_plain, d_ok, stream=0) -> None:
+        self._check(fastrack_decrypt_verify_samples(self.handle, d_iv_bases, sample_bytes, n_samples, d_cipher, d_tags,
+                                                    d_plain, d_ok, stream))
+
+    def encrypt_tag_samples(self, d_iv_bases, sample_bytes, n_samples, d_plain, d_cipher, d_tags, stream=0) -> None:
+        self._check(fastrack_encrypt_tag_samples(self.handle, d_iv_bases, sample_bytes, n_samples, d_plain, d_cipher,
+                                                 d_tags, stream))
 
     def ctr_crypt(self, iv_base, d_in, length, d_out, stream=0) -> None:
         self._check(fastrack_ctr_crypt(self.handle, iv_base, d_in, length, d_out, stream))

@@ -133,7 +133,8 @@ void run_pass(Setup& S, uint32_t n_chunks, std::vector<uint4>& acc)
 // One pass of mode `mode` (FrMode) over a buffer; seg_rows as the host planner would choose it (any value >= 1).
 extern "C" int emu_pass(int mode, const uint8_t* key, const uint8_t* iv_base, size_t cb, const uint8_t* in, size_t len,
                         uint8_t* out, const uint8_t* pad, uint8_t* mask, const uint8_t* tags_in, uint8_t* tags_out,
-                        uint32_t* ok, uint32_t seg_rows, uint32_t first_chunk, uint32_t aad_mod)
+                        uint32_t* ok, uint32_t seg_rows, uint32_t first_chunk, uint32_t aad_mod, size_t sample_bytes,
+                        const uint8_t* ivs)
 {
     Setup S;
     setup(S, key, cb);
@@ -147,15 +148,20 @@ extern "C" int emu_pass(int mode, const uint8_t* key, const uint8_t* iv_base, si
     P.aad_mod = aad_mod;
     P.len = len;
     P.chunk_bytes = cb;
-    const size_t n_chunks = (len + cb - 1) / cb;
-    const size_t first_len = std::min(len, cb);
+    if (sample_bytes == 0) sample_bytes = len;                                   // a plain buffer is one sample
+    const size_t cps = (sample_bytes + cb - 1) / cb;
+    const size_t n_chunks = (len / sample_bytes) * cps;
+    const size_t first_len = std::min(sample_bytes, cb);
+    P.sample_bytes = sample_bytes;
+    P.chunks_per_sample = (uint32_t)cps;
+    P.ivs = ivs;
     const size_t rows_ref = ((first_len + 15) / 16 + 2 + 31) / 32;
     P.seg_rows = seg_rows ? seg_rows : 8;
     P.segs_per_chunk = (uint32_t)((rows_ref + P.seg_rows - 1) / P.seg_rows);
     P.n_chunks = (uint32_t)n_chunks;
     P.n_items = (uint32_t)(P.segs_per_chunk * n_chunks);
     P.lenh_full = length_term(S, first_len, aad_mod);
-    P.lenh_last = length_term(S, len - (n_chunks - 1) * cb, aad_mod);
+    P.lenh_last = length_term(S, sample_bytes - (cps - 1) * cb, aad_mod);
     P.in = in;
     P.out = out;
     P.pad = pad;
@@ -171,7 +177,7 @@ extern "C" int emu_pass(int mode, const uint8_t* key, const uint8_t* iv_base, si
         default: return -1;
     }
     for (uint32_t kk = 0; kk < n_chunks; kk++) {                            // the finishing warp's part
-        const uint4 tag = fr_xor4(acc[kk], (kk + 1 == n_chunks) ? P.lenh_last : P.lenh_full);
+        const uint4 tag = fr_xor4(acc[kk], ((kk + 1) % P.chunks_per_sample == 0) ? P.lenh_last : P.lenh_full);
         if (mode == FR_MODE_ENC) memcpy(tags_out + 16 * kk, &tag, 16);
         else ok[kk] = memcmp(&tag, tags_in + 16 * kk, 16) == 0;
     }

@@ -21,7 +21,7 @@ def emu(tmp_path_factory):
                            os.path.join(ROOT, "tests", "device_on_host", "emulate.cpp")])
     lib = ctypes.CDLL(str(so))
     V, Z, U = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_uint32
-    lib.emu_pass.argtypes = [ctypes.c_int, V, V, Z, V, Z, V, V, V, V, V, V, U, U, U]
+    lib.emu_pass.argtypes = [ctypes.c_int, V, V, Z, V, Z, V, V, V, V, V, V, U, U, U, Z, V]
     lib.emu_pass.restype = ctypes.c_int
     for name in ("emu_gf128_mul_device", "emu_gf128_mul_keysetup"):
         getattr(lib, name).argtypes = [ctypes.c_char_p] * 3
@@ -29,8 +29,8 @@ def emu(tmp_path_factory):
     return lib
 
 
-def run(lib, mode, key, iv, cb, data, n, pad=None, mask=None, tags=None, seg=8, first=0, aad=0):
-    K = (n + cb - 1) // cb
+def run(lib, mode, key, iv, cb, data, n, pad=None, mask=None, tags=None, seg=8, first=0, aad=0, sample_bytes=0, ivs=None):
+    K = (n + cb - 1) // cb if not sample_bytes else (n // sample_bytes) * ((sample_bytes + cb - 1) // cb)
     k = np.frombuffer(key, np.uint8).copy()
     v = np.frombuffer(iv, np.uint8).copy()
     src = np.ascontiguousarray(data, np.uint8) if data is not None else np.zeros(n, np.uint8)
@@ -43,7 +43,8 @@ def run(lib, mode, key, iv, cb, data, n, pad=None, mask=None, tags=None, seg=8, 
     if mode == VERIFY:
         out[:n] = src                                   # the pass does not store; keep the guard check meaningful
     rc = lib.emu_pass(mode, k.ctypes.data, v.ctypes.data, cb, src.ctypes.data, n, out.ctypes.data, pad_a.ctypes.data,
-                      mask_a.ctypes.data, tin.ctypes.data, tout.ctypes.data, ok.ctypes.data, seg, first, aad)
+                      mask_a.ctypes.data, tin.ctypes.data, tout.ctypes.data, ok.ctypes.data, seg, first, aad, sample_bytes,
+                      ivs.ctypes.data if ivs is not None else None)
     assert rc == 0 and (out[n:] == 0xA5).all()
     return out[:n], tout, ok, mask_a
 
@@ -126,3 +127,30 @@ def test_a_stage_that_starts_at_a_later_chunk(emu):
     c_ref, t_ref = oracle.mc_encrypt_framed(key, iv, cb, aad, p, 4)
     c, t, _, _ = run(emu, ENC, key, iv, cb, p[cb * first:], n, seg=8, first=first, aad=aad)
     assert np.array_equal(c, c_ref[cb * first:]) and np.array_equal(t, t_ref[first:])
+
+
+@pytest.mark.parametrize("sample_bytes,cb,n_samples,aad,seg", [(64, 16, 3, 0, 8), (1024, 1024, 5, 0, 2), (1040, 1024, 4, 16, 8),
+                                                              (3 * 4096 + 160, 4096, 6, 4, 4), (301056, 65536, 2, 16, 8)])
+def test_batch_of_samples_each_under_its_own_iv(emu, sample_bytes, cb, n_samples, aad, seg):
+    """Paper Section 4.2: every sample is its own multi-chain message; a batch is many of them in one launch."""
+    rng = np.random.default_rng(sample_bytes + n_samples)
+    key = rng.bytes(32)
+    ivs = np.frombuffer(rng.bytes(12 * n_samples), np.uint8).copy()
+    n = sample_bytes * n_samples
+    p = np.frombuffer(rng.bytes(n), np.uint8)
+    cs, ts = [], []
+    for s in range(n_samples):
+        part = p[s * sample_bytes:(s + 1) * sample_bytes]
+        iv = ivs[12 * s:12 * s + 12].tobytes()
+        c1, t1 = oracle.mc_encrypt_framed(key, iv, cb, aad, part, 2) if aad else oracle.mc_encrypt(key, iv, cb, part, 2)
+        cs.append(c1)
+        ts.append(t1)
+    c_ref, t_ref = np.concatenate(cs), np.concatenate(ts)
+    c, t, _, _ = run(emu, ENC, key, bytes(12), cb, p, n, seg=seg, aad=aad, sample_bytes=sample_bytes, ivs=ivs)
+    assert np.array_equal(c, c_ref) and np.array_equal(t, t_ref)
+    bad_t = t_ref.copy()
+    bad_t[len(bad_t) // 2, 0] ^= 1
+    out, _, ok, _ = run(emu, DEC, key, bytes(12), cb, c_ref, n, tags=bad_t, seg=seg, aad=aad, sample_bytes=sample_bytes, ivs=ivs)
+    exp = np.ones(len(bad_t), np.uint32)
+    exp[len(bad_t) // 2] = 0
+    assert np.array_equal(out, p) and np.array_equal(ok, exp)

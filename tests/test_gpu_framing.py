@@ -122,3 +122,80 @@ def test_framing_argument_range():
     assert fastrack.fastrack_ctx_set_framing(ctx, 256) == fastrack.OK
     assert fastrack.fastrack_ctx_set_framing(ctx, 0) == fastrack.OK
     fastrack.fastrack_ctx_destroy(ctx)
+
+
+@pytest.mark.parametrize("sample_bytes,cb,n_samples,chains", [(16, 16, 1, 0), (64, 16, 3, 0), (1040, 1024, 5, 16),
+                                                               (301056, 301056 // 16 // 16 * 16, 64, 16),     # ResNet-style batch
+                                                               (301056, 65536, 64, 0), (1 << 20, 1 << 16, 9, 16)])
+def test_batch_of_samples_each_under_its_own_iv(sample_bytes, cb, n_samples, chains):
+    """Paper Section 4.2: every input sample is split into n chunks with n tags, and the user encrypted every
+    sample on its own.  One launch over the batch must equal one oracle multi-chain call per sample."""
+    key, _ = synth.key_and_iv(3)
+    rng = np.random.Generator(np.random.PCG64(sample_bytes + n_samples))
+    ivs = np.frombuffer(rng.bytes(12 * n_samples), np.uint8).copy()
+    n = sample_bytes * n_samples
+    plain = synth.random_bytes(n, 3, salt=n_samples)
+    cs, ts = [], []
+    for s in range(n_samples):
+        part, iv = plain[s * sample_bytes:(s + 1) * sample_bytes], ivs[12 * s:12 * s + 12].tobytes()
+        c1, t1 = (oracle.mc_encrypt_framed(key, iv, cb, chains, part, NT) if chains else oracle.mc_encrypt(key, iv, cb, part, NT))
+        cs.append(c1)
+        ts.append(t1)
+    c_ref, t_ref = np.concatenate(cs), np.concatenate(ts)
+    K = t_ref.shape[0]
+    with fastrack.Context(key, cb) as ctx:
+        ctx.set_framing(chains)
+        st = torch.cuda.current_stream().cuda_stream
+        d_iv = dev(ivs)
+        d_p = dev(plain)
+        d_c = torch.empty_like(d_p)
+        d_t = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
+        ctx.encrypt_tag_samples(d_iv.data_ptr(), sample_bytes, n_samples, d_p.data_ptr(), d_c.data_ptr(), d_t.data_ptr(), st)
+        torch.cuda.synchronize()
+        assert np.array_equal(d_c.cpu().numpy(), c_ref)
+        assert np.array_equal(d_t.cpu().numpy().reshape(K, 16), t_ref)
+
+        bad_c, bad_t = c_ref.copy(), t_ref.copy()
+        hits = sorted({0, K // 2, K - 1})
+        for i, k in enumerate(hits):
+            if i % 2:
+                bad_t[k, 5] ^= 0x40
+            else:
+                sample, kk = divmod(k, K // n_samples)
+                bad_c[sample * sample_bytes + kk * cb] ^= 1
+        d_bc, d_bt = dev(bad_c), dev(bad_t)
+        d_ok = torch.full((K,), 7, dtype=torch.int32, device="cuda")
+        ctx.decrypt_verify_samples(d_iv.data_ptr(), sample_bytes, n_samples, d_bc.data_ptr(), d_bt.data_ptr(), d_bc.data_ptr(),
+                                   d_ok.data_ptr(), st)                                       # in place
+        torch.cuda.synchronize()
+        ok = d_ok.cpu().numpy().view(np.uint32)
+        assert [int(k) for k in np.flatnonzero(ok == 0)] == hits
+        out = d_bc.cpu().numpy()
+        diff = np.flatnonzero(out != plain)
+        assert diff.size == len([1 for i in range(len(hits)) if i % 2 == 0])                   # one flipped bit per ciphertext hit
+        # the oracle agrees sample by sample
+        for s in (0, n_samples - 1):
+            iv = ivs[12 * s:12 * s + 12].tobytes()
+            lo, cps = s * sample_bytes, K // n_samples
+            args = (key, iv, cb) + ((chains,) if chains else ()) + (bad_c[lo:lo + sample_bytes], bad_t[s * cps:(s + 1) * cps], NT)
+            p_s, ok_s = (oracle.mc_decrypt_framed(*args) if chains else oracle.mc_decrypt(*args))
+            assert np.array_equal(ok_s, ok[s * cps:(s + 1) * cps]) and np.array_equal(p_s, out[lo:lo + sample_bytes])
+
+
+def test_sample_batch_argument_errors():
+    rc, ctx = fastrack.fastrack_ctx_create(bytes(32), 1024)
+    assert rc == fastrack.OK
+    buf = torch.zeros(8192, dtype=torch.uint8, device="cuda")
+    ivs = torch.zeros(96, dtype=torch.uint8, device="cuda")
+    tags = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    ok = torch.zeros(16, dtype=torch.int32, device="cuda")
+    b, i, t, o = buf.data_ptr(), ivs.data_ptr(), tags.data_ptr(), ok.data_ptr()
+    D = fastrack.fastrack_decrypt_verify_samples
+    assert D(ctx, i, 1024, 0, b, t, b, o, 0) == fastrack.OK                 # empty batch
+    assert D(ctx, 0, 1024, 2, b, t, b, o, 0) == fastrack.ERR_ARG            # no IVs
+    assert D(ctx, i, 1000, 2, b, t, b, o, 0) == fastrack.ERR_ARG            # sample size not a multiple of 16
+    assert D(ctx, i, 0, 2, b, t, b, o, 0) == fastrack.ERR_ARG
+    assert D(ctx, i, 1024, 2, b, t, b + 16, o, 0) == fastrack.ERR_ARG       # partial overlap
+    assert D(ctx, i, 1536, 2, b, t, b + 4096, o, 0) == fastrack.OK          # 2 samples x 2 chunks (1024 + 512)
+    torch.cuda.synchronize()
+    fastrack.fastrack_ctx_destroy(ctx)

@@ -16,7 +16,7 @@ def declared_functions():
 
 def test_header_and_binding_agree():
     names = declared_functions()
-    assert len(names) >= 20
+    assert len(names) >= 22
     assert sorted(fastrack.EXPORTS) == names
 
 
@@ -54,6 +54,8 @@ def test_argument_checks_that_need_no_device():
     assert fastrack.fastrack_decrypt_verify(None, bytes(12), 0, 16, 0, 0, 0, 0) == fastrack.ERR_ARG
     assert fastrack.fastrack_encrypt_tag(None, bytes(12), 0, 16, 0, 0, 0) == fastrack.ERR_ARG
     assert fastrack.fastrack_decrypt_verify_noalloc(None, bytes(12), 0, 16, 0, 0, 0, 0) == fastrack.ERR_ARG
+    assert fastrack.fastrack_decrypt_verify_samples(None, 0, 16, 1, 0, 0, 0, 0, 0) == fastrack.ERR_ARG
+    assert fastrack.fastrack_encrypt_tag_samples(None, 0, 16, 1, 0, 0, 0, 0) == fastrack.ERR_ARG
     assert fastrack.fastrack_ctr_crypt(None, bytes(12), 0, 16, 0, 0) == fastrack.ERR_ARG
     assert fastrack.fastrack_verify(None, bytes(12), 0, 16, 0, 0, 0) == fastrack.ERR_ARG
     assert fastrack.fastrack_keystream(None, bytes(12), 16, 0, 0, 0) == fastrack.ERR_ARG
