@@ -493,6 +493,37 @@ def run_sweep(args):
             assert bool((d_ok == 1).all())
         print(json.dumps(out), flush=True)
 
+    def samples_cell(sample_bytes, n_samples, chains, label):
+        """The paper's data model: a batch of samples, each split into `chains` chunks under its own IV."""
+        cb = (sample_bytes // chains + 15) // 16 * 16
+        with fastrack.Context(key, cb) as ctx:
+            ctx.set_framing(chains)
+            st = stream.cuda_stream
+            n = sample_bytes * n_samples
+            K = n_samples * ((sample_bytes + cb - 1) // cb)
+            d_iv = torch.randint(0, 256, (12 * n_samples,), dtype=torch.uint8, device="cuda")
+            d_p = torch.randint(0, 256, (n,), dtype=torch.uint8, device="cuda")
+            d_c, d_o = torch.empty_like(d_p), torch.empty_like(d_p)
+            d_t = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
+            d_ok = torch.zeros(K, dtype=torch.int32, device="cuda")
+            ctx.encrypt_tag_samples(d_iv.data_ptr(), sample_bytes, n_samples, d_p.data_ptr(), d_c.data_ptr(), d_t.data_ptr(), st)
+            t_batch = timed(lambda: ctx.decrypt_verify_samples(d_iv.data_ptr(), sample_bytes, n_samples, d_c.data_ptr(),
+                                                               d_t.data_ptr(), d_o.data_ptr(), d_ok.data_ptr(), st), 100)
+            assert bool((d_ok == 1).all()) and bool((d_o == d_p).all())
+            ivs_h = d_iv.cpu().numpy().tobytes()
+            cps = K // n_samples
+
+            def one_by_one():
+                for s in range(n_samples):
+                    ctx.decrypt_verify(ivs_h[12 * s:12 * s + 12], d_c.data_ptr() + s * sample_bytes, sample_bytes,
+                                       d_t.data_ptr() + 16 * cps * s, d_o.data_ptr() + s * sample_bytes,
+                                       d_ok.data_ptr() + 4 * cps * s, st)
+            t_each = timed(one_by_one, 20)
+            assert bool((d_ok == 1).all()) and bool((d_o == d_p).all())
+        print(json.dumps({"cell": label, "sample_bytes": sample_bytes, "n_samples": n_samples, "chains_per_sample": chains,
+                          "chunk": cb, "batch_call_us": t_batch * 1e6, "batch_call_gbs": n / t_batch / 1e9,
+                          "one_call_per_sample_us": t_each * 1e6}), flush=True)
+
     for K in (1, 4, 16, 64, 256, 1024):                                   # config 1
         device_cell(64 << 20, (64 << 20) // K, "config1")
     for cb in (256 << 10, 1 << 20, 4 << 20, 8 << 20):                     # config 2
@@ -501,6 +532,8 @@ def run_sweep(args):
     device_cell(670_000_000, 4 << 20, "config3")
     for ns in (2, 4):
         d2h_cell(670_000_000, 4 << 20, ns, "config3_d2h")
+    samples_cell(3 * 224 * 224 * 2, 64, 16, "sample_batch")        # a ResNet-style batch: 64 fp16 images, 16 tags each
+    samples_cell(3 * 224 * 224 * 2, 256, 16, "sample_batch")
     modes_cell(256 << 20, 4 << 20, "split_passes")
     for K in (16, 64, 256, 1024, 4096):
         modes_cell(64 << 20, (64 << 20) // K, "split_passes_vs_K")
