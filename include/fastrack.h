@@ -165,6 +165,13 @@ FASTRACK_API int fastrack_encrypt_tag_samples(fastrack_ctx* ctx, const void* d_i
                                               size_t n_samples, const void* d_plain, void* d_cipher, void* d_tags,
                                               void* stream);
 
+/* fastrack_pipelined_h2d for such a batch (Sections 4.2 + 4.3 together): the batch sits in pinned host memory, its
+ * IV bases (HOST pointer here, 12 * n_samples bytes, pinned or pageable) and tags travel with it; stages are whole
+ * samples.  Blocking; everything else as in fastrack_pipelined_h2d and fastrack_decrypt_verify_samples. */
+FASTRACK_API int fastrack_pipelined_h2d_samples(fastrack_ctx* ctx, const void* h_iv_bases, size_t sample_bytes,
+                                                size_t n_samples, const void* h_cipher_pinned, const void* h_tags,
+                                                void* d_plain, uint32_t* d_ok, int n_streams);
+
 /* ---- Split passes (paper Section 4.3, "Eager evaluation") -------------------------------------------------
  * The paper lets the consumer start on the decrypted data before authentication has finished and runs the
  * authentication kernel later, in parallel with the next batch's PCIe transfer; results are discarded if the

@@ -594,9 +594,9 @@ extern "C" int fastrack_encrypt_tag(fastrack_ctx* ctx, const uint8_t iv_base[12]
 // the buffer, then three quarters of the rest, ... down to about 2 MiB (never less than one chunk) -- few copies,
 // and a short exposed kernel.  A stage's kernel is 6-9 times faster than a copy of the same size, so it still
 // finishes under the next stage's copy, which is a quarter as large.  Returns the stage sizes in descending order (host->device order).
-static size_t plan_stages(const fastrack_ctx* ctx, size_t len, size_t out[FR_MAX_STAGES])
+static size_t plan_stages(const fastrack_ctx* ctx, size_t len, size_t unit, size_t out[FR_MAX_STAGES])
 {
-    const size_t cb = ctx->chunk_bytes;
+    const size_t cb = unit;        // stages are whole multiples of this (a chunk, or a sample in a batch of samples)
     const size_t floor_bytes = (size_t)2 << 20;
     const size_t min_stage = cb >= floor_bytes ? cb : (floor_bytes + cb - 1) / cb * cb;
     size_t off = 0, count = 0;
@@ -621,9 +621,10 @@ static size_t plan_stages(const fastrack_ctx* ctx, size_t len, size_t out[FR_MAX
 // d_pad != nullptr: the keystream for the whole buffer is produced first, on a stream of its own, while the
 // first copy is in flight; the stages then only XOR and authenticate.
 static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* h_cipher_pinned, size_t len,
-                          const void* h_tags, void* d_pad, void* d_plain, uint32_t* d_ok, int n_streams)
+                          const void* h_tags, void* d_pad, void* d_plain, uint32_t* d_ok, int n_streams,
+                          const void* h_iv_bases = nullptr, size_t sample_bytes = 0)
 {
-    if (!ctx || !iv_base) return FASTRACK_ERR_ARG;
+    if (!ctx || (!iv_base && !h_iv_bases)) return FASTRACK_ERR_ARG;
     if (n_streams < 1 || n_streams > 8) return FASTRACK_ERR_ARG;
     if (len == 0) return FASTRACK_OK;
     if (!h_cipher_pinned || !h_tags || !d_plain || !d_ok) return FASTRACK_ERR_ARG;
@@ -633,18 +634,21 @@ static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const vo
     cudaError_t e = cudaPointerGetAttributes(&attr, h_cipher_pinned);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return FASTRACK_ERR_NOT_PINNED; }
     if (attr.type != cudaMemoryTypeHost) return FASTRACK_ERR_NOT_PINNED;
-    const size_t K = fastrack_num_chunks(ctx, len);
+    const size_t cps = sample_bytes ? (sample_bytes + ctx->chunk_bytes - 1) / ctx->chunk_bytes : 0;
+    const size_t n_samples = sample_bytes ? len / sample_bytes : 0;
+    const size_t K = sample_bytes ? cps * n_samples : fastrack_num_chunks(ctx, len);
     if (K > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
     int rc = ensure_scratch(ctx, K);
     if (rc != FASTRACK_OK) return rc;
-    if (K > ctx->tags_stage_chunks) {
+    const size_t need_slots = K + (12 * n_samples + 15) / 16;      // tags, then (batch of samples) the IV bases
+    if (need_slots > ctx->tags_stage_chunks) {
         size_t cap = ctx->tags_stage_chunks ? ctx->tags_stage_chunks : 1024;
-        while (cap < K) cap *= 2;
+        while (cap < need_slots) cap *= 2;
         FR_CUDA(ctx, cudaDeviceSynchronize());
         cudaFree(ctx->d_tags_stage);
         ctx->d_tags_stage = nullptr;
         ctx->tags_stage_chunks = 0;
-        e = cudaMalloc(&ctx->d_tags_stage, cap * 32);       // tags, then the E_K(J0) masks of the keystream-ahead variant
+        e = cudaMalloc(&ctx->d_tags_stage, cap * 32);       // tags (+ IV bases), then the E_K(J0) masks of the keystream-ahead variant
         if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); return FASTRACK_ERR_NOMEM; }
         ctx->tags_stage_chunks = cap;
     }
@@ -657,12 +661,13 @@ static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const vo
     bool waited[8] = {false, false, false, false, false, false, false, false};   // per working stream: events already awaited
 
     size_t stage_bytes[FR_MAX_STAGES];
-    const size_t n_stages = plan_stages(ctx, len, stage_bytes);
     const size_t cb = ctx->chunk_bytes;
+    const size_t n_stages = plan_stages(ctx, len, sample_bytes ? sample_bytes : cb, stage_bytes);
+    uint8_t* d_ivs = (uint8_t*)(ctx->d_tags_stage + K);            // batch of samples: device copy of the IV bases
     size_t off = 0;
     for (size_t stage = 0; stage < n_stages; stage++) {
         const size_t n = stage_bytes[stage];
-        const size_t k0 = off / cb;
+        const size_t k0 = sample_bytes ? (off / sample_bytes) * cps : off / cb;
         cudaStream_t st = ctx->streams[stage % (size_t)n_streams];
         uint8_t* dst = (uint8_t*)d_plain + off;
         rc = FASTRACK_OK;
@@ -673,6 +678,8 @@ static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const vo
         if (tracing) cudaEventRecord(ctx->trace_ev[3 * stage + 1], st);
         if (rc == FASTRACK_OK && stage == 0) {
             e = cudaMemcpyAsync(ctx->d_tags_stage, h_tags, K * 16, cudaMemcpyHostToDevice, tag_stream);
+            if (e == cudaSuccess && sample_bytes)
+                e = cudaMemcpyAsync(d_ivs, h_iv_bases, 12 * n_samples, cudaMemcpyHostToDevice, tag_stream);
             if (e == cudaSuccess) e = cudaEventRecord(ctx->tags_ready, tag_stream);
             if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); rc = FASTRACK_ERR_CUDA; }
             if (rc == FASTRACK_OK && d_pad) {
@@ -695,6 +702,7 @@ static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const vo
         if (rc == FASTRACK_OK) {
             PassBuffers b;
             b.in = dst; b.out = dst; b.tags_in = ctx->d_tags_stage + k0; b.ok = d_ok + k0;
+            if (sample_bytes) { b.ivs = d_ivs + 12 * (off / sample_bytes); b.sample_bytes = sample_bytes; }
             if (d_pad) { b.pad = (const uint8_t*)d_pad + off; b.mask = d_mask + k0; }
             rc = launch_pass(ctx, d_pad ? FR_MODE_PADDEC : FR_MODE_DEC, iv_base, k0, n, b, st);
         }
@@ -730,6 +738,17 @@ extern "C" int fastrack_pipelined_h2d(fastrack_ctx* ctx, const uint8_t iv_base[1
                                       const void* h_tags, void* d_plain, uint32_t* d_ok, int n_streams)
 {
     return pipelined_impl(ctx, iv_base, h_cipher_pinned, len, h_tags, nullptr, d_plain, d_ok, n_streams);
+}
+
+extern "C" int fastrack_pipelined_h2d_samples(fastrack_ctx* ctx, const void* h_iv_bases, size_t sample_bytes, size_t n_samples,
+                                              const void* h_cipher_pinned, const void* h_tags, void* d_plain, uint32_t* d_ok,
+                                              int n_streams)
+{
+    if (!ctx || !h_iv_bases) return FASTRACK_ERR_ARG;
+    if (sample_bytes == 0 || (sample_bytes & 15)) return FASTRACK_ERR_ARG;
+    if (n_samples > ((size_t)1 << 40) / sample_bytes) return FASTRACK_ERR_TOO_MANY;
+    return pipelined_impl(ctx, nullptr, h_cipher_pinned, sample_bytes * n_samples, h_tags, nullptr, d_plain, d_ok, n_streams,
+                          h_iv_bases, sample_bytes);
 }
 
 extern "C" int fastrack_pipelined_h2d_ahead(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* h_cipher_pinned,
@@ -772,7 +791,7 @@ extern "C" int fastrack_pipelined_d2h(fastrack_ctx* ctx, const uint8_t iv_base[1
     // short last chunk, if any, stays at the end of the last (largest) stage.
     size_t stage_bytes[FR_MAX_STAGES];
     const size_t cb = ctx->chunk_bytes;
-    const size_t n_stages = plan_stages(ctx, K * cb, stage_bytes);
+    const size_t n_stages = plan_stages(ctx, K * cb, cb, stage_bytes);
     size_t off = 0;
     for (size_t i = 0; i < n_stages; i++) {
         size_t n = stage_bytes[n_stages - 1 - i];

@@ -23,7 +23,7 @@ EXPORTS = ("fastrack_ctx_create", "fastrack_ctx_destroy", "fastrack_num_chunks",
            "fastrack_pipelined_h2d", "fastrack_launch_count", "fastrack_decrypt_verify_noalloc",
            "fastrack_ctr_crypt", "fastrack_verify", "fastrack_keystream", "fastrack_xor_verify",
            "fastrack_pipelined_h2d_ahead", "fastrack_ctx_set_framing", "fastrack_verify_sequential", "fastrack_pipelined_d2h", "fastrack_ctx_set_trace", "fastrack_ctx_get_trace",
-           "fastrack_decrypt_verify_samples", "fastrack_encrypt_tag_samples")
+           "fastrack_decrypt_verify_samples", "fastrack_encrypt_tag_samples", "fastrack_pipelined_h2d_samples")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2410_15240_b200.build` "
@@ -64,6 +64,8 @@ _lib.fastrack_decrypt_verify_samples.restype = _int
 _lib.fastrack_decrypt_verify_samples.argtypes = [_vp, _vp, _sz, _sz, _vp, _vp, _vp, _vp, _vp]
 _lib.fastrack_encrypt_tag_samples.restype = _int
 _lib.fastrack_encrypt_tag_samples.argtypes = [_vp, _vp, _sz, _sz, _vp, _vp, _vp, _vp]
+_lib.fastrack_pipelined_h2d_samples.restype = _int
+_lib.fastrack_pipelined_h2d_samples.argtypes = [_vp, _vp, _sz, _sz, _vp, _vp, _vp, _vp, _int]
 _lib.fastrack_ctr_crypt.restype = _int
 _lib.fastrack_ctr_crypt.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp]
 _lib.fastrack_verify.restype = _int
@@ -167,6 +169,12 @@ def fastrack_encrypt_tag_samples(ctx, d_iv_bases: int, sample_bytes: int, n_samp
     return _lib.fastrack_encrypt_tag_samples(ctx, d_iv_bases, sample_bytes, n_samples, d_plain, d_cipher, d_tags, stream)
 
 
+def fastrack_pipelined_h2d_samples(ctx, h_iv_bases: int, sample_bytes: int, n_samples: int, h_cipher_pinned: int,
+                                   h_tags: int, d_plain: int, d_ok: int, n_streams: int) -> int:
+    return _lib.fastrack_pipelined_h2d_samples(ctx, h_iv_bases, sample_bytes, n_samples, h_cipher_pinned, h_tags, d_plain,
+                                               d_ok, n_streams)
+
+
 def fastrack_ctr_crypt(ctx, iv_base: bytes, d_in: int, length: int, d_out: int, stream: int = 0) -> int:
     return _lib.fastrack_ctr_crypt(ctx, iv_base, d_in, length, d_out, stream)
 
@@ -250,6 +258,11 @@ class Context:
     def encrypt_tag_samples(self, d_iv_bases, sample_bytes, n_samples, d_plain, d_cipher, d_tags, stream=0) -> None:
         self._check(fastrack_encrypt_tag_samples(self.handle, d_iv_bases, sample_bytes, n_samples, d_plain, d_cipher,
                                                  d_tags, stream))
+
+    def pipelined_h2d_samples(self, h_iv_bases, sample_bytes, n_samples, h_cipher_pinned, h_tags, d_plain, d_ok,
+                              n_streams=4) -> None:
+        self._check(fastrack_pipelined_h2d_samples(self.handle, h_iv_bases, sample_bytes, n_samples, h_cipher_pinned, h_tags,
+                                                   d_plain, d_ok, n_streams))
 
     def ctr_crypt(self, iv_base, d_in, length, d_out, stream=0) -> None:
         self._check(fastrack_ctr_crypt(self.handle, iv_base, d_in, length, d_out, stream))

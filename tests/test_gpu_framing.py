@@ -199,3 +199,38 @@ def test_sample_batch_argument_errors():
     assert D(ctx, i, 1536, 2, b, t, b + 4096, o, 0) == fastrack.OK          # 2 samples x 2 chunks (1024 + 512)
     torch.cuda.synchronize()
     fastrack.fastrack_ctx_destroy(ctx)
+
+
+@pytest.mark.parametrize("sample_bytes,cb,n_samples,chains,n_streams", [(1040, 1024, 5, 16, 1), (301056, 18816, 64, 16, 3),
+                                                                        (1 << 20, 1 << 16, 9, 0, 2)])
+def test_pipelined_h2d_of_a_batch_of_samples(sample_bytes, cb, n_samples, chains, n_streams):
+    """The inference input path of the paper: an encrypted batch of samples arrives in pinned host memory."""
+    key, _ = synth.key_and_iv(3)
+    rng = np.random.Generator(np.random.PCG64(sample_bytes + n_samples + 1))
+    ivs = np.frombuffer(rng.bytes(12 * n_samples), np.uint8).copy()
+    n = sample_bytes * n_samples
+    plain = synth.random_bytes(n, 3, salt=n_samples + 100)
+    cs, ts = [], []
+    for s in range(n_samples):
+        part, iv = plain[s * sample_bytes:(s + 1) * sample_bytes], ivs[12 * s:12 * s + 12].tobytes()
+        c1, t1 = (oracle.mc_encrypt_framed(key, iv, cb, chains, part, NT) if chains else oracle.mc_encrypt(key, iv, cb, part, NT))
+        cs.append(c1)
+        ts.append(t1)
+    c, t = np.concatenate(cs), np.concatenate(ts)
+    K = t.shape[0]
+    t[K // 3, 2] ^= 8
+    c[n - 1] ^= 0x80
+    with fastrack.Context(key, cb) as ctx:
+        ctx.set_framing(chains)
+        h_c = torch.from_numpy(c).pin_memory()
+        h_t = torch.from_numpy(t.reshape(-1).copy())
+        d_p = torch.empty(n, dtype=torch.uint8, device="cuda")
+        d_ok = torch.full((K,), 7, dtype=torch.int32, device="cuda")
+        torch.cuda.synchronize()
+        for _ in range(2):
+            ctx.pipelined_h2d_samples(ivs.ctypes.data, sample_bytes, n_samples, h_c.data_ptr(), h_t.data_ptr(), d_p.data_ptr(),
+                                      d_ok.data_ptr(), n_streams)
+            ok = d_ok.cpu().numpy().view(np.uint32)
+            assert [int(k) for k in np.flatnonzero(ok == 0)] == sorted({K // 3, K - 1})
+            out = d_p.cpu().numpy()
+            assert np.flatnonzero(out != plain).tolist() == [n - 1]

@@ -16,7 +16,7 @@ def declared_functions():
 
 def test_header_and_binding_agree():
     names = declared_functions()
-    assert len(names) >= 22
+    assert len(names) >= 23
     assert sorted(fastrack.EXPORTS) == names
 
 
@@ -56,6 +56,7 @@ def test_argument_checks_that_need_no_device():
     assert fastrack.fastrack_decrypt_verify_noalloc(None, bytes(12), 0, 16, 0, 0, 0, 0) == fastrack.ERR_ARG
     assert fastrack.fastrack_decrypt_verify_samples(None, 0, 16, 1, 0, 0, 0, 0, 0) == fastrack.ERR_ARG
     assert fastrack.fastrack_encrypt_tag_samples(None, 0, 16, 1, 0, 0, 0, 0) == fastrack.ERR_ARG
+    assert fastrack.fastrack_pipelined_h2d_samples(None, 0, 16, 1, 0, 0, 0, 0, 2) == fastrack.ERR_ARG
     assert fastrack.fastrack_ctr_crypt(None, bytes(12), 0, 16, 0, 0) == fastrack.ERR_ARG
     assert fastrack.fastrack_verify(None, bytes(12), 0, 16, 0, 0, 0) == fastrack.ERR_ARG
     assert fastrack.fastrack_keystream(None, bytes(12), 16, 0, 0, 0) == fastrack.ERR_ARG
