@@ -1,23 +1,27 @@
 // fastrack_device.cuh -- per-lane device code of the fused AES-256-CTR + GHASH pass (sm_100a).
 //
-// One warp works on one "segment": a run of consecutive rows of one chunk, a row being 32 consecutive
-// 16-byte blocks (512 B, one block per lane, so global loads and stores are 128-bit and coalesced).
+// One warp works on one "segment": a run of consecutive rows of one chunk.  A row is 32 consecutive counter
+// values, lane = counter mod 32, and the block at counter c is data block c - 2 of the chunk (GCM keeps
+// counter 1 for the tag mask), so a row is 512 contiguous bytes and global loads and stores are 128-bit and
+// coalesced.  Counter 1 of row 0 is a spare lane: it yields E_K(J0), and with the serial-number framing it
+// also absorbs the one-byte AAD block.
 //
 // AES (paper Section 2.3, "The AES block cipher": AES in counter mode, every block independent):
 //   four round tables Te0..Te3 live in shared memory, each entry replicated 32 times so that lane l
 //   only ever touches bank l -- a table lookup is one conflict-free wavefront whatever the index.
 //   Row v of array T01 is [Te0[v] x32 | Te1[v] x32] (256 B), array T23 likewise; the byte address
 //   v*256 + 4*lane is produced by ONE byte-permute from the state word and the lane register.
+//   Rounds 1 and 2 are shared by the 256 counters that differ only in their last byte.
 //
 // GHASH (paper Section 2.3, "Authentication with Galois Field"; Section 4.2 shortens the chain by
 // chunking, here every chain is additionally evaluated as a power sum):
-//   lane l of the warp folds blocks l, l+32, l+64, ... with Horner's rule and the FIXED multiplier
+//   a lane folds its blocks (every 32nd block of the segment) with Horner's rule and the FIXED multiplier
 //   H^32, Y <- (Y xor X) * H^32, using byte tables of H^32 in shared memory (entry for byte position p
 //   and byte value v at v*256 + p*16).  Lanes walk the 16 byte positions in a lane-dependent order
 //   (position = step xor (lane & 7)) so that the eight lanes of a quarter-warp always hit eight
 //   different 16-byte bank groups: every 128-bit lookup is conflict-free.  The lane's last block is
 //   not multiplied by H^32 but by the power of H that its distance from the end of the chunk calls
-//   for, with a general (bit-serial) product; the 32 lane values are then XOR-reduced.
+//   for, with a general product built from integer multiplies; the 32 lane values are then XOR-reduced.
 #pragma once
 #include <stdint.h>
 
