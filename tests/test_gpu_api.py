@@ -85,3 +85,34 @@ def test_calls_are_asynchronous_and_ordered_on_the_stream():
         assert bool((d_back == d_p).all()) and bool((d_ok == 1).all())
         c_ref, t_ref = oracle.mc_encrypt(key, iv, cb, plain, oracle.host_threads())
         assert np.array_equal(d_c.cpu().numpy(), c_ref) and np.array_equal(d_t.cpu().numpy().reshape(K, 16), t_ref)
+
+
+def test_long_dependent_chain_without_host_synchronisation():
+    """100 x (encrypt A->B, decrypt B->A, verify-only, in place) queued on one stream with no host sync, on two
+    contexts with different keys taking turns: every kernel's table build may overlap its predecessor's tail,
+    the data dependencies must still hold."""
+    key1, iv = synth.key_and_iv(0)
+    key2, _ = synth.key_and_iv(1)
+    cb, n = 65536, (2 << 20) + 4096 + 16
+    K = (n + cb - 1) // cb
+    plain = synth.random_bytes(n, 0, salt=31)
+    with fastrack.Context(key1, cb) as c1, fastrack.Context(key2, cb) as c2:
+        st = torch.cuda.Stream()
+        a = torch.from_numpy(plain).cuda()
+        b = torch.empty_like(a)
+        tags = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
+        oks = torch.zeros(100, K, dtype=torch.int32, device="cuda")
+        oks2 = torch.zeros(100, K, dtype=torch.int32, device="cuda")
+        torch.cuda.synchronize()
+        with torch.cuda.stream(st):
+            for i in range(100):
+                ctx = c1 if i % 2 == 0 else c2
+                ctx.encrypt_tag(iv, a.data_ptr(), n, b.data_ptr(), tags.data_ptr(), st.cuda_stream)
+                ctx.verify(iv, b.data_ptr(), n, tags.data_ptr(), oks2[i].data_ptr(), st.cuda_stream)
+                a.zero_()                                                   # a torch kernel in between
+                ctx.decrypt_verify(iv, b.data_ptr(), n, tags.data_ptr(), a.data_ptr(), oks[i].data_ptr(), st.cuda_stream)
+        st.synchronize()
+        assert bool((oks == 1).all()) and bool((oks2 == 1).all())
+        assert np.array_equal(a.cpu().numpy(), plain)
+        c_ref, _ = oracle.mc_encrypt(key2, iv, cb, plain, oracle.host_threads())       # the last round used key 2
+        assert np.array_equal(b.cpu().numpy(), c_ref)
