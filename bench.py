@@ -570,6 +570,21 @@ def run_trace(args):
         print(json.dumps({"len": n, "chunk": cb, "streams": ns, "stages": best}), flush=True)
 
 
+def run_peaks(args):
+    """Unit rates behind the kernel roofline, measured on this GPU (integer pipes, shared-memory lookups, PCIe)."""
+    import ctypes
+    from paper_2410_15240_b200 import build as lib_build
+    lib_build.build()
+    lib = ctypes.CDLL(lib_build.PROBE_LIB)
+    lib.fastrack_probe_peaks.argtypes = [ctypes.c_char_p, ctypes.c_size_t]
+    lib.fastrack_probe_peaks.restype = ctypes.c_int
+    buf = ctypes.create_string_buffer(1 << 16)
+    rc = lib.fastrack_probe_peaks(buf, len(buf))
+    sys.stdout.write(buf.value.decode())
+    if rc != 0:
+        raise RuntimeError(f"probe failed with CUDA error {rc}")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -582,8 +597,11 @@ def main():
     ap.add_argument("--sweep", action="store_true",
                     help="print throughput over the benchmark configurations instead of the one bench line")
     ap.add_argument("--trace", action="store_true", help="print stage-level timelines of the pipelined H2D call")
+    ap.add_argument("--peaks", action="store_true", help="measure the unit rates the kernel roofline is derived from")
     args = ap.parse_args()
-    if args.trace:
+    if args.peaks:
+        run_peaks(args)
+    elif args.trace:
         run_trace(args)
     elif args.sweep:
         run_sweep(args)

@@ -16,15 +16,25 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", 
               "-shared", "-Xcompiler", "-fPIC,-fvisibility=hidden"]
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile libfastrack.so if it is missing or older than its sources.  Returns its path."""
-    stale = (not os.path.exists(LIB)) or any(os.path.getmtime(LIB) < os.path.getmtime(d) for d in DEPS)
+PROBE_LIB = os.path.join(HERE, "libfastrack_probe.so")
+PROBE_SRC = os.path.join(CSRC, "peaks_probe.cu")
+
+
+def _compile(target: str, sources, deps, force: bool, verbose: bool) -> None:
+    stale = (not os.path.exists(target)) or any(os.path.getmtime(target) < os.path.getmtime(d) for d in deps)
     if force or stale:
         nvcc = os.environ.get("NVCC", "nvcc")
-        tmp = LIB + f".{os.getpid()}.tmp"
-        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + SOURCES
+        tmp = target + f".{os.getpid()}.tmp"
+        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + list(sources)
         subprocess.check_call(cmd)
-        os.replace(tmp, LIB)
+        os.replace(tmp, target)
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    """Compile libfastrack.so (and the small peak-rate probe library) if missing or older than their sources.
+    Returns the path of libfastrack.so."""
+    _compile(LIB, SOURCES, DEPS, force, verbose)
+    _compile(PROBE_LIB, [PROBE_SRC], [PROBE_SRC], force, False)
     return LIB
 
 

@@ -1,0 +1,201 @@
+// peaks_probe.cu -- measures, on the GPU at hand, the unit rates the kernel roofline is derived from:
+// integer-pipe throughput (LOP3, PRMT, SHF on the ALU pipe; IMAD and 32x32->64 multiplies on the FMA pipe),
+// shared-memory lookup throughput (conflict-free and random, 32-bit and 128-bit), and pinned PCIe bandwidth.
+// Built into its own small library (libfastrack_probe.so); `python bench.py --peaks` prints its results.
+// It shares nothing with the data path and is not needed to use the library.
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+namespace {
+
+constexpr int ITERS = 2048;
+
+template <int MODE>
+__global__ void alu_kernel(uint32_t* out, uint32_t seed, long long* cyc)
+{
+    uint32_t a0 = threadIdx.x + seed, a1 = a0 * 3, a2 = a0 * 5, a3 = a0 * 7, a4 = a0 * 11, a5 = a0 * 13, a6 = a0 * 17, a7 = a0 * 19;
+    uint32_t b = seed ^ 0x9e3779b9u, c = seed * 0x85ebca6bu + blockIdx.x;
+    const long long t0 = clock64();
+#pragma unroll 1
+    for (int i = 0; i < ITERS; i++) {
+#pragma unroll
+        for (int u = 0; u < 4; u++) {
+#define FR_LOP(x) asm volatile("lop3.b32 %0, %0, %1, %2, 0x78;" : "+r"(x) : "r"(b), "r"(c));
+#define FR_PRM(x) asm volatile("prmt.b32 %0, %0, %1, 0x5140;" : "+r"(x) : "r"(b));
+#define FR_MAD(x) asm volatile("mad.lo.u32 %0, %0, %1, %2;" : "+r"(x) : "r"(b), "r"(c));
+#define FR_SHF(x) asm volatile("shf.r.wrap.b32 %0, %0, %1, 7;" : "+r"(x) : "r"(b));
+            if (MODE == 0) { FR_LOP(a0) FR_LOP(a1) FR_LOP(a2) FR_LOP(a3) FR_LOP(a4) FR_LOP(a5) FR_LOP(a6) FR_LOP(a7) }
+            else if (MODE == 1) { FR_PRM(a0) FR_PRM(a1) FR_PRM(a2) FR_PRM(a3) FR_PRM(a4) FR_PRM(a5) FR_PRM(a6) FR_PRM(a7) }
+            else if (MODE == 2) { FR_MAD(a0) FR_MAD(a1) FR_MAD(a2) FR_MAD(a3) FR_MAD(a4) FR_MAD(a5) FR_MAD(a6) FR_MAD(a7) }
+            else if (MODE == 3) { FR_SHF(a0) FR_SHF(a1) FR_SHF(a2) FR_SHF(a3) FR_SHF(a4) FR_SHF(a5) FR_SHF(a6) FR_SHF(a7) }
+            else if (MODE == 4) { FR_LOP(a0) FR_MAD(a1) FR_LOP(a2) FR_MAD(a3) FR_LOP(a4) FR_MAD(a5) FR_LOP(a6) FR_MAD(a7) }
+            else if (MODE == 5) { FR_LOP(a0) FR_PRM(a1) FR_LOP(a2) FR_PRM(a3) FR_LOP(a4) FR_PRM(a5) FR_LOP(a6) FR_PRM(a7) }
+            else {                                   // 32 x 32 -> 64 multiplies (four per pass, each result consumed)
+                unsigned long long w0, w1, w2, w3;
+                asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w0) : "r"(a0), "r"(b));
+                asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w1) : "r"(a2), "r"(b));
+                asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w2) : "r"(a4), "r"(b));
+                asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w3) : "r"(a6), "r"(b));
+                a0 = (uint32_t)w0; a1 ^= (uint32_t)(w0 >> 32); a2 = (uint32_t)w1; a3 ^= (uint32_t)(w1 >> 32);
+                a4 = (uint32_t)w2; a5 ^= (uint32_t)(w2 >> 32); a6 = (uint32_t)w3; a7 ^= (uint32_t)(w3 >> 32);
+            }
+#undef FR_LOP
+#undef FR_PRM
+#undef FR_MAD
+#undef FR_SHF
+        }
+    }
+    const long long t1 = clock64();
+    const uint32_t r = a0 ^ a1 ^ a2 ^ a3 ^ a4 ^ a5 ^ a6 ^ a7;
+    if (r == 0x12345678u) out[0] = r;
+    if (threadIdx.x == 0 && blockIdx.x == 0) cyc[0] = t1 - t0;
+}
+
+// Dependent lookups in a 64 KiB shared table.  MODE 0: 32-bit, row = data byte, bank = lane (conflict-free).
+// MODE 1: 32-bit, random word of a 1 KiB table.  MODE 2: 128-bit, row = data byte, 16-byte slot = lane & 7.
+// MODE 3: 128-bit, random entry.
+template <int MODE>
+__global__ void lds_kernel(uint32_t* out, uint32_t seed, long long* cyc)
+{
+    extern __shared__ __align__(16) uint32_t sm[];
+    for (int i = threadIdx.x; i < 65536 / 4; i += blockDim.x) sm[i] = (i * 2654435761u) ^ seed;
+    __syncthreads();
+    const uint32_t lane = threadIdx.x & 31;
+    uint32_t x0 = threadIdx.x * 2654435761u + seed, x1 = x0 * 3 + 1, x2 = x0 * 5 + 2, x3 = x0 * 7 + 3;
+    const char* base = (const char*)sm;
+    const long long t0 = clock64();
+#pragma unroll 1
+    for (int i = 0; i < ITERS; i++) {
+#pragma unroll
+        for (int u = 0; u < 4; u++) {
+            if (MODE == 0) {
+#define FR_OP(q) q = *(const uint32_t*)(base + __byte_perm(q, lane * 4, 0x5514));
+                FR_OP(x0) FR_OP(x1) FR_OP(x2) FR_OP(x3)
+#undef FR_OP
+            } else if (MODE == 1) {
+#define FR_OP(q) q = *(const uint32_t*)(base + (q & 0x3fc));
+                FR_OP(x0) FR_OP(x1) FR_OP(x2) FR_OP(x3)
+#undef FR_OP
+            } else if (MODE == 2) {
+#define FR_OP(q) { uint4 v = *(const uint4*)(base + __byte_perm(q, (lane & 7) << 4, 0x5514)); q = v.x ^ v.y ^ v.z ^ v.w; }
+                FR_OP(x0) FR_OP(x1) FR_OP(x2) FR_OP(x3)
+#undef FR_OP
+            } else {
+#define FR_OP(q) { uint4 v = *(const uint4*)(base + (q & 0xfff0)); q = v.x ^ v.y ^ v.z ^ v.w; }
+                FR_OP(x0) FR_OP(x1) FR_OP(x2) FR_OP(x3)
+#undef FR_OP
+            }
+        }
+    }
+    const long long t1 = clock64();
+    const uint32_t r = x0 ^ x1 ^ x2 ^ x3;
+    if (r == 0x12345678u) out[0] = r;
+    if (threadIdx.x == 0 && blockIdx.x == 0) cyc[0] = t1 - t0;
+}
+
+struct Out {
+    char* buf;
+    size_t cap, used;
+    void add(const char* line)
+    {
+        const size_t n = strlen(line);
+        if (used + n + 2 <= cap) { memcpy(buf + used, line, n); used += n; buf[used++] = '\n'; buf[used] = 0; }
+    }
+};
+
+template <typename F>
+void measure(Out& o, const char* name, F launch, double ops_per_thread, int threads_per_sm)
+{
+    cudaEvent_t e0, e1;
+    cudaEventCreate(&e0);
+    cudaEventCreate(&e1);
+    long long* d_cyc = nullptr;
+    cudaMalloc(&d_cyc, 8);
+    for (int i = 0; i < 3; i++) launch(d_cyc);
+    cudaDeviceSynchronize();
+    cudaEventRecord(e0);
+    const int reps = 5;
+    for (int i = 0; i < reps; i++) launch(d_cyc);
+    cudaEventRecord(e1);
+    cudaDeviceSynchronize();
+    float ms = 0;
+    cudaEventElapsedTime(&ms, e0, e1);
+    long long cyc = 1;
+    cudaMemcpy(&cyc, d_cyc, 8, cudaMemcpyDeviceToHost);
+    char line[256];
+    snprintf(line, sizeof line, "{\"probe\": \"%s\", \"us\": %.1f, \"sm_mhz\": %.0f, \"thread_ops_per_clk_per_sm\": %.2f}", name,
+             ms * 1e3 / reps, cyc / (ms * 1e-3 / reps) / 1e6, ops_per_thread * threads_per_sm / (double)cyc);
+    o.add(line);
+    cudaFree(d_cyc);
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+}
+
+}  // namespace
+
+// Runs every probe on the current device and writes one JSON object per line into `out` (NUL-terminated).
+// Returns 0, or a CUDA error code.  Takes a few seconds; allocates up to 256 MiB of device and pinned host memory.
+extern "C" __attribute__((visibility("default"))) int fastrack_probe_peaks(char* out, size_t cap)
+{
+    if (!out || cap < 64) return -1;
+    Out o = {out, cap, 0};
+    out[0] = 0;
+    cudaDeviceProp prop;
+    cudaError_t e = cudaGetDeviceProperties(&prop, 0);
+    if (e != cudaSuccess) return (int)e;
+    const int nsm = prop.multiProcessorCount, T = 1024;
+    char line[512];
+    snprintf(line, sizeof line, "{\"device\": \"%s\", \"sms\": %d, \"smem_optin_bytes\": %zu}", prop.name, nsm, prop.sharedMemPerBlockOptin);
+    o.add(line);
+    uint32_t* d_out = nullptr;
+    if ((e = cudaMalloc(&d_out, 4)) != cudaSuccess) return (int)e;
+    const double alu_ops = (double)ITERS * 4 * 8;
+#define FR_ALU(M, NAME, OPS) measure(o, NAME, [&](long long* c) { alu_kernel<M><<<nsm, T>>>(d_out, 1u, c); }, OPS, T)
+    FR_ALU(0, "lop3", alu_ops);
+    FR_ALU(1, "prmt", alu_ops);
+    FR_ALU(3, "shf", alu_ops);
+    FR_ALU(5, "lop3+prmt", alu_ops);
+    FR_ALU(2, "imad", alu_ops);
+    FR_ALU(4, "lop3+imad", alu_ops);
+    FR_ALU(6, "mul.wide", (double)ITERS * 4 * 4);
+#undef FR_ALU
+    const double lds_ops = (double)ITERS * 4 * 4;
+#define FR_LDS(M, NAME)                                                                              \
+    cudaFuncSetAttribute(lds_kernel<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536);         \
+    measure(o, NAME, [&](long long* c) { lds_kernel<M><<<nsm, T, 65536>>>(d_out, 1u, c); }, lds_ops, T)
+    FR_LDS(0, "lds32_bank_per_lane");
+    FR_LDS(1, "lds32_random_1KiB");
+    FR_LDS(2, "lds128_slot_per_lane");
+    FR_LDS(3, "lds128_random");
+#undef FR_LDS
+    cudaFree(d_out);
+    for (size_t sz : {(size_t)256 << 10, (size_t)1 << 20, (size_t)4 << 20, (size_t)8 << 20, (size_t)64 << 20, (size_t)256 << 20}) {
+        void *h = nullptr, *d = nullptr;
+        if (cudaMallocHost(&h, sz) != cudaSuccess || cudaMalloc(&d, sz) != cudaSuccess) { cudaFreeHost(h); cudaFree(d); (void)cudaGetLastError(); break; }
+        cudaEvent_t e0, e1;
+        cudaEventCreate(&e0);
+        cudaEventCreate(&e1);
+        for (int dir = 0; dir < 2; dir++) {
+            const int reps = sz >= ((size_t)64 << 20) ? 5 : 50;
+            const cudaMemcpyKind kind = dir ? cudaMemcpyDeviceToHost : cudaMemcpyHostToDevice;
+            for (int i = 0; i < 3; i++) cudaMemcpyAsync(dir ? h : d, dir ? d : h, sz, kind, 0);
+            cudaEventRecord(e0);
+            for (int i = 0; i < reps; i++) cudaMemcpyAsync(dir ? h : d, dir ? d : h, sz, kind, 0);
+            cudaEventRecord(e1);
+            cudaDeviceSynchronize();
+            float ms = 0;
+            cudaEventElapsedTime(&ms, e0, e1);
+            snprintf(line, sizeof line, "{\"probe\": \"%s\", \"bytes\": %zu, \"GBps\": %.2f}", dir ? "pinned_d2h" : "pinned_h2d", sz,
+                     sz * (double)reps / (ms * 1e-3) / 1e9);
+            o.add(line);
+        }
+        cudaEventDestroy(e0);
+        cudaEventDestroy(e1);
+        cudaFreeHost(h);
+        cudaFree(d);
+    }
+    e = cudaGetLastError();
+    return (int)e;
+}
