@@ -87,7 +87,11 @@ FASTRACK_API size_t fastrack_num_chunks(const fastrack_ctx* ctx, size_t len);
 
 /* Pre-sizes the per-chunk scratch (40 bytes per chunk: two banks of a 16-byte accumulator and a counter) for buffers up to max_len bytes so that later
  * calls allocate nothing.  Without it the first call that needs more chunks than any call before
- * grows the scratch (cudaMalloc + a device synchronisation) before launching. */
+ * grows the scratch (cudaMalloc + a device synchronisation) before launching.
+ * Stream capture: once the scratch is large enough, every asynchronous call below is a single kernel launch with
+ * all arguments passed by value, so it may be recorded into a CUDA graph and replayed.  A replay repeats the
+ * recorded arguments -- the IV base included, for the calls that take it by value; the *_samples calls read their IV
+ * bases from device memory and are the ones to capture when every replay needs fresh IVs (it does, under GCM). */
 FASTRACK_API int fastrack_ctx_reserve(fastrack_ctx* ctx, size_t max_len);
 
 /* Paper-faithful framing (Section 4.2: every chunk is "attached to one byte of additional authentication data

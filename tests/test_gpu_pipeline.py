@@ -105,7 +105,7 @@ def test_stage_trace_shows_copies_hiding_kernels():
         assert b["offset"] == a["offset"] + a["bytes"] and b["bytes"] <= a["bytes"]          # shrinking stages
         assert a["copy_start_ms"] <= a["copy_end_ms"] <= a["kernel_end_ms"]
         assert b["copy_start_ms"] >= a["copy_start_ms"]
-        assert a["kernel_end_ms"] <= b["copy_end_ms"] + 0.02, "a stage's kernel should finish under the next copy"
+        assert a["kernel_end_ms"] <= b["copy_end_ms"] + 0.05, "a stage's kernel should finish under the next copy"
     total = tr[-1]["kernel_end_ms"]
     copies = sum(s["copy_end_ms"] - s["copy_start_ms"] for s in tr)
-    assert total < 1.15 * copies                                                              # the kernels are hidden
+    assert total < 1.25 * copies                                                              # the kernels are hidden
