@@ -206,3 +206,74 @@ extern "C" void emu_keysetup(const uint8_t* key, uint8_t* round_keys, uint8_t* h
     memcpy(round_keys, S.P.rk, 240);
     memcpy(h, S.h, 16);
 }
+
+#ifdef EMU_SANITIZER_MAIN
+// Stand-alone driver for a build with -fsanitize=address,undefined (the GPU-side memory checker is not available
+// to this project, so the index arithmetic of the per-lane code is checked here instead): every buffer is a heap
+// block of exactly the size the C ABI asks the caller for, so a lane that reads or writes one byte outside the
+// payload, the tag / verdict / mask arrays, the power table or the shared-memory image stops the program.
+// Results are not compared here -- the Python tests do that -- only memory safety and the return code.
+#include <stdio.h>
+
+static uint32_t lcg(uint32_t& s) { return s = s * 1664525u + 1013904223u; }
+
+static size_t g_short_out = 0;      // self-test: allocate the output this many bytes short, which must be caught
+
+static int run_case(size_t cb, size_t len, uint32_t seg, uint32_t first, uint32_t aad, size_t sample_bytes)
+{
+    const size_t sb = sample_bytes ? sample_bytes : len;
+    const size_t n_samples = len / sb, cps = (sb + cb - 1) / cb, K = n_samples * cps;
+    uint32_t s = (uint32_t)(cb * 31 + len * 7 + seg + first + aad);
+    uint8_t key[32], iv[12];
+    for (auto& b : key) b = (uint8_t)(lcg(s) >> 24);
+    for (auto& b : iv) b = (uint8_t)(lcg(s) >> 24);
+    int bad = 0;
+    for (int mode = 0; mode < 6; mode++) {
+        uint8_t* in = new uint8_t[len];
+        uint8_t* out = new uint8_t[len - g_short_out];
+        uint8_t* pad = new uint8_t[len];
+        uint8_t* mask = new uint8_t[16 * K];
+        uint8_t* tin = new uint8_t[16 * K];
+        uint8_t* tout = new uint8_t[16 * K];
+        uint32_t* ok = new uint32_t[K];
+        uint8_t* ivs = sample_bytes ? new uint8_t[12 * n_samples] : nullptr;
+        for (size_t i = 0; i < len; i++) { in[i] = (uint8_t)(lcg(s) >> 24); pad[i] = (uint8_t)(lcg(s) >> 16); }
+        for (size_t i = 0; i < 16 * K; i++) { mask[i] = (uint8_t)(lcg(s) >> 24); tin[i] = (uint8_t)(lcg(s) >> 24); tout[i] = 0; }
+        for (size_t i = 0; i < K; i++) ok[i] = 9;
+        if (ivs) for (size_t i = 0; i < 12 * n_samples; i++) ivs[i] = (uint8_t)(lcg(s) >> 24);
+        bad |= emu_pass(mode, key, iv, cb, in, len, out, pad, mask, tin, tout, ok, seg, first, aad, sample_bytes, ivs);
+        delete[] in; delete[] out; delete[] pad; delete[] mask; delete[] tin; delete[] tout; delete[] ok; delete[] ivs;
+    }
+    return bad;
+}
+
+int main(int argc, char** argv)
+{
+    if (argc > 1 && !strcmp(argv[1], "short-output")) {     // must die inside the sanitizer: proves the check has teeth
+        g_short_out = 1;
+        return run_case(512, 1041, 2, 0, 0, 0);
+    }
+    int bad = 0, cases = 0;
+    const size_t cbs[] = {16, 32, 496, 512, 528, 1024, 4112};
+    for (size_t cb : cbs) {
+        const size_t lens[] = {1, 15, 16, 17, 31, 33, cb - 1, cb, cb + 1, 2 * cb, 3 * cb + 5, 7 * cb + cb / 2 + 3};
+        for (size_t len : lens) {
+            if (len == 0 || len > 40000) continue;
+            for (uint32_t seg : {1u, 2u, 8u}) {
+                bad |= run_case(cb, len, seg, 0, 0, 0);
+                cases++;
+            }
+            bad |= run_case(cb, len, 4, 0xfffffffeu, 3, 0);                 // wrapping chunk index, framing on
+            cases++;
+        }
+        for (size_t sb : {(size_t)16, (size_t)48, cb, cb + 16, 3 * cb - 16}) {  // batches of samples
+            if (sb * 5 > 40000) continue;
+            bad |= run_case(cb, sb * 5, 2, 0, 0, sb);
+            bad |= run_case(cb, sb * 5, 8, 0, 16, sb);
+            cases += 2;
+        }
+    }
+    printf("%d cases, status %d\n", cases, bad);
+    return bad ? 1 : 0;
+}
+#endif

@@ -154,3 +154,18 @@ def test_batch_of_samples_each_under_its_own_iv(emu, sample_bytes, cb, n_samples
     exp = np.ones(len(bad_t), np.uint32)
     exp[len(bad_t) // 2] = 0
     assert np.array_equal(out, p) and np.array_equal(ok, exp)
+
+
+def test_index_arithmetic_under_address_and_ub_sanitizers(tmp_path):
+    """The per-lane code again, as a stand-alone program built with -fsanitize=address,undefined over heap buffers of
+    exactly the sizes the C ABI asks for: 400+ shapes x 6 pass modes must run clean, and the same program given an
+    output buffer one byte short must be stopped by the sanitizer."""
+    exe = tmp_path / "emulate_sanitized"
+    src = os.path.join(ROOT, "tests", "device_on_host", "emulate.cpp")
+    subprocess.check_call(["g++", "-O1", "-g", "-std=c++17", "-fsanitize=address,undefined", "-fno-sanitize-recover=all",
+                           "-DEMU_SANITIZER_MAIN", "-o", str(exe), src])
+    ok = subprocess.run([str(exe)], capture_output=True, text=True, timeout=600)
+    assert ok.returncode == 0, ok.stderr[-2000:]
+    assert "status 0" in ok.stdout
+    short = subprocess.run([str(exe), "short-output"], capture_output=True, text=True, timeout=600)
+    assert short.returncode != 0 and "AddressSanitizer" in short.stderr
