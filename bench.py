@@ -598,7 +598,17 @@ def main():
                     help="print throughput over the benchmark configurations instead of the one bench line")
     ap.add_argument("--trace", action="store_true", help="print stage-level timelines of the pipelined H2D call")
     ap.add_argument("--peaks", action="store_true", help="measure the unit rates the kernel roofline is derived from")
+    ap.add_argument("--shape", default=None, metavar="LEN_BYTES,CHUNK_BYTES",
+                    help="with --kernel-only: time another buffer / chunk size than the headline one (profiling aid)")
     args = ap.parse_args()
+    if args.shape:
+        if not args.kernel_only:
+            ap.error("--shape only applies to --kernel-only; the metric line is always the headline workload")
+        global LEN, CHUNK, WORKLOAD
+        LEN, CHUNK = (int(x) for x in args.shape.split(","))
+        if LEN % CHUNK:
+            ap.error("--shape: LEN_BYTES must be a multiple of CHUNK_BYTES")
+        WORKLOAD = f"AES-256-GCM multi-chain decrypt+verify, {LEN} uniform random bytes, chunk {CHUNK} (K={LEN // CHUNK})"
     if args.peaks:
         run_peaks(args)
     elif args.trace:

@@ -17,6 +17,7 @@ using namespace fr_host;
 #define FR_THREADS 1024
 #define FR_MAX_STAGES 96      // most stages a pipelined call is cut into
 #define FR_WARPS (FR_THREADS / 32)
+#define FR_PACK_MAX_BLOCKS 4096   // chunks of more blocks than this never take the packed-row kernels
 
 // ------------------------------------------------------------------------------------ kernels ----
 
@@ -106,6 +107,70 @@ __global__ void __launch_bounds__(FR_THREADS, 1) fr_crypt_kernel(const __grid_co
     else fr_crypt_body<MODE, false>(P, sm, L);
 }
 
+// Packed rows (many short chains, see the device header): a warp takes pack_chunks whole chunks and walks their
+// slots 32 at a time; the per-chunk XOR of the lane terms is a segmented inclusive scan over the row (a lane adds
+// the lane d below it only if that lane belongs to the same chunk), a chunk that continues into the next row hands
+// its running sum to that row's lane 0, and the lane holding a chunk's last slot finishes the tag.  No chunk is
+// shared between warps.  The shared-memory GHASH tables hold H here, not H^32.
+template <int MODE, bool ABS>
+__device__ __forceinline__ void fr_packed_body(const FrParams& P, const char* sm, FrLane L)
+{
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const uint32_t total_warps = gridDim.x * (blockDim.x >> 5);
+    const FrPackGeom g = fr_pack_geom(P);
+
+    for (uint32_t item = warp * gridDim.x + blockIdx.x; item < P.n_items; item += total_warps) {
+        const uint32_t kk0 = item * P.pack_chunks;
+        const uint32_t kk1 = (P.n_chunks - kk0 < P.pack_chunks) ? P.n_chunks : kk0 + P.pack_chunks;
+        const uint32_t slot_end = fr_pack_slot_begin(P, g, kk1);
+        uint4 carry = make_uint4(0, 0, 0, 0);
+        for (uint32_t base = fr_pack_slot_begin(P, g, kk0); base < slot_end; base += 32u) {
+            const uint32_t slot = base + lane;
+            const bool valid = slot < slot_end;               // only the item's last row has idle lanes, at its top
+            FrSlot si = {0u, lane, 0xFFFFFFFFu};
+            uint4 z = make_uint4(0, 0, 0, 0);
+            if (valid) z = fr_packed_slot_lane<MODE, ABS>(P, sm, L, g, slot, si);
+            if (lane == 0u && si.i != 0u) z = fr_xor4(z, carry);
+            const uint32_t first = lane >= si.i ? lane - si.i : 0u;      // lowest lane of this row in the same chunk
+#pragma unroll
+            for (uint32_t d = 1; d < 32u; d <<= 1) {
+                const uint32_t tx = __shfl_up_sync(0xFFFFFFFFu, z.x, d), ty = __shfl_up_sync(0xFFFFFFFFu, z.y, d);
+                const uint32_t tz = __shfl_up_sync(0xFFFFFFFFu, z.z, d), tw = __shfl_up_sync(0xFFFFFFFFu, z.w, d);
+                if (lane >= first + d) { z.x ^= tx; z.y ^= ty; z.z ^= tz; z.w ^= tw; }
+            }
+            carry.x = __shfl_sync(0xFFFFFFFFu, z.x, 31); carry.y = __shfl_sync(0xFFFFFFFFu, z.y, 31);
+            carry.z = __shfl_sync(0xFFFFFFFFu, z.z, 31); carry.w = __shfl_sync(0xFFFFFFFFu, z.w, 31);
+            if (valid && si.i == si.last) {
+                const uint4 lenh = ((si.kk + 1u) % P.chunks_per_sample == 0u) ? P.lenh_last : P.lenh_full;
+                const uint4 tag = fr_xor4(z, lenh);
+                if (MODE == FR_MODE_ENC) {
+                    P.tags_out[si.kk] = tag;
+                } else {
+                    const uint4 t = P.tags_in[si.kk];
+                    const uint32_t diff = (tag.x ^ t.x) | (tag.y ^ t.y) | (tag.z ^ t.z) | (tag.w ^ t.w);
+                    P.ok[si.kk] = diff == 0u ? 1u : 0u;
+                }
+            }
+        }
+    }
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(FR_THREADS, 1) fr_packed_kernel(const __grid_constant__ FrParams P)
+{
+    extern __shared__ __align__(256) char sm[];
+    fr_build_smem<FR_THREADS>(sm, threadIdx.x, P.te0, P.gh_tab);
+    asm volatile("griddepcontrol.wait;" ::: "memory");           // as in fr_crypt_kernel
+    asm volatile("griddepcontrol.launch_dependents;");
+    __syncthreads();
+    uint32_t after_barrier;
+    asm volatile("mov.u32 %0, 0;" : "=r"(after_barrier)::"memory");
+    FrLane L = fr_make_lane(threadIdx.x & 31u);
+    L.lane4 |= after_barrier;
+    if ((uint32_t)__cvta_generic_to_shared(sm) == FR_SMEM_ABS_BASE && !P.generic_smem) fr_packed_body<MODE, true>(P, sm, L);
+    else fr_packed_body<MODE, false>(P, sm, L);
+}
+
 // pow[i] = pow[i - half] * pow[half] for i in (half, min(2*half, n - 1)]: one doubling pass of the table
 // of powers (pow[half] itself was the last entry of the previous pass; pow[0] = 1 and pow[1] = H are given).
 __global__ void fr_pow_double_kernel(uint4* pow, uint32_t half, uint32_t n)
@@ -189,6 +254,9 @@ struct fastrack_ctx {
     size_t stage_bytes_override;  // 0 = automatic (FASTRACK_STAGE_BYTES, for experiments)
     uint32_t generic_smem;        // FASTRACK_GENERIC_SMEM=1: exercise the portable addressing path (tests)
     uint32_t no_overlap_launch;   // FASTRACK_NO_OVERLAP_LAUNCH=1: plain stream-ordered launches (experiments)
+    uint32_t pack_max_blocks;     // chunks of at most this many blocks may take the packed-row kernels (FASTRACK_PACK_MAX_BLOCKS; 0 = never)
+    uint32_t pack_run_override;   // 0 = automatic; else packed rows with this run length wherever they apply (FASTRACK_PACK_RUN, tests)
+    uint32_t pack_group_override; // 0 = automatic; else this many chunks per packed work item (FASTRACK_PACK_GROUP, tests)
 };
 
 #define FR_CUDA(ctx, call)                                              \
@@ -243,6 +311,10 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
     if (const char* env = getenv("FASTRACK_GENERIC_SMEM")) ctx->generic_smem = (uint32_t)(strtoul(env, nullptr, 10) != 0);
     if (const char* env = getenv("FASTRACK_NO_OVERLAP_LAUNCH")) ctx->no_overlap_launch = (uint32_t)(strtoul(env, nullptr, 10) != 0);
     if (const char* env = getenv("FASTRACK_STAGE_BYTES")) ctx->stage_bytes_override = (size_t)strtoull(env, nullptr, 10);
+    ctx->pack_max_blocks = FR_PACK_MAX_BLOCKS;
+    if (const char* env = getenv("FASTRACK_PACK_MAX_BLOCKS")) ctx->pack_max_blocks = (uint32_t)strtoul(env, nullptr, 10);
+    if (const char* env = getenv("FASTRACK_PACK_RUN")) ctx->pack_run_override = (uint32_t)strtoul(env, nullptr, 10);
+    if (const char* env = getenv("FASTRACK_PACK_GROUP")) ctx->pack_group_override = (uint32_t)strtoul(env, nullptr, 10);
 
     // key material on the host: S-box, Te0, round keys, H, byte tables of H^32
     uint8_t sbox[256];
@@ -304,6 +376,8 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
         if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_PADGEN>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
         if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_PADDEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
         if ((e = cudaFuncSetAttribute(fr_verify_sequential_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_DEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_ENC>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
         for (int i = 0; i < 8 && e == cudaSuccess; i++) e = cudaStreamCreateWithFlags(&ctx->streams[i], cudaStreamNonBlocking);
         if (e != cudaSuccess) break;
         if ((e = cudaEventCreateWithFlags(&ctx->tags_ready, cudaEventDisableTiming)) != cudaSuccess) break;
@@ -460,6 +534,64 @@ static void plan_segments(const fastrack_ctx* ctx, size_t sample_bytes, size_t n
     P.lenh_last = length_term(ctx, last_len);
 }
 
+// Decides between the row kernels (plan_segments has filled P) and the packed-row kernels for a fused pass, and
+// in the latter case picks the run length and the work-item size.  Both are judged by the same kind of estimate, in
+// SM clocks: the shared-memory work of the busiest SM plus, for the packed form, the latency of one row (its rows
+// are long, so pipeline fill and drain show).  Fitted to measurements on B200: a row kernel costs about 285 clocks
+// per row plus 400 per segment; a packed row costs about 280 plus, per counter of its run, 258 clocks for runs up to
+// 3 counters and more beyond (a lane's 16-byte loads and stores are 16 * run bytes apart, so longer runs touch more
+// cache lines per request).
+static bool plan_packed(const fastrack_ctx* ctx, size_t sample_bytes, size_t n_chunks, FrParams& P)
+{
+    if (!ctx->pack_max_blocks) return false;
+    const size_t first_len = sample_bytes < ctx->chunk_bytes ? sample_bytes : ctx->chunk_bytes;
+    const size_t counters = (first_len + 15) / 16 + 1;
+    if (counters - 1 > ctx->pack_max_blocks) return false;
+    const size_t sms = (size_t)ctx->num_sms, warps = sms * FR_WARPS;
+
+    const size_t rows_ref = (counters + 1 + FR_ROW_BLOCKS - 1) / FR_ROW_BLOCKS;
+    const size_t waves = ((size_t)P.n_items + warps - 1) / warps;
+    const size_t row_thr = (n_chunks * rows_ref + sms - 1) / sms * 285 + ((size_t)P.n_items + sms - 1) / sms * 400;
+    const size_t row_lat = waves * ((size_t)P.seg_rows * 1000 + 4000);
+    const size_t row_cost = row_thr > row_lat ? row_thr : row_lat;
+
+    // clocks per counter of a run, by run length (runs whose byte stride is a power of two do worst: the lanes'
+    // 16-byte pieces then fall on the same few cache banks)
+    static const size_t step_clocks[14] = {0, 258, 257, 256, 289, 264, 281, 330, 396, 302, 304, 304, 327, 305};
+    size_t best_run = 0, best_group = 1, best_cost = ~(size_t)0;
+    const size_t cand[] = {1, 2, 3, 4, 5, 6, 9, 10, 11, 13, counters <= 64 ? counters : 5};
+    for (size_t run : cand) {
+        if (ctx->pack_run_override) run = ctx->pack_run_override;
+        if (run > counters) run = counters;
+        const size_t slots = (counters + run - 1) / run;
+        if (n_chunks * slots >= ((size_t)1 << 32)) continue;                       // slots are counted in 32 bits
+        const size_t per_row = 280 + run * (run < 14 ? step_clocks[run] : 335);
+        const size_t row_latency = 2500 + run * 2250;       // one warp alone on its SM partition
+        // a work item is `group` whole chunks.  Its last row is only partly filled, and an instruction costs the same
+        // with idle lanes; on the other hand a launch with fewer items than warps leaves warps idle.  Try a range of
+        // item sizes and count the rows each really takes.
+        const size_t sizes[] = {1, 2, 3, 4, 5, 6, 8, 10, 12, 16, 24, 32, 48, 64, 96, 128, 256, 512,
+                                32 / slots, 64 / slots, 128 / slots, 256 / slots, 512 / slots};
+        for (size_t group : sizes) {
+            if (ctx->pack_group_override) group = ctx->pack_group_override;
+            if (group < 1 || group * slots > 1024) continue;
+            if (group > n_chunks) group = n_chunks;
+            const size_t rows_per_item = (group * slots + 31) / 32;
+            const size_t items = (n_chunks + group - 1) / group;
+            const size_t thr = (items * rows_per_item + sms - 1) / sms * per_row;
+            const size_t lat = (items + warps - 1) / warps * rows_per_item * row_latency;
+            const size_t cost = thr > lat ? thr + lat / 4 : lat + thr / 4;      // between the two regimes both show
+            if (cost < best_cost) { best_cost = cost; best_run = run; best_group = group; }
+        }
+    }
+    if (!best_run) return false;
+    if (!ctx->pack_run_override && best_cost >= row_cost) return false;
+    P.pack_run = (uint32_t)best_run;
+    P.pack_chunks = (uint32_t)best_group;
+    P.n_items = (uint32_t)((n_chunks + best_group - 1) / best_group);
+    return true;
+}
+
 // Buffers of one pass (which ones are used depends on the mode, see FrMode).
 struct PassBuffers {
     const void* in = nullptr;
@@ -498,6 +630,8 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
     P.n_chunks = (uint32_t)n_chunks;
 
     plan_segments(ctx, sample_bytes, n_chunks, P);
+    // Many short chains: one run of counters per lane (see fr_packed_body) when that is predicted to be faster.
+    const bool packed = (mode == FR_MODE_DEC || mode == FR_MODE_ENC) && plan_packed(ctx, sample_bytes, n_chunks, P);
 
     P.in = (const uint8_t*)b.in;
     P.out = (uint8_t*)b.out;
@@ -507,7 +641,7 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
     P.tags_out = (uint4*)b.tags_out;
     P.ok = b.ok;
     P.te0 = ctx->d_te0;
-    P.gh_tab = ctx->d_gh_tab;
+    P.gh_tab = packed ? ctx->d_gh1_tab : ctx->d_gh_tab;
     P.pow = ctx->d_pow;
     uint32_t* bank = ctx->d_scratch + (size_t)b.bank * 5 * ctx->scratch_chunks;
     P.acc = bank + 4 * first_chunk;
@@ -531,8 +665,10 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
     }
     cudaError_t le;
     switch (mode) {
-        case FR_MODE_DEC:    le = cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_DEC>, P); break;
-        case FR_MODE_ENC:    le = cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_ENC>, P); break;
+        case FR_MODE_DEC:    le = packed ? cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_DEC>, P)
+                                         : cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_DEC>, P); break;
+        case FR_MODE_ENC:    le = packed ? cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_ENC>, P)
+                                         : cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_ENC>, P); break;
         case FR_MODE_CTR:    le = cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_CTR>, P); break;
         case FR_MODE_VERIFY: le = cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_VERIFY>, P); break;
         case FR_MODE_PADGEN: le = cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_PADGEN>, P); break;

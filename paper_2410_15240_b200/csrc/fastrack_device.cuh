@@ -60,7 +60,9 @@ struct FrParams {
     uint64_t chunk_bytes;
     uint64_t sample_bytes;     // the launch is a sequence of equal samples of this many bytes (one sample: = len)
     uint32_t chunks_per_sample;  // ceil(sample_bytes / chunk_bytes); only a sample's last chunk may be short
-    uint32_t pad1;
+    uint32_t pack_chunks;        // packed rows: chunks per work item; then n_items = ceil(n_chunks / pack_chunks)
+    uint32_t pack_run;           // packed rows: consecutive counters per slot (lane)
+    uint32_t pad2;
     const uint8_t* ivs;        // per-sample 12-byte IV bases (device), or null: one IV base for the whole launch
     const uint8_t* in;
     uint8_t* out;
@@ -538,4 +540,92 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
     if (!DO_GHASH) return make_uint4(0, 0, 0, 0);
     if (c_last == 0u) return extra;
     return fr_xor4(fr_gf128_mul(pend, hpow), extra);
+}
+
+// ---- Packed rows: many short chains -----------------------------------------------------------------------
+// The row layout above gives one warp 32 consecutive blocks of ONE chunk; a 16-byte chunk would keep 2 of its 32
+// lanes busy, and every chunk pays a closing product, a warp reduction and a ticket.  When a launch has many
+// chunks that are not large, it is laid out the other way round: a chunk's counters 1 .. nblk+1 (counter 1 = the
+// tag mask E_K(J0) and, under the serial-number framing, the AAD block; counter c >= 2 = data block c - 2) are cut
+// into runs of `pack_run` consecutive counters, one run = one SLOT = one lane.  A lane walks its run block by
+// block -- counter mode with the first two rounds shared as above, Horner's rule with the FIXED multiplier H
+// (byte tables of H in shared memory, same conflict-free lane rotation) -- and multiplies the result by the power
+// of H that aligns it to the end of the chunk.  Slots of a chunk are consecutive, a warp takes a run of whole chunks
+// and walks their slots 32 at a time; the per-chunk XOR of the lane terms is a segmented scan in the calling
+// kernel.  No chunk is shared between warps, so this path needs neither atomics nor scratch memory.  Lanes read
+// and write 16 bytes at a stride of 16 * pack_run bytes: short runs keep those accesses in few cache lines, long runs
+// amortise the closing product; the host picks the run length.
+struct FrPackGeom {
+    uint32_t run;               // counters per slot
+    uint32_t slots_full;        // slots of a full-size chunk
+    uint32_t slots_sample;      // slots of a whole sample
+};
+
+__device__ __forceinline__ FrPackGeom fr_pack_geom(const FrParams& P)
+{
+    const uint64_t first_len = P.sample_bytes < P.chunk_bytes ? P.sample_bytes : P.chunk_bytes;
+    const uint64_t last_len = P.sample_bytes - (uint64_t)(P.chunks_per_sample - 1u) * P.chunk_bytes;
+    FrPackGeom g;
+    g.run = P.pack_run;
+    g.slots_full = ((uint32_t)((first_len + 15) >> 4) + g.run) / g.run;                  // ceil((nblk + 1) / run)
+    g.slots_sample = (P.chunks_per_sample - 1u) * g.slots_full + ((uint32_t)((last_len + 15) >> 4) + g.run) / g.run;
+    return g;
+}
+
+// First slot of chunk kk (kk = n_chunks gives the total).
+__device__ __forceinline__ uint32_t fr_pack_slot_begin(const FrParams& P, const FrPackGeom& g, uint32_t kk)
+{
+    const uint32_t sample = kk / P.chunks_per_sample, k = kk - sample * P.chunks_per_sample;
+    return sample * g.slots_sample + k * g.slots_full;
+}
+
+struct FrSlot {
+    uint32_t kk;        // chunk the slot belongs to
+    uint32_t i;         // index of the slot inside the chunk
+    uint32_t last;      // index of the chunk's last slot
+};
+
+// One slot: encrypt or decrypt the blocks of its run (counter 1: produce the tag mask) and return the slot's
+// term of the tag, sum over its counters c of block_c * H^(nblk + 3 - c), plus E_K(J0) from counter 1.
+// XOR over a chunk's slots, plus the length term, is its tag.
+template <int MODE, bool ABS>
+__device__ __forceinline__ uint4 fr_packed_slot_lane(const FrParams& P, const char* sm, const FrLane& L,
+                                                     const FrPackGeom& g, uint32_t slot, FrSlot& si)
+{
+    static_assert(MODE == FR_MODE_DEC || MODE == FR_MODE_ENC, "packed rows exist for the fused passes");
+    const uint32_t sample = slot / g.slots_sample, t = slot - sample * g.slots_sample;
+    const uint32_t k = t / g.slots_full, i = t - k * g.slots_full;
+    const uint32_t kk = sample * P.chunks_per_sample + k;
+    const FrChunk ck = fr_chunk_info(P, kk);
+    const uint32_t nblk = (uint32_t)((ck.len + 15) >> 4);
+    si.kk = kk; si.i = i; si.last = nblk / g.run;                        // ceil((nblk + 1) / run) - 1
+    const uint32_t c0 = i * g.run + 1u;                                  // the run's counters are c0 .. c1 - 1
+    uint32_t c1 = c0 + g.run;
+    if (c1 > nblk + 2u) c1 = nblk + 2u;
+    const uint4 hpow = P.pow[nblk + 4u - c1];                            // for the run's last block, counter c1 - 1
+    const uint8_t* in = P.in + ck.off;
+    uint8_t* out = P.out + ck.off;
+    const FrCtrChunk cc = fr_ctr_chunk<ABS>(sm, L.lane4, P, ck.iv_w0, ck.iv_w1, fr_bswap(ck.iv_ctr));
+    FrCtrGroup cg = fr_ctr_group<ABS>(sm, L.lane4, P, cc, c0);
+    uint4 y = make_uint4(0, 0, 0, 0), extra = make_uint4(0, 0, 0, 0);
+    for (uint32_t c = c0; c < c1; c++) {
+        if ((c & 255u) == 0u && c != c0) cg = fr_ctr_group<ABS>(sm, L.lane4, P, cc, c);      // entered the next 256-counter group
+        const uint4 ks = fr_aes256_ctr_block<ABS>(sm, L.lane4, P, cc, cg, c);
+        uint4 gblk;
+        if (c == 1u) {
+            extra = ks;                                                                      // E_K(J0)
+            gblk = make_uint4(P.aad_mod ? ck.serial % P.aad_mod : 0u, 0, 0, 0);               // the one-byte AAD block, or nothing
+        } else {
+            const uint64_t boff = (uint64_t)(c - 2u) << 4;
+            const bool full = ck.len - boff >= 16;
+            const uint32_t nvalid = full ? 16u : (uint32_t)(ck.len - boff);
+            const uint4 x = full ? *(const uint4*)(in + boff) : fr_load_partial(in + boff, nvalid);
+            const uint4 o = fr_xor4(x, ks);
+            if (full) *(uint4*)(out + boff) = o; else fr_store_partial(out + boff, o, nvalid);
+            gblk = (MODE == FR_MODE_ENC) ? (full ? o : fr_mask_bytes(o, nvalid)) : x;
+        }
+        y = fr_xor4(y, gblk);
+        if (c + 1u != c1) y = fr_ghash_tabmul<ABS>(sm, L, y);                                // Horner step with the fixed multiplier H
+    }
+    return fr_xor4(fr_gf128_mul(y, hpow), extra);
 }

@@ -58,7 +58,7 @@ struct Setup {
 };
 
 // The same derivation fastrack_ctx_create performs (host part) plus the power table and the shared-memory fill.
-void setup(Setup& S, const uint8_t key[32], size_t cb)
+void setup(Setup& S, const uint8_t key[32], size_t cb, int squarings = 5)   // byte tables of H^(2^squarings): H^32, or H for the packed rows
 {
     memset(&S.P, 0, sizeof S.P);
     uint8_t sbox[256];
@@ -71,7 +71,7 @@ void setup(Setup& S, const uint8_t key[32], size_t cb)
     const uint8_t zero[16] = {0};
     encrypt_block_host(S.P.rk, S.te0, sbox, zero, S.h);
     Gf128 G = gf_load(S.h);
-    for (int i = 0; i < 5; i++) G = gf_mul(G, G);
+    for (int i = 0; i < squarings; i++) G = gf_mul(G, G);
     S.gh_tab.assign(65536, 0);
     for (int p = 0; p < 16; p++) {
         Gf128 basis[8];
@@ -184,6 +184,87 @@ extern "C" int emu_pass(int mode, const uint8_t* key, const uint8_t* iv_base, si
     return 0;
 }
 
+// The packed-row kernels (small chunks): the lane function from the header, and the kernel body's segmented scan,
+// carry and finishing step written out over an array of 32 lane values, shuffle by shuffle.
+template <int MODE>
+static void run_packed(Setup& S, const uint8_t* tags_in, uint8_t* tags_out, uint32_t* ok)
+{
+    FrParams& P = S.P;
+    const FrPackGeom g = fr_pack_geom(P);
+    for (uint32_t item = 0; item < P.n_items; item++) {
+        const uint32_t kk0 = item * P.pack_chunks;
+        const uint32_t kk1 = (P.n_chunks - kk0 < P.pack_chunks) ? P.n_chunks : kk0 + P.pack_chunks;
+        const uint32_t slot_end = fr_pack_slot_begin(P, g, kk1);
+        uint4 carry = {0, 0, 0, 0};
+        for (uint32_t base = fr_pack_slot_begin(P, g, kk0); base < slot_end; base += 32u) {
+            uint4 z[32];
+            FrSlot si[32];
+            bool valid[32];
+            for (uint32_t lane = 0; lane < 32; lane++) {
+                const FrLane L = fr_make_lane(lane);
+                valid[lane] = base + lane < slot_end;
+                si[lane] = FrSlot{0u, lane, 0xFFFFFFFFu};
+                z[lane] = uint4{0, 0, 0, 0};
+                if (valid[lane]) z[lane] = fr_packed_slot_lane<MODE, false>(P, S.sm.data(), L, g, base + lane, si[lane]);
+            }
+            if (si[0].i != 0u) z[0] = fr_xor4(z[0], carry);
+            for (uint32_t d = 1; d < 32; d <<= 1) {
+                uint4 up[32];
+                for (uint32_t lane = 0; lane < 32; lane++) up[lane] = z[lane >= d ? lane - d : lane];   // shfl_up
+                for (uint32_t lane = 0; lane < 32; lane++) {
+                    const uint32_t first = lane >= si[lane].i ? lane - si[lane].i : 0u;
+                    if (lane >= first + d) z[lane] = fr_xor4(z[lane], up[lane]);
+                }
+            }
+            carry = z[31];
+            for (uint32_t lane = 0; lane < 32; lane++) {
+                if (!(valid[lane] && si[lane].i == si[lane].last)) continue;
+                const uint32_t kk = si[lane].kk;
+                const uint4 tag = fr_xor4(z[lane], ((kk + 1u) % P.chunks_per_sample == 0u) ? P.lenh_last : P.lenh_full);
+                if (MODE == FR_MODE_ENC) memcpy(tags_out + 16 * (size_t)kk, &tag, 16);
+                else ok[kk] = memcmp(&tag, tags_in + 16 * (size_t)kk, 16) == 0;
+            }
+        }
+    }
+}
+
+// One packed-row pass (mode 0 = decrypt + verify, 1 = encrypt + tag): pack_run counters per slot, pack_chunks chunks per work item.
+extern "C" int emu_packed(int mode, const uint8_t* key, const uint8_t* iv_base, size_t cb, const uint8_t* in, size_t len,
+                          uint8_t* out, const uint8_t* tags_in, uint8_t* tags_out, uint32_t* ok, uint32_t pack_chunks,
+                          uint32_t pack_run, uint32_t first_chunk, uint32_t aad_mod, size_t sample_bytes, const uint8_t* ivs)
+{
+    Setup S;
+    setup(S, key, cb, 0);
+    FrParams& P = S.P;
+    auto be32 = [](const uint8_t* p) { return ((uint32_t)p[0] << 24) | ((uint32_t)p[1] << 16) | ((uint32_t)p[2] << 8) | p[3]; };
+    auto le32 = [](const uint8_t* p) { return ((uint32_t)p[3] << 24) | ((uint32_t)p[2] << 16) | ((uint32_t)p[1] << 8) | p[0]; };
+    P.iv_w0 = le32(iv_base);
+    P.iv_w1 = le32(iv_base + 4);
+    P.iv_ctr = be32(iv_base + 8) + first_chunk;
+    P.first_chunk = first_chunk;
+    P.aad_mod = aad_mod;
+    P.len = len;
+    P.chunk_bytes = cb;
+    if (sample_bytes == 0) sample_bytes = len;
+    const size_t cps = (sample_bytes + cb - 1) / cb;
+    const size_t n_chunks = (len / sample_bytes) * cps;
+    P.sample_bytes = sample_bytes;
+    P.chunks_per_sample = (uint32_t)cps;
+    P.ivs = ivs;
+    P.n_chunks = (uint32_t)n_chunks;
+    P.pack_chunks = pack_chunks ? pack_chunks : 1;
+    P.pack_run = pack_run ? pack_run : 1;
+    P.n_items = (uint32_t)((n_chunks + P.pack_chunks - 1) / P.pack_chunks);
+    P.lenh_full = length_term(S, std::min(sample_bytes, cb), aad_mod);
+    P.lenh_last = length_term(S, sample_bytes - (cps - 1) * cb, aad_mod);
+    P.in = in;
+    P.out = out;
+    if (mode == FR_MODE_DEC) run_packed<FR_MODE_DEC>(S, tags_in, tags_out, ok);
+    else if (mode == FR_MODE_ENC) run_packed<FR_MODE_ENC>(S, tags_in, tags_out, ok);
+    else return -1;
+    return 0;
+}
+
 extern "C" void emu_gf128_mul_device(const uint8_t* a, const uint8_t* b, uint8_t* o)
 {
     uint4 x, y;
@@ -242,6 +323,9 @@ static int run_case(size_t cb, size_t len, uint32_t seg, uint32_t first, uint32_
         for (size_t i = 0; i < K; i++) ok[i] = 9;
         if (ivs) for (size_t i = 0; i < 12 * n_samples; i++) ivs[i] = (uint8_t)(lcg(s) >> 24);
         bad |= emu_pass(mode, key, iv, cb, in, len, out, pad, mask, tin, tout, ok, seg, first, aad, sample_bytes, ivs);
+        if (mode <= FR_MODE_ENC)                        // the packed-row form of the same pass, seg doubling as group size and run length
+            for (uint32_t run : {1u, seg + 1u, 40u})
+                bad |= emu_packed(mode, key, iv, cb, in, len, out, tin, tout, ok, seg * 3 - 2, run, first, aad, sample_bytes, ivs);
         delete[] in; delete[] out; delete[] pad; delete[] mask; delete[] tin; delete[] tout; delete[] ok; delete[] ivs;
     }
     return bad;

@@ -26,6 +26,8 @@ def emu(tmp_path_factory):
     for name in ("emu_gf128_mul_device", "emu_gf128_mul_keysetup"):
         getattr(lib, name).argtypes = [ctypes.c_char_p] * 3
     lib.emu_keysetup.argtypes = [ctypes.c_char_p, V, V]
+    lib.emu_packed.argtypes = [ctypes.c_int, V, V, Z, V, Z, V, V, V, V, U, U, U, U, Z, V]
+    lib.emu_packed.restype = ctypes.c_int
     return lib
 
 
@@ -154,6 +156,82 @@ def test_batch_of_samples_each_under_its_own_iv(emu, sample_bytes, cb, n_samples
     exp = np.ones(len(bad_t), np.uint32)
     exp[len(bad_t) // 2] = 0
     assert np.array_equal(out, p) and np.array_equal(ok, exp)
+
+
+def run_packed(lib, mode, key, iv, cb, data, n, tags=None, group=1, run_len=1, first=0, aad=0, sample_bytes=0, ivs=None):
+    K = (n + cb - 1) // cb if not sample_bytes else (n // sample_bytes) * ((sample_bytes + cb - 1) // cb)
+    k = np.frombuffer(key, np.uint8).copy()
+    v = np.frombuffer(iv, np.uint8).copy()
+    src = np.ascontiguousarray(data, np.uint8)
+    out = np.full(n + 64, 0xA5, np.uint8)
+    tin = np.ascontiguousarray(tags, np.uint8) if tags is not None else np.zeros((K, 16), np.uint8)
+    tout = np.zeros((K, 16), np.uint8)
+    ok = np.full(K, 7, np.uint32)
+    rc = lib.emu_packed(mode, k.ctypes.data, v.ctypes.data, cb, src.ctypes.data, n, out.ctypes.data, tin.ctypes.data,
+                        tout.ctypes.data, ok.ctypes.data, group, run_len, first, aad, sample_bytes,
+                        ivs.ctypes.data if ivs is not None else None)
+    assert rc == 0 and (out[n:] == 0xA5).all()
+    return out[:n], tout, ok
+
+
+PACKED_SHAPES = [(1, 16, 1), (16, 16, 1), (16 * 100, 16, 7), (16 * 100 + 5, 16, 300), (32 * 37 + 17, 32, 5), (48 * 50, 48, 4),
+                 (112 * 9 + 1, 112, 2), (240 * 33, 240, 3), (496 * 5 + 495, 496, 2), (512 * 6 + 16, 512, 1), (528 * 4, 528, 3),
+                 (1024 * 5 + 1000, 1024, 2), (2048 * 3 + 31, 2048, 1), (700, 4096, 1),
+                 (4096 * 3 + 100, 4096, 2), (65536 + 17, 16384, 1)]        # runs that cross a 256-counter group
+
+
+@pytest.mark.parametrize("n,cb,group", PACKED_SHAPES)
+@pytest.mark.parametrize("aad,run_len", [(0, 1), (5, 1), (0, 2), (5, 4), (0, 8), (0, 3), (5, 32), (0, 300)])
+def test_packed_rows_match_oracle(emu, n, cb, group, aad, run_len):
+    """Small chunks, several to a row: ciphertext, tags, plaintext and verdicts (with tampering) equal the oracle's."""
+    rng = np.random.default_rng(n * 31 + cb + aad)
+    key, iv = rng.bytes(32), rng.bytes(8) + bytes([0xFF, 0xFF, 0xFF, 0xFD])          # the chunk index wraps the IV's counter
+    p = np.frombuffer(rng.bytes(n), np.uint8)
+    enc = (lambda q: oracle.mc_encrypt_framed(key, iv, cb, aad, q, 4)) if aad else (lambda q: oracle.mc_encrypt(key, iv, cb, q, 4))
+    c_ref, t_ref = enc(p)
+    K = t_ref.shape[0]
+    c, t, _ = run_packed(emu, ENC, key, iv, cb, p, n, group=group, run_len=run_len, aad=aad)
+    assert np.array_equal(c, c_ref) and np.array_equal(t, t_ref)
+    bad_c, bad_t = c_ref.copy(), t_ref.copy()
+    bad_c[n // 2] ^= 0x10
+    if K > 1:
+        bad_t[K - 1, 3] ^= 4
+    if K > 4:
+        bad_t[1, 15] ^= 0x80
+    if aad:
+        p_ref, ok_ref = oracle.mc_decrypt_framed(key, iv, cb, aad, bad_c, bad_t, 4)
+    else:
+        p_ref, ok_ref = oracle.mc_decrypt(key, iv, cb, bad_c, bad_t, 4)
+    assert 0 < int(ok_ref.sum()) < K or K <= 2
+    out, _, ok = run_packed(emu, DEC, key, iv, cb, bad_c, n, tags=bad_t, group=group, run_len=run_len, aad=aad)
+    assert np.array_equal(out, p_ref) and np.array_equal(ok, ok_ref)
+
+
+@pytest.mark.parametrize("run_len", [1, 4, 7])
+@pytest.mark.parametrize("sample_bytes,cb,n_samples,aad,group", [(16, 16, 40, 0, 3), (48, 16, 9, 0, 4), (400, 400, 11, 0, 2),
+                                                                (400, 112, 7, 16, 5), (1040, 1024, 4, 16, 1), (208, 64, 6, 3, 100)])
+def test_packed_rows_over_a_batch_of_samples(emu, sample_bytes, cb, n_samples, aad, group, run_len):
+    rng = np.random.default_rng(sample_bytes * 7 + n_samples)
+    key = rng.bytes(32)
+    ivs = np.frombuffer(rng.bytes(12 * n_samples), np.uint8).copy()
+    n = sample_bytes * n_samples
+    p = np.frombuffer(rng.bytes(n), np.uint8)
+    c_ref, t_ref = [], []
+    for s_ in range(n_samples):
+        q = p[s_ * sample_bytes:(s_ + 1) * sample_bytes]
+        iv_s = ivs[12 * s_:12 * s_ + 12].tobytes()
+        c_s, t_s = (oracle.mc_encrypt_framed(key, iv_s, cb, aad, q, 2) if aad else oracle.mc_encrypt(key, iv_s, cb, q, 2))
+        c_ref.append(c_s)
+        t_ref.append(t_s)
+    c_ref, t_ref = np.concatenate(c_ref), np.concatenate(t_ref)
+    c, t, _ = run_packed(emu, ENC, key, bytes(12), cb, p, n, group=group, run_len=run_len, aad=aad, sample_bytes=sample_bytes, ivs=ivs)
+    assert np.array_equal(c, c_ref) and np.array_equal(t, t_ref)
+    bad_t = t_ref.copy()
+    bad_t[len(bad_t) // 2, 0] ^= 1
+    out, _, ok = run_packed(emu, DEC, key, bytes(12), cb, c_ref, n, tags=bad_t, group=group, run_len=run_len, aad=aad, sample_bytes=sample_bytes, ivs=ivs)
+    expect = np.ones(len(bad_t), np.uint32)
+    expect[len(bad_t) // 2] = 0
+    assert np.array_equal(out, p) and np.array_equal(ok, expect)
 
 
 def test_index_arithmetic_under_address_and_ub_sanitizers(tmp_path):
