@@ -130,6 +130,7 @@ __device__ __forceinline__ void fr_packed_body(const FrParams& P, const char* sm
             FrSlot si = {0u, lane, 0xFFFFFFFFu};
             uint4 z = make_uint4(0, 0, 0, 0);
             if (valid) z = fr_packed_slot_lane<MODE, ABS>(P, sm, L, g, slot, si);
+            if (MODE == FR_MODE_CTR) continue;                   // nothing to authenticate
             if (lane == 0u && si.i != 0u) z = fr_xor4(z, carry);
             const uint32_t first = lane >= si.i ? lane - si.i : 0u;      // lowest lane of this row in the same chunk
 #pragma unroll
@@ -378,6 +379,8 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
         if ((e = cudaFuncSetAttribute(fr_verify_sequential_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
         if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_DEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
         if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_ENC>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_CTR>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_VERIFY>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
         for (int i = 0; i < 8 && e == cudaSuccess; i++) e = cudaStreamCreateWithFlags(&ctx->streams[i], cudaStreamNonBlocking);
         if (e != cudaSuccess) break;
         if ((e = cudaEventCreateWithFlags(&ctx->tags_ready, cudaEventDisableTiming)) != cudaSuccess) break;
@@ -631,7 +634,8 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
 
     plan_segments(ctx, sample_bytes, n_chunks, P);
     // Many short chains: one run of counters per lane (see fr_packed_body) when that is predicted to be faster.
-    const bool packed = (mode == FR_MODE_DEC || mode == FR_MODE_ENC) && plan_packed(ctx, sample_bytes, n_chunks, P);
+    const bool packed = (mode == FR_MODE_DEC || mode == FR_MODE_ENC || mode == FR_MODE_CTR || mode == FR_MODE_VERIFY) &&
+                        plan_packed(ctx, sample_bytes, n_chunks, P);
 
     P.in = (const uint8_t*)b.in;
     P.out = (uint8_t*)b.out;
@@ -669,8 +673,10 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
                                          : cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_DEC>, P); break;
         case FR_MODE_ENC:    le = packed ? cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_ENC>, P)
                                          : cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_ENC>, P); break;
-        case FR_MODE_CTR:    le = cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_CTR>, P); break;
-        case FR_MODE_VERIFY: le = cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_VERIFY>, P); break;
+        case FR_MODE_CTR:    le = packed ? cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_CTR>, P)
+                                         : cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_CTR>, P); break;
+        case FR_MODE_VERIFY: le = packed ? cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_VERIFY>, P)
+                                         : cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_VERIFY>, P); break;
         case FR_MODE_PADGEN: le = cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_PADGEN>, P); break;
         case FR_MODE_PADDEC: le = cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_PADDEC>, P); break;
         default: return FASTRACK_ERR_ARG;

@@ -592,7 +592,10 @@ template <int MODE, bool ABS>
 __device__ __forceinline__ uint4 fr_packed_slot_lane(const FrParams& P, const char* sm, const FrLane& L,
                                                      const FrPackGeom& g, uint32_t slot, FrSlot& si)
 {
-    static_assert(MODE == FR_MODE_DEC || MODE == FR_MODE_ENC, "packed rows exist for the fused passes");
+    static_assert(MODE == FR_MODE_DEC || MODE == FR_MODE_ENC || MODE == FR_MODE_CTR || MODE == FR_MODE_VERIFY,
+                  "packed rows exist for the fused passes and their two halves");
+    constexpr bool DO_AES = MODE != FR_MODE_VERIFY;       // VERIFY still needs E_K(J0), counter 1
+    constexpr bool DO_GHASH = MODE != FR_MODE_CTR;
     const uint32_t sample = slot / g.slots_sample, t = slot - sample * g.slots_sample;
     const uint32_t k = t / g.slots_full, i = t - k * g.slots_full;
     const uint32_t kk = sample * P.chunks_per_sample + k;
@@ -602,15 +605,21 @@ __device__ __forceinline__ uint4 fr_packed_slot_lane(const FrParams& P, const ch
     const uint32_t c0 = i * g.run + 1u;                                  // the run's counters are c0 .. c1 - 1
     uint32_t c1 = c0 + g.run;
     if (c1 > nblk + 2u) c1 = nblk + 2u;
-    const uint4 hpow = P.pow[nblk + 4u - c1];                            // for the run's last block, counter c1 - 1
+    uint4 hpow = make_uint4(0, 0, 0, 0);
+    if (DO_GHASH) hpow = P.pow[nblk + 4u - c1];                          // for the run's last block, counter c1 - 1
     const uint8_t* in = P.in + ck.off;
     uint8_t* out = P.out + ck.off;
-    const FrCtrChunk cc = fr_ctr_chunk<ABS>(sm, L.lane4, P, ck.iv_w0, ck.iv_w1, fr_bswap(ck.iv_ctr));
-    FrCtrGroup cg = fr_ctr_group<ABS>(sm, L.lane4, P, cc, c0);
+    FrCtrChunk cc = {0, 0, 0, 0};
+    FrCtrGroup cg = {0, 0, 0, 0};
+    if (DO_AES || c0 == 1u) {
+        cc = fr_ctr_chunk<ABS>(sm, L.lane4, P, ck.iv_w0, ck.iv_w1, fr_bswap(ck.iv_ctr));
+        cg = fr_ctr_group<ABS>(sm, L.lane4, P, cc, c0);
+    }
     uint4 y = make_uint4(0, 0, 0, 0), extra = make_uint4(0, 0, 0, 0);
     for (uint32_t c = c0; c < c1; c++) {
-        if ((c & 255u) == 0u && c != c0) cg = fr_ctr_group<ABS>(sm, L.lane4, P, cc, c);      // entered the next 256-counter group
-        const uint4 ks = fr_aes256_ctr_block<ABS>(sm, L.lane4, P, cc, cg, c);
+        if (DO_AES && (c & 255u) == 0u && c != c0) cg = fr_ctr_group<ABS>(sm, L.lane4, P, cc, c);   // entered the next 256-counter group
+        uint4 ks = make_uint4(0, 0, 0, 0);
+        if (DO_AES ? (DO_GHASH || c != 1u) : (c == 1u)) ks = fr_aes256_ctr_block<ABS>(sm, L.lane4, P, cc, cg, c);
         uint4 gblk;
         if (c == 1u) {
             extra = ks;                                                                      // E_K(J0)
@@ -621,11 +630,14 @@ __device__ __forceinline__ uint4 fr_packed_slot_lane(const FrParams& P, const ch
             const uint32_t nvalid = full ? 16u : (uint32_t)(ck.len - boff);
             const uint4 x = full ? *(const uint4*)(in + boff) : fr_load_partial(in + boff, nvalid);
             const uint4 o = fr_xor4(x, ks);
-            if (full) *(uint4*)(out + boff) = o; else fr_store_partial(out + boff, o, nvalid);
+            if (MODE != FR_MODE_VERIFY) { if (full) *(uint4*)(out + boff) = o; else fr_store_partial(out + boff, o, nvalid); }
             gblk = (MODE == FR_MODE_ENC) ? (full ? o : fr_mask_bytes(o, nvalid)) : x;
         }
-        y = fr_xor4(y, gblk);
-        if (c + 1u != c1) y = fr_ghash_tabmul<ABS>(sm, L, y);                                // Horner step with the fixed multiplier H
+        if (DO_GHASH) {
+            y = fr_xor4(y, gblk);
+            if (c + 1u != c1) y = fr_ghash_tabmul<ABS>(sm, L, y);                            // Horner step with the fixed multiplier H
+        }
     }
+    if (!DO_GHASH) return make_uint4(0, 0, 0, 0);
     return fr_xor4(fr_gf128_mul(y, hpow), extra);
 }

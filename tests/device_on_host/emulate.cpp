@@ -207,6 +207,7 @@ static void run_packed(Setup& S, const uint8_t* tags_in, uint8_t* tags_out, uint
                 z[lane] = uint4{0, 0, 0, 0};
                 if (valid[lane]) z[lane] = fr_packed_slot_lane<MODE, false>(P, S.sm.data(), L, g, base + lane, si[lane]);
             }
+            if (MODE == FR_MODE_CTR) continue;
             if (si[0].i != 0u) z[0] = fr_xor4(z[0], carry);
             for (uint32_t d = 1; d < 32; d <<= 1) {
                 uint4 up[32];
@@ -228,7 +229,7 @@ static void run_packed(Setup& S, const uint8_t* tags_in, uint8_t* tags_out, uint
     }
 }
 
-// One packed-row pass (mode 0 = decrypt + verify, 1 = encrypt + tag): pack_run counters per slot, pack_chunks chunks per work item.
+// One packed-row pass (mode 0 = decrypt + verify, 1 = encrypt + tag, 2 = counter mode only, 3 = verify only): pack_run counters per slot, pack_chunks chunks per work item.
 extern "C" int emu_packed(int mode, const uint8_t* key, const uint8_t* iv_base, size_t cb, const uint8_t* in, size_t len,
                           uint8_t* out, const uint8_t* tags_in, uint8_t* tags_out, uint32_t* ok, uint32_t pack_chunks,
                           uint32_t pack_run, uint32_t first_chunk, uint32_t aad_mod, size_t sample_bytes, const uint8_t* ivs)
@@ -261,6 +262,8 @@ extern "C" int emu_packed(int mode, const uint8_t* key, const uint8_t* iv_base, 
     P.out = out;
     if (mode == FR_MODE_DEC) run_packed<FR_MODE_DEC>(S, tags_in, tags_out, ok);
     else if (mode == FR_MODE_ENC) run_packed<FR_MODE_ENC>(S, tags_in, tags_out, ok);
+    else if (mode == FR_MODE_CTR) run_packed<FR_MODE_CTR>(S, tags_in, tags_out, ok);
+    else if (mode == FR_MODE_VERIFY) run_packed<FR_MODE_VERIFY>(S, tags_in, tags_out, ok);
     else return -1;
     return 0;
 }
@@ -323,7 +326,7 @@ static int run_case(size_t cb, size_t len, uint32_t seg, uint32_t first, uint32_
         for (size_t i = 0; i < K; i++) ok[i] = 9;
         if (ivs) for (size_t i = 0; i < 12 * n_samples; i++) ivs[i] = (uint8_t)(lcg(s) >> 24);
         bad |= emu_pass(mode, key, iv, cb, in, len, out, pad, mask, tin, tout, ok, seg, first, aad, sample_bytes, ivs);
-        if (mode <= FR_MODE_ENC)                        // the packed-row form of the same pass, seg doubling as group size and run length
+        if (mode <= FR_MODE_VERIFY)                     // the packed-row form of the same pass, seg doubling as group size and run length
             for (uint32_t run : {1u, seg + 1u, 40u})
                 bad |= emu_packed(mode, key, iv, cb, in, len, out, tin, tout, ok, seg * 3 - 2, run, first, aad, sample_bytes, ivs);
         delete[] in; delete[] out; delete[] pad; delete[] mask; delete[] tin; delete[] tout; delete[] ok; delete[] ivs;

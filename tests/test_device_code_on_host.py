@@ -174,6 +174,22 @@ def run_packed(lib, mode, key, iv, cb, data, n, tags=None, group=1, run_len=1, f
     return out[:n], tout, ok
 
 
+def run_packed_verify(lib, key, iv, cb, cipher, n, tags, group, run_len, aad):
+    """Verify-only pass: `out` is never written, so hand it the ciphertext's own buffer with guard bytes behind it."""
+    K = (n + cb - 1) // cb
+    buf = np.full(n + 64, 0xA5, np.uint8)
+    buf[:n] = cipher
+    k = np.frombuffer(key, np.uint8).copy()
+    v = np.frombuffer(iv, np.uint8).copy()
+    tin = np.ascontiguousarray(tags, np.uint8)
+    tout = np.zeros((K, 16), np.uint8)
+    ok = np.full(K, 7, np.uint32)
+    rc = lib.emu_packed(VERIFY, k.ctypes.data, v.ctypes.data, cb, buf.ctypes.data, n, buf.ctypes.data, tin.ctypes.data,
+                        tout.ctypes.data, ok.ctypes.data, group, run_len, 0, aad, 0, None)
+    assert rc == 0 and (buf[n:] == 0xA5).all() and np.array_equal(buf[:n], cipher)
+    return buf[:n], tout, ok
+
+
 PACKED_SHAPES = [(1, 16, 1), (16, 16, 1), (16 * 100, 16, 7), (16 * 100 + 5, 16, 300), (32 * 37 + 17, 32, 5), (48 * 50, 48, 4),
                  (112 * 9 + 1, 112, 2), (240 * 33, 240, 3), (496 * 5 + 495, 496, 2), (512 * 6 + 16, 512, 1), (528 * 4, 528, 3),
                  (1024 * 5 + 1000, 1024, 2), (2048 * 3 + 31, 2048, 1), (700, 4096, 1),
@@ -205,6 +221,11 @@ def test_packed_rows_match_oracle(emu, n, cb, group, aad, run_len):
     assert 0 < int(ok_ref.sum()) < K or K <= 2
     out, _, ok = run_packed(emu, DEC, key, iv, cb, bad_c, n, tags=bad_t, group=group, run_len=run_len, aad=aad)
     assert np.array_equal(out, p_ref) and np.array_equal(ok, ok_ref)
+    out, _, _ = run_packed(emu, CTR, key, iv, cb, bad_c, n, group=group, run_len=run_len, aad=aad)
+    assert np.array_equal(out, p_ref)
+    keep = bad_c.copy()
+    _, _, ok = run_packed_verify(emu, key, iv, cb, keep, n, bad_t, group, run_len, aad)
+    assert np.array_equal(ok, ok_ref)
 
 
 @pytest.mark.parametrize("run_len", [1, 4, 7])

@@ -64,6 +64,20 @@ def test_small_chunks_match_oracle(family, n, cb):
             assert np.array_equal(p[keep], p_ref[keep]) and np.array_equal(p, p_ref)
         p, ok = g.pipelined(iv, bad_c, bad_t, 3)
         assert np.array_equal(ok, ok_ref) and np.array_equal(p, p_ref)
+        # the two halves of the fused pass (eager evaluation: plaintext first, verdicts later)
+        K = t_ref.shape[0]
+        d_c = torch.from_numpy(bad_c).cuda()
+        d_t = torch.from_numpy(bad_t.reshape(-1).copy()).cuda()
+        d_o = torch.full((n + 32,), 0xA5, dtype=torch.uint8, device="cuda")
+        d_ok = torch.full((K + 8,), 0x5A5A5A5A, dtype=torch.int32, device="cuda")
+        g.ctx.ctr_crypt(iv, d_c.data_ptr(), n, d_o[16:].data_ptr(), 0)
+        g.ctx.verify(iv, d_c.data_ptr(), n, d_t.data_ptr(), d_ok[4:].data_ptr(), 0)
+        torch.cuda.synchronize()
+        assert np.array_equal(d_o[16:16 + n].cpu().numpy(), p_ref)
+        assert bool((d_o[:16] == 0xA5).all()) and bool((d_o[16 + n:] == 0xA5).all())
+        okh = d_ok.cpu().numpy().view(np.uint32)
+        assert np.array_equal(okh[4:4 + K], ok_ref) and (okh[:4] == 0x5A5A5A5A).all() and (okh[4 + K:] == 0x5A5A5A5A).all()
+        assert np.array_equal(d_c.cpu().numpy(), bad_c)                       # verify-only leaves the ciphertext alone
 
 
 def test_two_million_sixteen_byte_chunks(family):
