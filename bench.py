@@ -518,11 +518,11 @@ def run_sweep(args):
                     ctx.decrypt_verify(ivs_h[12 * s:12 * s + 12], d_c.data_ptr() + s * sample_bytes, sample_bytes,
                                        d_t.data_ptr() + 16 * cps * s, d_o.data_ptr() + s * sample_bytes,
                                        d_ok.data_ptr() + 4 * cps * s, st)
-            t_each = timed(one_by_one, 20)
+            t_each = timed(one_by_one, 20) if n_samples <= 1024 else None        # a call per sample is pointless beyond that
             assert bool((d_ok == 1).all()) and bool((d_o == d_p).all())
         print(json.dumps({"cell": label, "sample_bytes": sample_bytes, "n_samples": n_samples, "chains_per_sample": chains,
                           "chunk": cb, "batch_call_us": t_batch * 1e6, "batch_call_gbs": n / t_batch / 1e9,
-                          "one_call_per_sample_us": t_each * 1e6}), flush=True)
+                          "one_call_per_sample_us": None if t_each is None else t_each * 1e6}), flush=True)
 
     for K in (1, 4, 16, 64, 256, 1024):                                   # config 1
         device_cell(64 << 20, (64 << 20) // K, "config1")
@@ -534,6 +534,11 @@ def run_sweep(args):
         d2h_cell(670_000_000, 4 << 20, ns, "config3_d2h")
     samples_cell(3 * 224 * 224 * 2, 64, 16, "sample_batch")        # a ResNet-style batch: 64 fp16 images, 16 tags each
     samples_cell(3 * 224 * 224 * 2, 256, 16, "sample_batch")
+    samples_cell(400, 1 << 18, 1, "small_sample_batch")             # 262 144 feature rows of 100 floats, one tag each
+    samples_cell(64, 1 << 20, 1, "small_sample_batch")              # a million 64-byte records
+    samples_cell(4096, 1 << 14, 16, "small_sample_batch")           # 4 KiB samples cut into 16 chunks of 256 bytes
+    for cb in (16, 64, 256, 1024, 4096, 16384):                    # many small chunks (packed-row kernels below about 8 KiB)
+        device_cell(256 << 20, cb, "small_chunks")
     modes_cell(256 << 20, 4 << 20, "split_passes")
     for K in (16, 64, 256, 1024, 4096):
         modes_cell(64 << 20, (64 << 20) // K, "split_passes_vs_K")

@@ -258,6 +258,7 @@ struct fastrack_ctx {
     uint32_t pack_max_blocks;     // chunks of at most this many blocks may take the packed-row kernels (FASTRACK_PACK_MAX_BLOCKS; 0 = never)
     uint32_t pack_run_override;   // 0 = automatic; else packed rows with this run length wherever they apply (FASTRACK_PACK_RUN, tests)
     uint32_t pack_group_override; // 0 = automatic; else this many chunks per packed work item (FASTRACK_PACK_GROUP, tests)
+    struct { size_t sample_bytes, n_chunks; uint32_t run, group; bool valid; } pack_memo;   // the planner's last answer (callers repeat shapes)
 };
 
 #define FR_CUDA(ctx, call)                                              \
@@ -544,13 +545,25 @@ static void plan_segments(const fastrack_ctx* ctx, size_t sample_bytes, size_t n
 // per row plus 400 per segment; a packed row costs about 280 plus, per counter of its run, 258 clocks for runs up to
 // 3 counters and more beyond (a lane's 16-byte loads and stores are 16 * run bytes apart, so longer runs touch more
 // cache lines per request).
-static bool plan_packed(const fastrack_ctx* ctx, size_t sample_bytes, size_t n_chunks, FrParams& P)
+static bool plan_packed(fastrack_ctx* ctx, size_t sample_bytes, size_t n_chunks, FrParams& P)
 {
     if (!ctx->pack_max_blocks) return false;
     const size_t first_len = sample_bytes < ctx->chunk_bytes ? sample_bytes : ctx->chunk_bytes;
     const size_t counters = (first_len + 15) / 16 + 1;
     if (counters - 1 > ctx->pack_max_blocks) return false;
     const size_t sms = (size_t)ctx->num_sms, warps = sms * FR_WARPS;
+    if (!ctx->pack_run_override && counters > 32 && n_chunks * 8 < warps) return false;   // a few long chains: rows, no search needed
+    if (ctx->pack_memo.valid && ctx->pack_memo.sample_bytes == sample_bytes && ctx->pack_memo.n_chunks == n_chunks) {
+        if (!ctx->pack_memo.run) return false;
+        P.pack_run = ctx->pack_memo.run;
+        P.pack_chunks = ctx->pack_memo.group;
+        P.n_items = (uint32_t)((n_chunks + P.pack_chunks - 1) / P.pack_chunks);
+        return true;
+    }
+    ctx->pack_memo.valid = true;
+    ctx->pack_memo.sample_bytes = sample_bytes;
+    ctx->pack_memo.n_chunks = n_chunks;
+    ctx->pack_memo.run = 0;
 
     const size_t rows_ref = (counters + 1 + FR_ROW_BLOCKS - 1) / FR_ROW_BLOCKS;
     const size_t waves = ((size_t)P.n_items + warps - 1) / warps;
@@ -592,6 +605,8 @@ static bool plan_packed(const fastrack_ctx* ctx, size_t sample_bytes, size_t n_c
     P.pack_run = (uint32_t)best_run;
     P.pack_chunks = (uint32_t)best_group;
     P.n_items = (uint32_t)((n_chunks + best_group - 1) / best_group);
+    ctx->pack_memo.run = P.pack_run;
+    ctx->pack_memo.group = P.pack_chunks;
     return true;
 }
 
