@@ -87,7 +87,8 @@ FASTRACK_API size_t fastrack_num_chunks(const fastrack_ctx* ctx, size_t len);
 
 /* Pre-sizes the per-chunk scratch (40 bytes per chunk: two banks of a 16-byte accumulator and a counter) for buffers up to max_len bytes so that later
  * calls allocate nothing.  Without it the first call that needs more chunks than any call before
- * grows the scratch (cudaMalloc + a device synchronisation) before launching.
+ * grows the scratch (cudaMalloc + a device synchronisation) before launching.  Contexts whose chunk_bytes is at
+ * most 992 never need more than the scratch they are created with (such chunks are never split between warps).
  * Stream capture: once the scratch is large enough, every asynchronous call below is a single kernel launch with
  * all arguments passed by value, so it may be recorded into a CUDA graph and replayed.  A replay repeats the
  * recorded arguments -- the IV base included, for the calls that take it by value; the *_samples calls read their IV

@@ -281,6 +281,10 @@ static void secure_zero(void* p, size_t n)
 static int ensure_scratch(fastrack_ctx* ctx, size_t chunks)
 {
     if (chunks <= ctx->scratch_chunks) return FASTRACK_OK;
+    // A chunk of at most 62 blocks is two rows, and no segment is shorter than two rows: such chunks are never split
+    // between warps, so neither kernel family touches the scratch (40 bytes per chunk would exceed the data itself
+    // at 16-byte chunks).  launch_pass checks this assumption.
+    if (!ctx->seg_rows_override && ctx->chunk_bytes <= 62 * 16) return FASTRACK_OK;
     size_t cap = ctx->scratch_chunks ? ctx->scratch_chunks : 1024;
     while (cap < chunks) cap *= 2;
     FR_CUDA(ctx, cudaDeviceSynchronize());       // nothing may still be using the old scratch
@@ -662,6 +666,7 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
     P.te0 = ctx->d_te0;
     P.gh_tab = packed ? ctx->d_gh1_tab : ctx->d_gh_tab;
     P.pow = ctx->d_pow;
+    if (!packed && P.segs_per_chunk > 1 && first_chunk + n_chunks > ctx->scratch_chunks) return FASTRACK_ERR_NOMEM;   // cannot happen, see ensure_scratch
     uint32_t* bank = ctx->d_scratch + (size_t)b.bank * 5 * ctx->scratch_chunks;
     P.acc = bank + 4 * first_chunk;
     P.cnt = bank + 4 * ctx->scratch_chunks + first_chunk;
