@@ -113,8 +113,19 @@ def test_portable_shared_addressing_path(monkeypatch):
     expects, and falls back to ordinary pointer arithmetic otherwise.  FASTRACK_GENERIC_SMEM=1 forces the
     fallback so that it is exercised on hardware where the fast form applies."""
     monkeypatch.setenv("FASTRACK_GENERIC_SMEM", "1")
+    _every_pass_on([(1, 16, 0), (70001, 4096, 0), ((1 << 20) + 33, 65536, 16), ((5 << 20) + 7, 1 << 20, 0)])
+
+
+def test_portable_shared_addressing_path_packed_rows(monkeypatch):
+    """The same fallback in the packed-row kernels (forced here by fixing the run length)."""
+    monkeypatch.setenv("FASTRACK_GENERIC_SMEM", "1")
+    monkeypatch.setenv("FASTRACK_PACK_RUN", "3")
+    _every_pass_on([(1, 16, 0), (80009, 16, 0), (154128, 512, 4), (70001, 4096, 0), (300000, 16384, 16)])
+
+
+def _every_pass_on(cases):
     key, iv = synth.key_and_iv(7)
-    for n, cb, chains in [(1, 16, 0), (70001, 4096, 0), ((1 << 20) + 33, 65536, 16), ((5 << 20) + 7, 1 << 20, 0)]:
+    for n, cb, chains in cases:
         plain = synth.random_bytes(n, 7, salt=n)
         c, t = (oracle.mc_encrypt_framed(key, iv, cb, chains, plain, NT) if chains else oracle.mc_encrypt(key, iv, cb, plain, NT))
         K = t.shape[0]
