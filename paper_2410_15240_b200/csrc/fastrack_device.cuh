@@ -22,6 +22,10 @@
 //   different 16-byte bank groups: every 128-bit lookup is conflict-free.  The lane's last block is
 //   not multiplied by H^32 but by the power of H that its distance from the end of the chunk calls
 //   for, with a general product built from integer multiplies; the 32 lane values are then XOR-reduced.
+//
+// A second layout for launches with many chunks that are not large ("packed rows", at the end of this file)
+// gives every lane a short run of one chunk's counters instead; it uses the same tables and the same lane code
+// for the cipher, the table multiply and the general product.
 #pragma once
 #include <stdint.h>
 
