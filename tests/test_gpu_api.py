@@ -116,3 +116,38 @@ def test_long_dependent_chain_without_host_synchronisation():
         assert np.array_equal(a.cpu().numpy(), plain)
         c_ref, _ = oracle.mc_encrypt(key2, iv, cb, plain, oracle.host_threads())       # the last round used key 2
         assert np.array_equal(b.cpu().numpy(), c_ref)
+
+
+def test_contexts_on_concurrent_streams_do_not_interfere():
+    """Four contexts (own keys, chunk sizes in both kernel families), each on its own stream, 30 rounds of
+    encrypt -> decrypt queued without host synchronisation so that their kernels overlap on the device; every
+    context's result must equal the oracle's for its key."""
+    shapes = [(65536, (3 << 20) + 100), (1 << 20, (5 << 20) + 16), (256, (1 << 20) + 7), (4096, 2 << 20)]
+    iv = synth.key_and_iv(0)[1]
+    ctxs, streams, bufs = [], [], []
+    try:
+        for i, (cb, n) in enumerate(shapes):
+            key = synth.key_and_iv(20 + i)[0]
+            ctx = fastrack.Context(key, cb)
+            K = ctx.num_chunks(n)
+            ctx.reserve(n)
+            plain = synth.random_bytes(n, 20 + i, salt=41)
+            ctxs.append((ctx, key, cb, n, K, plain))
+            streams.append(torch.cuda.Stream())
+            bufs.append((torch.from_numpy(plain).cuda(), torch.empty(n, dtype=torch.uint8, device="cuda"),
+                         torch.empty(n, dtype=torch.uint8, device="cuda"), torch.empty(16 * K, dtype=torch.uint8, device="cuda"),
+                         torch.zeros(30, K, dtype=torch.int32, device="cuda")))
+        torch.cuda.synchronize()
+        for r in range(30):
+            for (ctx, key, cb, n, K, plain), st, (d_p, d_c, d_o, d_t, d_ok) in zip(ctxs, streams, bufs):
+                ctx.encrypt_tag(iv, d_p.data_ptr(), n, d_c.data_ptr(), d_t.data_ptr(), st.cuda_stream)
+                ctx.decrypt_verify(iv, d_c.data_ptr(), n, d_t.data_ptr(), d_o.data_ptr(), d_ok[r].data_ptr(), st.cuda_stream)
+        torch.cuda.synchronize()
+        for (ctx, key, cb, n, K, plain), (d_p, d_c, d_o, d_t, d_ok) in zip(ctxs, bufs):
+            c_ref, t_ref = oracle.mc_encrypt(key, iv, cb, plain, oracle.host_threads())
+            assert bool((d_ok == 1).all())
+            assert np.array_equal(d_o.cpu().numpy(), plain)
+            assert np.array_equal(d_c.cpu().numpy(), c_ref) and np.array_equal(d_t.cpu().numpy().reshape(K, 16), t_ref)
+    finally:
+        for c in ctxs:
+            c[0].close()
