@@ -584,7 +584,7 @@ static bool plan_packed(fastrack_ctx* ctx, size_t sample_bytes, size_t n_chunks,
         if (ctx->pack_run_override) run = ctx->pack_run_override;
         if (run > counters) run = counters;
         const size_t slots = (counters + run - 1) / run;
-        if (n_chunks * slots >= ((size_t)1 << 32) - 64) continue;                  // slots are counted in 32 bits, a row may overshoot by 31
+        if (n_chunks * slots >= ((size_t)1 << 32) - 2048) continue;                // slots and chunks are counted in 32 bits; a row may overshoot by 31, an item's first chunk index by its size
         const size_t per_row = 280 + run * (run < 14 ? step_clocks[run] : 335);
         const size_t row_latency = 2500 + run * 2250;       // one warp alone on its SM partition
         // a work item is `group` whole chunks.  Its last row is only partly filled, and an instruction costs the same
