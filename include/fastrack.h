@@ -265,6 +265,15 @@ FASTRACK_API int fastrack_decrypt_verify_noalloc(fastrack_ctx* ctx, const uint8_
 FASTRACK_API int fastrack_pipelined_d2h(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_plain, size_t len,
                                         void* d_cipher, void* h_cipher_pinned, void* h_tags, int n_streams);
 
+/* fastrack_pipelined_d2h for a batch of samples, each encrypted as its own multi-chain message under its own IV base
+ * (Sections 4.2 + 4.3, outbound): n_samples samples of sample_bytes bytes (a multiple of 16) back to back in d_plain;
+ * h_iv_bases is a HOST pointer to 12 * n_samples bytes (pinned or pageable; copied in once, up front); tags leave in
+ * the order of fastrack_encrypt_tag_samples.  Stages are whole samples.  Blocking; everything else as in
+ * fastrack_pipelined_d2h. */
+FASTRACK_API int fastrack_pipelined_d2h_samples(fastrack_ctx* ctx, const void* h_iv_bases, size_t sample_bytes,
+                                                size_t n_samples, const void* d_plain, void* d_cipher,
+                                                void* h_cipher_pinned, void* h_tags, int n_streams);
+
 /* Stage-level trace of pipelined host->device calls (paper Section 4.3 argues that the copy of one piece hides
  * the kernels of the previous one; this shows it).  While enabled, every fastrack_pipelined_h2d /
  * fastrack_pipelined_h2d_ahead call records three CUDA events per stage on the stage's stream -- before its copy,

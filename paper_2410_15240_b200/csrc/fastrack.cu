@@ -921,10 +921,11 @@ extern "C" int fastrack_pipelined_h2d_ahead(fastrack_ctx* ctx, const uint8_t iv_
     return pipelined_impl(ctx, iv_base, h_cipher_pinned, len, h_tags, d_pad, d_plain, d_ok, n_streams);
 }
 
-extern "C" int fastrack_pipelined_d2h(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_plain, size_t len,
-                                      void* d_cipher, void* h_cipher_pinned, void* h_tags, int n_streams)
+static int pipelined_d2h_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_plain, size_t len, void* d_cipher,
+                              void* h_cipher_pinned, void* h_tags, int n_streams, const void* h_iv_bases = nullptr,
+                              size_t sample_bytes = 0)
 {
-    if (!ctx || !iv_base) return FASTRACK_ERR_ARG;
+    if (!ctx || (!iv_base && !h_iv_bases)) return FASTRACK_ERR_ARG;
     if (n_streams < 1 || n_streams > 8) return FASTRACK_ERR_ARG;
     if (len == 0) return FASTRACK_OK;
     if (!d_plain || !d_cipher || !h_cipher_pinned || !h_tags) return FASTRACK_ERR_ARG;
@@ -933,13 +934,17 @@ extern "C" int fastrack_pipelined_d2h(fastrack_ctx* ctx, const uint8_t iv_base[1
     cudaError_t e = cudaPointerGetAttributes(&attr, h_cipher_pinned);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return FASTRACK_ERR_NOT_PINNED; }
     if (attr.type != cudaMemoryTypeHost) return FASTRACK_ERR_NOT_PINNED;
-    const size_t K = fastrack_num_chunks(ctx, len);
+    const size_t cb = ctx->chunk_bytes;
+    const size_t cps = sample_bytes ? (sample_bytes + cb - 1) / cb : 0;
+    const size_t n_samples = sample_bytes ? len / sample_bytes : 0;
+    const size_t K = sample_bytes ? cps * n_samples : fastrack_num_chunks(ctx, len);
     if (K > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
     int rc = ensure_scratch(ctx, K);
     if (rc != FASTRACK_OK) return rc;
-    if (K > ctx->tags_stage_chunks) {
+    const size_t need_slots = K + (12 * n_samples + 15) / 16;      // tags, then (batch of samples) the IV bases
+    if (need_slots > ctx->tags_stage_chunks) {
         size_t cap = ctx->tags_stage_chunks ? ctx->tags_stage_chunks : 1024;
-        while (cap < K) cap *= 2;
+        while (cap < need_slots) cap *= 2;
         FR_CUDA(ctx, cudaDeviceSynchronize());
         cudaFree(ctx->d_tags_stage);
         ctx->d_tags_stage = nullptr;
@@ -948,24 +953,42 @@ extern "C" int fastrack_pipelined_d2h(fastrack_ctx* ctx, const uint8_t iv_base[1
         if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); return FASTRACK_ERR_NOMEM; }
         ctx->tags_stage_chunks = cap;
     }
+    uint8_t* d_ivs = (uint8_t*)(ctx->d_tags_stage + K);
+    cudaStream_t iv_stream = ctx->streams[7];
+    if (sample_bytes) {                          // the IV bases go in first: one small copy, every working stream waits for it
+        e = cudaMemcpyAsync(d_ivs, h_iv_bases, 12 * n_samples, cudaMemcpyHostToDevice, iv_stream);
+        if (e == cudaSuccess) e = cudaEventRecord(ctx->tags_ready, iv_stream);
+        if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); return FASTRACK_ERR_CUDA; }
+    }
     // On the way out the FIRST stage's kernel is the exposed one: smallest stage first.  The plan is made on
-    // whole chunks (K * chunk_bytes) and walked backwards, so every stage starts on a chunk boundary and the
-    // short last chunk, if any, stays at the end of the last (largest) stage.
+    // whole chunks (K * chunk_bytes), or whole samples, and walked backwards, so every stage starts on a chunk
+    // (sample) boundary and the short last chunk, if any, stays at the end of the last (largest) stage.
     size_t stage_bytes[FR_MAX_STAGES];
-    const size_t cb = ctx->chunk_bytes;
-    const size_t n_stages = plan_stages(ctx, K * cb, cb, stage_bytes);
+    const size_t unit = sample_bytes ? sample_bytes : cb;
+    const size_t n_stages = plan_stages(ctx, sample_bytes ? len : K * cb, unit, stage_bytes);
+    bool waited[8] = {false, false, false, false, false, false, false, false};
     size_t off = 0;
     for (size_t i = 0; i < n_stages; i++) {
         size_t n = stage_bytes[n_stages - 1 - i];
         if (n > len - off) n = len - off;
-        const size_t k0 = off / cb;
-        cudaStream_t st = ctx->streams[i % (size_t)n_streams];
+        const size_t k0 = sample_bytes ? (off / sample_bytes) * cps : off / cb;
+        const size_t k_here = sample_bytes ? (n / sample_bytes) * cps : (n + cb - 1) / cb;
+        const size_t si = i % (size_t)n_streams;
+        cudaStream_t st = ctx->streams[si];
+        rc = FASTRACK_OK;
+        if (sample_bytes && !waited[si]) {
+            waited[si] = true;
+            if (st != iv_stream && (e = cudaStreamWaitEvent(st, ctx->tags_ready, 0)) != cudaSuccess) {
+                ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); rc = FASTRACK_ERR_CUDA;
+            }
+        }
         PassBuffers b;
         b.in = (const uint8_t*)d_plain + off; b.out = (uint8_t*)d_cipher + off; b.tags_out = ctx->d_tags_stage + k0;
-        rc = launch_pass(ctx, FR_MODE_ENC, iv_base, k0, n, b, st);
+        if (sample_bytes) { b.ivs = d_ivs + 12 * (off / sample_bytes); b.sample_bytes = sample_bytes; }
+        if (rc == FASTRACK_OK) rc = launch_pass(ctx, FR_MODE_ENC, iv_base, k0, n, b, st);
         if (rc == FASTRACK_OK) {
             e = cudaMemcpyAsync((uint8_t*)h_cipher_pinned + off, (const uint8_t*)d_cipher + off, n, cudaMemcpyDeviceToHost, st);
-            if (e == cudaSuccess) e = cudaMemcpyAsync((uint8_t*)h_tags + 16 * k0, ctx->d_tags_stage + k0, 16 * ((n + cb - 1) / cb),
+            if (e == cudaSuccess) e = cudaMemcpyAsync((uint8_t*)h_tags + 16 * k0, ctx->d_tags_stage + k0, 16 * k_here,
                                                       cudaMemcpyDeviceToHost, st);
             if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); rc = FASTRACK_ERR_CUDA; }
         }
@@ -976,8 +999,27 @@ extern "C" int fastrack_pipelined_d2h(fastrack_ctx* ctx, const uint8_t iv_base[1
         }
         off += n;
     }
+    if (sample_bytes) FR_CUDA(ctx, cudaStreamSynchronize(iv_stream));
     for (int i = 0; i < n_streams; i++) FR_CUDA(ctx, cudaStreamSynchronize(ctx->streams[i]));
     return FASTRACK_OK;
+}
+
+extern "C" int fastrack_pipelined_d2h(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_plain, size_t len,
+                                      void* d_cipher, void* h_cipher_pinned, void* h_tags, int n_streams)
+{
+    if (!iv_base) return FASTRACK_ERR_ARG;
+    return pipelined_d2h_impl(ctx, iv_base, d_plain, len, d_cipher, h_cipher_pinned, h_tags, n_streams);
+}
+
+extern "C" int fastrack_pipelined_d2h_samples(fastrack_ctx* ctx, const void* h_iv_bases, size_t sample_bytes, size_t n_samples,
+                                              const void* d_plain, void* d_cipher, void* h_cipher_pinned, void* h_tags,
+                                              int n_streams)
+{
+    if (!ctx || !h_iv_bases) return FASTRACK_ERR_ARG;
+    if (sample_bytes == 0 || (sample_bytes & 15)) return FASTRACK_ERR_ARG;
+    if (n_samples > ((size_t)1 << 40) / sample_bytes) return FASTRACK_ERR_TOO_MANY;
+    return pipelined_d2h_impl(ctx, nullptr, d_plain, sample_bytes * n_samples, d_cipher, h_cipher_pinned, h_tags, n_streams,
+                              h_iv_bases, sample_bytes);
 }
 
 // Argument checks shared by the two batch-of-samples entry points.

@@ -23,7 +23,8 @@ EXPORTS = ("fastrack_ctx_create", "fastrack_ctx_destroy", "fastrack_num_chunks",
            "fastrack_pipelined_h2d", "fastrack_launch_count", "fastrack_decrypt_verify_noalloc",
            "fastrack_ctr_crypt", "fastrack_verify", "fastrack_keystream", "fastrack_xor_verify",
            "fastrack_pipelined_h2d_ahead", "fastrack_ctx_set_framing", "fastrack_verify_sequential", "fastrack_pipelined_d2h", "fastrack_ctx_set_trace", "fastrack_ctx_get_trace",
-           "fastrack_decrypt_verify_samples", "fastrack_encrypt_tag_samples", "fastrack_pipelined_h2d_samples")
+           "fastrack_decrypt_verify_samples", "fastrack_encrypt_tag_samples", "fastrack_pipelined_h2d_samples",
+           "fastrack_pipelined_d2h_samples")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2410_15240_b200.build` "
@@ -80,6 +81,8 @@ _lib.fastrack_pipelined_h2d_ahead.restype = _int
 _lib.fastrack_pipelined_h2d_ahead.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp, _vp, _int]
 _lib.fastrack_pipelined_d2h.restype = _int
 _lib.fastrack_pipelined_d2h.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp, _int]
+_lib.fastrack_pipelined_d2h_samples.restype = _int
+_lib.fastrack_pipelined_d2h_samples.argtypes = [_vp, _vp, _sz, _sz, _vp, _vp, _vp, _vp, _int]
 _lib.fastrack_pipelined_h2d.restype = _int
 _lib.fastrack_pipelined_h2d.argtypes = [_vp, ctypes.c_char_p, _vp, _sz, _vp, _vp, _vp, _int]
 
@@ -203,6 +206,12 @@ def fastrack_pipelined_h2d_ahead(ctx, iv_base: bytes, h_cipher_pinned: int, leng
                                              n_streams)
 
 
+def fastrack_pipelined_d2h_samples(ctx, h_iv_bases: int, sample_bytes: int, n_samples: int, d_plain: int, d_cipher: int,
+                                   h_cipher_pinned: int, h_tags: int, n_streams: int) -> int:
+    return _lib.fastrack_pipelined_d2h_samples(ctx, h_iv_bases, sample_bytes, n_samples, d_plain, d_cipher, h_cipher_pinned,
+                                               h_tags, n_streams)
+
+
 def fastrack_pipelined_d2h(ctx, iv_base: bytes, d_plain: int, length: int, d_cipher: int, h_cipher_pinned: int,
                            h_tags: int, n_streams: int) -> int:
     return _lib.fastrack_pipelined_d2h(ctx, iv_base, d_plain, length, d_cipher, h_cipher_pinned, h_tags, n_streams)
@@ -287,6 +296,11 @@ class Context:
     def pipelined_d2h(self, iv_base, d_plain, length, d_cipher, h_cipher_pinned, h_tags, n_streams=4) -> None:
         self._check(fastrack_pipelined_d2h(self.handle, iv_base, d_plain, length, d_cipher, h_cipher_pinned, h_tags,
                                            n_streams))
+
+    def pipelined_d2h_samples(self, h_iv_bases, sample_bytes, n_samples, d_plain, d_cipher, h_cipher_pinned, h_tags,
+                              n_streams=4) -> None:
+        self._check(fastrack_pipelined_d2h_samples(self.handle, h_iv_bases, sample_bytes, n_samples, d_plain, d_cipher,
+                                                   h_cipher_pinned, h_tags, n_streams))
 
     @property
     def launches(self) -> int:

@@ -234,3 +234,54 @@ def test_pipelined_h2d_of_a_batch_of_samples(sample_bytes, cb, n_samples, chains
             assert [int(k) for k in np.flatnonzero(ok == 0)] == sorted({K // 3, K - 1})
             out = d_p.cpu().numpy()
             assert np.flatnonzero(out != plain).tolist() == [n - 1]
+
+
+@pytest.mark.parametrize("sample_bytes,cb,n_samples,chains,n_streams,in_place",
+                         [(1040, 1024, 5, 16, 1, False), (301056, 18816, 64, 16, 3, False), (1 << 20, 1 << 16, 9, 0, 2, True),
+                          (400, 400, 30000, 0, 4, False), (4096, 256, 3000, 16, 2, True)])
+def test_pipelined_d2h_of_a_batch_of_samples(sample_bytes, cb, n_samples, chains, n_streams, in_place):
+    """The outbound mirror: a batch of results leaves the GPU, every sample encrypted and tagged under its own IV base,
+    the device-to-host copies overlapped with the kernels.  Ciphertext and tags must equal the oracle's per sample."""
+    key, _ = synth.key_and_iv(3)
+    rng = np.random.Generator(np.random.PCG64(sample_bytes + n_samples + 2))
+    ivs = np.frombuffer(rng.bytes(12 * n_samples), np.uint8).copy()
+    n = sample_bytes * n_samples
+    plain = synth.random_bytes(n, 3, salt=n_samples + 200)
+    cs, ts = [], []
+    for s in range(n_samples):
+        part, iv = plain[s * sample_bytes:(s + 1) * sample_bytes], ivs[12 * s:12 * s + 12].tobytes()
+        c1, t1 = (oracle.mc_encrypt_framed(key, iv, cb, chains, part, 1) if chains else oracle.mc_encrypt(key, iv, cb, part, 1))
+        cs.append(c1)
+        ts.append(t1)
+    c_ref, t_ref = np.concatenate(cs), np.concatenate(ts)
+    K = t_ref.shape[0]
+    with fastrack.Context(key, cb) as ctx:
+        ctx.set_framing(chains)
+        h_c = torch.full((n + 64,), 0xA5, dtype=torch.uint8).pin_memory()
+        h_t = np.full(16 * K + 64, 0xA5, np.uint8)
+        for rep in range(2):
+            d_p = torch.from_numpy(plain).cuda()
+            d_c = d_p if in_place else torch.empty_like(d_p)
+            torch.cuda.synchronize()
+            ctx.pipelined_d2h_samples(ivs.ctypes.data, sample_bytes, n_samples, d_p.data_ptr(), d_c.data_ptr(),
+                                      h_c[32:].data_ptr(), h_t[32:].ctypes.data, n_streams)
+            # blocking call: the host buffers are complete now
+            assert np.array_equal(h_c[32:32 + n].numpy(), c_ref), f"rep {rep}"
+            assert np.array_equal(h_t[32:32 + 16 * K].reshape(K, 16), t_ref), f"rep {rep}"
+            assert bool((h_c[:32] == 0xA5).all()) and bool((h_c[32 + n:] == 0xA5).all())
+            assert (h_t[:32] == 0xA5).all() and (h_t[32 + 16 * K:] == 0xA5).all()
+            if not in_place:
+                assert np.array_equal(d_p.cpu().numpy(), plain)
+            h_c[32:32 + n] = 0
+            h_t[32:32 + 16 * K] = 0
+    rc, raw = fastrack.fastrack_ctx_create(key, cb)
+    assert rc == fastrack.OK
+    buf = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    pinned = torch.zeros(4096, dtype=torch.uint8).pin_memory()
+    tags = np.zeros(4096, np.uint8)
+    D = fastrack.fastrack_pipelined_d2h_samples
+    assert D(raw, None, 1024, 2, buf.data_ptr(), buf.data_ptr(), pinned.data_ptr(), tags.ctypes.data, 2) == fastrack.ERR_ARG
+    assert D(raw, ivs.ctypes.data, 1000, 2, buf.data_ptr(), buf.data_ptr(), pinned.data_ptr(), tags.ctypes.data, 2) == fastrack.ERR_ARG
+    assert D(raw, ivs.ctypes.data, 1024, 2, buf.data_ptr(), buf.data_ptr(), tags.ctypes.data, tags.ctypes.data, 2) == fastrack.ERR_NOT_PINNED
+    assert D(raw, ivs.ctypes.data, 1024, 0, buf.data_ptr(), buf.data_ptr(), pinned.data_ptr(), tags.ctypes.data, 2) == fastrack.OK
+    fastrack.fastrack_ctx_destroy(raw)
