@@ -666,7 +666,8 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
     P.te0 = ctx->d_te0;
     P.gh_tab = packed ? ctx->d_gh1_tab : ctx->d_gh_tab;
     P.pow = ctx->d_pow;
-    if (!packed && P.segs_per_chunk > 1 && first_chunk + n_chunks > ctx->scratch_chunks) return FASTRACK_ERR_NOMEM;   // cannot happen, see ensure_scratch
+    if (!packed && mode != FR_MODE_CTR && mode != FR_MODE_PADGEN && P.segs_per_chunk > 1 &&
+        first_chunk + n_chunks > ctx->scratch_chunks) return FASTRACK_ERR_NOMEM;                // cannot happen, see ensure_scratch
     uint32_t* bank = ctx->d_scratch + (size_t)b.bank * 5 * ctx->scratch_chunks;
     P.acc = bank + 4 * first_chunk;
     P.cnt = bank + 4 * ctx->scratch_chunks + first_chunk;
