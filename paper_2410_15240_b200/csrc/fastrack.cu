@@ -674,8 +674,7 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
 
     unsigned grid = (unsigned)ctx->num_sms;
     if (P.n_items < grid) grid = P.n_items;
-    cudaLaunchConfig_t cfg;
-    memset(&cfg, 0, sizeof cfg);
+    cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(FR_THREADS);
     cfg.dynamicSmemBytes = FR_SMEM_BYTES;
