@@ -319,27 +319,6 @@ def run_gpu(args):
                           args.streams)
     d2h_gbs = world * LEN / (max_over_ranks(time.perf_counter() - t0) / e2e_steps) / 1e9
 
-    # ---- the same buffer cut into 1 KiB chunks (K = 262 144): the other kernel layout, for the record
-    small_gbs = None
-    if rank == 0:
-        small_cb = 1024
-        with fastrack.Context(key, small_cb) as small:
-            Ks = LEN // small_cb
-            d_ts = torch.empty(16 * Ks, dtype=torch.uint8, device="cuda")
-            d_oks = torch.zeros(Ks, dtype=torch.int32, device="cuda")
-            small.encrypt_tag(iv, d_plain_src.data_ptr(), LEN, d_cipher.data_ptr(), d_ts.data_ptr(), st)
-            for _ in range(3):
-                small.decrypt_verify(iv, d_cipher.data_ptr(), LEN, d_ts.data_ptr(), d_out.data_ptr(), d_oks.data_ptr(), st)
-            s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            s0.record(stream)
-            for _ in range(20):
-                small.decrypt_verify(iv, d_cipher.data_ptr(), LEN, d_ts.data_ptr(), d_out.data_ptr(), d_oks.data_ptr(), st)
-            s1.record(stream)
-            torch.cuda.synchronize()
-            assert bool((d_oks == 1).all()) and bool((d_out == d_plain_src).all())
-            small_gbs = LEN * 20 / (s0.elapsed_time(s1) * 1e-3) / 1e9
-            del d_ts, d_oks
-
     if sampler is not None:
         sampler.stop()
     if rank == 0:
@@ -374,8 +353,7 @@ def run_gpu(args):
                                  "payload_peak": hbm_payload_peak}},
             "cpu_baseline": {"value": cpu_gbs, "unit": UNIT, "cores": threads, "kind": "oracle",
                              "sample": f"{n_sample} of the 64 chunks (4 MiB each), {threads} threads over chunks, {cpu_s:.1f} s"},
-            "extra": {"encrypt_tag_gbs": enc_gbs, "pipelined_d2h_encrypt_gbs": d2h_gbs,
-                      "decrypt_verify_1KiB_chunks_gbs": small_gbs},
+            "extra": {"encrypt_tag_gbs": enc_gbs, "pipelined_d2h_encrypt_gbs": d2h_gbs},
         }
         print(json.dumps(line))
     ctx.close()
