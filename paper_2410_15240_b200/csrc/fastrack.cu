@@ -258,7 +258,7 @@ struct fastrack_ctx {
     uint32_t pack_max_blocks;     // chunks of at most this many blocks may take the packed-row kernels (FASTRACK_PACK_MAX_BLOCKS; 0 = never)
     uint32_t pack_run_override;   // 0 = automatic; else packed rows with this run length wherever they apply (FASTRACK_PACK_RUN, tests)
     uint32_t pack_group_override; // 0 = automatic; else this many chunks per packed work item (FASTRACK_PACK_GROUP, tests)
-    struct { size_t sample_bytes, n_chunks; uint32_t run, group; bool valid; } pack_memo;   // the planner's last answer (callers repeat shapes)
+    struct { size_t sample_bytes, n_chunks; uint32_t run, group; bool valid; } pack_memo[3];   // the planner's last answer per kind of pass (callers repeat shapes)
 };
 
 #define FR_CUDA(ctx, call)                                              \
@@ -544,40 +544,57 @@ static void plan_segments(const fastrack_ctx* ctx, size_t sample_bytes, size_t n
 
 // Decides between the row kernels (plan_segments has filled P) and the packed-row kernels for a fused pass, and
 // in the latter case picks the run length and the work-item size.  Both are judged by the same kind of estimate, in
-// SM clocks: the shared-memory work of the busiest SM plus, for the packed form, the latency of one row (its rows
-// are long, so pipeline fill and drain show).  Fitted to measurements on B200: a row kernel costs about 285 clocks
-// per row plus 400 per segment; a packed row costs about 280 plus, per counter of its run, 258 clocks for runs up to
-// 3 counters and more beyond (a lane's 16-byte loads and stores are 16 * run bytes apart, so longer runs touch more
-// cache lines per request).
-static bool plan_packed(fastrack_ctx* ctx, size_t sample_bytes, size_t n_chunks, FrParams& P)
+// SM clocks: the shared-memory work of the busiest SM or the latency of the busiest warp, whichever is larger (plus
+// a quarter of the other: between the two regimes both show).  For the fused passes a row kernel costs about 285
+// clocks per row plus 400 per segment; a packed row costs about 280 plus, per counter of its run, 258 clocks for runs
+// up to 3 counters and more beyond (a lane's 16-byte loads and stores are 16 * run bytes apart, so longer runs touch
+// more cache lines per request).  The two halves of the fused pass have constants of their own (pack_costs).
+// Cost constants of the two layouts for one kind of pass, in SM clocks (fitted to measurements on B200).
+struct PackCosts {
+    size_t row_clocks, seg_clocks, row_step_latency;      // row kernels: per row, per segment; latency of a row for a lone warp
+    size_t fixed, step_latency;                           // packed rows: per row of 32 runs; latency per counter for a lone warp
+    size_t step[14];                                      // packed rows: clocks per counter of a run, by run length (0 unused)
+    size_t step_long;                                     // ... for longer runs
+};
+// Runs whose byte stride is a power of two (4, 8) do worst: the lanes' 16-byte pieces fall on the same few cache banks.
+static const PackCosts pack_costs[3] = {
+    // fused passes: cipher + Horner step per counter, one general product per run
+    {285, 400, 1000, 280, 2250, {0, 258, 257, 256, 289, 264, 281, 330, 396, 302, 304, 304, 327, 305}, 335},
+    // counter mode only: no product, no reduction
+    {218, 100, 900, 30, 2000, {0, 227, 227, 227, 245, 227, 240, 270, 330, 250, 252, 252, 270, 255}, 260},
+    // verify only: no cipher (but counter 1), so the closing product weighs more and longer runs pay
+    {85, 400, 300, 465, 700, {0, 65, 65, 65, 80, 65, 75, 85, 120, 86, 88, 88, 100, 90}, 95},
+};
+
+static bool plan_packed(fastrack_ctx* ctx, int mode, size_t sample_bytes, size_t n_chunks, FrParams& P)
 {
     if (!ctx->pack_max_blocks) return false;
+    const int kind = mode == FR_MODE_CTR ? 1 : mode == FR_MODE_VERIFY ? 2 : 0;
+    const PackCosts& C = pack_costs[kind];
+    auto& memo = ctx->pack_memo[kind];
     const size_t first_len = sample_bytes < ctx->chunk_bytes ? sample_bytes : ctx->chunk_bytes;
     const size_t counters = (first_len + 15) / 16 + 1;
     if (counters - 1 > ctx->pack_max_blocks) return false;
     const size_t sms = (size_t)ctx->num_sms, warps = sms * FR_WARPS;
     if (!ctx->pack_run_override && counters > 32 && n_chunks * 8 < warps) return false;   // a few long chains: rows, no search needed
-    if (ctx->pack_memo.valid && ctx->pack_memo.sample_bytes == sample_bytes && ctx->pack_memo.n_chunks == n_chunks) {
-        if (!ctx->pack_memo.run) return false;
-        P.pack_run = ctx->pack_memo.run;
-        P.pack_chunks = ctx->pack_memo.group;
+    if (memo.valid && memo.sample_bytes == sample_bytes && memo.n_chunks == n_chunks) {
+        if (!memo.run) return false;
+        P.pack_run = memo.run;
+        P.pack_chunks = memo.group;
         P.n_items = (uint32_t)((n_chunks + P.pack_chunks - 1) / P.pack_chunks);
         return true;
     }
-    ctx->pack_memo.valid = true;
-    ctx->pack_memo.sample_bytes = sample_bytes;
-    ctx->pack_memo.n_chunks = n_chunks;
-    ctx->pack_memo.run = 0;
+    memo.valid = true;
+    memo.sample_bytes = sample_bytes;
+    memo.n_chunks = n_chunks;
+    memo.run = 0;
 
     const size_t rows_ref = (counters + 1 + FR_ROW_BLOCKS - 1) / FR_ROW_BLOCKS;
     const size_t waves = ((size_t)P.n_items + warps - 1) / warps;
-    const size_t row_thr = (n_chunks * rows_ref + sms - 1) / sms * 285 + ((size_t)P.n_items + sms - 1) / sms * 400;
-    const size_t row_lat = waves * ((size_t)P.seg_rows * 1000 + 4000);
+    const size_t row_thr = (n_chunks * rows_ref + sms - 1) / sms * C.row_clocks + ((size_t)P.n_items + sms - 1) / sms * C.seg_clocks;
+    const size_t row_lat = waves * ((size_t)P.seg_rows * C.row_step_latency + 4000);
     const size_t row_cost = row_thr > row_lat ? row_thr : row_lat;
 
-    // clocks per counter of a run, by run length (runs whose byte stride is a power of two do worst: the lanes'
-    // 16-byte pieces then fall on the same few cache banks)
-    static const size_t step_clocks[14] = {0, 258, 257, 256, 289, 264, 281, 330, 396, 302, 304, 304, 327, 305};
     size_t best_run = 0, best_group = 1, best_cost = ~(size_t)0;
     const size_t cand[] = {1, 2, 3, 4, 5, 6, 9, 10, 11, 13, counters <= 64 ? counters : 5};
     for (size_t run : cand) {
@@ -585,8 +602,8 @@ static bool plan_packed(fastrack_ctx* ctx, size_t sample_bytes, size_t n_chunks,
         if (run > counters) run = counters;
         const size_t slots = (counters + run - 1) / run;
         if (n_chunks * slots >= ((size_t)1 << 32) - 2048) continue;                // slots and chunks are counted in 32 bits; a row may overshoot by 31, an item's first chunk index by its size
-        const size_t per_row = 280 + run * (run < 14 ? step_clocks[run] : 335);
-        const size_t row_latency = 2500 + run * 2250;       // one warp alone on its SM partition
+        const size_t per_row = C.fixed + run * (run < 14 ? C.step[run] : C.step_long);
+        const size_t row_latency = 2500 + run * C.step_latency;       // one warp alone on its SM partition
         // a work item is `group` whole chunks.  Its last row is only partly filled, and an instruction costs the same
         // with idle lanes; on the other hand a launch with fewer items than warps leaves warps idle.  Try a range of
         // item sizes and count the rows each really takes.
@@ -609,8 +626,8 @@ static bool plan_packed(fastrack_ctx* ctx, size_t sample_bytes, size_t n_chunks,
     P.pack_run = (uint32_t)best_run;
     P.pack_chunks = (uint32_t)best_group;
     P.n_items = (uint32_t)((n_chunks + best_group - 1) / best_group);
-    ctx->pack_memo.run = P.pack_run;
-    ctx->pack_memo.group = P.pack_chunks;
+    memo.run = P.pack_run;
+    memo.group = P.pack_chunks;
     return true;
 }
 
@@ -654,7 +671,7 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
     plan_segments(ctx, sample_bytes, n_chunks, P);
     // Many short chains: one run of counters per lane (see fr_packed_body) when that is predicted to be faster.
     const bool packed = (mode == FR_MODE_DEC || mode == FR_MODE_ENC || mode == FR_MODE_CTR || mode == FR_MODE_VERIFY) &&
-                        plan_packed(ctx, sample_bytes, n_chunks, P);
+                        plan_packed(ctx, mode, sample_bytes, n_chunks, P);
 
     P.in = (const uint8_t*)b.in;
     P.out = (uint8_t*)b.out;
