@@ -33,6 +33,9 @@
  *   - K is derived from `len`; dropping trailing chunks is invisible to this layer, so `len` must
  *     come from a trusted source.
  *   - There is no CPU implementation behind these calls: without a usable CUDA device they fail.
+ *   - chunk_bytes may be anything from 16 bytes to 1 GiB.  Two kernel layouts serve that range -- a warp per run
+ *     of 32 consecutive blocks of a chunk, or, when a launch has many chunks that are not large, a lane per short
+ *     run of one chunk's blocks -- and the library picks per launch; results do not depend on the choice.
  */
 #ifndef FASTRACK_H
 #define FASTRACK_H
@@ -72,7 +75,7 @@ typedef struct fastrack_ctx fastrack_ctx;
  * authentication process"; Section 4.2: every chain uses the same H).
  * Copies the 32-byte AES-256 key (host pointer), expands it into the 15 round keys, derives H, and
  * builds on the current device the tables the kernels need, sized for `chunk_bytes`: the byte tables
- * of the fixed multiplier H^32 (and of H, for the sequential comparator) and the powers
+ * of the fixed multiplier H^32 (and of H, for launches with many small chunks and for the sequential comparator) and the powers
  * H^0 .. H^(chunk_bytes/16 + 65), 16 bytes each, i.e. a table as large as one chunk.  Allocates device
  * memory and synchronises the device once.  chunk_bytes: multiple of 16, 16 .. FASTRACK_MAX_CHUNK_BYTES.
  * On success *out is a new context; on failure *out is NULL. */
