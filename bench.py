@@ -333,6 +333,7 @@ def run_gpu(args):
         n_sample = max(1, min(64, threads))
         cpu_s = OracleSample(n_sample, CHUNK, threads).step()
         cpu_gbs = n_sample * CHUNK / cpu_s / 1e9
+        cpu_one_gbs = CHUNK / OracleSample(1, CHUNK, 1).step() / 1e9       # the same oracle on one thread, one chunk
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -352,7 +353,8 @@ def run_gpu(args):
                                  "unit": "GB/s", "peak_source": f"{pk['source']} copy bandwidth",
                                  "payload_peak": hbm_payload_peak}},
             "cpu_baseline": {"value": cpu_gbs, "unit": UNIT, "cores": threads, "kind": "oracle",
-                             "sample": f"{n_sample} of the 64 chunks (4 MiB each), {threads} threads over chunks, {cpu_s:.1f} s"},
+                             "sample": f"{n_sample} of the 64 chunks (4 MiB each), {threads} threads over chunks, {cpu_s:.1f} s",
+                             "one_thread_value": cpu_one_gbs},
             "extra": {"encrypt_tag_gbs": enc_gbs, "pipelined_d2h_encrypt_gbs": d2h_gbs},
         }
         print(json.dumps(line))
