@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfastrack.so")
 SOURCES = [os.path.join(CSRC, "fastrack.cu")]
-DEPS = SOURCES + [os.path.join(CSRC, "fastrack_device.cuh"), os.path.join(CSRC, "fastrack_keysetup.h"),
+DEPS = SOURCES + [os.path.join(CSRC, "fastrack_device.cuh"), os.path.join(CSRC, "fastrack_keysetup.h"), os.path.join(CSRC, "fastrack_plan.h"),
                   os.path.join(os.path.dirname(HERE), "include", "fastrack.h")]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -11,13 +11,9 @@
 #include "../../include/fastrack.h"
 #include "fastrack_device.cuh"
 #include "fastrack_keysetup.h"
+#include "fastrack_plan.h"
 
 using namespace fr_host;
-
-#define FR_THREADS 1024
-#define FR_MAX_STAGES 96      // most stages a pipelined call is cut into
-#define FR_WARPS (FR_THREADS / 32)
-#define FR_PACK_MAX_BLOCKS 4096   // chunks of more blocks than this never take the packed-row kernels
 
 // ------------------------------------------------------------------------------------ kernels ----
 
@@ -231,6 +227,7 @@ struct fastrack_ctx {
     int device;
     int num_sms;
     size_t chunk_bytes;
+    FrPlanConfig plan;            // what the host-side planners need (fastrack_plan.h); num_sms and chunk_bytes repeated
     uint32_t rk[60];
     uint8_t h[16];
     uint32_t* d_te0;
@@ -251,14 +248,9 @@ struct fastrack_ctx {
     int last_cuda_error;
     uint64_t launches;
     uint32_t aad_mod;             // 0 = no AAD, else chains per sample of the serial-number framing
-    uint32_t seg_rows_override;   // 0 = automatic (FASTRACK_SEG_ROWS, for experiments)
-    size_t stage_bytes_override;  // 0 = automatic (FASTRACK_STAGE_BYTES, for experiments)
     uint32_t generic_smem;        // FASTRACK_GENERIC_SMEM=1: exercise the portable addressing path (tests)
     uint32_t no_overlap_launch;   // FASTRACK_NO_OVERLAP_LAUNCH=1: plain stream-ordered launches (experiments)
-    uint32_t pack_max_blocks;     // chunks of at most this many blocks may take the packed-row kernels (FASTRACK_PACK_MAX_BLOCKS; 0 = never)
-    uint32_t pack_run_override;   // 0 = automatic; else packed rows with this run length wherever they apply (FASTRACK_PACK_RUN, tests)
-    uint32_t pack_group_override; // 0 = automatic; else this many chunks per packed work item (FASTRACK_PACK_GROUP, tests)
-    struct { size_t sample_bytes, n_chunks; uint32_t run, group; bool valid; } pack_memo[3];   // the planner's last answer per kind of pass (callers repeat shapes)
+    struct { size_t sample_bytes, n_chunks; FrPackPlan plan; bool valid; } pack_memo[3];   // fr_plan_packed's last answer per kind of pass (callers repeat shapes)
 };
 
 #define FR_CUDA(ctx, call)                                              \
@@ -284,7 +276,7 @@ static int ensure_scratch(fastrack_ctx* ctx, size_t chunks)
     // A chunk of at most 62 blocks is two rows, and no segment is shorter than two rows: such chunks are never split
     // between warps, so neither kernel family touches the scratch (40 bytes per chunk would exceed the data itself
     // at 16-byte chunks).  launch_pass checks this assumption.
-    if (!ctx->seg_rows_override && ctx->chunk_bytes <= 62 * 16) return FASTRACK_OK;
+    if (!ctx->plan.seg_rows_override && ctx->chunk_bytes <= 62 * 16) return FASTRACK_OK;
     size_t cap = ctx->scratch_chunks ? ctx->scratch_chunks : 1024;
     while (cap < chunks) cap *= 2;
     FR_CUDA(ctx, cudaDeviceSynchronize());       // nothing may still be using the old scratch
@@ -313,14 +305,16 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
     cudaError_t e = cudaGetDevice(&ctx->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, ctx->device);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return fail(FASTRACK_ERR_CUDA); }
-    if (const char* env = getenv("FASTRACK_SEG_ROWS")) ctx->seg_rows_override = (uint32_t)strtoul(env, nullptr, 10);
+    ctx->plan.num_sms = ctx->num_sms;
+    ctx->plan.chunk_bytes = chunk_bytes;
+    if (const char* env = getenv("FASTRACK_SEG_ROWS")) ctx->plan.seg_rows_override = (uint32_t)strtoul(env, nullptr, 10);
     if (const char* env = getenv("FASTRACK_GENERIC_SMEM")) ctx->generic_smem = (uint32_t)(strtoul(env, nullptr, 10) != 0);
     if (const char* env = getenv("FASTRACK_NO_OVERLAP_LAUNCH")) ctx->no_overlap_launch = (uint32_t)(strtoul(env, nullptr, 10) != 0);
-    if (const char* env = getenv("FASTRACK_STAGE_BYTES")) ctx->stage_bytes_override = (size_t)strtoull(env, nullptr, 10);
-    ctx->pack_max_blocks = FR_PACK_MAX_BLOCKS;
-    if (const char* env = getenv("FASTRACK_PACK_MAX_BLOCKS")) ctx->pack_max_blocks = (uint32_t)strtoul(env, nullptr, 10);
-    if (const char* env = getenv("FASTRACK_PACK_RUN")) ctx->pack_run_override = (uint32_t)strtoul(env, nullptr, 10);
-    if (const char* env = getenv("FASTRACK_PACK_GROUP")) ctx->pack_group_override = (uint32_t)strtoul(env, nullptr, 10);
+    if (const char* env = getenv("FASTRACK_STAGE_BYTES")) ctx->plan.stage_bytes_override = (size_t)strtoull(env, nullptr, 10);
+    ctx->plan.pack_max_blocks = FR_PACK_MAX_BLOCKS;
+    if (const char* env = getenv("FASTRACK_PACK_MAX_BLOCKS")) ctx->plan.pack_max_blocks = (uint32_t)strtoul(env, nullptr, 10);
+    if (const char* env = getenv("FASTRACK_PACK_RUN")) ctx->plan.pack_run_override = (uint32_t)strtoul(env, nullptr, 10);
+    if (const char* env = getenv("FASTRACK_PACK_GROUP")) ctx->plan.pack_group_override = (uint32_t)strtoul(env, nullptr, 10);
 
     // key material on the host: S-box, Te0, round keys, H, byte tables of H^32
     uint8_t sbox[256];
@@ -491,49 +485,14 @@ static uint4 length_term(const fastrack_ctx* ctx, uint64_t bytes)
     return r;
 }
 
-// Segment geometry of a launch over n_chunks chunks of samples of `sample_bytes` bytes (a plain buffer is one
-// sample): rows are aligned to the counter (block j sits at counter
-// j + 2), segments are whole multiples of 8 rows so that they start on a 256-counter group.
+// Fills the geometry of a launch into P: the row kernels' segment plan (fastrack_plan.h) and the per-sample layout.
 static void plan_segments(const fastrack_ctx* ctx, size_t sample_bytes, size_t n_chunks, FrParams& P)
 {
+    const FrSegPlan seg = fr_plan_segments(ctx->plan, sample_bytes, n_chunks);
+    P.seg_rows = seg.seg_rows;
+    P.segs_per_chunk = seg.segs_per_chunk;
+    P.n_items = seg.n_items;
     const size_t first_len = sample_bytes < ctx->chunk_bytes ? sample_bytes : ctx->chunk_bytes;
-    const size_t rows_ref = ((first_len + 15) / 16 + 2 + FR_ROW_BLOCKS - 1) / FR_ROW_BLOCKS;
-    const size_t warps = (size_t)ctx->num_sms * FR_WARPS;
-    // Segments are dealt round-robin to the resident warps.  Two things bound a launch: the latency of the
-    // busiest warp (about 1000 cycles per row when few warps run, plus about 4000 per segment for the closing
-    // GF(2^128) product, the atomics and the tag), and the shared-memory work of the busiest SM (about 270
-    // wavefront-cycles per row plus about 300 per segment).  Try short segments (2 or 4 rows, for small buffers)
-    // and 1..8 segments per warp in whole 8-row groups, and keep the split with the smaller bound.
-    size_t seg_rows = 8, spc = (rows_ref + 7) / 8;
-    if (ctx->seg_rows_override) {
-        seg_rows = ctx->seg_rows_override;
-        spc = (rows_ref + seg_rows - 1) / seg_rows;
-    } else {
-        size_t best_cost = ~(size_t)0;
-        for (int cand = 0; cand < 10; cand++) {
-            size_t rows;
-            if (cand < 2) {
-                rows = cand == 0 ? 2 : 4;
-            } else {
-                size_t want = (size_t)(cand - 1) * warps / n_chunks;
-                if (want < 1) want = 1;
-                rows = ((rows_ref + want - 1) / want + 7) / 8 * 8;
-                if (rows > 1024) rows = 1024;
-            }
-            const size_t per_chunk = (rows_ref + rows - 1) / rows;
-            const size_t items = per_chunk * n_chunks;
-            const size_t waves = (items + warps - 1) / warps;
-            const size_t per_sm = (items + (size_t)ctx->num_sms - 1) / (size_t)ctx->num_sms;
-            const size_t latency = waves * (rows * 1000 + 4000);
-            const size_t throughput = per_sm * (rows * 270 + 300);
-            const size_t cost = latency > throughput ? latency : throughput;
-            if (cost < best_cost) { best_cost = cost; seg_rows = rows; spc = per_chunk; }
-        }
-    }
-    while (spc * n_chunks >= ((size_t)1 << 31)) { seg_rows *= 2; spc = (rows_ref + seg_rows - 1) / seg_rows; }
-    P.seg_rows = (uint32_t)seg_rows;
-    P.segs_per_chunk = (uint32_t)spc;
-    P.n_items = (uint32_t)(spc * n_chunks);
     const size_t cps = (sample_bytes + ctx->chunk_bytes - 1) / ctx->chunk_bytes;
     const size_t last_len = sample_bytes - (cps - 1) * ctx->chunk_bytes;     // a sample's last chunk may be short
     P.sample_bytes = sample_bytes;
@@ -542,92 +501,23 @@ static void plan_segments(const fastrack_ctx* ctx, size_t sample_bytes, size_t n
     P.lenh_last = length_term(ctx, last_len);
 }
 
-// Decides between the row kernels (plan_segments has filled P) and the packed-row kernels for a fused pass, and
-// in the latter case picks the run length and the work-item size.  Both are judged by the same kind of estimate, in
-// SM clocks: the shared-memory work of the busiest SM or the latency of the busiest warp, whichever is larger (plus
-// a quarter of the other: between the two regimes both show).  For the fused passes a row kernel costs about 285
-// clocks per row plus 400 per segment; a packed row costs about 280 plus, per counter of its run, 258 clocks for runs
-// up to 3 counters and more beyond (a lane's 16-byte loads and stores are 16 * run bytes apart, so longer runs touch
-// more cache lines per request).  The two halves of the fused pass have constants of their own (pack_costs).
-// Cost constants of the two layouts for one kind of pass, in SM clocks (fitted to measurements on B200).
-struct PackCosts {
-    size_t row_clocks, seg_clocks, row_step_latency;      // row kernels: per row, per segment; latency of a row for a lone warp
-    size_t fixed, step_latency;                           // packed rows: per row of 32 runs; latency per counter for a lone warp
-    size_t step[14];                                      // packed rows: clocks per counter of a run, by run length (0 unused)
-    size_t step_long;                                     // ... for longer runs
-};
-// Runs whose byte stride is a power of two (4, 8) do worst: the lanes' 16-byte pieces fall on the same few cache banks.
-static const PackCosts pack_costs[3] = {
-    // fused passes: cipher + Horner step per counter, one general product per run
-    {285, 400, 1000, 280, 2250, {0, 258, 257, 256, 289, 264, 281, 330, 396, 302, 304, 304, 327, 305}, 335},
-    // counter mode only: no product, no reduction
-    {218, 100, 900, 30, 2000, {0, 227, 227, 227, 245, 227, 240, 270, 330, 250, 252, 252, 270, 255}, 260},
-    // verify only: no cipher (but counter 1), so the closing product weighs more and longer runs pay
-    {85, 400, 300, 465, 700, {0, 65, 65, 65, 80, 65, 75, 85, 120, 86, 88, 88, 100, 90}, 95},
-};
-
+// Row kernels (false; plan_segments has filled P) or packed-row kernels (true; P is switched over to them)?
+// fr_plan_packed decides; its last answer per kind of pass is kept, since callers repeat shapes.
 static bool plan_packed(fastrack_ctx* ctx, int mode, size_t sample_bytes, size_t n_chunks, FrParams& P)
 {
-    if (!ctx->pack_max_blocks) return false;
-    const int kind = mode == FR_MODE_CTR ? 1 : mode == FR_MODE_VERIFY ? 2 : 0;
-    const PackCosts& C = pack_costs[kind];
+    const int kind = mode == FR_MODE_CTR ? FR_PASS_CTR : mode == FR_MODE_VERIFY ? FR_PASS_VERIFY : FR_PASS_FUSED;
     auto& memo = ctx->pack_memo[kind];
-    const size_t first_len = sample_bytes < ctx->chunk_bytes ? sample_bytes : ctx->chunk_bytes;
-    const size_t counters = (first_len + 15) / 16 + 1;
-    if (counters - 1 > ctx->pack_max_blocks) return false;
-    const size_t sms = (size_t)ctx->num_sms, warps = sms * FR_WARPS;
-    if (!ctx->pack_run_override && counters > 32 && n_chunks * 8 < warps) return false;   // a few long chains: rows, no search needed
-    if (memo.valid && memo.sample_bytes == sample_bytes && memo.n_chunks == n_chunks) {
-        if (!memo.run) return false;
-        P.pack_run = memo.run;
-        P.pack_chunks = memo.group;
-        P.n_items = (uint32_t)((n_chunks + P.pack_chunks - 1) / P.pack_chunks);
-        return true;
+    if (!(memo.valid && memo.sample_bytes == sample_bytes && memo.n_chunks == n_chunks)) {
+        const FrSegPlan seg = {P.seg_rows, P.segs_per_chunk, P.n_items};
+        memo.plan = fr_plan_packed(ctx->plan, kind, sample_bytes, n_chunks, seg);
+        memo.sample_bytes = sample_bytes;
+        memo.n_chunks = n_chunks;
+        memo.valid = true;
     }
-    memo.valid = true;
-    memo.sample_bytes = sample_bytes;
-    memo.n_chunks = n_chunks;
-    memo.run = 0;
-
-    const size_t rows_ref = (counters + 1 + FR_ROW_BLOCKS - 1) / FR_ROW_BLOCKS;
-    const size_t waves = ((size_t)P.n_items + warps - 1) / warps;
-    const size_t row_thr = (n_chunks * rows_ref + sms - 1) / sms * C.row_clocks + ((size_t)P.n_items + sms - 1) / sms * C.seg_clocks;
-    const size_t row_lat = waves * ((size_t)P.seg_rows * C.row_step_latency + 4000);
-    const size_t row_cost = row_thr > row_lat ? row_thr : row_lat;
-
-    size_t best_run = 0, best_group = 1, best_cost = ~(size_t)0;
-    const size_t cand[] = {1, 2, 3, 4, 5, 6, 9, 10, 11, 13, counters <= 64 ? counters : 5};
-    for (size_t run : cand) {
-        if (ctx->pack_run_override) run = ctx->pack_run_override;
-        if (run > counters) run = counters;
-        const size_t slots = (counters + run - 1) / run;
-        if (n_chunks * slots >= ((size_t)1 << 32) - 2048) continue;                // slots and chunks are counted in 32 bits; a row may overshoot by 31, an item's first chunk index by its size
-        const size_t per_row = C.fixed + run * (run < 14 ? C.step[run] : C.step_long);
-        const size_t row_latency = 2500 + run * C.step_latency;       // one warp alone on its SM partition
-        // a work item is `group` whole chunks.  Its last row is only partly filled, and an instruction costs the same
-        // with idle lanes; on the other hand a launch with fewer items than warps leaves warps idle.  Try a range of
-        // item sizes and count the rows each really takes.
-        const size_t sizes[] = {1, 2, 3, 4, 5, 6, 8, 10, 12, 16, 24, 32, 48, 64, 96, 128, 256, 512,
-                                32 / slots, 64 / slots, 128 / slots, 256 / slots, 512 / slots};
-        for (size_t group : sizes) {
-            if (ctx->pack_group_override) group = ctx->pack_group_override;
-            if (group < 1 || group * slots > 1024) continue;
-            if (group > n_chunks) group = n_chunks;
-            const size_t rows_per_item = (group * slots + 31) / 32;
-            const size_t items = (n_chunks + group - 1) / group;
-            const size_t thr = (items * rows_per_item + sms - 1) / sms * per_row;
-            const size_t lat = (items + warps - 1) / warps * rows_per_item * row_latency;
-            const size_t cost = thr > lat ? thr + lat / 4 : lat + thr / 4;      // between the two regimes both show
-            if (cost < best_cost) { best_cost = cost; best_run = run; best_group = group; }
-        }
-    }
-    if (!best_run) return false;
-    if (!ctx->pack_run_override && best_cost >= row_cost) return false;
-    P.pack_run = (uint32_t)best_run;
-    P.pack_chunks = (uint32_t)best_group;
-    P.n_items = (uint32_t)((n_chunks + best_group - 1) / best_group);
-    memo.run = P.pack_run;
-    memo.group = P.pack_chunks;
+    if (!memo.plan.run) return false;
+    P.pack_run = memo.plan.run;
+    P.pack_chunks = memo.plan.group;
+    P.n_items = memo.plan.n_items;
     return true;
 }
 
@@ -775,25 +665,7 @@ extern "C" int fastrack_encrypt_tag(fastrack_ctx* ctx, const uint8_t iv_base[12]
 // finishes under the next stage's copy, which is a quarter as large.  Returns the stage sizes in descending order (host->device order).
 static size_t plan_stages(const fastrack_ctx* ctx, size_t len, size_t unit, size_t out[FR_MAX_STAGES])
 {
-    const size_t cb = unit;        // stages are whole multiples of this (a chunk, or a sample in a batch of samples)
-    const size_t floor_bytes = (size_t)2 << 20;
-    const size_t min_stage = cb >= floor_bytes ? cb : (floor_bytes + cb - 1) / cb * cb;
-    size_t off = 0, count = 0;
-    while (off < len) {
-        const size_t remaining = len - off;
-        size_t n;
-        if (ctx->stage_bytes_override) {
-            n = (ctx->stage_bytes_override + cb - 1) / cb * cb;
-        } else {
-            n = (remaining / 4 * 3) / cb * cb;
-            if (n < min_stage) n = min_stage;
-            if (remaining < n + min_stage / 2) n = remaining;      // do not leave a sliver behind
-        }
-        if (n > remaining || count == FR_MAX_STAGES - 1) n = remaining;
-        out[count++] = n;
-        off += n;
-    }
-    return count;
+    return fr_plan_stages(ctx->plan, len, unit, out);
 }
 
 // Common body of the two pipelined entry points.  d_pad == nullptr: fused decrypt+verify per stage.

@@ -1,0 +1,36 @@
+// plan_check.cpp -- TEST INFRASTRUCTURE: the library's host-side planners (paper_2410_15240_b200/csrc/fastrack_plan.h,
+// plain C++) behind a C interface, so that the CPU-only tests can check their invariants over many shapes.
+#include "../../paper_2410_15240_b200/csrc/fastrack_plan.h"
+
+extern "C" {
+
+static FrPlanConfig make(int num_sms, size_t chunk_bytes, uint32_t seg_rows, uint32_t pack_max, uint32_t run, uint32_t group,
+                         size_t stage_bytes)
+{
+    FrPlanConfig c;
+    c.num_sms = num_sms; c.chunk_bytes = chunk_bytes; c.seg_rows_override = seg_rows; c.pack_max_blocks = pack_max;
+    c.pack_run_override = run; c.pack_group_override = group; c.stage_bytes_override = stage_bytes;
+    return c;
+}
+
+// out[0..2] = seg_rows, segs_per_chunk, n_items of the row kernels; out[3..5] = run, group, n_items of the packed rows
+void plan_launch(int num_sms, size_t chunk_bytes, uint32_t seg_rows, uint32_t pack_max, uint32_t run, uint32_t group, int kind,
+                 size_t sample_bytes, size_t n_chunks, uint32_t out[6])
+{
+    const FrPlanConfig c = make(num_sms, chunk_bytes, seg_rows, pack_max, run, group, 0);
+    const FrSegPlan s = fr_plan_segments(c, sample_bytes, n_chunks);
+    const FrPackPlan p = fr_plan_packed(c, kind, sample_bytes, n_chunks, s);
+    out[0] = s.seg_rows; out[1] = s.segs_per_chunk; out[2] = s.n_items;
+    out[3] = p.run; out[4] = p.group; out[5] = p.n_items;
+}
+
+size_t plan_stages(size_t chunk_bytes, size_t stage_bytes, size_t len, size_t unit, size_t* out)
+{
+    const FrPlanConfig c = make(148, chunk_bytes, 0, FR_PACK_MAX_BLOCKS, 0, 0, stage_bytes);
+    return fr_plan_stages(c, len, unit, out);
+}
+
+int plan_max_stages(void) { return FR_MAX_STAGES; }
+int plan_max_item_slots(void) { return FR_PACK_MAX_ITEM_SLOTS; }
+
+}

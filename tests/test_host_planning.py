@@ -1,0 +1,128 @@
+"""Host-side planning logic of the library (segments, packed rows, pipeline stages), compiled as plain C++ and checked
+on the CPU for the invariants the kernels and the pipelined calls rely on.  No GPU, no oracle: pure host arithmetic."""
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+WARPS = 148 * 32
+
+
+@pytest.fixture(scope="module")
+def plan(tmp_path_factory):
+    so = tmp_path_factory.mktemp("host_logic") / "libplan.so"
+    subprocess.check_call(["g++", "-O1", "-std=c++17", "-Wall", "-Wextra", "-Werror", "-shared", "-fPIC", "-o", str(so),
+                           os.path.join(ROOT, "tests", "host_logic", "plan_check.cpp")])
+    lib = ctypes.CDLL(str(so))
+    Z, U = ctypes.c_size_t, ctypes.c_uint32
+    lib.plan_launch.argtypes = [ctypes.c_int, Z, U, U, U, U, ctypes.c_int, Z, Z, ctypes.c_void_p]
+    lib.plan_stages.argtypes = [Z, Z, Z, Z, ctypes.c_void_p]
+    lib.plan_stages.restype = Z
+    return lib
+
+
+def launch(lib, cb, sample_bytes, n_chunks, kind=0, seg_rows=0, pack_max=4096, run=0, group=0, sms=148):
+    out = np.zeros(6, np.uint32)
+    lib.plan_launch(sms, cb, seg_rows, pack_max, run, group, kind, sample_bytes, n_chunks, out.ctypes.data)
+    return [int(x) for x in out]
+
+
+CHUNKS = [16, 32, 48, 64, 112, 256, 496, 512, 528, 992, 1008, 1024, 4096, 16384, 65536, 1 << 20, 4 << 20, 1 << 30]
+COUNTS = [1, 2, 3, 17, 100, 591, 592, 593, 4735, 4736, 4737, 65536, 1 << 20, (1 << 24) + 1, (1 << 28) + 7]
+
+
+@pytest.mark.parametrize("kind", [0, 1, 2])
+def test_launch_plans_are_consistent(plan, kind):
+    for cb in CHUNKS:
+        blocks = cb // 16
+        rows = (blocks + 2 + 31) // 32
+        for n_chunks in COUNTS:
+            if cb * n_chunks > 1 << 42:
+                continue
+            seg_rows, spc, n_items, run, group, p_items = launch(plan, cb, cb * n_chunks, n_chunks, kind)
+            # row kernels: segments tile the chunk, items fit 31 bits
+            assert seg_rows >= 2 and (seg_rows <= 4 or seg_rows % 8 == 0), (cb, n_chunks, seg_rows)
+            assert spc == -(-rows // seg_rows) and n_items == spc * n_chunks and n_items < 1 << 31
+            if blocks <= 62:
+                assert spc == 1, "chunks of two rows are never split between warps (they then need no scratch)"
+            # packed rows: whole chunks per item, bounded item size, everything within 32 bits
+            if run:
+                counters = blocks + 1
+                assert 1 <= run <= counters and blocks <= 4096
+                slots = -(-counters // run)
+                assert 1 <= group <= n_chunks and group * slots <= 1024
+                assert p_items == -(-n_chunks // group)
+                assert n_chunks * slots < (1 << 32) - 2048
+            else:
+                assert group == 0 and p_items == 0
+            # a few long chains stay with the row kernels
+            if blocks > 31 and n_chunks * 8 < WARPS:
+                assert run == 0
+
+
+def test_packed_rows_can_be_switched_off_and_forced(plan):
+    for cb in (16, 256, 1024, 4096):
+        for n_chunks in (1, 1000, 1 << 20):
+            assert launch(plan, cb, cb * n_chunks, n_chunks, pack_max=0)[3:] == [0, 0, 0]
+            for run in (1, 2, 5, 300):
+                got = launch(plan, cb, cb * n_chunks, n_chunks, run=run)
+                assert got[3] == min(run, cb // 16 + 1) or got[3] == 0          # 0: no admissible item size
+                forced = launch(plan, cb, cb * n_chunks, n_chunks, run=run, group=7)
+                if forced[3]:
+                    assert forced[4] == min(7, n_chunks)
+    assert launch(plan, 65552, 65552 * 100000, 100000)[3] == 0                 # 4097 blocks: above the packed limit
+    assert launch(plan, 65536, 65536 * 100000, 100000, run=5)[3] == 5          # 4096 blocks: still admissible
+
+
+def test_small_chunks_in_large_numbers_take_the_packed_rows(plan):
+    """The planner's raison d'etre: where the row layout would idle most lanes, the packed one is chosen."""
+    for cb in (16, 32, 64, 256, 1024):
+        for n_chunks in (1 << 16, 1 << 20, 1 << 24):
+            run = launch(plan, cb, cb * n_chunks, n_chunks)[3]
+            assert run >= 1, (cb, n_chunks)
+    for cb in (65536, 1 << 20, 4 << 20):                                        # the benchmark's sizes stay with the rows
+        for n_chunks in (1, 64, 4096):
+            assert launch(plan, cb, cb * n_chunks, n_chunks)[3] == 0
+
+
+def test_sample_batches_plan_on_the_sample_geometry(plan):
+    # samples shorter than a chunk: the chunk that exists is the sample
+    seg = launch(plan, 4096, 400, 262144)
+    assert seg[1] == 1 and seg[3] >= 1
+    # samples of several chunks
+    seg = launch(plan, 1024, 3 * 1024 + 16, 4 * 50000)
+    assert seg[0] >= 2 and seg[2] == seg[1] * 4 * 50000
+
+
+def stages(lib, cb, length, unit=None, stage_bytes=0):
+    out = np.zeros(96, np.uint64)
+    n = lib.plan_stages(cb, stage_bytes, length, unit or cb, out.ctypes.data)
+    return [int(x) for x in out[:n]]
+
+
+def test_pipeline_stages_cover_the_buffer_in_whole_units(plan):
+    rng = np.random.default_rng(3)
+    cases = [(65536, 1), (65536, 65536), (65536, 77_070_336), (4 << 20, 256 << 20), (4 << 20, 670_000_000), (1 << 30, 5 << 30),
+             (16, 4 << 20), (1 << 20, (1 << 20) * 1000 + 5)]
+    cases += [(int(16 * rng.integers(1, 1 << 16)), int(rng.integers(1, 1 << 32))) for _ in range(300)]
+    for cb, length in cases:
+        whole = -(-length // cb) * cb                       # the pipelined calls plan on whole units and clip the last stage
+        st = stages(plan, cb, whole)
+        assert 1 <= len(st) <= 96 and sum(st) == whole, (cb, length)
+        assert all(s % cb == 0 and s > 0 for s in st)
+        if len(st) < 96:
+            assert all(a >= b for a, b in zip(st, st[1:-1])), "stages shrink (the last may absorb a sliver)"
+            if len(st) > 1:
+                assert min(st) >= min(2 << 20, whole) // 2 or cb >= (2 << 20)
+
+
+def test_pipeline_stage_override_and_sample_units(plan):
+    st = stages(plan, 4096, 1 << 24, stage_bytes=300000)
+    assert all(s == -(-300000 // 4096) * 4096 for s in st[:-1]) and sum(st) == 1 << 24
+    st = stages(plan, 256, 301056 * 64, unit=301056)        # a batch of 64 samples: stages of whole samples
+    assert sum(st) == 301056 * 64 and all(s % 301056 == 0 for s in st)
+    st = stages(plan, 65536, 1 << 40, stage_bytes=65536)    # more pieces than stages: the last stage takes the rest
+    assert len(st) == 96 and sum(st) == 1 << 40
