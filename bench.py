@@ -235,6 +235,19 @@ def run_gpu(args):
     def step():
         ctx.decrypt_verify(iv, d_cipher.data_ptr(), LEN, d_tags.data_ptr(), d_out.data_ptr(), d_ok.data_ptr(), st)
 
+    if args.kernel_only and args.kernel_pass != "decrypt_verify":       # profiling aid: another pass over the same buffers
+        if args.kernel_pass == "encrypt_tag":
+            d_tags2 = torch.empty_like(d_tags)
+
+            def step():
+                ctx.encrypt_tag(iv, d_plain_src.data_ptr(), LEN, d_out.data_ptr(), d_tags2.data_ptr(), st)
+        elif args.kernel_pass == "ctr_crypt":
+            def step():
+                ctx.ctr_crypt(iv, d_cipher.data_ptr(), LEN, d_out.data_ptr(), st)
+        else:
+            def step():
+                ctx.verify(iv, d_cipher.data_ptr(), LEN, d_tags.data_ptr(), d_ok.data_ptr(), st)
+
     def e2e_step():
         ctx.pipelined_h2d(iv, h_cipher.data_ptr(), LEN, h_tags.data_ptr(), d_out.data_ptr(), d_ok.data_ptr(), args.streams)
         h_ok.copy_(d_ok, non_blocking=True)
@@ -260,8 +273,12 @@ def run_gpu(args):
     ms_this_rank = e0.elapsed_time(e1)
     ms_total = max_over_ranks(ms_this_rank)
     ms_per_step = ms_total / args.steps
-    assert bool((d_ok == 1).all()), "verification failed inside the benchmark"
-    assert bool((d_out == d_plain_src).all()), "decryption mismatch inside the benchmark"
+    if not (args.kernel_only and args.kernel_pass in ("encrypt_tag", "ctr_crypt")):
+        assert bool((d_ok == 1).all()), "verification failed inside the benchmark"
+    if not (args.kernel_only and args.kernel_pass in ("encrypt_tag", "verify")):
+        assert bool((d_out == d_plain_src).all()), "decryption mismatch inside the benchmark"
+    if args.kernel_only and args.kernel_pass == "encrypt_tag":
+        assert bool((d_out == d_cipher).all()) and bool((d_tags2 == d_tags).all()), "encryption mismatch inside the benchmark"
     value = ranks.aggregate_throughput(LEN * args.steps, ms_this_rank * 1e-3) / 1e9
 
     if args.kernel_only:
@@ -270,7 +287,7 @@ def run_gpu(args):
         if rank == 0:
             print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                               "warmup": args.warmup, "ms_per_step": ms_per_step, "gpu_launches": gpu_launches,
-                              "config": {"workload": WORKLOAD}, "kernel_only": True}))
+                              "config": {"workload": WORKLOAD, "pass": args.kernel_pass}, "kernel_only": True}))
         ctx.close()
         ranks.close()
         return
@@ -605,6 +622,9 @@ def main():
                     help="print throughput over the benchmark configurations instead of the one bench line")
     ap.add_argument("--trace", action="store_true", help="print stage-level timelines of the pipelined H2D call")
     ap.add_argument("--peaks", action="store_true", help="measure the unit rates the kernel roofline is derived from")
+    ap.add_argument("--pass", dest="kernel_pass", default="decrypt_verify",
+                    choices=["decrypt_verify", "encrypt_tag", "ctr_crypt", "verify"],
+                    help="with --kernel-only: which device-resident pass to time (profiling aid)")
     ap.add_argument("--shape", default=None, metavar="LEN_BYTES,CHUNK_BYTES",
                     help="with --kernel-only: time another buffer / chunk size than the headline one (profiling aid)")
     args = ap.parse_args()
