@@ -639,7 +639,10 @@ __device__ __forceinline__ uint4 fr_packed_slot_lane(const FrParams& P, const ch
         }
         if (DO_GHASH) {
             y = fr_xor4(y, gblk);
-            if (c + 1u != c1) y = fr_ghash_tabmul<ABS>(sm, L, y);                            // Horner step with the fixed multiplier H
+            // Horner step with the fixed multiplier H -- not after the run's last block (the closing product follows),
+            // and not at counter 1 without AAD, where y is still zero (when every lane of a warp starts its run
+            // there -- one lane per small chunk -- the whole step is skipped)
+            if (c + 1u != c1 && (c != 1u || P.aad_mod)) y = fr_ghash_tabmul<ABS>(sm, L, y);
         }
     }
     if (!DO_GHASH) return make_uint4(0, 0, 0, 0);
