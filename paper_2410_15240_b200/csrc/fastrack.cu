@@ -108,7 +108,7 @@ __global__ void __launch_bounds__(FR_THREADS, 1) fr_crypt_kernel(const __grid_co
 // the lane d below it only if that lane belongs to the same chunk), a chunk that continues into the next row hands
 // its running sum to that row's lane 0, and the lane holding a chunk's last slot finishes the tag.  No chunk is
 // shared between warps.  The shared-memory GHASH tables hold H here, not H^32.
-template <int MODE, bool ABS>
+template <int MODE, bool ABS, bool WHOLE>
 __device__ __forceinline__ void fr_packed_body(const FrParams& P, const char* sm, FrLane L)
 {
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
@@ -125,8 +125,9 @@ __device__ __forceinline__ void fr_packed_body(const FrParams& P, const char* sm
             const bool valid = slot < slot_end;               // only the item's last row has idle lanes, at its top
             FrSlot si = {0u, lane, 0xFFFFFFFFu};
             uint4 z = make_uint4(0, 0, 0, 0);
-            if (valid) z = fr_packed_slot_lane<MODE, ABS>(P, sm, L, g, slot, si);
+            if (valid) z = fr_packed_slot_lane<MODE, ABS, WHOLE>(P, sm, L, g, slot, si);
             if (MODE == FR_MODE_CTR) continue;                   // nothing to authenticate
+            if (!WHOLE) {                                        // (one lane per chunk: z is the chunk's sum already)
             if (lane == 0u && si.i != 0u) z = fr_xor4(z, carry);
             const uint32_t first = lane >= si.i ? lane - si.i : 0u;      // lowest lane of this row in the same chunk
 #pragma unroll
@@ -137,6 +138,7 @@ __device__ __forceinline__ void fr_packed_body(const FrParams& P, const char* sm
             }
             carry.x = __shfl_sync(0xFFFFFFFFu, z.x, 31); carry.y = __shfl_sync(0xFFFFFFFFu, z.y, 31);
             carry.z = __shfl_sync(0xFFFFFFFFu, z.z, 31); carry.w = __shfl_sync(0xFFFFFFFFu, z.w, 31);
+            }
             if (valid && si.i == si.last) {
                 const uint4 lenh = ((si.kk + 1u) % P.chunks_per_sample == 0u) ? P.lenh_last : P.lenh_full;
                 const uint4 tag = fr_xor4(z, lenh);
@@ -152,7 +154,7 @@ __device__ __forceinline__ void fr_packed_body(const FrParams& P, const char* sm
     }
 }
 
-template <int MODE>
+template <int MODE, bool WHOLE>
 __global__ void __launch_bounds__(FR_THREADS, 1) fr_packed_kernel(const __grid_constant__ FrParams P)
 {
     extern __shared__ __align__(256) char sm[];
@@ -164,8 +166,8 @@ __global__ void __launch_bounds__(FR_THREADS, 1) fr_packed_kernel(const __grid_c
     asm volatile("mov.u32 %0, 0;" : "=r"(after_barrier)::"memory");
     FrLane L = fr_make_lane(threadIdx.x & 31u);
     L.lane4 |= after_barrier;
-    if ((uint32_t)__cvta_generic_to_shared(sm) == FR_SMEM_ABS_BASE && !P.generic_smem) fr_packed_body<MODE, true>(P, sm, L);
-    else fr_packed_body<MODE, false>(P, sm, L);
+    if ((uint32_t)__cvta_generic_to_shared(sm) == FR_SMEM_ABS_BASE && !P.generic_smem) fr_packed_body<MODE, true, WHOLE>(P, sm, L);
+    else fr_packed_body<MODE, false, WHOLE>(P, sm, L);
 }
 
 // pow[i] = pow[i - half] * pow[half] for i in (half, min(2*half, n - 1)]: one doubling pass of the table
@@ -376,10 +378,14 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
         if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_PADGEN>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
         if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_PADDEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
         if ((e = cudaFuncSetAttribute(fr_verify_sequential_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
-        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_DEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
-        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_ENC>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
-        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_CTR>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
-        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_VERIFY>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_DEC, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_DEC, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_ENC, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_ENC, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_CTR, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_CTR, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_VERIFY, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_VERIFY, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
         for (int i = 0; i < 8 && e == cudaSuccess; i++) e = cudaStreamCreateWithFlags(&ctx->streams[i], cudaStreamNonBlocking);
         if (e != cudaSuccess) break;
         if ((e = cudaEventCreateWithFlags(&ctx->tags_ready, cudaEventDisableTiming)) != cudaSuccess) break;
@@ -572,6 +578,12 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
     P.ok = b.ok;
     P.te0 = ctx->d_te0;
     P.gh_tab = packed ? ctx->d_gh1_tab : ctx->d_gh_tab;
+    // One lane per chunk (run >= blocks + 1) has a kernel variant of its own that closes with two table steps and needs
+    // no reduction across lanes.  It wins while the integer pipes are the busier ones (up to 3 blocks per chunk) or the
+    // launch is short enough for the reduction's latency to show; beyond that the general product is the better closing.
+    const size_t full_blocks = ((sample_bytes < ctx->chunk_bytes ? sample_bytes : ctx->chunk_bytes) + 15) / 16;
+    const bool whole = packed && P.pack_run > full_blocks &&
+                       (full_blocks <= 3 || n_chunks <= 2 * (size_t)ctx->num_sms * FR_THREADS);
     P.pow = ctx->d_pow;
     if (!packed && mode != FR_MODE_CTR && mode != FR_MODE_PADGEN && P.segs_per_chunk > 1 &&
         first_chunk + n_chunks > ctx->scratch_chunks) return FASTRACK_ERR_NOMEM;                // cannot happen, see ensure_scratch
@@ -596,13 +608,17 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
     }
     cudaError_t le;
     switch (mode) {
-        case FR_MODE_DEC:    le = packed ? cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_DEC>, P)
+        case FR_MODE_DEC:    le = packed ? (whole ? cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_DEC, true>, P)
+                                                  : cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_DEC, false>, P))
                                          : cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_DEC>, P); break;
-        case FR_MODE_ENC:    le = packed ? cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_ENC>, P)
+        case FR_MODE_ENC:    le = packed ? (whole ? cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_ENC, true>, P)
+                                                  : cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_ENC, false>, P))
                                          : cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_ENC>, P); break;
-        case FR_MODE_CTR:    le = packed ? cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_CTR>, P)
+        case FR_MODE_CTR:    le = packed ? (whole ? cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_CTR, true>, P)
+                                                  : cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_CTR, false>, P))
                                          : cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_CTR>, P); break;
-        case FR_MODE_VERIFY: le = packed ? cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_VERIFY>, P)
+        case FR_MODE_VERIFY: le = packed ? (whole ? cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_VERIFY, true>, P)
+                                                  : cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_VERIFY, false>, P))
                                          : cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_VERIFY>, P); break;
         case FR_MODE_PADGEN: le = cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_PADGEN>, P); break;
         case FR_MODE_PADDEC: le = cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_PADDEC>, P); break;

@@ -592,7 +592,11 @@ struct FrSlot {
 // One slot: encrypt or decrypt the blocks of its run (counter 1: produce the tag mask) and return the slot's
 // term of the tag, sum over its counters c of block_c * H^(nblk + 3 - c), plus E_K(J0) from counter 1.
 // XOR over a chunk's slots, plus the length term, is its tag.
-template <int MODE, bool ABS>
+// WHOLE: every run is a whole chunk (one lane per chunk).  The run then always ends with the chunk's last block,
+// whose factor is H^2, so the closing product is two more table steps instead of the general product (the lookup
+// pipe has room for them where the integer pipes, busy with two ciphers per handful of bytes, do not), and the
+// value returned is the chunk's complete tag sum: the caller needs no reduction across lanes.
+template <int MODE, bool ABS, bool WHOLE>
 __device__ __forceinline__ uint4 fr_packed_slot_lane(const FrParams& P, const char* sm, const FrLane& L,
                                                      const FrPackGeom& g, uint32_t slot, FrSlot& si)
 {
@@ -610,7 +614,7 @@ __device__ __forceinline__ uint4 fr_packed_slot_lane(const FrParams& P, const ch
     uint32_t c1 = c0 + g.run;
     if (c1 > nblk + 2u) c1 = nblk + 2u;
     uint4 hpow = make_uint4(0, 0, 0, 0);
-    if (DO_GHASH) hpow = P.pow[nblk + 4u - c1];                          // for the run's last block, counter c1 - 1
+    if (DO_GHASH && !WHOLE) hpow = P.pow[nblk + 4u - c1];                // for the run's last block, counter c1 - 1
     const uint8_t* in = P.in + ck.off;
     uint8_t* out = P.out + ck.off;
     FrCtrChunk cc = {0, 0, 0, 0};
@@ -646,5 +650,7 @@ __device__ __forceinline__ uint4 fr_packed_slot_lane(const FrParams& P, const ch
         }
     }
     if (!DO_GHASH) return make_uint4(0, 0, 0, 0);
-    return fr_xor4(fr_gf128_mul(y, hpow), extra);
+    if (WHOLE) y = fr_ghash_tabmul<ABS>(sm, L, fr_ghash_tabmul<ABS>(sm, L, y));
+    else y = fr_gf128_mul(y, hpow);
+    return fr_xor4(y, extra);
 }

@@ -228,6 +228,27 @@ def test_packed_rows_match_oracle(emu, n, cb, group, aad, run_len):
     assert np.array_equal(ok, ok_ref)
 
 
+@pytest.mark.parametrize("cb,n_chunks,run_len,aad", [(16, 70, 2, 0), (16, 70, 9, 3), (48, 33, 4, 0), (112, 40, 8, 5), (1024, 5, 65, 0)])
+def test_packed_rows_on_a_stage_that_starts_at_a_later_chunk(emu, cb, n_chunks, run_len, aad):
+    """One lane per chunk, launched from chunk 1 and from chunk 2 of a buffer (pipelined calls do that): the IV index
+    and the serial number continue, and both closing variants of the whole-chunk layout are exercised (the emulation
+    picks the general product for odd starts)."""
+    rng = np.random.default_rng(cb + n_chunks)
+    key, iv = rng.bytes(32), rng.bytes(12)
+    for first in (1, 2):
+        n = cb * n_chunks - 5
+        p = np.frombuffer(rng.bytes(cb * first + n), np.uint8)
+        c_ref, t_ref = (oracle.mc_encrypt_framed(key, iv, cb, aad, p, 4) if aad else oracle.mc_encrypt(key, iv, cb, p, 4))
+        c, t, _ = run_packed(emu, ENC, key, iv, cb, p[cb * first:], n, group=3, run_len=run_len, first=first, aad=aad)
+        assert np.array_equal(c, c_ref[cb * first:]) and np.array_equal(t, t_ref[first:])
+        bad_t = t_ref[first:].copy()
+        bad_t[n_chunks // 2, 5] ^= 1
+        out, _, ok = run_packed(emu, DEC, key, iv, cb, c_ref[cb * first:], n, tags=bad_t, group=3, run_len=run_len, first=first, aad=aad)
+        expect = np.ones(n_chunks, np.uint32)
+        expect[n_chunks // 2] = 0
+        assert np.array_equal(out, p[cb * first:]) and np.array_equal(ok, expect)
+
+
 @pytest.mark.parametrize("run_len", [1, 4, 7])
 @pytest.mark.parametrize("sample_bytes,cb,n_samples,aad,group", [(16, 16, 40, 0, 3), (48, 16, 9, 0, 4), (400, 400, 11, 0, 2),
                                                                 (400, 112, 7, 16, 5), (1040, 1024, 4, 16, 1), (208, 64, 6, 3, 100)])
