@@ -397,10 +397,17 @@ __device__ __forceinline__ FrChunk fr_chunk_info(const FrParams& P, uint32_t kk)
     c.last_of_sample = (k + 1u == P.chunks_per_sample);
     if (P.ivs) {                 // a batch of samples, each encrypted under its own IV base: chunk k of the sample
         const uint8_t* iv = P.ivs + 12ull * sample;
-        c.iv_w0 = (uint32_t)iv[0] | ((uint32_t)iv[1] << 8) | ((uint32_t)iv[2] << 16) | ((uint32_t)iv[3] << 24);
-        c.iv_w1 = (uint32_t)iv[4] | ((uint32_t)iv[5] << 8) | ((uint32_t)iv[6] << 16) | ((uint32_t)iv[7] << 24);
         c.serial = k;
-        c.iv_ctr = (((uint32_t)iv[8] << 24) | ((uint32_t)iv[9] << 16) | ((uint32_t)iv[10] << 8) | (uint32_t)iv[11]) + k;
+        if ((((size_t)P.ivs) & 3u) == 0u) {          // the usual case: three word loads (12 * sample keeps the alignment)
+            const uint32_t* w = (const uint32_t*)iv;
+            c.iv_w0 = w[0];
+            c.iv_w1 = w[1];
+            c.iv_ctr = fr_bswap(w[2]) + k;
+        } else {
+            c.iv_w0 = (uint32_t)iv[0] | ((uint32_t)iv[1] << 8) | ((uint32_t)iv[2] << 16) | ((uint32_t)iv[3] << 24);
+            c.iv_w1 = (uint32_t)iv[4] | ((uint32_t)iv[5] << 8) | ((uint32_t)iv[6] << 16) | ((uint32_t)iv[7] << 24);
+            c.iv_ctr = (((uint32_t)iv[8] << 24) | ((uint32_t)iv[9] << 16) | ((uint32_t)iv[10] << 8) | (uint32_t)iv[11]) + k;
+        }
     } else {
         c.iv_w0 = P.iv_w0;
         c.iv_w1 = P.iv_w1;

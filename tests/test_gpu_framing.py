@@ -146,7 +146,12 @@ def test_batch_of_samples_each_under_its_own_iv(sample_bytes, cb, n_samples, cha
     with fastrack.Context(key, cb) as ctx:
         ctx.set_framing(chains)
         st = torch.cuda.current_stream().cuda_stream
-        d_iv = dev(ivs)
+        # the IV bases need no alignment: odd sample counts get them at an odd address (byte loads), the others at an
+        # aligned one (word loads)
+        iv_store = torch.zeros(12 * n_samples + 4, dtype=torch.uint8, device="cuda")
+        d_iv = iv_store[n_samples % 2:n_samples % 2 + 12 * n_samples]
+        d_iv.copy_(torch.from_numpy(ivs))
+        assert d_iv.data_ptr() % 4 == n_samples % 2
         d_p = dev(plain)
         d_c = torch.empty_like(d_p)
         d_t = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
