@@ -18,10 +18,11 @@ def _fresh_ivs(n, rep):
     return [synth.fresh_iv(7, 100 * rep + s + 1) for s in range(n)]
 
 
-def test_sample_batch_round_trip_replayed_from_a_graph():
+@pytest.mark.parametrize("cb,sample_bytes,n_samples", [(64 << 10, 150528, 6),      # 3 chunks per sample, the last one 19 456 bytes
+                                                       (256, 4096 + 48, 700)])      # many small chunks: the packed-row kernels
+def test_sample_batch_round_trip_replayed_from_a_graph(cb, sample_bytes, n_samples):
     from paper_2410_15240_b200 import fastrack
     key, _ = synth.key_and_iv(7)
-    cb, sample_bytes, n_samples = 64 << 10, 150528, 6            # 3 chunks per sample, the last one 19 456 bytes
     n = sample_bytes * n_samples
     with fastrack.Context(key, cb) as ctx:
         cps = ctx.num_chunks(sample_bytes)
