@@ -147,6 +147,8 @@ FASTRACK_API int fastrack_encrypt_tag(fastrack_ctx* ctx, const uint8_t iv_base[1
  *   h_tags          host, 16*K bytes, pinned or pageable (copied once, up front).
  *   d_plain, d_ok   device outputs as in fastrack_decrypt_verify.
  *   n_streams       1..8.
+ * A transfer too small to be cut (one stage, up to about 3 MiB) is not copied at all: the kernel reads the
+ * page-locked host buffer itself (and page-locked tags), which saves the copy engine's start-up latency.
  * BLOCKING: returns after every internal stream has completed, so wall-clock time around the call is
  * the effective transfer time.  Work already queued by the caller on other streams is not waited for. */
 FASTRACK_API int fastrack_pipelined_h2d(fastrack_ctx* ctx, const uint8_t iv_base[12],

@@ -252,6 +252,7 @@ struct fastrack_ctx {
     uint32_t aad_mod;             // 0 = no AAD, else chains per sample of the serial-number framing
     uint32_t generic_smem;        // FASTRACK_GENERIC_SMEM=1: exercise the portable addressing path (tests)
     uint32_t no_overlap_launch;   // FASTRACK_NO_OVERLAP_LAUNCH=1: plain stream-ordered launches (experiments)
+    uint32_t direct_small_h2d;    // single-stage pipelined transfers read the host buffer from the kernel (FASTRACK_DIRECT_SMALL=0 switches it off)
     struct { size_t sample_bytes, n_chunks; FrPackPlan plan; bool valid; } pack_memo[3];   // fr_plan_packed's last answer per kind of pass (callers repeat shapes)
 };
 
@@ -313,6 +314,8 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
     if (const char* env = getenv("FASTRACK_GENERIC_SMEM")) ctx->generic_smem = (uint32_t)(strtoul(env, nullptr, 10) != 0);
     if (const char* env = getenv("FASTRACK_NO_OVERLAP_LAUNCH")) ctx->no_overlap_launch = (uint32_t)(strtoul(env, nullptr, 10) != 0);
     if (const char* env = getenv("FASTRACK_STAGE_BYTES")) ctx->plan.stage_bytes_override = (size_t)strtoull(env, nullptr, 10);
+    ctx->direct_small_h2d = 1;
+    if (const char* env = getenv("FASTRACK_DIRECT_SMALL")) ctx->direct_small_h2d = (uint32_t)(strtoul(env, nullptr, 10) != 0);
     ctx->plan.pack_max_blocks = FR_PACK_MAX_BLOCKS;
     if (const char* env = getenv("FASTRACK_PACK_MAX_BLOCKS")) ctx->plan.pack_max_blocks = (uint32_t)strtoul(env, nullptr, 10);
     if (const char* env = getenv("FASTRACK_PACK_RUN")) ctx->plan.pack_run_override = (uint32_t)strtoul(env, nullptr, 10);
@@ -731,6 +734,48 @@ static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const vo
     const size_t cb = ctx->chunk_bytes;
     const size_t n_stages = plan_stages(ctx, len, sample_bytes ? sample_bytes : cb, stage_bytes);
     uint8_t* d_ivs = (uint8_t*)(ctx->d_tags_stage + K);            // batch of samples: device copy of the IV bases
+
+    // A transfer of a single stage has nothing to overlap: copy, then kernel, each with its own start-up latency.
+    // There the kernel reads the ciphertext straight from the page-locked host buffer instead (every block is read
+    // exactly once, 512 contiguous bytes per warp request), so the transfer IS the kernel: no copy engine set-up,
+    // no copy-to-kernel dependency.  Larger transfers keep the copy engine, which leaves the SMs free.
+    // (Measured: a gain of 3-10 us up to 1 MiB whatever the chunk size; from there to the 3 MiB a single stage can
+    // have, only while a lane's reads stay wide -- small chunks in the packed layout read 16 bytes at a stride, which
+    // the link serves poorly.)
+    if (n_stages == 1 && !d_pad && ctx->direct_small_h2d && attr.devicePointer && !misaligned(attr.devicePointer, 16) &&
+        (len <= ((size_t)1 << 20) || cb >= 4096)) {
+        cudaStream_t st = ctx->streams[0];
+        const uint4* tags_src = ctx->d_tags_stage;
+        cudaPointerAttributes ta;
+        if (cudaPointerGetAttributes(&ta, h_tags) == cudaSuccess && ta.type == cudaMemoryTypeHost && ta.devicePointer &&
+            !misaligned(ta.devicePointer, 16)) {
+            tags_src = (const uint4*)ta.devicePointer;             // page-locked tags are read in place too
+        } else {
+            (void)cudaGetLastError();
+            FR_CUDA(ctx, cudaMemcpyAsync(ctx->d_tags_stage, h_tags, K * 16, cudaMemcpyHostToDevice, st));
+        }
+        if (sample_bytes) FR_CUDA(ctx, cudaMemcpyAsync(d_ivs, h_iv_bases, 12 * n_samples, cudaMemcpyHostToDevice, st));
+        const bool tracing = ctx->trace_on;
+        if (tracing) { cudaEventRecord(ctx->trace_ev[0], st); cudaEventRecord(ctx->trace_ev[1], st); }
+        PassBuffers b;
+        b.in = attr.devicePointer; b.out = d_plain; b.tags_in = tags_src; b.ok = d_ok;
+        if (sample_bytes) { b.ivs = d_ivs; b.sample_bytes = sample_bytes; }
+        rc = launch_pass(ctx, FR_MODE_DEC, iv_base, 0, len, b, st);
+        if (tracing) cudaEventRecord(ctx->trace_ev[2], st);
+        cudaError_t se = cudaStreamSynchronize(st);
+        if (rc != FASTRACK_OK) return rc;
+        FR_CUDA(ctx, se);
+        if (tracing) {
+            ctx->trace_count = 1;
+            ctx->trace[0].offset = 0; ctx->trace[0].bytes = len; ctx->trace[0].stream = 0;
+            cudaEventElapsedTime(&ctx->trace[0].copy_start_ms, ctx->trace_ev[0], ctx->trace_ev[0]);
+            cudaEventElapsedTime(&ctx->trace[0].copy_end_ms, ctx->trace_ev[0], ctx->trace_ev[1]);
+            cudaEventElapsedTime(&ctx->trace[0].kernel_end_ms, ctx->trace_ev[0], ctx->trace_ev[2]);
+            (void)cudaGetLastError();
+        }
+        return FASTRACK_OK;
+    }
+
     size_t off = 0;
     for (size_t stage = 0; stage < n_stages; stage++) {
         const size_t n = stage_bytes[stage];

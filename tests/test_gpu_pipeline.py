@@ -16,11 +16,15 @@ from gpu_harness import Gpu  # noqa: E402
 NT = oracle.host_threads()
 
 
-@pytest.mark.parametrize("n,cb", [(1, 16), (100, 1024), (1 << 20, 65536), ((1 << 20) + 17, 65536),
+@pytest.mark.parametrize("n,cb", [(1, 16), (100, 1024), (1 << 20, 65536), ((1 << 20) + 17, 65536), (700001, 256), (2500000, 4096),
                                   (3 * (1 << 20) + 5, 1 << 20), (9 * (1 << 20) + 12345, 256 * 1024),
                                   ((5 << 20) - 16, 48 * 1024), (2 * (1 << 22) + 999, 1 << 22)])
 @pytest.mark.parametrize("n_streams", [1, 3])
-def test_pipelined_matches_oracle_small(n, cb, n_streams):
+@pytest.mark.parametrize("direct", ["1", "0"])
+def test_pipelined_matches_oracle_small(n, cb, n_streams, direct, monkeypatch):
+    """Single-stage transfers (up to about 3 MiB) are by default read from the page-locked host buffer by the kernel
+    itself, pinned tags included; FASTRACK_DIRECT_SMALL=0 keeps them on the copy engine.  Both must equal the oracle."""
+    monkeypatch.setenv("FASTRACK_DIRECT_SMALL", direct)
     key, iv = synth.key_and_iv(2)
     plain = synth.random_bytes(n, 2, salt=n)
     c, t = oracle.mc_encrypt(key, iv, cb, plain, NT)
