@@ -284,7 +284,8 @@ FASTRACK_API int fastrack_pipelined_d2h_samples(fastrack_ctx* ctx, const void* h
  * fastrack_pipelined_h2d_ahead call records three CUDA events per stage on the stage's stream -- before its copy,
  * after its copy, after its kernel -- and fastrack_ctx_get_trace returns, for the most recent call, each stage's
  * byte range, stream index and those three times in milliseconds since the first copy was started.
- * Enabling creates the events (allocation; do it at start-up); tracing adds about a microsecond per event.
+ * (A transfer small enough for the kernel to read the host buffer itself shows as one stage with an empty copy
+ * interval.)  Enabling creates the events (allocation; do it at start-up); tracing adds about a microsecond per event.
  * fastrack_ctx_get_trace copies at most `cap` entries to `out` (may be NULL) and returns the number of stages. */
 typedef struct {
     size_t offset, bytes;          /* byte range of the stage inside the buffer */
