@@ -165,7 +165,8 @@ __global__ void __launch_bounds__(FR_THREADS, 1) fr_packed_kernel(const __grid_c
     uint32_t after_barrier;
     asm volatile("mov.u32 %0, 0;" : "=r"(after_barrier)::"memory");
     FrLane L = fr_make_lane(threadIdx.x & 31u);
-    L.lane4 |= after_barrier;
+    L.lane4 |= after_barrier;          // no table load above the barrier, as in fr_crypt_kernel: every lookup address here
+                                       // derives from lane4, from loaded data, or (the AAD block) is tied to lane4 by the lane code
     if ((uint32_t)__cvta_generic_to_shared(sm) == FR_SMEM_ABS_BASE && !P.generic_smem) fr_packed_body<MODE, true, WHOLE>(P, sm, L);
     else fr_packed_body<MODE, false, WHOLE>(P, sm, L);
 }

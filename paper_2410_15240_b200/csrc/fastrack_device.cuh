@@ -638,7 +638,10 @@ __device__ __forceinline__ uint4 fr_packed_slot_lane(const FrParams& P, const ch
         uint4 gblk;
         if (c == 1u) {
             extra = ks;                                                                      // E_K(J0)
-            gblk = make_uint4(P.aad_mod ? ck.serial % P.aad_mod : 0u, 0, 0, 0);               // the one-byte AAD block, or nothing
+            // the one-byte AAD block, or nothing.  (lane4 >> 8 is zero; the kernel makes lane4 opaque to the compiler after
+            // the barrier that follows the table build, and this ties the only table step whose input is not loaded data or
+            // cipher output to it, so that the step cannot be scheduled above that barrier.)
+            gblk = make_uint4(P.aad_mod ? (ck.serial % P.aad_mod) | (L.lane4 >> 8) : 0u, 0, 0, 0);
         } else {
             const uint64_t boff = (uint64_t)(c - 2u) << 4;
             const bool full = ck.len - boff >= 16;
