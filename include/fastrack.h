@@ -263,6 +263,8 @@ FASTRACK_API int fastrack_decrypt_verify_noalloc(fastrack_ctx* ctx, const uint8_
  * of stage i overlaps the kernel of stage i+1 and only the short first stage's kernel is exposed.
  *   d_plain         device, len bytes in (not modified unless d_cipher == d_plain).
  *   d_cipher        device, len bytes of ciphertext staging; d_cipher == d_plain (exactly) encrypts in place.
+ *                   Otherwise its contents after the call are unspecified: a transfer too small to be cut (one
+ *                   stage, up to about 3 MiB) is written to the host buffers by the kernel itself and skips it.
  *   h_cipher_pinned host, page-locked, len bytes out.
  *   h_tags          host, 16*K bytes out, pinned or pageable.
  *   n_streams       1..8.

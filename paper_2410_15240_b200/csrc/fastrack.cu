@@ -917,6 +917,32 @@ static int pipelined_d2h_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], cons
     size_t stage_bytes[FR_MAX_STAGES];
     const size_t unit = sample_bytes ? sample_bytes : cb;
     const size_t n_stages = plan_stages(ctx, sample_bytes ? len : K * cb, unit, stage_bytes);
+    // A transfer of a single stage: the kernel writes ciphertext (and tags, if their buffer is page-locked too) straight
+    // into the host buffers instead of into d_cipher followed by two copies -- the mirror of the small host-to-device case.
+    // Not when encrypting in place: the caller then expects d_plain to hold the ciphertext afterwards.
+    if (n_stages == 1 && ctx->direct_small_h2d && d_cipher != d_plain && attr.devicePointer && !misaligned(attr.devicePointer, 16) &&
+        (len <= ((size_t)1 << 20) || cb >= 4096)) {
+        cudaStream_t st = ctx->streams[0];
+        if (sample_bytes) FR_CUDA(ctx, cudaStreamWaitEvent(st, ctx->tags_ready, 0));          // the IV bases
+        cudaPointerAttributes ta;
+        void* tags_dst = nullptr;
+        if (cudaPointerGetAttributes(&ta, h_tags) == cudaSuccess && ta.type == cudaMemoryTypeHost && ta.devicePointer &&
+            !misaligned(ta.devicePointer, 16)) tags_dst = ta.devicePointer;
+        (void)cudaGetLastError();
+        PassBuffers b;
+        b.in = d_plain; b.out = attr.devicePointer; b.tags_out = tags_dst ? tags_dst : (void*)ctx->d_tags_stage;
+        if (sample_bytes) { b.ivs = d_ivs; b.sample_bytes = sample_bytes; }
+        rc = launch_pass(ctx, FR_MODE_ENC, iv_base, 0, len, b, st);
+        if (rc == FASTRACK_OK && !tags_dst) {
+            e = cudaMemcpyAsync(h_tags, ctx->d_tags_stage, 16 * K, cudaMemcpyDeviceToHost, st);
+            if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); rc = FASTRACK_ERR_CUDA; }
+        }
+        cudaError_t se = cudaStreamSynchronize(st);
+        if (sample_bytes) cudaStreamSynchronize(iv_stream);
+        if (rc != FASTRACK_OK) return rc;
+        FR_CUDA(ctx, se);
+        return FASTRACK_OK;
+    }
     bool waited[8] = {false, false, false, false, false, false, false, false};
     size_t off = 0;
     for (size_t i = 0; i < n_stages; i++) {

@@ -54,11 +54,16 @@ def test_config2_fp16_image_batch(cb, n_streams):
 
 
 @pytest.mark.parametrize("n,cb,n_streams,in_place", [(1, 16, 1, False), (100, 1024, 2, True), ((1 << 20) + 17, 65536, 2, False),
+                                                      (700001, 256, 2, False), (2500000, 4096, 1, False), (2500000, 4096, 1, True),
                                                       ((9 << 20) + 12345, 256 * 1024, 3, True),
                                                       (2 * (1 << 22) + 999, 1 << 22, 4, False), (77_070_336, 4 << 20, 4, False)])
-def test_pipelined_d2h_encrypt_matches_oracle(n, cb, n_streams, in_place):
-    """GPU encrypt+tag with overlapped device->host copies; the host side (oracle) verifies and decrypts."""
+@pytest.mark.parametrize("direct,pinned_tags", [("1", False), ("1", True), ("0", False)])
+def test_pipelined_d2h_encrypt_matches_oracle(n, cb, n_streams, in_place, direct, pinned_tags, monkeypatch):
+    """GPU encrypt+tag with overlapped device->host copies; the host side (oracle) verifies and decrypts.
+    Single-stage transfers are by default written to the page-locked host buffers by the kernel itself (tags too when
+    their buffer is page-locked); FASTRACK_DIRECT_SMALL=0 keeps them on the copy engine."""
     from paper_2410_15240_b200 import fastrack
+    monkeypatch.setenv("FASTRACK_DIRECT_SMALL", direct)
     key, iv = synth.key_and_iv(3)
     plain = synth.fp16_image_batch() if n == 77_070_336 else synth.random_bytes(n, 3, salt=n)
     c_ref, t_ref = oracle.mc_encrypt(key, iv, cb, plain, NT)
@@ -68,6 +73,8 @@ def test_pipelined_d2h_encrypt_matches_oracle(n, cb, n_streams, in_place):
         d_c = d_p if in_place else torch.empty_like(d_p)
         h_c = torch.full((n,), 0xEE, dtype=torch.uint8).pin_memory()
         h_t = torch.zeros(16 * K, dtype=torch.uint8)
+        if pinned_tags:
+            h_t = h_t.pin_memory()
         torch.cuda.synchronize()
         for _ in range(1 if in_place else 2):
             ctx.pipelined_d2h(iv, d_p.data_ptr(), n, d_c.data_ptr(), h_c.data_ptr(), h_t.data_ptr(), n_streams)
