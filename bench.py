@@ -48,6 +48,20 @@ ROW_BYTES = 512
 DRAM_TRAFFIC_BYTES_PER_LAUNCH = 501.9e6
 
 
+def build_bench_helper(source: str, target: str, shared: bool = False) -> str:
+    """Compile one of the measurement helpers under bench/ (they are not part of the library) if it is stale."""
+    src, out = os.path.join(ROOT, "bench", source), os.path.join(ROOT, "bench", target)
+    deps = [src, os.path.join(ROOT, "include", "fastrack.h")]
+    if not os.path.exists(out) or any(os.path.getmtime(out) < os.path.getmtime(d) for d in deps):
+        nvcc = os.environ.get("NVCC", "nvcc")
+        cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-o", out + ".tmp", src]
+        if shared:
+            cmd += ["-shared", "-Xcompiler", "-fPIC"]
+        subprocess.check_call(cmd)
+        os.replace(out + ".tmp", out)
+    return out
+
+
 def peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -597,9 +611,7 @@ def run_trace(args):
 def run_peaks(args):
     """Unit rates behind the kernel roofline, measured on this GPU (integer pipes, shared-memory lookups, PCIe)."""
     import ctypes
-    from paper_2410_15240_b200 import build as lib_build
-    lib_build.build()
-    lib = ctypes.CDLL(lib_build.PROBE_LIB)
+    lib = ctypes.CDLL(build_bench_helper("peaks_probe.cu", "libpeaks_probe.so", shared=True))
     lib.fastrack_probe_peaks.argtypes = [ctypes.c_char_p, ctypes.c_size_t]
     lib.fastrack_probe_peaks.restype = ctypes.c_int
     buf = ctypes.create_string_buffer(1 << 16)

@@ -25,9 +25,10 @@
  *     h_* are HOST pointers.  `key` and `iv_base` are always HOST pointers.  The caller owns every
  *     data buffer; the context owns only key-derived tables, per-chunk scratch and internal streams.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
- *   - A context is bound to the device that was current at creation and must not be used from two
- *     host threads, or on two streams, at the same time (calls share per-chunk scratch memory); the one
- *     exception is fastrack_verify, see there.
+ *   - A context is bound to the device that was current at creation.  That device must be the current device
+ *     of the calling thread at every call that launches work or touches device memory; otherwise the call returns
+ *     FASTRACK_ERR_ARG and does nothing.  A context must not be used from two host threads, or on two streams,
+ *     at the same time (calls share scratch memory); the one exception is fastrack_verify, see there.
  *   - IV discipline is the caller's: one call consumes the IV values iv_base .. iv_base + K - 1;
  *     reusing an IV under the same key voids GCM's guarantees.  The library does not track this.
  *   - K is derived from `len`; dropping trailing chunks is invisible to this layer, so `len` must
@@ -60,13 +61,13 @@ extern "C" {
 #define FASTRACK_ERR_CUDA        -4   /* a CUDA call failed; see fastrack_last_cuda_error */
 #define FASTRACK_ERR_NOMEM       -5   /* host or device allocation failed */
 #define FASTRACK_ERR_TOO_MANY    -6   /* more than 2^32 chunks in one call (the IV index is 32 bits) */
-#define FASTRACK_ERR_LIMIT       -7   /* more chunks than fastrack_decrypt_verify_noalloc's fixed scratch holds */
+#define FASTRACK_ERR_LIMIT       -7   /* beyond a fixed limit of fastrack_decrypt_verify_noalloc (chunks per call, SMs of the device) */
 
 /* Largest chunk: 1 GiB.  (GCM itself allows 2^36 - 32 bytes per message; the limit here keeps the
  * per-context table of powers of H, 16 bytes per 16-byte block of a chunk, at most 1 GiB.) */
 #define FASTRACK_MAX_CHUNK_BYTES ((size_t)1 << 30)
 
-/* Most chunks one fastrack_decrypt_verify_noalloc call may cover (its scratch is a fixed 320 KiB array). */
+/* Most chunks one fastrack_decrypt_verify_noalloc call may cover. */
 #define FASTRACK_NOALLOC_MAX_CHUNKS 16384
 
 typedef struct fastrack_ctx fastrack_ctx;
@@ -88,14 +89,10 @@ FASTRACK_API void fastrack_ctx_destroy(fastrack_ctx* ctx);
 /* K = ceil(len / chunk_bytes); 0 for len == 0 or ctx == NULL (Section 4.2: one tag per chunk). */
 FASTRACK_API size_t fastrack_num_chunks(const fastrack_ctx* ctx, size_t len);
 
-/* Pre-sizes the per-chunk scratch (40 bytes per chunk: two banks of a 16-byte accumulator and a counter) for buffers up to max_len bytes so that later
- * calls allocate nothing.  Without it the first call that needs more chunks than any call before
- * grows the scratch (cudaMalloc + a device synchronisation) before launching.  Contexts whose chunk_bytes is at
- * most 992 never need more than the scratch they are created with (such chunks are never split between warps).
- * Stream capture: once the scratch is large enough, every asynchronous call below is a single kernel launch with
- * all arguments passed by value, so it may be recorded into a CUDA graph and replayed.  A replay repeats the
- * recorded arguments -- the IV base included, for the calls that take it by value; the *_samples calls read their IV
- * bases from device memory and are the ones to capture when every replay needs fresh IVs (it does, under GCM). */
+/* Kept for callers written against earlier versions, in which the scratch memory grew with the number of chunks
+ * and this call pre-sized it.  The scratch is now a fixed set of records per context (the pieces of a chunk are
+ * first combined inside a CTA, and only one record per CTA of a launch is needed across CTAs), allocated by
+ * fastrack_ctx_create; no later call of any kind allocates device memory for it.  Returns FASTRACK_OK. */
 FASTRACK_API int fastrack_ctx_reserve(fastrack_ctx* ctx, size_t max_len);
 
 /* Paper-faithful framing (Section 4.2: every chunk is "attached to one byte of additional authentication data
@@ -106,6 +103,23 @@ FASTRACK_API int fastrack_ctx_reserve(fastrack_ctx* ctx, size_t max_len);
  * The IV rule is unchanged in both cases.  Applies to every later call on the context, of every kind; both
  * ends must use the same setting (a mismatch rejects every chunk).  Takes effect for calls issued afterwards. */
 FASTRACK_API int fastrack_ctx_set_framing(fastrack_ctx* ctx, unsigned chains_per_sample);
+
+/* Test and tuning controls.  Results never depend on them -- every setting computes the same bytes, tags and
+ * verdicts -- only the choice of kernel layout and launch geometry does, which the library otherwise makes by itself;
+ * the defaults are the ones to ship.  They exist so that tests can force each layout on any shape and so that the
+ * cost models can be re-fitted on new hardware.  The library reads no environment variable.
+ * A setting applies to every later call on the context.  Unknown option: FASTRACK_ERR_ARG. */
+enum {
+    FASTRACK_OPT_ROW_SLOTS = 1,         /* row layout: spread a launch over this many warps (0 = automatic) */
+    FASTRACK_OPT_GENERIC_SMEM = 2,      /* 1: portable shared-memory addressing even where the absolute form applies */
+    FASTRACK_OPT_NO_OVERLAP_LAUNCH = 3, /* 1: plain stream-ordered launches (no programmatic dependent launch) */
+    FASTRACK_OPT_STAGE_BYTES = 4,       /* pipelined calls: fixed stage size in bytes (0 = the shrinking / growing stages) */
+    FASTRACK_OPT_DIRECT_SMALL = 5,      /* 0: single-stage pipelined transfers use the copy engine too (default 1) */
+    FASTRACK_OPT_PACK_MAX_BLOCKS = 6,   /* packed layout only for chunks of at most this many blocks (0 = never; default and cap 4096) */
+    FASTRACK_OPT_PACK_RUN = 7,          /* packed layout with this many counters per lane wherever it applies (0 = automatic) */
+    FASTRACK_OPT_PACK_GROUP = 8         /* packed layout: whole chunks per work item (0 = automatic) */
+};
+FASTRACK_API int fastrack_ctx_set_option(fastrack_ctx* ctx, int option, uint64_t value);
 
 /* CUDA error code (cudaError_t as int) of the last failing CUDA call made through ctx, else 0. */
 FASTRACK_API int fastrack_last_cuda_error(const fastrack_ctx* ctx);

@@ -16,10 +16,6 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", 
               "-shared", "-Xcompiler", "-fPIC,-fvisibility=hidden"]
 
 
-PROBE_LIB = os.path.join(HERE, "libfastrack_probe.so")
-PROBE_SRC = os.path.join(CSRC, "peaks_probe.cu")
-
-
 def _compile(target: str, sources, deps, force: bool, verbose: bool) -> None:
     stale = (not os.path.exists(target)) or any(os.path.getmtime(target) < os.path.getmtime(d) for d in deps)
     if force or stale:
@@ -31,10 +27,8 @@ def _compile(target: str, sources, deps, force: bool, verbose: bool) -> None:
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile libfastrack.so (and the small peak-rate probe library) if missing or older than their sources.
-    Returns the path of libfastrack.so."""
+    """Compile libfastrack.so if it is missing or older than its sources.  Returns its path."""
     _compile(LIB, SOURCES, DEPS, force, verbose)
-    _compile(PROBE_LIB, [PROBE_SRC], [PROBE_SRC], force, False)
     return LIB
 
 

@@ -18,72 +18,99 @@ using namespace fr_host;
 // ------------------------------------------------------------------------------------ kernels ----
 
 template <int MODE, bool ABS>
-__device__ __forceinline__ void fr_crypt_body(const FrParams& P, const char* sm, FrLane L)
+__device__ __forceinline__ void fr_crypt_body(const FrParams& P, char* sm, FrLane L)
 {
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    const uint32_t total_warps = gridDim.x * (blockDim.x >> 5);
+    if (warp >= P.warps_used) return;
+    const uint32_t cta_first = blockIdx.x * P.warps_used, slot = cta_first + warp;
+    if (slot >= P.n_slots) return;
+    uint32_t cta_last = cta_first + P.warps_used - 1u;
+    if (cta_last >= P.n_slots) cta_last = P.n_slots - 1u;
+    uint32_t* const comb = (uint32_t*)(sm + FR_SM_COMB);
 
-    for (uint32_t item = warp * gridDim.x + blockIdx.x; item < P.n_items; item += total_warps) {
-        const uint32_t kk = item / P.segs_per_chunk, s = item - kk * P.segs_per_chunk;
-        const uint32_t nseg = fr_chunk_segs(P, kk);
-        if (s >= nseg) continue;                       // only the short last chunk has fewer segments
-
-        uint4 z = fr_process_segment_lane<MODE, ABS>(P, sm, L, lane, kk, s);
+    uint64_t g = fr_slot_begin(P, slot);
+    const uint64_t end = fr_slot_begin(P, slot + 1u);
+    while (g < end) {                                    // one segment per chunk that the warp's range touches
+        const FrRowPos pos = fr_locate_row(P, g);
+        uint32_t take = pos.rows_k - pos.r;
+        if (take > end - g) take = (uint32_t)(end - g);
+        uint4 z = fr_process_segment_lane<MODE, ABS>(P, sm, L, lane, pos.kk, pos.r, pos.r + take);
+        const uint64_t g0 = g - pos.r;                   // the chunk's first row in the row space
+        g += take;
         if (MODE != FR_MODE_CTR && MODE != FR_MODE_PADGEN) {                // the other passes authenticate
-    #pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                z.x ^= __shfl_xor_sync(0xFFFFFFFFu, z.x, off);
-                z.y ^= __shfl_xor_sync(0xFFFFFFFFu, z.y, off);
-                z.z ^= __shfl_xor_sync(0xFFFFFFFFu, z.z, off);
-                z.w ^= __shfl_xor_sync(0xFFFFFFFFu, z.w, off);
-            }
-            bool finisher = true;
-            if (nseg > 1) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            z.x ^= __shfl_xor_sync(0xFFFFFFFFu, z.x, off);
+            z.y ^= __shfl_xor_sync(0xFFFFFFFFu, z.y, off);
+            z.z ^= __shfl_xor_sync(0xFFFFFFFFu, z.z, off);
+            z.w ^= __shfl_xor_sync(0xFFFFFFFFu, z.w, off);
+        }
+        // A chunk covered by several warps: each XORs its part into a record and takes a ticket; whoever takes the
+        // last ticket carries the sum on (XOR commutes, so the result does not depend on the order of arrival).
+        // First among the warps of this CTA, in shared memory; then among CTAs, in the global record of the first
+        // CTA that works on the chunk.  Records are left zeroed.  No warp ever waits for another.
+        bool finisher = true;
+        if (take != pos.rows_k) {
+            const FrShare sh = fr_chunk_share(P, g0, pos.rows_k, cta_first, cta_last);
+            if (sh.n_in_cta > 1u) {
+                uint32_t* rec = comb + 8u * sh.rec;
                 uint32_t ticket = 0;
                 if (lane == 0) {
-                    atomicXor(&P.acc[4 * kk + 0], z.x);
-                    atomicXor(&P.acc[4 * kk + 1], z.y);
-                    atomicXor(&P.acc[4 * kk + 2], z.z);
-                    atomicXor(&P.acc[4 * kk + 3], z.w);
-                    __threadfence();
-                    ticket = atomicAdd(&P.cnt[kk], 1u);
+                    atomicXor(rec + 0, z.x); atomicXor(rec + 1, z.y); atomicXor(rec + 2, z.z); atomicXor(rec + 3, z.w);
+                    __threadfence_block();
+                    ticket = atomicAdd(rec + 4, 1u);
                 }
                 ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
-                finisher = (ticket == nseg - 1);
-                if (finisher) {
+                finisher = (ticket == sh.n_in_cta - 1u);
+                if (finisher && lane == 0) {
+                    __threadfence_block();
+                    z.x = atomicExch(rec + 0, 0u); z.y = atomicExch(rec + 1, 0u);
+                    z.z = atomicExch(rec + 2, 0u); z.w = atomicExch(rec + 3, 0u);
+                }
+            }
+            if (finisher && sh.n_ctas > 1u) {
+                uint32_t* rec = P.acc + 8u * sh.first_cta;
+                uint32_t ticket = 0;
+                if (lane == 0) {
+                    atomicXor(rec + 0, z.x); atomicXor(rec + 1, z.y); atomicXor(rec + 2, z.z); atomicXor(rec + 3, z.w);
                     __threadfence();
-                    if (lane == 0) {                       // read the sum and leave the scratch zeroed
-                        z.x = atomicExch(&P.acc[4 * kk + 0], 0u);
-                        z.y = atomicExch(&P.acc[4 * kk + 1], 0u);
-                        z.z = atomicExch(&P.acc[4 * kk + 2], 0u);
-                        z.w = atomicExch(&P.acc[4 * kk + 3], 0u);
-                        atomicExch(&P.cnt[kk], 0u);
-                    }
+                    ticket = atomicAdd(rec + 4, 1u);
+                }
+                ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
+                finisher = (ticket == sh.n_ctas - 1u);
+                if (finisher && lane == 0) {              // read the sum and leave the record zeroed
+                    __threadfence();
+                    z.x = atomicExch(rec + 0, 0u); z.y = atomicExch(rec + 1, 0u);
+                    z.z = atomicExch(rec + 2, 0u); z.w = atomicExch(rec + 3, 0u);
+                    atomicExch(rec + 4, 0u);
                 }
             }
-            if (finisher && lane == 0) {
-                const uint4 lenh = ((kk + 1u) % P.chunks_per_sample == 0u) ? P.lenh_last : P.lenh_full;
-                const uint4 tag = fr_xor4(z, lenh);           // z already holds GHASH of the data xor E_K(J0)
-                if (MODE == FR_MODE_ENC) {
-                    P.tags_out[kk] = tag;
-                } else {
-                    const uint4 t = P.tags_in[kk];
-                    const uint32_t diff = (tag.x ^ t.x) | (tag.y ^ t.y) | (tag.z ^ t.z) | (tag.w ^ t.w);
-                    P.ok[kk] = diff == 0u ? 1u : 0u;
-                }
+        }
+        if (finisher && lane == 0) {
+            const uint4 lenh = ((pos.kk + 1u) % P.chunks_per_sample == 0u) ? P.lenh_last : P.lenh_full;
+            const uint4 tag = fr_xor4(z, lenh);           // z already holds GHASH of the data xor E_K(J0)
+            if (MODE == FR_MODE_ENC) {
+                P.tags_out[pos.kk] = tag;
+            } else {
+                const uint4 t = P.tags_in[pos.kk];
+                const uint32_t diff = (tag.x ^ t.x) | (tag.y ^ t.y) | (tag.z ^ t.z) | (tag.w ^ t.w);
+                P.ok[pos.kk] = diff == 0u ? 1u : 0u;
             }
+        }
         }
     }
 }
 
-// Fused pass: keystream, XOR, per-segment GHASH partial, per-chunk tag.  Segments are dealt to warps
-// round-robin; a warp XORs its segment's partial into the chunk's accumulator and takes a ticket; the
-// warp that takes the chunk's last ticket finishes the tag (no warp ever waits for another).
+// Fused pass: keystream, XOR, per-segment GHASH partial, per-chunk tag.  Every warp that takes work walks one
+// contiguous range of the launch's rows (see fr_slot_begin in the device header).
 template <int MODE>
 __global__ void __launch_bounds__(FR_THREADS, 1) fr_crypt_kernel(const __grid_constant__ FrParams P)
 {
     extern __shared__ __align__(256) char sm[];
+    FR_STAMP_GT(0); FR_STAMP_SET(7);
     fr_build_smem<FR_THREADS>(sm, threadIdx.x, P.te0, P.gh_tab);
+    if (threadIdx.x < 33u * 8u) ((uint32_t*)(sm + FR_SM_COMB))[threadIdx.x] = 0u;      // the combine records start at zero
+    FR_STAMP_SET(1);
     // Programmatic dependent launch: the table build above touches only per-context constants, so it may run
     // while the previous kernel in the stream is still finishing; everything below waits until that kernel has
     // completed and its writes are visible (a no-op when the launch carries no such dependency).  Kernels queued
@@ -91,6 +118,7 @@ __global__ void __launch_bounds__(FR_THREADS, 1) fr_crypt_kernel(const __grid_co
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;");
     __syncthreads();
+    FR_STAMP_SET(2);
     // Lane constants are made to depend on a value the compiler cannot see through and that is produced
     // after the barrier, so that no table load can be scheduled above the barrier.
     uint32_t after_barrier;
@@ -101,6 +129,7 @@ __global__ void __launch_bounds__(FR_THREADS, 1) fr_crypt_kernel(const __grid_co
     L.qo |= after_barrier;
     if ((uint32_t)__cvta_generic_to_shared(sm) == FR_SMEM_ABS_BASE && !P.generic_smem) fr_crypt_body<MODE, true>(P, sm, L);
     else fr_crypt_body<MODE, false>(P, sm, L);
+    FR_STAMP_MAX(5); FR_STAMP_GTMAX(6);
 }
 
 // Packed rows (many short chains, see the device header): a warp takes pack_chunks whole chunks and walks their
@@ -224,6 +253,21 @@ __global__ void __launch_bounds__(32, 1) fr_verify_sequential_kernel(const __gri
     P.ok[kk] = ((tag.x ^ t.x) | (tag.y ^ t.y) | (tag.z ^ t.z) | (tag.w ^ t.w)) == 0u ? 1u : 0u;
 }
 
+#ifdef FR_STAMPS
+// Diagnostic build only: reset the probes (rows-done minimum to all ones, the rest to zero) / copy them out.
+extern "C" __attribute__((visibility("default"))) int fastrack_stamps_reset(void)
+{
+    static unsigned long long init[1024 * 8];
+    for (int b = 0; b < 1024; b++)
+        for (int i = 0; i < 8; i++) init[b * 8 + i] = (i == 3) ? ~0ull : 0ull;
+    return (int)cudaMemcpyToSymbol(fr_stamps, init, sizeof init);
+}
+extern "C" __attribute__((visibility("default"))) int fastrack_stamps_read(unsigned long long* out)
+{
+    return (int)cudaMemcpyFromSymbol(out, fr_stamps, sizeof(unsigned long long) * 1024 * 8);
+}
+#endif
+
 // ------------------------------------------------------------------------------------ context ----
 
 struct fastrack_ctx {
@@ -238,8 +282,7 @@ struct fastrack_ctx {
     uint4* d_gh1_tab;          // byte tables of H (sequential-chain comparator only)
     uint4* d_pow;
     size_t pow_entries;
-    uint32_t* d_scratch;       // two banks, each acc[4*cap] then cnt[cap]; bank 1 serves fastrack_verify
-    size_t scratch_chunks;
+    uint32_t* d_scratch;       // combine records of the row kernels: 2 banks x FR_SCRATCH_WINDOWS windows x num_sms records of 8 words
     uint4* d_tags_stage;       // pipelined calls: device copy of the tags, then (second half) the E_K(J0) masks
     size_t tags_stage_chunks;
     cudaStream_t streams[8];
@@ -251,9 +294,9 @@ struct fastrack_ctx {
     int last_cuda_error;
     uint64_t launches;
     uint32_t aad_mod;             // 0 = no AAD, else chains per sample of the serial-number framing
-    uint32_t generic_smem;        // FASTRACK_GENERIC_SMEM=1: exercise the portable addressing path (tests)
-    uint32_t no_overlap_launch;   // FASTRACK_NO_OVERLAP_LAUNCH=1: plain stream-ordered launches (experiments)
-    uint32_t direct_small_h2d;    // single-stage pipelined transfers read the host buffer from the kernel (FASTRACK_DIRECT_SMALL=0 switches it off)
+    uint32_t generic_smem;        // FASTRACK_OPT_GENERIC_SMEM: exercise the portable addressing path (tests)
+    uint32_t no_overlap_launch;   // FASTRACK_OPT_NO_OVERLAP_LAUNCH: plain stream-ordered launches (experiments)
+    uint32_t direct_small_h2d;    // single-stage pipelined transfers read / write the host buffer from the kernel (FASTRACK_OPT_DIRECT_SMALL)
     struct { size_t sample_bytes, n_chunks; FrPackPlan plan; bool valid; } pack_memo[3];   // fr_plan_packed's last answer per kind of pass (callers repeat shapes)
 };
 
@@ -274,24 +317,19 @@ static void secure_zero(void* p, size_t n)
     for (size_t i = 0; i < n; i++) q[i] = 0;
 }
 
-static int ensure_scratch(fastrack_ctx* ctx, size_t chunks)
+// The row kernels combine the pieces of a chunk that several CTAs worked on in one 32-byte record per CTA of the
+// launch (see fr_crypt_body).  Launches that may be in flight at the same time use different windows of
+// num_sms records: window 0 serves the caller's stream, window 1 + i the library's internal stream i (stages of
+// the pipelined calls), and fastrack_verify has a bank of its own.  The size does not depend on the data.
+#define FR_SCRATCH_WINDOWS 9
+static size_t scratch_words(const fastrack_ctx* ctx) { return (size_t)2 * FR_SCRATCH_WINDOWS * (size_t)ctx->num_sms * 8; }
+
+// Every entry point that launches work or touches device memory runs on the context's device only.
+static int check_device(fastrack_ctx* ctx)
 {
-    if (chunks <= ctx->scratch_chunks) return FASTRACK_OK;
-    // A chunk of at most 62 blocks is two rows, and no segment is shorter than two rows: such chunks are never split
-    // between warps, so neither kernel family touches the scratch (40 bytes per chunk would exceed the data itself
-    // at 16-byte chunks).  launch_pass checks this assumption.
-    if (!ctx->plan.seg_rows_override && ctx->chunk_bytes <= 62 * 16) return FASTRACK_OK;
-    size_t cap = ctx->scratch_chunks ? ctx->scratch_chunks : 1024;
-    while (cap < chunks) cap *= 2;
-    FR_CUDA(ctx, cudaDeviceSynchronize());       // nothing may still be using the old scratch
-    uint32_t* fresh = nullptr;
-    cudaError_t e = cudaMalloc(&fresh, cap * 10 * sizeof(uint32_t));
-    if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); return FASTRACK_ERR_NOMEM; }
-    FR_CUDA(ctx, cudaMemset(fresh, 0, cap * 10 * sizeof(uint32_t)));
-    if (ctx->d_scratch) cudaFree(ctx->d_scratch);
-    ctx->d_scratch = fresh;
-    ctx->scratch_chunks = cap;
-    return FASTRACK_OK;
+    int dev = -1;
+    FR_CUDA(ctx, cudaGetDevice(&dev));
+    return dev == ctx->device ? FASTRACK_OK : FASTRACK_ERR_ARG;
 }
 
 extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fastrack_ctx** out)
@@ -303,7 +341,6 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
     if (!ctx) return FASTRACK_ERR_NOMEM;
     memset(ctx, 0, sizeof *ctx);
     ctx->chunk_bytes = chunk_bytes;
-    int rc = FASTRACK_OK;
     auto fail = [&](int code) { fastrack_ctx_destroy(ctx); return code; };
 
     cudaError_t e = cudaGetDevice(&ctx->device);
@@ -311,16 +348,8 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
     if (e != cudaSuccess) { (void)cudaGetLastError(); return fail(FASTRACK_ERR_CUDA); }
     ctx->plan.num_sms = ctx->num_sms;
     ctx->plan.chunk_bytes = chunk_bytes;
-    if (const char* env = getenv("FASTRACK_SEG_ROWS")) ctx->plan.seg_rows_override = (uint32_t)strtoul(env, nullptr, 10);
-    if (const char* env = getenv("FASTRACK_GENERIC_SMEM")) ctx->generic_smem = (uint32_t)(strtoul(env, nullptr, 10) != 0);
-    if (const char* env = getenv("FASTRACK_NO_OVERLAP_LAUNCH")) ctx->no_overlap_launch = (uint32_t)(strtoul(env, nullptr, 10) != 0);
-    if (const char* env = getenv("FASTRACK_STAGE_BYTES")) ctx->plan.stage_bytes_override = (size_t)strtoull(env, nullptr, 10);
     ctx->direct_small_h2d = 1;
-    if (const char* env = getenv("FASTRACK_DIRECT_SMALL")) ctx->direct_small_h2d = (uint32_t)(strtoul(env, nullptr, 10) != 0);
     ctx->plan.pack_max_blocks = FR_PACK_MAX_BLOCKS;
-    if (const char* env = getenv("FASTRACK_PACK_MAX_BLOCKS")) ctx->plan.pack_max_blocks = (uint32_t)strtoul(env, nullptr, 10);
-    if (const char* env = getenv("FASTRACK_PACK_RUN")) ctx->plan.pack_run_override = (uint32_t)strtoul(env, nullptr, 10);
-    if (const char* env = getenv("FASTRACK_PACK_GROUP")) ctx->plan.pack_group_override = (uint32_t)strtoul(env, nullptr, 10);
 
     // key material on the host: S-box, Te0, round keys, H, byte tables of H^32
     uint8_t sbox[256];
@@ -362,6 +391,8 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
         if ((e = cudaMalloc(&ctx->d_gh_tab, 65536)) != cudaSuccess) break;
         if ((e = cudaMalloc(&ctx->d_gh1_tab, 65536)) != cudaSuccess) break;
         if ((e = cudaMalloc(&ctx->d_pow, ctx->pow_entries * 16)) != cudaSuccess) break;
+        if ((e = cudaMalloc(&ctx->d_scratch, scratch_words(ctx) * sizeof(uint32_t))) != cudaSuccess) break;
+        if ((e = cudaMemset(ctx->d_scratch, 0, scratch_words(ctx) * sizeof(uint32_t))) != cudaSuccess) break;
         if ((e = cudaMemcpy(ctx->d_te0, te0, sizeof te0, cudaMemcpyHostToDevice)) != cudaSuccess) break;
         if ((e = cudaMemcpy(ctx->d_gh_tab, tab, 65536, cudaMemcpyHostToDevice)) != cudaSuccess) break;
         if ((e = cudaMemcpy(ctx->d_gh1_tab, tab + 65536, 65536, cudaMemcpyHostToDevice)) != cudaSuccess) break;
@@ -375,12 +406,12 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
             fr_pow_double_kernel<<<(unsigned)((todo + 255) / 256), 256>>>(ctx->d_pow, (uint32_t)half, (uint32_t)ctx->pow_entries);
         }
         if ((e = cudaGetLastError()) != cudaSuccess) break;
-        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_DEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
-        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_ENC>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
-        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_CTR>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
-        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_VERIFY>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
-        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_PADGEN>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
-        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_PADDEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_DEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_ENC>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_CTR>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_VERIFY>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_PADGEN>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_PADDEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
         if ((e = cudaFuncSetAttribute(fr_verify_sequential_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
         if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_DEC, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
         if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_DEC, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
@@ -403,8 +434,6 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
         (void)cudaGetLastError();
         return fail(e == cudaErrorMemoryAllocation ? FASTRACK_ERR_NOMEM : FASTRACK_ERR_CUDA);
     }
-    rc = ensure_scratch(ctx, 1024);
-    if (rc != FASTRACK_OK) return fail(rc);
     *out = ctx;
     return FASTRACK_OK;
 }
@@ -442,8 +471,26 @@ extern "C" size_t fastrack_num_chunks(const fastrack_ctx* ctx, size_t len)
 
 extern "C" int fastrack_ctx_reserve(fastrack_ctx* ctx, size_t max_len)
 {
+    (void)max_len;                       // the scratch is a fixed set of records per context: nothing to grow
+    return ctx ? FASTRACK_OK : FASTRACK_ERR_ARG;
+}
+
+extern "C" int fastrack_ctx_set_option(fastrack_ctx* ctx, int option, uint64_t value)
+{
     if (!ctx) return FASTRACK_ERR_ARG;
-    return ensure_scratch(ctx, fastrack_num_chunks(ctx, max_len));
+    for (auto& memo : ctx->pack_memo) memo.valid = false;         // the planners' answers depend on these
+    switch (option) {
+        case FASTRACK_OPT_ROW_SLOTS:         ctx->plan.row_slots_override = (uint32_t)(value > 0xFFFFFFFFull ? 0xFFFFFFFFull : value); break;
+        case FASTRACK_OPT_GENERIC_SMEM:      ctx->generic_smem = value != 0; break;
+        case FASTRACK_OPT_NO_OVERLAP_LAUNCH: ctx->no_overlap_launch = value != 0; break;
+        case FASTRACK_OPT_STAGE_BYTES:       ctx->plan.stage_bytes_override = (size_t)value; break;
+        case FASTRACK_OPT_DIRECT_SMALL:      ctx->direct_small_h2d = value != 0; break;
+        case FASTRACK_OPT_PACK_MAX_BLOCKS:   ctx->plan.pack_max_blocks = (uint32_t)(value > FR_PACK_MAX_BLOCKS ? FR_PACK_MAX_BLOCKS : value); break;
+        case FASTRACK_OPT_PACK_RUN:          ctx->plan.pack_run_override = (uint32_t)(value > 0xFFFFFFFFull ? 0xFFFFFFFFull : value); break;
+        case FASTRACK_OPT_PACK_GROUP:        ctx->plan.pack_group_override = (uint32_t)(value > 0xFFFFFFFFull ? 0xFFFFFFFFull : value); break;
+        default: return FASTRACK_ERR_ARG;
+    }
+    return FASTRACK_OK;
 }
 
 extern "C" int fastrack_ctx_set_framing(fastrack_ctx* ctx, unsigned chains_per_sample)
@@ -495,13 +542,16 @@ static uint4 length_term(const fastrack_ctx* ctx, uint64_t bytes)
     return r;
 }
 
-// Fills the geometry of a launch into P: the row kernels' segment plan (fastrack_plan.h) and the per-sample layout.
-static void plan_segments(const fastrack_ctx* ctx, size_t sample_bytes, size_t n_chunks, FrParams& P)
+// Fills the geometry of a launch into P: the row kernels' plan (fastrack_plan.h) and the per-sample layout.
+static FrRowPlan plan_rows(const fastrack_ctx* ctx, size_t sample_bytes, size_t n_chunks, FrParams& P)
 {
-    const FrSegPlan seg = fr_plan_segments(ctx->plan, sample_bytes, n_chunks);
-    P.seg_rows = seg.seg_rows;
-    P.segs_per_chunk = seg.segs_per_chunk;
-    P.n_items = seg.n_items;
+    const FrRowPlan rows = fr_plan_rows(ctx->plan, sample_bytes, n_chunks);
+    P.n_slots = rows.n_slots;
+    P.warps_used = rows.warps_used;
+    P.rows_full = rows.rows_full;
+    P.rows_last = rows.rows_last;
+    P.rows_sample = rows.rows_sample;
+    P.total_rows = rows.total_rows;
     const size_t first_len = sample_bytes < ctx->chunk_bytes ? sample_bytes : ctx->chunk_bytes;
     const size_t cps = (sample_bytes + ctx->chunk_bytes - 1) / ctx->chunk_bytes;
     const size_t last_len = sample_bytes - (cps - 1) * ctx->chunk_bytes;     // a sample's last chunk may be short
@@ -509,17 +559,17 @@ static void plan_segments(const fastrack_ctx* ctx, size_t sample_bytes, size_t n
     P.chunks_per_sample = (uint32_t)cps;
     P.lenh_full = length_term(ctx, first_len);
     P.lenh_last = length_term(ctx, last_len);
+    return rows;
 }
 
-// Row kernels (false; plan_segments has filled P) or packed-row kernels (true; P is switched over to them)?
+// Row kernels (false) or packed-row kernels (true; P is switched over to them)?
 // fr_plan_packed decides; its last answer per kind of pass is kept, since callers repeat shapes.
-static bool plan_packed(fastrack_ctx* ctx, int mode, size_t sample_bytes, size_t n_chunks, FrParams& P)
+static bool plan_packed(fastrack_ctx* ctx, int mode, size_t sample_bytes, size_t n_chunks, const FrRowPlan& rows, FrParams& P)
 {
     const int kind = mode == FR_MODE_CTR ? FR_PASS_CTR : mode == FR_MODE_VERIFY ? FR_PASS_VERIFY : FR_PASS_FUSED;
     auto& memo = ctx->pack_memo[kind];
     if (!(memo.valid && memo.sample_bytes == sample_bytes && memo.n_chunks == n_chunks)) {
-        const FrSegPlan seg = {P.seg_rows, P.segs_per_chunk, P.n_items};
-        memo.plan = fr_plan_packed(ctx->plan, kind, sample_bytes, n_chunks, seg);
+        memo.plan = fr_plan_packed(ctx->plan, kind, sample_bytes, n_chunks, rows);
         memo.sample_bytes = sample_bytes;
         memo.n_chunks = n_chunks;
         memo.valid = true;
@@ -540,7 +590,11 @@ struct PassBuffers {
     const void* tags_in = nullptr;
     void* tags_out = nullptr;
     uint32_t* ok = nullptr;
-    int bank = 0;              // which half of the per-chunk scratch the pass uses
+    int bank = 0;              // which bank of combine records the pass uses (1: fastrack_verify)
+    int window = 0;            // which window of that bank: 0 = the caller's stream, 1 + i = internal stream i
+    uint32_t* acc_override = nullptr;   // combine records outside the context's own (fastrack_decrypt_verify_noalloc)
+    bool plain_launch = false;          // launch without the programmatic-dependency attribute
+    bool rows_only = false;             // never the packed-row kernels
     const void* ivs = nullptr; // batch of samples: per-sample IV bases on the device (then iv_base is unused)
     size_t sample_bytes = 0;   // batch of samples: bytes per sample (0: the launch is one plain buffer)
 };
@@ -568,10 +622,10 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
     const size_t n_chunks = (len / sample_bytes) * cps;            // len is a whole number of samples
     P.n_chunks = (uint32_t)n_chunks;
 
-    plan_segments(ctx, sample_bytes, n_chunks, P);
+    const FrRowPlan rows = plan_rows(ctx, sample_bytes, n_chunks, P);
     // Many short chains: one run of counters per lane (see fr_packed_body) when that is predicted to be faster.
-    const bool packed = (mode == FR_MODE_DEC || mode == FR_MODE_ENC || mode == FR_MODE_CTR || mode == FR_MODE_VERIFY) &&
-                        plan_packed(ctx, mode, sample_bytes, n_chunks, P);
+    const bool packed = !b.rows_only && (mode == FR_MODE_DEC || mode == FR_MODE_ENC || mode == FR_MODE_CTR || mode == FR_MODE_VERIFY) &&
+                        plan_packed(ctx, mode, sample_bytes, n_chunks, rows, P);
 
     P.in = (const uint8_t*)b.in;
     P.out = (uint8_t*)b.out;
@@ -589,21 +643,21 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
     const bool whole = packed && P.pack_run > full_blocks &&
                        (full_blocks <= 3 || n_chunks <= 2 * (size_t)ctx->num_sms * FR_THREADS);
     P.pow = ctx->d_pow;
-    if (!packed && mode != FR_MODE_CTR && mode != FR_MODE_PADGEN && P.segs_per_chunk > 1 &&
-        first_chunk + n_chunks > ctx->scratch_chunks) return FASTRACK_ERR_NOMEM;                // cannot happen, see ensure_scratch
-    uint32_t* bank = ctx->d_scratch + (size_t)b.bank * 5 * ctx->scratch_chunks;
-    P.acc = bank + 4 * first_chunk;
-    P.cnt = bank + 4 * ctx->scratch_chunks + first_chunk;
+    P.acc = b.acc_override ? b.acc_override
+                           : ctx->d_scratch + ((size_t)b.bank * FR_SCRATCH_WINDOWS + (size_t)b.window) * (size_t)ctx->num_sms * 8;
 
-    unsigned grid = (unsigned)ctx->num_sms;
-    if (P.n_items < grid) grid = P.n_items;
+    unsigned grid = rows.grid;
+    if (packed) {
+        grid = (unsigned)ctx->num_sms;
+        if (P.n_items < grid) grid = P.n_items;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(FR_THREADS);
-    cfg.dynamicSmemBytes = FR_SMEM_BYTES;
+    cfg.dynamicSmemBytes = packed ? FR_SMEM_BYTES : FR_SMEM_LAUNCH_BYTES;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
-    if (!ctx->no_overlap_launch) {
+    if (!ctx->no_overlap_launch && !b.plain_launch) {
         // let this kernel's table build overlap the tail of the previous kernel in the stream (see the kernel)
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -653,7 +707,7 @@ extern "C" int fastrack_decrypt_verify(fastrack_ctx* ctx, const uint8_t iv_base[
     if (bad_overlap(d_cipher, d_plain, len)) return FASTRACK_ERR_ARG;
     const size_t K = fastrack_num_chunks(ctx, len);
     if (K > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
-    int rc = ensure_scratch(ctx, K);
+    int rc = check_device(ctx);
     if (rc != FASTRACK_OK) return rc;
     PassBuffers b;
     b.in = d_cipher; b.out = d_plain; b.tags_in = d_tags; b.ok = d_ok;
@@ -670,7 +724,7 @@ extern "C" int fastrack_encrypt_tag(fastrack_ctx* ctx, const uint8_t iv_base[12]
     if (bad_overlap(d_cipher, d_plain, len)) return FASTRACK_ERR_ARG;
     const size_t K = fastrack_num_chunks(ctx, len);
     if (K > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
-    int rc = ensure_scratch(ctx, K);
+    int rc = check_device(ctx);
     if (rc != FASTRACK_OK) return rc;
     PassBuffers b;
     b.in = d_plain; b.out = d_cipher; b.tags_out = d_tags;
@@ -709,7 +763,7 @@ static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const vo
     const size_t n_samples = sample_bytes ? len / sample_bytes : 0;
     const size_t K = sample_bytes ? cps * n_samples : fastrack_num_chunks(ctx, len);
     if (K > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
-    int rc = ensure_scratch(ctx, K);
+    int rc = check_device(ctx);
     if (rc != FASTRACK_OK) return rc;
     const size_t need_slots = K + (12 * n_samples + 15) / 16;      // tags, then (batch of samples) the IV bases
     if (need_slots > ctx->tags_stage_chunks) {
@@ -759,6 +813,7 @@ static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const vo
         const bool tracing = ctx->trace_on;
         if (tracing) { cudaEventRecord(ctx->trace_ev[0], st); cudaEventRecord(ctx->trace_ev[1], st); }
         PassBuffers b;
+        b.window = 1;
         b.in = attr.devicePointer; b.out = d_plain; b.tags_in = tags_src; b.ok = d_ok;
         if (sample_bytes) { b.ivs = d_ivs; b.sample_bytes = sample_bytes; }
         rc = launch_pass(ctx, FR_MODE_DEC, iv_base, 0, len, b, st);
@@ -796,7 +851,7 @@ static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const vo
             if (e == cudaSuccess) e = cudaEventRecord(ctx->tags_ready, tag_stream);
             if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); rc = FASTRACK_ERR_CUDA; }
             if (rc == FASTRACK_OK && d_pad) {
-                PassBuffers pb;
+                PassBuffers pb;            // (no authentication in this pass: it uses no combine records)
                 pb.out = d_pad; pb.mask = d_mask;
                 rc = launch_pass(ctx, FR_MODE_PADGEN, iv_base, 0, len, pb, pad_stream);
                 if (rc == FASTRACK_OK && (e = cudaEventRecord(ctx->pad_ready, pad_stream)) != cudaSuccess) {
@@ -814,6 +869,7 @@ static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const vo
         }
         if (rc == FASTRACK_OK) {
             PassBuffers b;
+            b.window = 1 + (int)si;
             b.in = dst; b.out = dst; b.tags_in = ctx->d_tags_stage + k0; b.ok = d_ok + k0;
             if (sample_bytes) { b.ivs = d_ivs + 12 * (off / sample_bytes); b.sample_bytes = sample_bytes; }
             if (d_pad) { b.pad = (const uint8_t*)d_pad + off; b.mask = d_mask + k0; }
@@ -890,7 +946,7 @@ static int pipelined_d2h_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], cons
     const size_t n_samples = sample_bytes ? len / sample_bytes : 0;
     const size_t K = sample_bytes ? cps * n_samples : fastrack_num_chunks(ctx, len);
     if (K > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
-    int rc = ensure_scratch(ctx, K);
+    int rc = check_device(ctx);
     if (rc != FASTRACK_OK) return rc;
     const size_t need_slots = K + (12 * n_samples + 15) / 16;      // tags, then (batch of samples) the IV bases
     if (need_slots > ctx->tags_stage_chunks) {
@@ -930,6 +986,7 @@ static int pipelined_d2h_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], cons
             !misaligned(ta.devicePointer, 16)) tags_dst = ta.devicePointer;
         (void)cudaGetLastError();
         PassBuffers b;
+        b.window = 1;
         b.in = d_plain; b.out = attr.devicePointer; b.tags_out = tags_dst ? tags_dst : (void*)ctx->d_tags_stage;
         if (sample_bytes) { b.ivs = d_ivs; b.sample_bytes = sample_bytes; }
         rc = launch_pass(ctx, FR_MODE_ENC, iv_base, 0, len, b, st);
@@ -960,6 +1017,7 @@ static int pipelined_d2h_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], cons
             }
         }
         PassBuffers b;
+        b.window = 1 + (int)si;
         b.in = (const uint8_t*)d_plain + off; b.out = (uint8_t*)d_cipher + off; b.tags_out = ctx->d_tags_stage + k0;
         if (sample_bytes) { b.ivs = d_ivs + 12 * (off / sample_bytes); b.sample_bytes = sample_bytes; }
         if (rc == FASTRACK_OK) rc = launch_pass(ctx, FR_MODE_ENC, iv_base, k0, n, b, st);
@@ -1023,7 +1081,7 @@ extern "C" int fastrack_decrypt_verify_samples(fastrack_ctx* ctx, const void* d_
     if (!d_cipher || !d_tags || !d_plain || !d_ok) return FASTRACK_ERR_ARG;
     if (misaligned(d_cipher, 16) || misaligned(d_plain, 16) || misaligned(d_tags, 16) || misaligned(d_ok, 4)) return FASTRACK_ERR_ARG;
     if (bad_overlap(d_cipher, d_plain, len)) return FASTRACK_ERR_ARG;
-    rc = ensure_scratch(ctx, K);
+    rc = check_device(ctx);
     if (rc != FASTRACK_OK) return rc;
     PassBuffers b;
     b.in = d_cipher; b.out = d_plain; b.tags_in = d_tags; b.ok = d_ok; b.ivs = d_iv_bases; b.sample_bytes = sample_bytes;
@@ -1041,7 +1099,7 @@ extern "C" int fastrack_encrypt_tag_samples(fastrack_ctx* ctx, const void* d_iv_
     if (!d_plain || !d_cipher || !d_tags) return FASTRACK_ERR_ARG;
     if (misaligned(d_cipher, 16) || misaligned(d_plain, 16) || misaligned(d_tags, 16)) return FASTRACK_ERR_ARG;
     if (bad_overlap(d_cipher, d_plain, len)) return FASTRACK_ERR_ARG;
-    rc = ensure_scratch(ctx, K);
+    rc = check_device(ctx);
     if (rc != FASTRACK_OK) return rc;
     PassBuffers b;
     b.in = d_plain; b.out = d_cipher; b.tags_out = d_tags; b.ivs = d_iv_bases; b.sample_bytes = sample_bytes;
@@ -1056,6 +1114,8 @@ extern "C" int fastrack_ctr_crypt(fastrack_ctx* ctx, const uint8_t iv_base[12], 
     if (!d_in || !d_out) return FASTRACK_ERR_ARG;
     if (misaligned(d_in, 16) || misaligned(d_out, 16) || bad_overlap(d_in, d_out, len)) return FASTRACK_ERR_ARG;
     if (fastrack_num_chunks(ctx, len) > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
+    int rc = check_device(ctx);
+    if (rc != FASTRACK_OK) return rc;
     PassBuffers b;
     b.in = d_in; b.out = d_out;
     return launch_pass(ctx, FR_MODE_CTR, iv_base, 0, len, b, (cudaStream_t)stream);
@@ -1070,7 +1130,7 @@ extern "C" int fastrack_verify(fastrack_ctx* ctx, const uint8_t iv_base[12], con
     if (misaligned(d_cipher, 16) || misaligned(d_tags, 16) || misaligned(d_ok, 4)) return FASTRACK_ERR_ARG;
     const size_t K = fastrack_num_chunks(ctx, len);
     if (K > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
-    int rc = ensure_scratch(ctx, K);
+    int rc = check_device(ctx);
     if (rc != FASTRACK_OK) return rc;
     PassBuffers b;
     b.in = d_cipher; b.out = const_cast<void*>(d_cipher); b.tags_in = d_tags; b.ok = d_ok; b.bank = 1;
@@ -1086,6 +1146,8 @@ extern "C" int fastrack_verify_sequential(fastrack_ctx* ctx, const uint8_t iv_ba
     if (misaligned(d_cipher, 16) || misaligned(d_tags, 16) || misaligned(d_ok, 4)) return FASTRACK_ERR_ARG;
     const size_t K = fastrack_num_chunks(ctx, len);
     if (K > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
+    int rc = check_device(ctx);
+    if (rc != FASTRACK_OK) return rc;
     FrParams P;
     memset(&P, 0, sizeof P);
     memcpy(P.rk, ctx->rk, sizeof P.rk);
@@ -1117,6 +1179,8 @@ extern "C" int fastrack_keystream(fastrack_ctx* ctx, const uint8_t iv_base[12], 
     if (!d_pad || !d_mask) return FASTRACK_ERR_ARG;
     if (misaligned(d_pad, 16) || misaligned(d_mask, 16)) return FASTRACK_ERR_ARG;
     if (fastrack_num_chunks(ctx, len) > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
+    int rc = check_device(ctx);
+    if (rc != FASTRACK_OK) return rc;
     PassBuffers b;
     b.out = d_pad; b.mask = d_mask;
     return launch_pass(ctx, FR_MODE_PADGEN, iv_base, 0, len, b, (cudaStream_t)stream);
@@ -1134,7 +1198,7 @@ extern "C" int fastrack_xor_verify(fastrack_ctx* ctx, const uint8_t iv_base[12],
     if (bad_overlap(d_cipher, d_plain, len) || d_pad == d_plain || bad_overlap(d_pad, d_plain, len)) return FASTRACK_ERR_ARG;
     const size_t K = fastrack_num_chunks(ctx, len);
     if (K > 0xFFFFFFFFull) return FASTRACK_ERR_TOO_MANY;
-    int rc = ensure_scratch(ctx, K);
+    int rc = check_device(ctx);
     if (rc != FASTRACK_OK) return rc;
     PassBuffers b;
     b.in = d_cipher; b.out = d_plain; b.pad = d_pad; b.mask = const_cast<void*>(d_mask); b.tags_in = d_tags; b.ok = d_ok;
@@ -1143,10 +1207,11 @@ extern "C" int fastrack_xor_verify(fastrack_ctx* ctx, const uint8_t iv_base[12],
 
 // ------------------------------------------------------------- entry point that allocates nothing ----
 //
-// Per-chunk scratch for fastrack_decrypt_verify_noalloc: FASTRACK_NOALLOC_MAX_CHUNKS accumulators of four
-// words, then as many arrival counters.  It is part of the library image, so every GPU that loads the
-// library holds these 320 KiB until the process exits, and every call on a device shares them.
-static __device__ __align__(256) uint32_t fr_static_scratch[5 * FASTRACK_NOALLOC_MAX_CHUNKS];
+// Combine records for fastrack_decrypt_verify_noalloc: one 32-byte record per CTA of a launch (a launch has one
+// CTA per SM), FR_NOALLOC_MAX_CTAS of them.  The array is part of the library image, so every GPU that loads the
+// library holds these 32 KiB until the process exits, and every call on a device shares them.
+#define FR_NOALLOC_MAX_CTAS 1024
+static __device__ __align__(256) uint32_t fr_static_scratch[8 * FR_NOALLOC_MAX_CTAS];
 
 // In host code the array's name above is only a handle for the runtime, not a device address; the real
 // address differs per device and is looked up once per device with that device current.
@@ -1163,11 +1228,12 @@ extern "C" int fastrack_decrypt_verify_noalloc(fastrack_ctx* ctx, const uint8_t 
     if (misaligned(d_cipher, 16) || misaligned(d_plain, 16) || misaligned(d_tags, 16) || misaligned(d_ok, 4)) return FASTRACK_ERR_ARG;
     if (bad_overlap(d_cipher, d_plain, len)) return FASTRACK_ERR_ARG;
     const size_t K = fastrack_num_chunks(ctx, len);
-    if (K > FASTRACK_NOALLOC_MAX_CHUNKS) return FASTRACK_ERR_LIMIT;
+    if (K > FASTRACK_NOALLOC_MAX_CHUNKS || ctx->num_sms > FR_NOALLOC_MAX_CTAS) return FASTRACK_ERR_LIMIT;
 
-    int dev = -1;
-    FR_CUDA(ctx, cudaGetDevice(&dev));
-    if (dev != ctx->device || dev < 0 || dev >= FR_MAX_DEVICES) return FASTRACK_ERR_ARG;
+    int rc = check_device(ctx);
+    if (rc != FASTRACK_OK) return rc;
+    const int dev = ctx->device;
+    if (dev < 0 || dev >= FR_MAX_DEVICES) return FASTRACK_ERR_ARG;
     if (!fr_static_scratch_addr[dev]) {                 // first call on this device: resolve the symbol
         uint32_t* ptr = nullptr;
         FR_CUDA(ctx, cudaGetSymbolAddress((void**)&ptr, fr_static_scratch));
@@ -1175,38 +1241,15 @@ extern "C" int fastrack_decrypt_verify_noalloc(fastrack_ctx* ctx, const uint8_t 
         fr_static_scratch_addr[dev] = ptr;
     }
     uint32_t* acc = fr_static_scratch_addr[dev];
-    uint32_t* cnt = acc + 4 * (size_t)FASTRACK_NOALLOC_MAX_CHUNKS;
     cudaStream_t st = (cudaStream_t)stream;
-    // the array keeps whatever the previous call (possibly a failed one) left: zero what this call will use
-    FR_CUDA(ctx, cudaMemsetAsync(acc, 0, K * 4 * sizeof(uint32_t), st));
-    FR_CUDA(ctx, cudaMemsetAsync(cnt, 0, K * sizeof(uint32_t), st));
-
-    // same launch geometry as the allocating entry point, scratch pointers aside
-    FrParams P;
-    memset(&P, 0, sizeof P);
-    memcpy(P.rk, ctx->rk, sizeof P.rk);
-    P.iv_w0 = load_le32(iv_base);
-    P.iv_w1 = load_le32(iv_base + 4);
-    P.iv_ctr = load_be32(iv_base + 8);
-    P.aad_mod = ctx->aad_mod;
-    P.generic_smem = ctx->generic_smem;
-    P.len = len;
-    P.chunk_bytes = ctx->chunk_bytes;
-    P.n_chunks = (uint32_t)K;
-    plan_segments(ctx, len, K, P);
-    P.in = (const uint8_t*)d_cipher;
-    P.out = (uint8_t*)d_plain;
-    P.tags_in = (const uint4*)d_tags;
-    P.ok = d_ok;
-    P.te0 = ctx->d_te0;
-    P.gh_tab = ctx->d_gh_tab;
-    P.pow = ctx->d_pow;
-    P.acc = acc;
-    P.cnt = cnt;
-    unsigned grid = (unsigned)ctx->num_sms;
-    if (P.n_items < grid) grid = P.n_items;
-    fr_crypt_kernel<FR_MODE_DEC><<<grid, FR_THREADS, FR_SMEM_BYTES, st>>>(P);
-    ctx->launches++;
-    FR_CUDA(ctx, cudaGetLastError());
-    return FASTRACK_OK;
+    // the array keeps whatever the previous call (possibly a failed one) left: zero what this call may use, one
+    // 32-byte record per CTA of the launch
+    FR_CUDA(ctx, cudaMemsetAsync(acc, 0, (size_t)ctx->num_sms * 8 * sizeof(uint32_t), st));
+    // same launch as the allocating entry point, combine records aside
+    PassBuffers b;
+    b.in = d_cipher; b.out = d_plain; b.tags_in = d_tags; b.ok = d_ok;
+    b.acc_override = acc;
+    b.plain_launch = true;
+    b.rows_only = true;
+    return launch_pass(ctx, FR_MODE_DEC, iv_base, 0, len, b, st);
 }

@@ -1,6 +1,6 @@
 // fastrack_device.cuh -- per-lane device code of the fused AES-256-CTR + GHASH pass (sm_100a).
 //
-// One warp works on one "segment": a run of consecutive rows of one chunk.  A row is 32 consecutive counter
+// One warp works on one "segment" at a time: a run of consecutive rows of one chunk.  A row is 32 consecutive counter
 // values, lane = counter mod 32, and the block at counter c is data block c - 2 of the chunk (GCM keeps
 // counter 1 for the tag mask), so a row is 512 contiguous bytes and global loads and stores are 128-bit and
 // coalesced.  Counter 1 of row 0 is a spare lane: it yields E_K(J0), and with the serial-number framing it
@@ -32,7 +32,9 @@
 #define FR_SM_T01 0u          // AES rows [Te0 x32 | Te1 x32]
 #define FR_SM_T23 65536u      // AES rows [Te2 x32 | Te3 x32]
 #define FR_SM_GH 131072u      // byte tables of H^32
-#define FR_SMEM_BYTES 196608u
+#define FR_SMEM_BYTES 196608u // the three tables
+#define FR_SM_COMB 196608u    // row kernels: 33 records of 8 words in which the warps of a CTA combine their pieces of a chunk
+#define FR_SMEM_LAUNCH_BYTES (FR_SMEM_BYTES + 2048u)   // dynamic shared memory of a launch: the tables and the records
 
 // What one pass does.  DEC / ENC are the fused passes.  CTR and VERIFY split them (paper Section 4.3, eager
 // evaluation: plaintext first, authentication later).  PADGEN / PADDEC split the keystream from the XOR
@@ -47,6 +49,24 @@ enum FrMode : int {
 };
 
 #define FR_ROW_BLOCKS 32u     // blocks per row (one per lane)
+
+// Timing probes of a diagnostic build (-DFR_STAMPS): per CTA, clock values at the phases of the kernel.  The
+// library proper is built without the flag and contains none of this.
+#ifdef FR_STAMPS
+__device__ unsigned long long fr_stamps[1024 * 8];
+__device__ __forceinline__ unsigned long long fr_gtime() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define FR_STAMP_SET(i) do { if (threadIdx.x == 0) fr_stamps[blockIdx.x * 8 + (i)] = (unsigned long long)clock64(); } while (0)
+#define FR_STAMP_GT(i) do { if (threadIdx.x == 0) fr_stamps[blockIdx.x * 8 + (i)] = fr_gtime(); } while (0)
+#define FR_STAMP_MIN(i) do { if ((threadIdx.x & 31u) == 0) atomicMin(&fr_stamps[blockIdx.x * 8 + (i)], (unsigned long long)clock64()); } while (0)
+#define FR_STAMP_MAX(i) do { if ((threadIdx.x & 31u) == 0) atomicMax(&fr_stamps[blockIdx.x * 8 + (i)], (unsigned long long)clock64()); } while (0)
+#define FR_STAMP_GTMAX(i) do { if ((threadIdx.x & 31u) == 0) atomicMax(&fr_stamps[blockIdx.x * 8 + (i)], fr_gtime()); } while (0)
+#else
+#define FR_STAMP_SET(i) do { } while (0)
+#define FR_STAMP_GT(i) do { } while (0)
+#define FR_STAMP_MIN(i) do { } while (0)
+#define FR_STAMP_MAX(i) do { } while (0)
+#define FR_STAMP_GTMAX(i) do { } while (0)
+#endif
 #define FR_HORNER_STRIDE 32u  // the fixed multiplier is H^32
 
 struct FrParams {
@@ -54,15 +74,19 @@ struct FrParams {
     uint32_t iv_w0, iv_w1;     // little-endian loads of iv_base[0..3], iv_base[4..7]
     uint32_t iv_ctr;           // BE32(iv_base[8..11]) + index of this launch's first chunk
     uint32_t first_chunk;      // index of this launch's first chunk in the caller's buffer
-    uint32_t seg_rows;         // rows per segment
-    uint32_t segs_per_chunk;   // segments of a full-size chunk
+    uint32_t n_slots;          // row kernels: warps that take work; slot j is warp j % warps_used of CTA j / warps_used
+    uint32_t warps_used;       // row kernels: slots per CTA
     uint32_t n_chunks;         // chunks in this launch
-    uint32_t n_items;          // n_chunks * segs_per_chunk
+    uint32_t n_items;          // packed rows: work items
     uint32_t generic_smem;     // 1: use the portable shared-memory addressing even where the absolute form would do
     uint32_t aad_mod;          // 0: no AAD; n: a chunk authenticates the one byte (its serial number mod n) as AAD
     uint64_t len;              // bytes in this launch
     uint64_t chunk_bytes;
     uint64_t sample_bytes;     // the launch is a sequence of equal samples of this many bytes (one sample: = len)
+    uint64_t total_rows;       // row kernels: rows of all chunks of the launch together
+    uint64_t rows_sample;      // rows of one sample: (chunks_per_sample - 1) * rows_full + rows_last
+    uint32_t rows_full;        // rows of a full-size chunk
+    uint32_t rows_last;        // rows of a sample's last chunk
     uint32_t chunks_per_sample;  // ceil(sample_bytes / chunk_bytes); only a sample's last chunk may be short
     uint32_t pack_chunks;        // packed rows: chunks per work item; then n_items = ceil(n_chunks / pack_chunks)
     uint32_t pack_run;           // packed rows: consecutive counters per slot (lane)
@@ -76,8 +100,7 @@ struct FrParams {
     const uint32_t* te0;       // 256 words
     const uint4* gh_tab;       // 4096 entries, same layout as shared memory
     const uint4* pow;          // pow[e] = H^e
-    uint32_t* acc;             // per chunk 4 words, zero between launches
-    uint32_t* cnt;             // per chunk arrival counter, zero between launches
+    uint32_t* acc;             // per CTA of the launch a record of 8 words (4-word XOR accumulator, arrival counter, 3 unused), zero between launches
     const uint8_t* pad;        // FR_MODE_PADDEC: keystream made ahead of time, same layout as the data
     uint4* mask;               // E_K(J0) per chunk: written by FR_MODE_PADGEN, read by FR_MODE_PADDEC
     uint4 lenh_full;           // (BE64(0) || BE64(8 * chunk_bytes)) * H: the length block's term of a full chunk
@@ -417,22 +440,65 @@ __device__ __forceinline__ FrChunk fr_chunk_info(const FrParams& P, uint32_t kk)
     return c;
 }
 
-__device__ __forceinline__ uint64_t fr_chunk_len(const FrParams& P, uint32_t kk)
-{
-    const uint32_t k = kk % P.chunks_per_sample;
-    const uint64_t rem = P.sample_bytes - (uint64_t)k * P.chunk_bytes;
-    return rem < P.chunk_bytes ? rem : P.chunk_bytes;
-}
-
 // Rows are aligned to the COUNTER, not to the block index: row r of a chunk holds counters 32r .. 32r+31,
 // lane = counter mod 32.  Data block j uses counter j + 2, so row 0 carries 30 data blocks; its lane 1
 // (counter 1) produces E_K(J0), the tag mask, as a by-product and lane 0 idles.
 __device__ __forceinline__ uint32_t fr_chunk_rows(uint32_t nblk) { return (nblk + 2u + FR_ROW_BLOCKS - 1) / FR_ROW_BLOCKS; }
 
-__device__ __forceinline__ uint32_t fr_chunk_segs(const FrParams& P, uint32_t kk)
+// Work distribution of the row kernels.  The rows of all chunks of a launch, one chunk after the other, form
+// one row space of total_rows rows; it is cut into n_slots contiguous, equally long (to within one row) ranges and
+// slot j -- warp j % warps_used of CTA j / warps_used -- walks range j.  Where a range crosses a chunk boundary the
+// warp closes one segment and opens the next, so a chunk may be covered by one warp, by several warps of one CTA
+// or by several CTAs; the kernel combines the pieces in shared memory and, across CTAs, in global memory.
+// Requires n_slots <= total_rows (no empty range).
+__device__ __forceinline__ uint64_t fr_slot_begin(const FrParams& P, uint32_t j)        // j in 0 .. n_slots
 {
-    uint32_t nblk = (uint32_t)((fr_chunk_len(P, kk) + 15) >> 4);
-    return (fr_chunk_rows(nblk) + P.seg_rows - 1) / P.seg_rows;
+    return (uint64_t)j * P.total_rows / P.n_slots;
+}
+
+__device__ __forceinline__ uint32_t fr_slot_of_row(const FrParams& P, uint64_t g)      // the j with begin(j) <= g < begin(j + 1)
+{
+    return (uint32_t)(((g + 1u) * P.n_slots - 1u) / P.total_rows);
+}
+
+struct FrRowPos {
+    uint32_t kk;        // chunk of the launch
+    uint32_t r;         // row inside the chunk
+    uint32_t rows_k;    // rows of that chunk
+};
+
+__device__ __forceinline__ FrRowPos fr_locate_row(const FrParams& P, uint64_t g)
+{
+    const uint64_t sample = g / P.rows_sample, rem = g - sample * P.rows_sample;
+    const uint32_t k = (uint32_t)(rem / P.rows_full);           // at most chunks_per_sample - 1: the last chunk is not longer than the others
+    FrRowPos p;
+    p.kk = (uint32_t)sample * P.chunks_per_sample + k;
+    p.r = (uint32_t)(rem - (uint64_t)k * P.rows_full);
+    p.rows_k = (k + 1u == P.chunks_per_sample) ? P.rows_last : P.rows_full;
+    return p;
+}
+
+// Who else works on the chunk whose rows are [g0, g0 + rows_k) of the row space, seen from a warp of the CTA that
+// holds slots cta_first .. cta_last: how many warps of this CTA (n_in_cta; they are consecutive), which of the CTA's
+// 33 shared-memory records they meet in (the warp in which the chunk begins, or record 32 if it began in an
+// earlier CTA), the first CTA that works on it (its record in global memory is the meeting point across CTAs) and
+// how many CTAs do.  A warp's range holds the beginning of at most one chunk that continues beyond it, and at most
+// one chunk reaches into a CTA from before, so no record is used by two chunks in one launch.
+struct FrShare {
+    uint32_t n_in_cta, rec, first_cta, n_ctas;
+};
+
+__device__ __forceinline__ FrShare fr_chunk_share(const FrParams& P, uint64_t g0, uint32_t rows_k, uint32_t cta_first,
+                                                  uint32_t cta_last)
+{
+    const uint32_t sa = fr_slot_of_row(P, g0), sb = fr_slot_of_row(P, g0 + rows_k - 1u);
+    const uint32_t a = sa > cta_first ? sa : cta_first, b = sb < cta_last ? sb : cta_last;
+    FrShare s;
+    s.n_in_cta = b - a + 1u;
+    s.rec = sa < cta_first ? 32u : sa - cta_first;
+    s.first_cta = sa / P.warps_used;
+    s.n_ctas = sb / P.warps_used - s.first_cta + 1u;
+    return s;
 }
 
 // Load / store the last, partial block of the buffer byte by byte (zero-padded in registers).
@@ -460,14 +526,14 @@ __device__ __forceinline__ uint4 fr_mask_bytes(uint4 v, uint32_t n)
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-// One lane's share of segment s of chunk kk: decrypt (or encrypt) its blocks, fold them into the
+// One lane's share of rows row0 .. row1 - 1 of chunk kk: decrypt (or encrypt) its blocks, fold them into the
 // lane's Horner value, and return that value multiplied by the power of H that aligns it to the end
 // of the chunk (lane 1 of the chunk's first segment adds E_K(J0)).  XOR of the 32 lanes' results over all
 // segments of the chunk = GHASH of the data blocks (before the length block) xor E_K(J0).
 // Modes without GHASH (CTR, PADGEN) return zero.
 template <int MODE, bool ABS>
 __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, const char* sm, const FrLane& L,
-                                                         uint32_t lane, uint32_t kk, uint32_t s)
+                                                         uint32_t lane, uint32_t kk, uint32_t row0, uint32_t row1)
 {
     constexpr bool DO_AES = MODE == FR_MODE_DEC || MODE == FR_MODE_ENC || MODE == FR_MODE_CTR || MODE == FR_MODE_PADGEN;
     constexpr bool DO_GHASH = MODE == FR_MODE_DEC || MODE == FR_MODE_ENC || MODE == FR_MODE_VERIFY || MODE == FR_MODE_PADDEC;
@@ -478,10 +544,6 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
     const uint64_t chunk_off = ck.off;
     const uint64_t len_k = ck.len;
     const uint32_t nblk = (uint32_t)((len_k + 15) >> 4);
-    const uint32_t rows = fr_chunk_rows(nblk);
-    const uint32_t row0 = s * P.seg_rows;
-    uint32_t row1 = row0 + P.seg_rows;
-    if (row1 > rows) row1 = rows;
     uint32_t seg_end = row1 * FR_ROW_BLOCKS - 2u;   // first block index after this segment
     if (seg_end > nblk) seg_end = nblk;
     const uint8_t* in = P.in + chunk_off;
@@ -548,6 +610,7 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
             }
         }
     }
+    FR_STAMP_MIN(3); FR_STAMP_MAX(4);
     if (!DO_GHASH) return make_uint4(0, 0, 0, 0);
     if (c_last == 0u) return extra;
     return fr_xor4(fr_gf128_mul(pend, hpow), extra);

@@ -1,6 +1,6 @@
 // fastrack_plan.h -- host-side planning of a launch and of a pipelined transfer: plain C++ without CUDA, so that
 // the CPU-only tests can include it and check its invariants (tests/host_logic).  Three decisions are made here:
-//   fr_plan_segments: how the row kernels cut chunks into segments (one warp per segment);
+//   fr_plan_rows:     how the row kernels spread the rows of a launch over warps;
 //   fr_plan_packed:   whether a launch takes the packed-row kernels instead, and with which run length and
 //                     work-item size;
 //   fr_plan_stages:   how a pipelined host<->device transfer is cut into stages.
@@ -19,17 +19,23 @@
 struct FrPlanConfig {
     int num_sms;
     size_t chunk_bytes;
-    uint32_t seg_rows_override;     // 0 = automatic (FASTRACK_SEG_ROWS, for experiments)
-    uint32_t pack_max_blocks;       // chunks of at most this many blocks may take the packed-row kernels (FASTRACK_PACK_MAX_BLOCKS; 0 = never)
-    uint32_t pack_run_override;     // 0 = automatic; else packed rows with this run length wherever they apply (FASTRACK_PACK_RUN, tests)
-    uint32_t pack_group_override;   // 0 = automatic; else this many chunks per packed work item (FASTRACK_PACK_GROUP, tests)
-    size_t stage_bytes_override;    // 0 = automatic (FASTRACK_STAGE_BYTES, for experiments)
+    uint32_t row_slots_override;    // 0 = automatic; else the row kernels spread a launch over this many warps (tests, tuning)
+    uint32_t pack_max_blocks;       // chunks of at most this many blocks may take the packed-row kernels (0 = never)
+    uint32_t pack_run_override;     // 0 = automatic; else packed rows with this run length wherever they apply (tests)
+    uint32_t pack_group_override;   // 0 = automatic; else this many chunks per packed work item (tests)
+    size_t stage_bytes_override;    // 0 = automatic; else the stage size of pipelined transfers (experiments)
 };
 
-struct FrSegPlan {
-    uint32_t seg_rows;          // rows per segment
-    uint32_t segs_per_chunk;    // segments of a full-size chunk
-    uint32_t n_items;           // segs_per_chunk * n_chunks
+// How the row kernels spread a launch over warps: the rows of all chunks, one chunk after the other, are cut into
+// n_slots contiguous ranges of equal length (to within a row); slot j is warp j % warps_used of CTA j / warps_used.
+struct FrRowPlan {
+    uint32_t grid;              // CTAs
+    uint32_t warps_used;        // slots per CTA (the other warps of a CTA only help to fill shared memory)
+    uint32_t n_slots;           // <= grid * warps_used and <= total_rows
+    uint32_t rows_full;         // rows of a full-size chunk
+    uint32_t rows_last;         // rows of a sample's last chunk
+    uint64_t rows_sample;       // rows of a sample
+    uint64_t total_rows;
 };
 
 struct FrPackPlan {
@@ -40,50 +46,41 @@ struct FrPackPlan {
 
 enum FrPassKind : int { FR_PASS_FUSED = 0, FR_PASS_CTR = 1, FR_PASS_VERIFY = 2 };
 
-// Segment geometry of a launch over n_chunks chunks of samples of `sample_bytes` bytes (a plain buffer is one
-// sample): rows are aligned to the counter (block j sits at counter j + 2), segments longer than four rows are
-// whole multiples of 8 rows so that they start on a 256-counter group.
-static inline FrSegPlan fr_plan_segments(const FrPlanConfig& cfg, size_t sample_bytes, size_t n_chunks)
+// Rows of a chunk of `bytes` bytes: rows are aligned to the counter and block j sits at counter j + 2.
+static inline uint32_t fr_rows_of(size_t bytes)
 {
+    return (uint32_t)(((bytes + 15) / 16 + 2 + FR_PLAN_ROW_BLOCKS - 1) / FR_PLAN_ROW_BLOCKS);
+}
+
+// Row-kernel geometry of a launch over n_chunks chunks of samples of `sample_bytes` bytes (a plain buffer is one
+// sample).  Every warp that takes work pays one closing GF(2^128) product per chunk it touches, at least one; a
+// warp's rows run one after the other.  So a launch of T rows on S SMs wants about sqrt(T / S) warps per SM: more
+// warps shorten the row sequence of each, fewer warps mean fewer closings -- up to the 32 a CTA has, from about
+// 64 MiB on.  (Fitted on B200: best rows per warp 3 / 4 / 6 / 9 / 13 at 1 / 2 / 4 / 8 / 16 MiB.)
+static inline FrRowPlan fr_plan_rows(const FrPlanConfig& cfg, size_t sample_bytes, size_t n_chunks)
+{
+    FrRowPlan p;
+    const size_t cps = (sample_bytes + cfg.chunk_bytes - 1) / cfg.chunk_bytes;
     const size_t first_len = sample_bytes < cfg.chunk_bytes ? sample_bytes : cfg.chunk_bytes;
-    const size_t rows_ref = ((first_len + 15) / 16 + 2 + FR_PLAN_ROW_BLOCKS - 1) / FR_PLAN_ROW_BLOCKS;
-    const size_t warps = (size_t)cfg.num_sms * FR_WARPS;
-    // Segments are dealt round-robin to the resident warps.  Two things bound a launch: the latency of the
-    // busiest warp (about 1000 cycles per row when few warps run, plus about 4000 per segment for the closing
-    // GF(2^128) product, the atomics and the tag), and the shared-memory work of the busiest SM (about 270
-    // wavefront-cycles per row plus about 300 per segment).  Try short segments (2 or 4 rows, for small buffers)
-    // and 1..8 segments per warp in whole 8-row groups, and keep the split with the smaller bound.
-    size_t seg_rows = 8, spc = (rows_ref + 7) / 8;
-    if (cfg.seg_rows_override) {
-        seg_rows = cfg.seg_rows_override;
-        spc = (rows_ref + seg_rows - 1) / seg_rows;
+    p.rows_full = fr_rows_of(first_len);
+    p.rows_last = fr_rows_of(sample_bytes - (cps - 1) * cfg.chunk_bytes);
+    p.rows_sample = (uint64_t)(cps - 1) * p.rows_full + p.rows_last;
+    p.total_rows = (uint64_t)(n_chunks / cps) * p.rows_sample;
+    const uint64_t sms = (uint64_t)cfg.num_sms, cap = sms * FR_WARPS;
+    uint64_t slots;
+    if (cfg.row_slots_override) {
+        slots = cfg.row_slots_override;
     } else {
-        size_t best_cost = ~(size_t)0;
-        for (int cand = 0; cand < 10; cand++) {
-            size_t rows;
-            if (cand < 2) {
-                rows = cand == 0 ? 2 : 4;
-            } else {
-                size_t want = (size_t)(cand - 1) * warps / n_chunks;
-                if (want < 1) want = 1;
-                rows = ((rows_ref + want - 1) / want + 7) / 8 * 8;
-                if (rows > 1024) rows = 1024;
-            }
-            const size_t per_chunk = (rows_ref + rows - 1) / rows;
-            const size_t items = per_chunk * n_chunks;
-            const size_t waves = (items + warps - 1) / warps;
-            const size_t per_sm = (items + (size_t)cfg.num_sms - 1) / (size_t)cfg.num_sms;
-            const size_t latency = waves * (rows * 1000 + 4000);
-            const size_t throughput = per_sm * (rows * 270 + 300);
-            const size_t cost = latency > throughput ? latency : throughput;
-            if (cost < best_cost) { best_cost = cost; seg_rows = rows; spc = per_chunk; }
-        }
+        uint64_t wu = 1;                                              // about 1.18 * sqrt(T / S), by squares
+        while (wu < FR_WARPS && (wu + 1) * (wu + 1) * 100 <= 139 * p.total_rows / sms) wu++;
+        slots = sms * wu;
     }
-    while (spc * n_chunks >= ((size_t)1 << 31)) { seg_rows *= 2; spc = (rows_ref + seg_rows - 1) / seg_rows; }
-    FrSegPlan p;
-    p.seg_rows = (uint32_t)seg_rows;
-    p.segs_per_chunk = (uint32_t)spc;
-    p.n_items = (uint32_t)(spc * n_chunks);
+    if (slots > cap) slots = cap;
+    if (slots > p.total_rows) slots = p.total_rows;
+    if (slots < 1) slots = 1;
+    p.n_slots = (uint32_t)slots;
+    p.warps_used = (uint32_t)((slots + sms - 1) / sms);
+    p.grid = (uint32_t)((slots + p.warps_used - 1) / p.warps_used);
     return p;
 }
 
@@ -95,7 +92,7 @@ struct FrPackCosts {
     size_t step_long;                                     // ... for longer runs
 };
 
-// Decides between the row kernels (`seg` is their plan) and the packed-row kernels, and in the latter case picks
+// Decides between the row kernels (`rows` is their plan) and the packed-row kernels, and in the latter case picks
 // the run length and the work-item size.  Both are judged by the same kind of estimate: the shared-memory work of
 // the busiest SM or the latency of the busiest warp, whichever is larger (plus a quarter of the other: between the
 // two regimes both show).  For the fused passes a row kernel costs about 285 clocks per row plus 400 per segment;
@@ -104,7 +101,7 @@ struct FrPackCosts {
 // whose byte stride is a power of two do worst: the lanes' pieces fall on the same few cache banks).  The two
 // halves of the fused pass have constants of their own.
 static inline FrPackPlan fr_plan_packed(const FrPlanConfig& cfg, int kind, size_t sample_bytes, size_t n_chunks,
-                                        const FrSegPlan& seg)
+                                        const FrRowPlan& rows)
 {
     static const FrPackCosts costs[3] = {
         // fused passes: cipher + Horner step per counter, one general product per run
@@ -123,10 +120,12 @@ static inline FrPackPlan fr_plan_packed(const FrPlanConfig& cfg, int kind, size_
     const size_t sms = (size_t)cfg.num_sms, warps = sms * FR_WARPS;
     if (!cfg.pack_run_override && counters > 32 && n_chunks * 8 < warps) return rows_kernels;   // a few long chains: rows, no search needed
 
-    const size_t rows_ref = (counters + 1 + FR_PLAN_ROW_BLOCKS - 1) / FR_PLAN_ROW_BLOCKS;
-    const size_t waves = ((size_t)seg.n_items + warps - 1) / warps;
-    const size_t row_thr = (n_chunks * rows_ref + sms - 1) / sms * C.row_clocks + ((size_t)seg.n_items + sms - 1) / sms * C.seg_clocks;
-    const size_t row_lat = waves * ((size_t)seg.seg_rows * C.row_step_latency + 4000);
+    // row kernels: every slot closes one segment per chunk it touches
+    const size_t pieces = (size_t)rows.n_slots + n_chunks;
+    const size_t rows_per_slot = (size_t)((rows.total_rows + rows.n_slots - 1) / rows.n_slots);
+    const size_t segs_per_slot = (pieces + rows.n_slots - 1) / rows.n_slots;
+    const size_t row_thr = (size_t)((rows.total_rows + sms - 1) / sms) * C.row_clocks + (pieces + sms - 1) / sms * C.seg_clocks;
+    const size_t row_lat = rows_per_slot * C.row_step_latency + segs_per_slot * 4000;
     const size_t row_cost = row_thr > row_lat ? row_thr : row_lat;
 
     size_t best_run = 0, best_group = 1, best_cost = ~(size_t)0;

@@ -18,7 +18,11 @@ ERR_ARG, ERR_CHUNK, ERR_NOT_PINNED, ERR_CUDA, ERR_NOMEM, ERR_TOO_MANY, ERR_LIMIT
 NOALLOC_MAX_CHUNKS = 16384
 MAX_CHUNK_BYTES = 1 << 30
 
-EXPORTS = ("fastrack_ctx_create", "fastrack_ctx_destroy", "fastrack_num_chunks", "fastrack_ctx_reserve",
+# fastrack_ctx_set_option: test and tuning controls (the library reads no environment variable)
+OPT_ROW_SLOTS, OPT_GENERIC_SMEM, OPT_NO_OVERLAP_LAUNCH, OPT_STAGE_BYTES = 1, 2, 3, 4
+OPT_DIRECT_SMALL, OPT_PACK_MAX_BLOCKS, OPT_PACK_RUN, OPT_PACK_GROUP = 5, 6, 7, 8
+
+EXPORTS = ("fastrack_ctx_create", "fastrack_ctx_destroy", "fastrack_num_chunks", "fastrack_ctx_reserve", "fastrack_ctx_set_option",
            "fastrack_last_cuda_error", "fastrack_decrypt_verify", "fastrack_encrypt_tag",
            "fastrack_pipelined_h2d", "fastrack_launch_count", "fastrack_decrypt_verify_noalloc",
            "fastrack_ctr_crypt", "fastrack_verify", "fastrack_keystream", "fastrack_xor_verify",
@@ -40,6 +44,8 @@ _lib.fastrack_num_chunks.restype = _sz
 _lib.fastrack_num_chunks.argtypes = [_vp, _sz]
 _lib.fastrack_ctx_reserve.restype = _int
 _lib.fastrack_ctx_reserve.argtypes = [_vp, _sz]
+_lib.fastrack_ctx_set_option.restype = _int
+_lib.fastrack_ctx_set_option.argtypes = [_vp, _int, ctypes.c_uint64]
 _lib.fastrack_ctx_set_framing.restype = _int
 _lib.fastrack_ctx_set_framing.argtypes = [_vp, ctypes.c_uint]
 class StageTrace(ctypes.Structure):
@@ -111,6 +117,10 @@ def fastrack_num_chunks(ctx, length: int) -> int:
 
 def fastrack_ctx_reserve(ctx, max_len: int) -> int:
     return _lib.fastrack_ctx_reserve(ctx, max_len)
+
+
+def fastrack_ctx_set_option(ctx, option: int, value: int) -> int:
+    return _lib.fastrack_ctx_set_option(ctx, option, value)
 
 
 def fastrack_ctx_set_framing(ctx, chains_per_sample: int) -> int:
@@ -220,12 +230,18 @@ def fastrack_pipelined_d2h(ctx, iv_base: bytes, d_plain: int, length: int, d_cip
 class Context:
     """RAII wrapper: ``with Context(key, chunk_bytes) as ctx: ctx.decrypt_verify(...)``; raises FastrackError."""
 
-    def __init__(self, key: bytes, chunk_bytes: int):
+    def __init__(self, key: bytes, chunk_bytes: int, options=None):
+        """options: {OPT_*: value} passed to fastrack_ctx_set_option right after creation (tests, tuning)."""
         rc, handle = fastrack_ctx_create(key, chunk_bytes)
         if rc != OK:
             raise FastrackError(rc)
         self.handle = handle
         self.chunk_bytes = chunk_bytes
+        for option, value in (options or {}).items():
+            self.set_option(option, value)
+
+    def set_option(self, option: int, value: int) -> None:
+        self._check(fastrack_ctx_set_option(self.handle, option, value))
 
     def _check(self, rc: int) -> None:
         if rc != OK:

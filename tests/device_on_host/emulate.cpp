@@ -11,6 +11,9 @@
 #include <string.h>
 
 #include <algorithm>
+#include <map>
+#include <set>
+#include <utility>
 #include <vector>
 
 // ---- what the device header needs from CUDA, as plain C++ ----
@@ -44,6 +47,7 @@ static inline uint32_t __brev(uint32_t x)
 
 #include "../../paper_2410_15240_b200/csrc/fastrack_device.cuh"
 #include "../../paper_2410_15240_b200/csrc/fastrack_keysetup.h"
+#include "../../paper_2410_15240_b200/csrc/fastrack_plan.h"
 using namespace fr_host;
 
 namespace {
@@ -114,27 +118,77 @@ uint4 length_term(const Setup& S, uint64_t bytes, uint32_t aad_mod)
     return r;
 }
 
+// The row kernels' work distribution, slot by slot as fr_crypt_body walks it (the slots stand for warps), with
+// the XOR of the pieces of a chunk done in a plain array instead of the shared-memory and global records.  What the
+// kernel derives from fr_chunk_share -- how many warps of the CTA and how many CTAs meet on a chunk, and in which
+// record -- is checked here against what the walk really does.  Returns 0, or a code that says which check failed.
 template <int MODE>
-void run_pass(Setup& S, uint32_t n_chunks, std::vector<uint4>& acc)
+int run_pass(Setup& S, std::vector<uint4>& acc)
 {
-    for (uint32_t item = 0; item < S.P.n_items; item++) {
-        const uint32_t kk = item / S.P.segs_per_chunk, s = item - kk * S.P.segs_per_chunk;
-        if (s >= fr_chunk_segs(S.P, kk)) continue;
-        for (uint32_t lane = 0; lane < 32; lane++) {                        // the warp, one lane after the other
-            const FrLane L = fr_make_lane(lane);
-            acc[kk] = fr_xor4(acc[kk], fr_process_segment_lane<MODE, false>(S.P, S.sm.data(), L, lane, kk, s));
+    const FrParams& P = S.P;
+    struct Piece { uint32_t slot; uint64_t g0; uint32_t rows_k; };
+    std::map<uint32_t, std::vector<Piece>> partial;          // chunk -> pieces of it that are not the whole chunk
+    std::vector<uint32_t> pieces_of(P.n_chunks, 0);
+    std::vector<uint64_t> rows_done(P.n_chunks, 0);
+    if (P.n_slots == 0 || P.n_slots > P.total_rows) return 10;
+    for (uint32_t slot = 0; slot < P.n_slots; slot++) {
+        uint64_t g = fr_slot_begin(P, slot);
+        const uint64_t end = fr_slot_begin(P, slot + 1u);
+        if (end <= g) return 11;                                                     // no empty range
+        if (fr_slot_of_row(P, g) != slot || fr_slot_of_row(P, end - 1) != slot) return 12;
+        while (g < end) {
+            const FrRowPos pos = fr_locate_row(P, g);
+            if (pos.kk >= P.n_chunks || pos.r >= pos.rows_k) return 13;
+            uint32_t take = pos.rows_k - pos.r;
+            if (take > end - g) take = (uint32_t)(end - g);
+            for (uint32_t lane = 0; lane < 32; lane++) {                             // the warp, one lane after the other
+                const FrLane L = fr_make_lane(lane);
+                acc[pos.kk] = fr_xor4(acc[pos.kk], fr_process_segment_lane<MODE, false>(P, S.sm.data(), L, lane, pos.kk, pos.r, pos.r + take));
+            }
+            pieces_of[pos.kk]++;
+            rows_done[pos.kk] += take;
+            if (take != pos.rows_k) partial[pos.kk].push_back(Piece{slot, g - pos.r, pos.rows_k});
+            g += take;
         }
     }
-    (void)n_chunks;
+    if (fr_slot_begin(P, P.n_slots) != P.total_rows) return 14;
+    for (uint32_t kk = 0; kk < P.n_chunks; kk++)
+        if (rows_done[kk] == 0 || (pieces_of[kk] > 1) != (partial.count(kk) != 0)) return 15;
+    std::set<std::pair<uint32_t, uint32_t>> shared_recs;     // (CTA, record) pairs in use
+    std::set<uint32_t> global_recs;
+    for (const auto& kv : partial) {
+        const std::vector<Piece>& v = kv.second;
+        std::map<uint32_t, uint32_t> per_cta;
+        for (const Piece& pc : v) per_cta[pc.slot / P.warps_used]++;
+        for (const Piece& pc : v) {
+            const uint32_t cta = pc.slot / P.warps_used, cta_first = cta * P.warps_used;
+            uint32_t cta_last = cta_first + P.warps_used - 1u;
+            if (cta_last >= P.n_slots) cta_last = P.n_slots - 1u;
+            const FrShare sh = fr_chunk_share(P, pc.g0, pc.rows_k, cta_first, cta_last);
+            if (sh.n_in_cta != per_cta[cta]) return 16;
+            if (sh.n_ctas != per_cta.size() || sh.first_cta != per_cta.begin()->first) return 17;
+            if (sh.rec > 32u || (sh.rec < 32u && sh.rec >= P.warps_used)) return 18;
+        }
+        for (const auto& c : per_cta) {
+            const uint32_t cta_first = c.first * P.warps_used;
+            uint32_t cta_last = cta_first + P.warps_used - 1u;
+            if (cta_last >= P.n_slots) cta_last = P.n_slots - 1u;
+            const FrShare sh = fr_chunk_share(P, v[0].g0, v[0].rows_k, cta_first, cta_last);
+            if (c.second > 1 && !shared_recs.insert({c.first, sh.rec}).second) return 19;      // one chunk per shared record
+        }
+        if (per_cta.size() > 1 && !global_recs.insert(per_cta.begin()->first).second) return 20;   // one chunk per global record
+    }
+    return 0;
 }
 
 }  // namespace
 
-// One pass of mode `mode` (FrMode) over a buffer; seg_rows as the host planner would choose it (any value >= 1).
+// One pass of mode `mode` (FrMode) over a buffer, laid out by the library's own planner (fr_plan_rows) for a GPU of
+// `num_sms` SMs; rows_per_slot > 0 asks for that many rows per warp instead of the planner's choice (any value >= 1).
 extern "C" int emu_pass(int mode, const uint8_t* key, const uint8_t* iv_base, size_t cb, const uint8_t* in, size_t len,
                         uint8_t* out, const uint8_t* pad, uint8_t* mask, const uint8_t* tags_in, uint8_t* tags_out,
-                        uint32_t* ok, uint32_t seg_rows, uint32_t first_chunk, uint32_t aad_mod, size_t sample_bytes,
-                        const uint8_t* ivs)
+                        uint32_t* ok, uint32_t rows_per_slot, uint32_t num_sms, uint32_t first_chunk, uint32_t aad_mod,
+                        size_t sample_bytes, const uint8_t* ivs)
 {
     Setup S;
     setup(S, key, cb);
@@ -155,11 +209,23 @@ extern "C" int emu_pass(int mode, const uint8_t* key, const uint8_t* iv_base, si
     P.sample_bytes = sample_bytes;
     P.chunks_per_sample = (uint32_t)cps;
     P.ivs = ivs;
-    const size_t rows_ref = ((first_len + 15) / 16 + 2 + 31) / 32;
-    P.seg_rows = seg_rows ? seg_rows : 8;
-    P.segs_per_chunk = (uint32_t)((rows_ref + P.seg_rows - 1) / P.seg_rows);
     P.n_chunks = (uint32_t)n_chunks;
-    P.n_items = (uint32_t)(P.segs_per_chunk * n_chunks);
+    FrPlanConfig cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.num_sms = (int)(num_sms ? num_sms : 148);
+    cfg.chunk_bytes = cb;
+    FrRowPlan rows = fr_plan_rows(cfg, sample_bytes, n_chunks);
+    if (rows_per_slot) {
+        cfg.row_slots_override = (uint32_t)((rows.total_rows + rows_per_slot - 1) / rows_per_slot);
+        rows = fr_plan_rows(cfg, sample_bytes, n_chunks);
+    }
+    P.n_slots = rows.n_slots;
+    P.warps_used = rows.warps_used;
+    P.rows_full = rows.rows_full;
+    P.rows_last = rows.rows_last;
+    P.rows_sample = rows.rows_sample;
+    P.total_rows = rows.total_rows;
+    if ((uint64_t)rows.grid * rows.warps_used < rows.n_slots || rows.warps_used > 32 || rows.grid > (uint32_t)cfg.num_sms) return -2;
     P.lenh_full = length_term(S, first_len, aad_mod);
     P.lenh_last = length_term(S, sample_bytes - (cps - 1) * cb, aad_mod);
     P.in = in;
@@ -167,15 +233,17 @@ extern "C" int emu_pass(int mode, const uint8_t* key, const uint8_t* iv_base, si
     P.pad = pad;
     P.mask = (uint4*)mask;
     std::vector<uint4> acc(n_chunks, uint4{0, 0, 0, 0});
+    int rc;
     switch (mode) {
-        case FR_MODE_DEC: run_pass<FR_MODE_DEC>(S, P.n_chunks, acc); break;
-        case FR_MODE_ENC: run_pass<FR_MODE_ENC>(S, P.n_chunks, acc); break;
-        case FR_MODE_CTR: run_pass<FR_MODE_CTR>(S, P.n_chunks, acc); return 0;
-        case FR_MODE_VERIFY: run_pass<FR_MODE_VERIFY>(S, P.n_chunks, acc); break;
-        case FR_MODE_PADGEN: run_pass<FR_MODE_PADGEN>(S, P.n_chunks, acc); return 0;
-        case FR_MODE_PADDEC: run_pass<FR_MODE_PADDEC>(S, P.n_chunks, acc); break;
+        case FR_MODE_DEC: rc = run_pass<FR_MODE_DEC>(S, acc); break;
+        case FR_MODE_ENC: rc = run_pass<FR_MODE_ENC>(S, acc); break;
+        case FR_MODE_CTR: return run_pass<FR_MODE_CTR>(S, acc);
+        case FR_MODE_VERIFY: rc = run_pass<FR_MODE_VERIFY>(S, acc); break;
+        case FR_MODE_PADGEN: return run_pass<FR_MODE_PADGEN>(S, acc);
+        case FR_MODE_PADDEC: rc = run_pass<FR_MODE_PADDEC>(S, acc); break;
         default: return -1;
     }
+    if (rc) return rc;
     for (uint32_t kk = 0; kk < n_chunks; kk++) {                            // the finishing warp's part
         const uint4 tag = fr_xor4(acc[kk], ((kk + 1) % P.chunks_per_sample == 0) ? P.lenh_last : P.lenh_full);
         if (mode == FR_MODE_ENC) memcpy(tags_out + 16 * kk, &tag, 16);
@@ -330,7 +398,8 @@ static int run_case(size_t cb, size_t len, uint32_t seg, uint32_t first, uint32_
         for (size_t i = 0; i < 16 * K; i++) { mask[i] = (uint8_t)(lcg(s) >> 24); tin[i] = (uint8_t)(lcg(s) >> 24); tout[i] = 0; }
         for (size_t i = 0; i < K; i++) ok[i] = 9;
         if (ivs) for (size_t i = 0; i < 12 * n_samples; i++) ivs[i] = (uint8_t)(lcg(s) >> 24);
-        bad |= emu_pass(mode, key, iv, cb, in, len, out, pad, mask, tin, tout, ok, seg, first, aad, sample_bytes, ivs);
+        bad |= emu_pass(mode, key, iv, cb, in, len, out, pad, mask, tin, tout, ok, seg, 2 + seg % 3, first, aad, sample_bytes, ivs);
+        bad |= emu_pass(mode, key, iv, cb, in, len, out, pad, mask, tin, tout, ok, 0, 148, first, aad, sample_bytes, ivs);
         if (mode <= FR_MODE_VERIFY)                     // the packed-row form of the same pass, seg doubling as group size and run length
             for (uint32_t run : {1u, seg + 1u, 40u})
                 bad |= emu_packed(mode, key, iv, cb, in, len, out, tin, tout, ok, seg * 3 - 2, run, first, aad, sample_bytes, ivs);

@@ -36,8 +36,8 @@ def to_dev(a: np.ndarray) -> torch.Tensor:
 class Gpu:
     """One library context plus numpy-in / numpy-out wrappers around the three data-path calls."""
 
-    def __init__(self, key: bytes, chunk_bytes: int):
-        self.ctx = fastrack.Context(key, chunk_bytes)
+    def __init__(self, key: bytes, chunk_bytes: int, options=None):
+        self.ctx = fastrack.Context(key, chunk_bytes, options)
         self.cb = chunk_bytes
 
     def close(self):

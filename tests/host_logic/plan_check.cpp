@@ -4,24 +4,26 @@
 
 extern "C" {
 
-static FrPlanConfig make(int num_sms, size_t chunk_bytes, uint32_t seg_rows, uint32_t pack_max, uint32_t run, uint32_t group,
+static FrPlanConfig make(int num_sms, size_t chunk_bytes, uint32_t row_slots, uint32_t pack_max, uint32_t run, uint32_t group,
                          size_t stage_bytes)
 {
     FrPlanConfig c;
-    c.num_sms = num_sms; c.chunk_bytes = chunk_bytes; c.seg_rows_override = seg_rows; c.pack_max_blocks = pack_max;
+    c.num_sms = num_sms; c.chunk_bytes = chunk_bytes; c.row_slots_override = row_slots; c.pack_max_blocks = pack_max;
     c.pack_run_override = run; c.pack_group_override = group; c.stage_bytes_override = stage_bytes;
     return c;
 }
 
-// out[0..2] = seg_rows, segs_per_chunk, n_items of the row kernels; out[3..5] = run, group, n_items of the packed rows
-void plan_launch(int num_sms, size_t chunk_bytes, uint32_t seg_rows, uint32_t pack_max, uint32_t run, uint32_t group, int kind,
-                 size_t sample_bytes, size_t n_chunks, uint32_t out[6])
+// out[0..2] = grid, warps_used, n_slots of the row kernels; out[3..5] = run, group, n_items of the packed rows;
+// out[6..9] = rows_full, rows_last, rows_sample, total_rows
+void plan_launch(int num_sms, size_t chunk_bytes, uint32_t row_slots, uint32_t pack_max, uint32_t run, uint32_t group, int kind,
+                 size_t sample_bytes, size_t n_chunks, uint64_t out[10])
 {
-    const FrPlanConfig c = make(num_sms, chunk_bytes, seg_rows, pack_max, run, group, 0);
-    const FrSegPlan s = fr_plan_segments(c, sample_bytes, n_chunks);
-    const FrPackPlan p = fr_plan_packed(c, kind, sample_bytes, n_chunks, s);
-    out[0] = s.seg_rows; out[1] = s.segs_per_chunk; out[2] = s.n_items;
+    const FrPlanConfig c = make(num_sms, chunk_bytes, row_slots, pack_max, run, group, 0);
+    const FrRowPlan r = fr_plan_rows(c, sample_bytes, n_chunks);
+    const FrPackPlan p = fr_plan_packed(c, kind, sample_bytes, n_chunks, r);
+    out[0] = r.grid; out[1] = r.warps_used; out[2] = r.n_slots;
     out[3] = p.run; out[4] = p.group; out[5] = p.n_items;
+    out[6] = r.rows_full; out[7] = r.rows_last; out[8] = r.rows_sample; out[9] = r.total_rows;
 }
 
 size_t plan_stages(size_t chunk_bytes, size_t stage_bytes, size_t len, size_t unit, size_t* out)

@@ -21,7 +21,7 @@ def emu(tmp_path_factory):
                            os.path.join(ROOT, "tests", "device_on_host", "emulate.cpp")])
     lib = ctypes.CDLL(str(so))
     V, Z, U = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_uint32
-    lib.emu_pass.argtypes = [ctypes.c_int, V, V, Z, V, Z, V, V, V, V, V, V, U, U, U, Z, V]
+    lib.emu_pass.argtypes = [ctypes.c_int, V, V, Z, V, Z, V, V, V, V, V, V, U, U, U, U, Z, V]
     lib.emu_pass.restype = ctypes.c_int
     for name in ("emu_gf128_mul_device", "emu_gf128_mul_keysetup"):
         getattr(lib, name).argtypes = [ctypes.c_char_p] * 3
@@ -31,7 +31,9 @@ def emu(tmp_path_factory):
     return lib
 
 
-def run(lib, mode, key, iv, cb, data, n, pad=None, mask=None, tags=None, seg=8, first=0, aad=0, sample_bytes=0, ivs=None):
+def run(lib, mode, key, iv, cb, data, n, pad=None, mask=None, tags=None, seg=8, first=0, aad=0, sample_bytes=0, ivs=None, sms=3):
+    """seg = rows per warp (0: the planner's own choice) on an emulated GPU of `sms` SMs: few SMs, so that chunks are
+    shared between warps of one CTA and between CTAs even in small cases."""
     K = (n + cb - 1) // cb if not sample_bytes else (n // sample_bytes) * ((sample_bytes + cb - 1) // cb)
     k = np.frombuffer(key, np.uint8).copy()
     v = np.frombuffer(iv, np.uint8).copy()
@@ -45,9 +47,10 @@ def run(lib, mode, key, iv, cb, data, n, pad=None, mask=None, tags=None, seg=8, 
     if mode == VERIFY:
         out[:n] = src                                   # the pass does not store; keep the guard check meaningful
     rc = lib.emu_pass(mode, k.ctypes.data, v.ctypes.data, cb, src.ctypes.data, n, out.ctypes.data, pad_a.ctypes.data,
-                      mask_a.ctypes.data, tin.ctypes.data, tout.ctypes.data, ok.ctypes.data, seg, first, aad, sample_bytes,
+                      mask_a.ctypes.data, tin.ctypes.data, tout.ctypes.data, ok.ctypes.data, seg, sms, first, aad, sample_bytes,
                       ivs.ctypes.data if ivs is not None else None)
-    assert rc == 0 and (out[n:] == 0xA5).all()
+    assert rc == 0, f"emulation reports inconsistency {rc}"
+    assert (out[n:] == 0xA5).all()
     return out[:n], tout, ok, mask_a
 
 
@@ -81,7 +84,8 @@ def test_both_gf128_products_match_oracle(emu):
 
 SHAPES = [(1, 16, 8), (16, 16, 8), (15, 64, 2), (17, 64, 4), (33, 32, 8), (480, 480, 8), (512, 512, 1), (513, 1024, 8),
           (1000, 256, 2), (4096, 1024, 8), (5000, 2048, 4), (70000, 16384, 8), (70001, 65536, 16), (200000, 65536, 24),
-          (100, 65536, 8), (300000, 100000 // 16 * 16, 3)]
+          (100, 65536, 8), (300000, 100000 // 16 * 16, 3), (300000, 100000 // 16 * 16, 0), (150000, 496, 1), (150000, 1008, 5),
+          (99999, 16, 7), (400000, 4096, 13)]
 
 
 @pytest.mark.parametrize("n,cb,seg", SHAPES)

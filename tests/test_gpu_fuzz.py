@@ -108,22 +108,21 @@ def test_random_shapes_all_entry_points(seed):
             check(d_o, d_ok, "pipelined_h2d")
 
 
-def test_portable_shared_addressing_path(monkeypatch):
+def test_portable_shared_addressing_path():
     """The kernel puts table base addresses into load immediates when the shared window starts where it
-    expects, and falls back to ordinary pointer arithmetic otherwise.  FASTRACK_GENERIC_SMEM=1 forces the
-    fallback so that it is exercised on hardware where the fast form applies."""
-    monkeypatch.setenv("FASTRACK_GENERIC_SMEM", "1")
-    _every_pass_on([(1, 16, 0), (70001, 4096, 0), ((1 << 20) + 33, 65536, 16), ((5 << 20) + 7, 1 << 20, 0)])
+    expects, and falls back to ordinary pointer arithmetic otherwise.  The option forces the fallback so that it
+    is exercised on hardware where the fast form applies."""
+    _every_pass_on([(1, 16, 0), (70001, 4096, 0), ((1 << 20) + 33, 65536, 16), ((5 << 20) + 7, 1 << 20, 0)],
+                   {fastrack.OPT_GENERIC_SMEM: 1})
 
 
-def test_portable_shared_addressing_path_packed_rows(monkeypatch):
+def test_portable_shared_addressing_path_packed_rows():
     """The same fallback in the packed-row kernels (forced here by fixing the run length)."""
-    monkeypatch.setenv("FASTRACK_GENERIC_SMEM", "1")
-    monkeypatch.setenv("FASTRACK_PACK_RUN", "3")
-    _every_pass_on([(1, 16, 0), (80009, 16, 0), (154128, 512, 4), (70001, 4096, 0), (300000, 16384, 16)])
+    _every_pass_on([(1, 16, 0), (80009, 16, 0), (154128, 512, 4), (70001, 4096, 0), (300000, 16384, 16)],
+                   {fastrack.OPT_GENERIC_SMEM: 1, fastrack.OPT_PACK_RUN: 3})
 
 
-def _every_pass_on(cases):
+def _every_pass_on(cases, options):
     key, iv = synth.key_and_iv(7)
     for n, cb, chains in cases:
         plain = synth.random_bytes(n, 7, salt=n)
@@ -133,7 +132,7 @@ def _every_pass_on(cases):
         synth.apply_tamper(bad_c, bad_t, cb, synth.tamper_plan(n, cb, 7, fraction=0.3, salt=n))
         p_ref, ok_ref = (oracle.mc_decrypt_framed(key, iv, cb, chains, bad_c, bad_t, NT) if chains
                          else oracle.mc_decrypt(key, iv, cb, bad_c, bad_t, NT))
-        with fastrack.Context(key, cb) as ctx:                      # the variable is read at context creation
+        with fastrack.Context(key, cb, options) as ctx:
             ctx.set_framing(chains)
             st = torch.cuda.current_stream().cuda_stream
             d_p = dev(plain)

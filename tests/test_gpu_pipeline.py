@@ -21,17 +21,18 @@ NT = oracle.host_threads()
                                   ((5 << 20) - 16, 48 * 1024), (2 * (1 << 22) + 999, 1 << 22)])
 @pytest.mark.parametrize("n_streams", [1, 3])
 @pytest.mark.parametrize("direct", ["1", "0"])
-def test_pipelined_matches_oracle_small(n, cb, n_streams, direct, monkeypatch):
+def test_pipelined_matches_oracle_small(n, cb, n_streams, direct):
     """Single-stage transfers (up to about 3 MiB) are by default read from the page-locked host buffer by the kernel
-    itself, pinned tags included; FASTRACK_DIRECT_SMALL=0 keeps them on the copy engine.  Both must equal the oracle."""
-    monkeypatch.setenv("FASTRACK_DIRECT_SMALL", direct)
+    itself, pinned tags included; the option set to 0 keeps them on the copy engine.  Both must equal the oracle."""
+    from paper_2410_15240_b200 import fastrack
+    options = {fastrack.OPT_DIRECT_SMALL: int(direct)}
     key, iv = synth.key_and_iv(2)
     plain = synth.random_bytes(n, 2, salt=n)
     c, t = oracle.mc_encrypt(key, iv, cb, plain, NT)
     plan = synth.tamper_plan(n, cb, 2, fraction=0.1, salt=n)
     synth.apply_tamper(c, t, cb, plan)
     p_ref, ok_ref = oracle.mc_decrypt(key, iv, cb, c, t, NT)
-    with Gpu(key, cb) as g:
+    with Gpu(key, cb, options) as g:
         p, ok = g.pipelined(iv, c, t, n_streams)
         assert np.array_equal(ok, ok_ref)
         assert np.array_equal(p, p_ref)
@@ -58,17 +59,16 @@ def test_config2_fp16_image_batch(cb, n_streams):
                                                       ((9 << 20) + 12345, 256 * 1024, 3, True),
                                                       (2 * (1 << 22) + 999, 1 << 22, 4, False), (77_070_336, 4 << 20, 4, False)])
 @pytest.mark.parametrize("direct,pinned_tags", [("1", False), ("1", True), ("0", False)])
-def test_pipelined_d2h_encrypt_matches_oracle(n, cb, n_streams, in_place, direct, pinned_tags, monkeypatch):
+def test_pipelined_d2h_encrypt_matches_oracle(n, cb, n_streams, in_place, direct, pinned_tags):
     """GPU encrypt+tag with overlapped device->host copies; the host side (oracle) verifies and decrypts.
     Single-stage transfers are by default written to the page-locked host buffers by the kernel itself (tags too when
-    their buffer is page-locked); FASTRACK_DIRECT_SMALL=0 keeps them on the copy engine."""
+    their buffer is page-locked); the option set to 0 keeps them on the copy engine."""
     from paper_2410_15240_b200 import fastrack
-    monkeypatch.setenv("FASTRACK_DIRECT_SMALL", direct)
     key, iv = synth.key_and_iv(3)
     plain = synth.fp16_image_batch() if n == 77_070_336 else synth.random_bytes(n, 3, salt=n)
     c_ref, t_ref = oracle.mc_encrypt(key, iv, cb, plain, NT)
     K = t_ref.shape[0]
-    with fastrack.Context(key, cb) as ctx:
+    with fastrack.Context(key, cb, {fastrack.OPT_DIRECT_SMALL: int(direct)}) as ctx:
         d_p = torch.from_numpy(plain).cuda()
         d_c = d_p if in_place else torch.empty_like(d_p)
         h_c = torch.full((n,), 0xEE, dtype=torch.uint8).pin_memory()

@@ -19,23 +19,21 @@ if not torch.cuda.is_available():
 NT = oracle.host_threads()
 
 
-FAMILIES = {
-    "general": {"FASTRACK_PACK_MAX_BLOCKS": "0"},                                   # row kernels only
+FAMILIES = {      # kernel layouts forced through fastrack_ctx_set_option
+    "general": {fastrack.OPT_PACK_MAX_BLOCKS: 0},                                  # row kernels only
+    "general-every-warp": {fastrack.OPT_PACK_MAX_BLOCKS: 0, fastrack.OPT_ROW_SLOTS: 148 * 32},   # ... rows spread as thinly as they go
+    "general-37-warps": {fastrack.OPT_PACK_MAX_BLOCKS: 0, fastrack.OPT_ROW_SLOTS: 37},   # ... chunks shared between warps and CTAs
     "auto": {},                                                                   # the planner decides
-    "run1": {"FASTRACK_PACK_RUN": "1"},                                           # packed rows, one counter per lane
-    "run5": {"FASTRACK_PACK_RUN": "5"},                                           # packed rows, five counters per lane
-    "run3-group7": {"FASTRACK_PACK_RUN": "3", "FASTRACK_PACK_GROUP": "7"},        # odd item size: rows that straddle chunks
-    "run300": {"FASTRACK_PACK_RUN": "300"},                                       # one lane per chunk, crossing 256-counter groups
+    "run1": {fastrack.OPT_PACK_RUN: 1},                                           # packed rows, one counter per lane
+    "run5": {fastrack.OPT_PACK_RUN: 5},                                           # packed rows, five counters per lane
+    "run3-group7": {fastrack.OPT_PACK_RUN: 3, fastrack.OPT_PACK_GROUP: 7},        # odd item size: rows that straddle chunks
+    "run300": {fastrack.OPT_PACK_RUN: 300},                                       # one lane per chunk, crossing 256-counter groups
 }
 
 
 @pytest.fixture(params=list(FAMILIES))
-def family(request, monkeypatch):
-    for name in ("FASTRACK_PACK_MAX_BLOCKS", "FASTRACK_PACK_RUN", "FASTRACK_PACK_GROUP"):
-        monkeypatch.delenv(name, raising=False)
-    for name, value in FAMILIES[request.param].items():
-        monkeypatch.setenv(name, value)
-    return request.param
+def family(request):
+    return FAMILIES[request.param]
 
 
 SHAPES = [(1, 16), (15, 16), (16, 16), (17, 16), (16 * 31, 16), (16 * 32 + 3, 16), (16 * 5000 + 9, 16), (32 * 777 + 31, 32),
@@ -52,7 +50,7 @@ def test_small_chunks_match_oracle(family, n, cb):
     bad_c, bad_t = c_ref.copy(), t_ref.copy()
     synth.apply_tamper(bad_c, bad_t, cb, synth.tamper_plan(n, cb, 4, fraction=0.2, salt=n))
     p_ref, ok_ref = oracle.mc_decrypt(key, iv, cb, bad_c, bad_t, NT)
-    with Gpu(key, cb) as g:
+    with Gpu(key, cb, family) as g:
         c, t = g.encrypt(iv, plain)
         assert np.array_equal(c, c_ref) and np.array_equal(t, t_ref)
         c, t = g.encrypt(iv, plain, in_place=True)
@@ -91,7 +89,7 @@ def test_two_million_sixteen_byte_chunks(family):
     bad_t[rej, 7] ^= 0x20
     expect = np.ones(K, np.uint32)
     expect[rej] = 0
-    with fastrack.Context(key, cb) as ctx:
+    with fastrack.Context(key, cb, family) as ctx:
         d_p = torch.from_numpy(plain).cuda()
         d_c = torch.empty_like(d_p)
         d_t = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
@@ -123,7 +121,7 @@ def test_batches_of_small_samples(family, sample_bytes, cb, n_samples, chains):
         t_ref.append(t_s)
     c_ref, t_ref = np.concatenate(c_ref), np.concatenate(t_ref)
     K = t_ref.shape[0]
-    with fastrack.Context(key, cb) as ctx:
+    with fastrack.Context(key, cb, family) as ctx:
         if chains:
             ctx.set_framing(chains)
         d_iv = torch.from_numpy(np.frombuffer(b"".join(ivs), np.uint8).copy()).cuda()

@@ -186,15 +186,14 @@ def test_sequential_chain_comparator_gives_the_same_verdicts(n, cb, chains):
         assert np.array_equal(d_c.cpu().numpy(), c)
 
 
-def test_counter_mode_only_needs_no_scratch(monkeypatch):
-    """A fresh context holds scratch for 1024 chunks; the pass without authentication must not ask for more, even
-    when its chunks are cut into several segments (row kernels forced) and there are thousands of them."""
-    monkeypatch.setenv("FASTRACK_PACK_MAX_BLOCKS", "0")
+def test_counter_mode_only_as_first_call_on_a_context():
+    """The pass without authentication as the very first call on a fresh context, with thousands of chunks that are
+    cut between warps (row kernels forced): it needs nothing that an earlier call would have set up."""
     key, iv = synth.key_and_iv(6)
     cb, n = 4096, 4096 * 3000 + 77
     plain = synth.random_bytes(n, 6, salt=5)
     c_ref, _ = oracle.mc_encrypt(key, iv, cb, plain, oracle.host_threads())
-    with fastrack.Context(key, cb) as ctx:
+    with fastrack.Context(key, cb, {fastrack.OPT_PACK_MAX_BLOCKS: 0}) as ctx:
         d_p = torch.from_numpy(plain).cuda()
         d_c = torch.empty_like(d_p)
         ctx.ctr_crypt(iv, d_p.data_ptr(), n, d_c.data_ptr(), 0)          # first call on the context

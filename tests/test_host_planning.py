@@ -24,10 +24,10 @@ def plan(tmp_path_factory):
     return lib
 
 
-def launch(lib, cb, sample_bytes, n_chunks, kind=0, seg_rows=0, pack_max=4096, run=0, group=0, sms=148):
-    out = np.zeros(6, np.uint32)
-    lib.plan_launch(sms, cb, seg_rows, pack_max, run, group, kind, sample_bytes, n_chunks, out.ctypes.data)
-    return [int(x) for x in out]
+def launch(lib, cb, sample_bytes, n_chunks, kind=0, row_slots=0, pack_max=4096, run=0, group=0, sms=148, geometry=False):
+    out = np.zeros(10, np.uint64)
+    lib.plan_launch(sms, cb, row_slots, pack_max, run, group, kind, sample_bytes, n_chunks, out.ctypes.data)
+    return [int(x) for x in (out if geometry else out[:6])]
 
 
 CHUNKS = [16, 32, 48, 64, 112, 256, 496, 512, 528, 992, 1008, 1024, 4096, 16384, 65536, 1 << 20, 4 << 20, 1 << 30]
@@ -42,12 +42,13 @@ def test_launch_plans_are_consistent(plan, kind):
         for n_chunks in COUNTS:
             if cb * n_chunks > 1 << 42:
                 continue
-            seg_rows, spc, n_items, run, group, p_items = launch(plan, cb, cb * n_chunks, n_chunks, kind)
-            # row kernels: segments tile the chunk, items fit 31 bits
-            assert seg_rows >= 2 and (seg_rows <= 4 or seg_rows % 8 == 0), (cb, n_chunks, seg_rows)
-            assert spc == -(-rows // seg_rows) and n_items == spc * n_chunks and n_items < 1 << 31
-            if blocks <= 62:
-                assert spc == 1, "chunks of two rows are never split between warps (they then need no scratch)"
+            grid, wu, n_slots, run, group, p_items, rows_full, rows_last, rows_sample, total = launch(
+                plan, cb, cb * n_chunks, n_chunks, kind, geometry=True)
+            # row kernels: the slots cover the row space without an empty range, on at most one CTA per SM
+            assert rows_full == rows and rows_last == rows and rows_sample == rows * n_chunks == total
+            assert 1 <= n_slots <= min(total, WARPS) and 1 <= grid <= 148 and 1 <= wu <= 32
+            assert (grid - 1) * wu < n_slots <= grid * wu, "every CTA of the grid holds at least one slot"
+            assert n_slots * total < 1 << 63, "slot boundaries are computed in 64 bits"
             # packed rows: whole chunks per item, bounded item size, everything within 32 bits
             if run:
                 counters = blocks + 1
@@ -90,11 +91,22 @@ def test_small_chunks_in_large_numbers_take_the_packed_rows(plan):
 
 def test_sample_batches_plan_on_the_sample_geometry(plan):
     # samples shorter than a chunk: the chunk that exists is the sample
-    seg = launch(plan, 4096, 400, 262144)
-    assert seg[1] == 1 and seg[3] >= 1
-    # samples of several chunks
-    seg = launch(plan, 1024, 3 * 1024 + 16, 4 * 50000)
-    assert seg[0] >= 2 and seg[2] == seg[1] * 4 * 50000
+    got = launch(plan, 4096, 400, 262144, geometry=True)
+    assert got[3] >= 1 and got[6] == got[7] == 1 and got[9] == 262144
+    # samples of several chunks: three full ones and a 16-byte one
+    got = launch(plan, 1024, 3 * 1024 + 16, 4 * 50000, geometry=True)
+    assert got[6] == 3 and got[7] == 1 and got[8] == 10 and got[9] == 10 * 50000
+
+
+def test_row_slots_follow_the_size_of_the_launch(plan):
+    """Small launches use few warps per SM (every warp pays a closing product), large ones all 32; a forced slot count
+    is honoured up to the number of rows and of warps."""
+    used = [launch(plan, 4 << 20, n, -(-n // (4 << 20)))[1] for n in (1 << 20, 4 << 20, 16 << 20, 64 << 20, 256 << 20)]
+    assert used == sorted(used) and used[0] <= 8 and used[-1] == 32
+    for want in (1, 2, 147, 148, 149, 1000, 4736, 10 ** 6):
+        grid, wu, n_slots = launch(plan, 65536, 1 << 24, 256, row_slots=want)[:3]
+        assert n_slots == min(want, WARPS) and (grid - 1) * wu < n_slots <= grid * wu
+    assert launch(plan, 16, 16 * 5, 5, row_slots=4736)[2] == 5          # one row per chunk: never more slots than rows
 
 
 def stages(lib, cb, length, unit=None, stage_bytes=0):

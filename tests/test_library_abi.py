@@ -49,6 +49,7 @@ def test_argument_checks_that_need_no_device():
     assert fastrack.fastrack_launch_count(None) == 0
     assert fastrack.fastrack_ctx_reserve(None, 1) == fastrack.ERR_ARG
     assert fastrack.fastrack_ctx_set_framing(None, 16) == fastrack.ERR_ARG
+    assert fastrack.fastrack_ctx_set_option(None, fastrack.OPT_PACK_RUN, 3) == fastrack.ERR_ARG
     assert fastrack.fastrack_ctx_set_trace(None, 1) == fastrack.ERR_ARG
     assert fastrack.fastrack_ctx_get_trace(None) == []
     assert fastrack.fastrack_decrypt_verify(None, bytes(12), 0, 16, 0, 0, 0, 0) == fastrack.ERR_ARG
@@ -75,14 +76,3 @@ def test_no_cpu_fallback_without_a_device():
         return
     rc, handle = fastrack.fastrack_ctx_create(bytes(32), 65536)
     assert rc == fastrack.ERR_CUDA and handle is None
-
-
-def test_probe_library_builds_and_exports_its_entry_point():
-    import ctypes
-    from paper_2410_15240_b200 import build as lib_build
-    lib_build.build()
-    lib = ctypes.CDLL(lib_build.PROBE_LIB)
-    assert hasattr(lib, "fastrack_probe_peaks")
-    lib.fastrack_probe_peaks.argtypes = [ctypes.c_char_p, ctypes.c_size_t]
-    lib.fastrack_probe_peaks.restype = ctypes.c_int
-    assert lib.fastrack_probe_peaks(None, 0) == -1        # argument check only: no device call
