@@ -9,6 +9,9 @@
 #include <new>
 
 #include "../../include/fastrack.h"
+// Waits (whole warp) until the bulk copy of the H-power byte tables has landed in shared memory; defined below.
+__device__ __forceinline__ void fr_await_tables(const char* sm, const uint4* gh_tab, uint32_t* timeouts);
+#define FR_AWAIT_TABLES(sm, P) fr_await_tables((sm), (P).gh_tab, (P).timeouts)
 #include "fastrack_device.cuh"
 #include "fastrack_keysetup.h"
 #include "fastrack_plan.h"
@@ -16,6 +19,64 @@
 using namespace fr_host;
 
 // ------------------------------------------------------------------------------------ kernels ----
+
+// Te0 (AES S-box folded with MixColumns; the same for every key).  Written once per device by fastrack_ctx_create.
+// (Tried instead: the 256 words as immediates in the code of the warp that stores them -- slower, 2.0 against
+// 1.4 us for the fill, because then every warp runs code of its own and the instruction fetch becomes the cost.)
+__constant__ uint32_t fr_te0_const[256];
+
+// Fills shared memory at the start of a kernel, up to but not including the barrier that publishes it.
+//   AES rows: every thread replicates eight entries of Te0 (and its byte rotations) across the 32 banks; the
+//     entries come from constant memory with a warp-uniform index.
+//   H-power byte tables (64 KiB, per context): two bulk asynchronous copies, global -> shared, issued by thread 0
+//     before anything else and signalled on an mbarrier.  Nobody waits for them here: every lane starts with a
+//     cipher block, which needs the AES rows only, and waits in front of its first table multiply
+//     (fr_await_tables), by which time the 64 KiB have long arrived.
+//     (Passes that do not authenticate have no use for them and start no copy: a CTA must not exit with a copy
+//     into its shared memory still in flight, and only the table multiply waits for it.)
+template <uint32_t NTHREADS, bool WITH_H_TABLES>
+__device__ __forceinline__ void fr_fill_smem(char* sm, const uint4* __restrict__ gh_tab)
+{
+    const uint32_t tid = threadIdx.x;
+    if (WITH_H_TABLES && tid == 0) {
+        const uint32_t mbar = (uint32_t)__cvta_generic_to_shared(sm + FR_SM_MBAR);
+        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(sm + FR_SM_GH);
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(mbar) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mbar), "r"(65536u) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(dst), "l"(gh_tab), "r"(32768u), "r"(mbar) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(dst + 32768u), "l"((const char*)gh_tab + 32768), "r"(32768u), "r"(mbar) : "memory");
+    }
+    constexpr uint32_t N_AES = 256u * 4u * 8u / NTHREADS;     // 256 rows x 2 arrays x 2 tables x 8 uint4 (32 words)
+    static_assert(N_AES * NTHREADS == 8192u, "thread count must divide the tables");
+#pragma unroll
+    for (uint32_t n = 0; n < N_AES; n++) {
+        const uint32_t i = tid + n * NTHREADS, q = i & 7u, t = (i >> 3) & 3u, v = i >> 5;
+        const uint32_t e = fr_te0_const[v];
+        const uint32_t w = __funnelshift_l(e, e, 8u * t);                 // Te1..Te3 are Te0 rotated left by 1..3 bytes
+        const uint32_t off = ((t >> 1) ? FR_SM_T23 : FR_SM_T01) + v * 256u + (t & 1u) * 128u + q * 16u;
+        *(uint4*)(sm + off) = make_uint4(w, w, w, w);
+    }
+    if (tid < 33u * 8u) ((uint32_t*)(sm + FR_SM_COMB))[tid] = 0u;        // the combine records start at zero
+}
+
+// Every thread calls this once, in front of its first table multiply: it polls the copy's mbarrier a bounded
+// number of times (each attempt gives up by itself after a while; in practice the first one succeeds, the copy
+// having had a whole cipher block's time to land).  Should the copy never arrive, the thread counts the event in
+// *timeouts and goes on: the tags it computes from an incomplete table do not match, so every chunk it touches
+// is rejected (or, when encrypting, will be rejected by the receiver) -- wrong towards refusal, never acceptance.
+__device__ __forceinline__ void fr_await_tables(const char* sm, const uint4* gh_tab, uint32_t* timeouts)
+{
+    (void)gh_tab;
+    const uint32_t mbar = (uint32_t)__cvta_generic_to_shared(sm + FR_SM_MBAR);
+    uint32_t done = 0;
+    for (uint32_t attempt = 0; attempt < 4096u && !done; attempt++)
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(mbar) : "memory");
+    if (!done) atomicAdd(timeouts, 1u);
+}
 
 template <int MODE, bool ABS>
 __device__ __forceinline__ void fr_crypt_body(const FrParams& P, char* sm, FrLane L)
@@ -30,11 +91,12 @@ __device__ __forceinline__ void fr_crypt_body(const FrParams& P, char* sm, FrLan
 
     uint64_t g = fr_slot_begin(P, slot);
     const uint64_t end = fr_slot_begin(P, slot + 1u);
+    bool await_tables = true;                            // the H tables may still be on their way into shared memory (per thread)
     while (g < end) {                                    // one segment per chunk that the warp's range touches
         const FrRowPos pos = fr_locate_row(P, g);
         uint32_t take = pos.rows_k - pos.r;
         if (take > end - g) take = (uint32_t)(end - g);
-        uint4 z = fr_process_segment_lane<MODE, ABS>(P, sm, L, lane, pos.kk, pos.r, pos.r + take);
+        uint4 z = fr_process_segment_lane<MODE, ABS>(P, sm, L, lane, pos.kk, pos.r, pos.r + take, await_tables);
         const uint64_t g0 = g - pos.r;                   // the chunk's first row in the row space
         g += take;
         if (MODE != FR_MODE_CTR && MODE != FR_MODE_PADGEN) {                // the other passes authenticate
@@ -108,8 +170,7 @@ __global__ void __launch_bounds__(FR_THREADS, 1) fr_crypt_kernel(const __grid_co
 {
     extern __shared__ __align__(256) char sm[];
     FR_STAMP_GT(0); FR_STAMP_SET(7);
-    fr_build_smem<FR_THREADS>(sm, threadIdx.x, P.te0, P.gh_tab);
-    if (threadIdx.x < 33u * 8u) ((uint32_t*)(sm + FR_SM_COMB))[threadIdx.x] = 0u;      // the combine records start at zero
+    fr_fill_smem<FR_THREADS, MODE != FR_MODE_CTR && MODE != FR_MODE_PADGEN>(sm, P.gh_tab);
     FR_STAMP_SET(1);
     // Programmatic dependent launch: the table build above touches only per-context constants, so it may run
     // while the previous kernel in the stream is still finishing; everything below waits until that kernel has
@@ -187,10 +248,11 @@ template <int MODE, bool WHOLE>
 __global__ void __launch_bounds__(FR_THREADS, 1) fr_packed_kernel(const __grid_constant__ FrParams P)
 {
     extern __shared__ __align__(256) char sm[];
-    fr_build_smem<FR_THREADS>(sm, threadIdx.x, P.te0, P.gh_tab);
+    fr_fill_smem<FR_THREADS, MODE != FR_MODE_CTR>(sm, P.gh_tab);
     asm volatile("griddepcontrol.wait;" ::: "memory");           // as in fr_crypt_kernel
     asm volatile("griddepcontrol.launch_dependents;");
     __syncthreads();
+    if (MODE != FR_MODE_CTR) fr_await_tables(sm, P.gh_tab, P.timeouts);      // (a packed row may start with a table step: wait here)
     uint32_t after_barrier;
     asm volatile("mov.u32 %0, 0;" : "=r"(after_barrier)::"memory");
     FrLane L = fr_make_lane(threadIdx.x & 31u);
@@ -266,6 +328,10 @@ extern "C" __attribute__((visibility("default"))) int fastrack_stamps_read(unsig
 {
     return (int)cudaMemcpyFromSymbol(out, fr_stamps, sizeof(unsigned long long) * 1024 * 8);
 }
+extern "C" __attribute__((visibility("default"))) int fastrack_warp_stamps_read(unsigned long long* out)
+{
+    return (int)cudaMemcpyFromSymbol(out, fr_warp_stamps, sizeof(unsigned long long) * 1024 * 32);
+}
 #endif
 
 // ------------------------------------------------------------------------------------ context ----
@@ -282,6 +348,7 @@ struct fastrack_ctx {
     uint4* d_gh1_tab;          // byte tables of H (sequential-chain comparator only)
     uint4* d_pow;
     size_t pow_entries;
+    uint32_t* d_timeouts;      // one word: how often a kernel's bulk copy of the H tables did not arrive in time (see fr_fill_smem)
     uint32_t* d_scratch;       // combine records of the row kernels: 2 banks x FR_SCRATCH_WINDOWS windows x num_sms records of 8 words
     uint4* d_tags_stage;       // pipelined calls: device copy of the tags, then (second half) the E_K(J0) masks
     size_t tags_stage_chunks;
@@ -394,6 +461,9 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
         if ((e = cudaMalloc(&ctx->d_scratch, scratch_words(ctx) * sizeof(uint32_t))) != cudaSuccess) break;
         if ((e = cudaMemset(ctx->d_scratch, 0, scratch_words(ctx) * sizeof(uint32_t))) != cudaSuccess) break;
         if ((e = cudaMemcpy(ctx->d_te0, te0, sizeof te0, cudaMemcpyHostToDevice)) != cudaSuccess) break;
+        if ((e = cudaMemcpyToSymbol(fr_te0_const, te0, sizeof te0)) != cudaSuccess) break;       // key-independent: every context writes the same words
+        if ((e = cudaMalloc(&ctx->d_timeouts, 256)) != cudaSuccess) break;
+        if ((e = cudaMemset(ctx->d_timeouts, 0, 256)) != cudaSuccess) break;
         if ((e = cudaMemcpy(ctx->d_gh_tab, tab, 65536, cudaMemcpyHostToDevice)) != cudaSuccess) break;
         if ((e = cudaMemcpy(ctx->d_gh1_tab, tab + 65536, 65536, cudaMemcpyHostToDevice)) != cudaSuccess) break;
         uint8_t seed[32] = {0};
@@ -413,14 +483,14 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
         if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_PADGEN>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
         if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_PADDEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
         if ((e = cudaFuncSetAttribute(fr_verify_sequential_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
-        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_DEC, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
-        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_DEC, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
-        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_ENC, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
-        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_ENC, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
-        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_CTR, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
-        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_CTR, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
-        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_VERIFY, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
-        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_VERIFY, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_DEC, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_DEC, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_ENC, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_ENC, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_CTR, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_CTR, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_VERIFY, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_packed_kernel<FR_MODE_VERIFY, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
         for (int i = 0; i < 8 && e == cudaSuccess; i++) e = cudaStreamCreateWithFlags(&ctx->streams[i], cudaStreamNonBlocking);
         if (e != cudaSuccess) break;
         if ((e = cudaEventCreateWithFlags(&ctx->tags_ready, cudaEventDisableTiming)) != cudaSuccess) break;
@@ -451,6 +521,7 @@ extern "C" void fastrack_ctx_destroy(fastrack_ctx* ctx)
     cudaFree(ctx->d_gh1_tab);
     cudaFree(ctx->d_pow);
     cudaFree(ctx->d_scratch);
+    cudaFree(ctx->d_timeouts);
     cudaFree(ctx->d_tags_stage);
     for (int i = 0; i < 8; i++)
         if (ctx->streams[i]) cudaStreamDestroy(ctx->streams[i]);
@@ -635,6 +706,7 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
     P.tags_out = (uint4*)b.tags_out;
     P.ok = b.ok;
     P.te0 = ctx->d_te0;
+    P.timeouts = ctx->d_timeouts;
     P.gh_tab = packed ? ctx->d_gh1_tab : ctx->d_gh_tab;
     // One lane per chunk (run >= blocks + 1) has a kernel variant of its own that closes with two table steps and needs
     // no reduction across lanes.  It wins while the integer pipes are the busier ones (up to 3 blocks per chunk) or the
@@ -654,7 +726,7 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(FR_THREADS);
-    cfg.dynamicSmemBytes = packed ? FR_SMEM_BYTES : FR_SMEM_LAUNCH_BYTES;
+    cfg.dynamicSmemBytes = FR_SMEM_LAUNCH_BYTES;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     if (!ctx->no_overlap_launch && !b.plain_launch) {

@@ -34,6 +34,7 @@
 #define FR_SM_GH 131072u      // byte tables of H^32
 #define FR_SMEM_BYTES 196608u // the three tables
 #define FR_SM_COMB 196608u    // row kernels: 33 records of 8 words in which the warps of a CTA combine their pieces of a chunk
+#define FR_SM_MBAR (FR_SM_COMB + 33u * 32u)   // arrival barrier of the bulk copy that brings in the H-power byte tables
 #define FR_SMEM_LAUNCH_BYTES (FR_SMEM_BYTES + 2048u)   // dynamic shared memory of a launch: the tables and the records
 
 // What one pass does.  DEC / ENC are the fused passes.  CTR and VERIFY split them (paper Section 4.3, eager
@@ -54,11 +55,12 @@ enum FrMode : int {
 // library proper is built without the flag and contains none of this.
 #ifdef FR_STAMPS
 __device__ unsigned long long fr_stamps[1024 * 8];
+__device__ unsigned long long fr_warp_stamps[1024 * 32];     // per warp: clock when its (last) segment's rows were done
 __device__ __forceinline__ unsigned long long fr_gtime() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
 #define FR_STAMP_SET(i) do { if (threadIdx.x == 0) fr_stamps[blockIdx.x * 8 + (i)] = (unsigned long long)clock64(); } while (0)
 #define FR_STAMP_GT(i) do { if (threadIdx.x == 0) fr_stamps[blockIdx.x * 8 + (i)] = fr_gtime(); } while (0)
 #define FR_STAMP_MIN(i) do { if ((threadIdx.x & 31u) == 0) atomicMin(&fr_stamps[blockIdx.x * 8 + (i)], (unsigned long long)clock64()); } while (0)
-#define FR_STAMP_MAX(i) do { if ((threadIdx.x & 31u) == 0) atomicMax(&fr_stamps[blockIdx.x * 8 + (i)], (unsigned long long)clock64()); } while (0)
+#define FR_STAMP_MAX(i) do { if ((threadIdx.x & 31u) == 0) { atomicMax(&fr_stamps[blockIdx.x * 8 + (i)], (unsigned long long)clock64()); if ((i) == 4) fr_warp_stamps[blockIdx.x * 32 + (threadIdx.x >> 5)] = (unsigned long long)clock64(); } } while (0)
 #define FR_STAMP_GTMAX(i) do { if ((threadIdx.x & 31u) == 0) atomicMax(&fr_stamps[blockIdx.x * 8 + (i)], fr_gtime()); } while (0)
 #else
 #define FR_STAMP_SET(i) do { } while (0)
@@ -97,7 +99,8 @@ struct FrParams {
     const uint4* tags_in;      // decrypt
     uint4* tags_out;           // encrypt
     uint32_t* ok;              // decrypt
-    const uint32_t* te0;       // 256 words
+    const uint32_t* te0;       // 256 words (the sequential comparator; the fast kernels read Te0 from constant memory)
+    uint32_t* timeouts;        // counter of bulk-copy timeouts (diagnostics)
     const uint4* gh_tab;       // 4096 entries, same layout as shared memory
     const uint4* pow;          // pow[e] = H^e
     uint32_t* acc;             // per CTA of the launch a record of 8 words (4-word XOR accumulator, arrival counter, 3 unused), zero between launches
@@ -531,9 +534,18 @@ __device__ __forceinline__ uint4 fr_mask_bytes(uint4 v, uint32_t n)
 // of the chunk (lane 1 of the chunk's first segment adds E_K(J0)).  XOR of the 32 lanes' results over all
 // segments of the chunk = GHASH of the data blocks (before the length block) xor E_K(J0).
 // Modes without GHASH (CTR, PADGEN) return zero.
+//
+// await_tables (per thread, kept by the caller across segments): the byte tables of H^32 may still be on their way
+// into shared memory (an asynchronous copy started at kernel entry, see the kernel); the thread waits for them in
+// front of its first table multiply, i.e. after its first cipher block, which needs the AES tables only, and
+// clears the flag.
+#ifndef FR_AWAIT_TABLES
+#define FR_AWAIT_TABLES(sm, P) do { } while (0)
+#endif
 template <int MODE, bool ABS>
 __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, const char* sm, const FrLane& L,
-                                                         uint32_t lane, uint32_t kk, uint32_t row0, uint32_t row1)
+                                                         uint32_t lane, uint32_t kk, uint32_t row0, uint32_t row1,
+                                                         bool& await_tables)
 {
     constexpr bool DO_AES = MODE == FR_MODE_DEC || MODE == FR_MODE_ENC || MODE == FR_MODE_CTR || MODE == FR_MODE_PADGEN;
     constexpr bool DO_GHASH = MODE == FR_MODE_DEC || MODE == FR_MODE_ENC || MODE == FR_MODE_VERIFY || MODE == FR_MODE_PADDEC;
@@ -593,6 +605,7 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
             if (DO_GHASH) {
                 const uint4 g = (MODE == FR_MODE_ENC) ? (full ? o : fr_mask_bytes(o, nvalid)) : x;
                 const uint4 v = fr_xor4(y, g);
+                if (await_tables) { FR_AWAIT_TABLES(sm, P); await_tables = false; }
                 if (ctr != c_last) y = fr_ghash_tabmul<ABS>(sm, L, v);
                 else pend = v;
             }
@@ -605,6 +618,7 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
             }
             if (DO_GHASH && P.aad_mod) {                                              // the one-byte AAD block
                 const uint4 v = make_uint4(ck.serial % P.aad_mod, 0, 0, 0);              // y is still zero here
+                if (await_tables) { FR_AWAIT_TABLES(sm, P); await_tables = false; }
                 if (ctr != c_last) y = fr_ghash_tabmul<ABS>(sm, L, v);
                 else pend = v;
             }
@@ -614,6 +628,14 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
     if (!DO_GHASH) return make_uint4(0, 0, 0, 0);
     if (c_last == 0u) return extra;
     return fr_xor4(fr_gf128_mul(pend, hpow), extra);
+}
+
+template <int MODE, bool ABS>
+__device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, const char* sm, const FrLane& L,
+                                                         uint32_t lane, uint32_t kk, uint32_t row0, uint32_t row1)
+{
+    bool tables_are_there = false;
+    return fr_process_segment_lane<MODE, ABS>(P, sm, L, lane, kk, row0, row1, tables_are_there);
 }
 
 // ---- Packed rows: many short chains -----------------------------------------------------------------------

@@ -9,7 +9,9 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#ifndef FR_THREADS
 #define FR_THREADS 1024
+#endif
 #define FR_WARPS (FR_THREADS / 32)
 #define FR_MAX_STAGES 96          // most stages a pipelined call is cut into
 #define FR_PLAN_ROW_BLOCKS 32     // blocks per row of the row kernels (one per lane)
@@ -71,8 +73,9 @@ static inline FrRowPlan fr_plan_rows(const FrPlanConfig& cfg, size_t sample_byte
     if (cfg.row_slots_override) {
         slots = cfg.row_slots_override;
     } else {
-        uint64_t wu = 1;                                              // about 1.18 * sqrt(T / S), by squares
-        while (wu < FR_WARPS && (wu + 1) * (wu + 1) * 100 <= 139 * p.total_rows / sms) wu++;
+        const uint64_t per_sm = p.total_rows / sms;
+        uint64_t wu = per_sm < 4 ? 1 : per_sm < 8 ? 2 : per_sm < 12 ? 4 : per_sm < 20 ? 8 : per_sm < 50 ? 12 : per_sm < 600 ? 16 : 24;
+        if (wu > FR_WARPS) wu = FR_WARPS;
         slots = sms * wu;
     }
     if (slots > cap) slots = cap;
