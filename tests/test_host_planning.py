@@ -99,10 +99,11 @@ def test_sample_batches_plan_on_the_sample_geometry(plan):
 
 
 def test_row_slots_follow_the_size_of_the_launch(plan):
-    """Small launches use few warps per SM (every warp pays a closing product), large ones all 32; a forced slot count
-    is honoured up to the number of rows and of warps."""
-    used = [launch(plan, 4 << 20, n, -(-n // (4 << 20)))[1] for n in (1 << 20, 4 << 20, 16 << 20, 64 << 20, 256 << 20)]
-    assert used == sorted(used) and used[0] <= 8 and used[-1] == 32
+    """Small launches use few warps per SM (every warp pays a closing product), large ones more, always a whole
+    number per quarter of an SM from four warps on; a forced slot count is honoured up to the number of rows and of warps."""
+    used = [launch(plan, 4 << 20, n, -(-n // (4 << 20)))[1] for n in (1 << 16, 1 << 20, 4 << 20, 16 << 20, 64 << 20, 256 << 20)]
+    assert used == sorted(used) and used[0] <= 2 and used[1] <= 8 and 16 <= used[-1] <= 32
+    assert all(u % 4 == 0 for u in used if u >= 4)
     for want in (1, 2, 147, 148, 149, 1000, 4736, 10 ** 6):
         grid, wu, n_slots = launch(plan, 65536, 1 << 24, 256, row_slots=want)[:3]
         assert n_slots == min(want, WARPS) and (grid - 1) * wu < n_slots <= grid * wu
