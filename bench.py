@@ -214,6 +214,43 @@ class Ranks:
             self.dist.destroy_process_group()
 
 
+def build_pipeline_timing() -> str:
+    """Compile bench/pipeline_timing.c (plain C: the library header and the CUDA runtime only) if it is stale."""
+    from paper_2410_15240_b200 import build as lib_build
+    lib = lib_build.build()
+    cuda = os.environ.get("CUDA_HOME", "/usr/local/cuda")
+    src, out = os.path.join(ROOT, "bench", "pipeline_timing.c"), os.path.join(ROOT, "bench", "pipeline_timing")
+    deps = [src, os.path.join(ROOT, "include", "fastrack.h"), lib]
+    if not os.path.exists(out) or any(os.path.getmtime(out) < os.path.getmtime(d) for d in deps):
+        subprocess.check_call(["gcc", "-std=c99", "-O2", "-Wall", "-I", os.path.join(ROOT, "include"), "-I", os.path.join(cuda, "include"),
+                               src, "-o", out + ".tmp", lib, "-L", os.path.join(cuda, "lib64"), "-lcudart",
+                               "-Wl,-rpath," + os.path.dirname(lib), "-Wl,-rpath," + os.path.join(cuda, "lib64")])
+        os.replace(out + ".tmp", out)
+    return out
+
+
+def pipeline_timing(direction: str, length: int, cells, reps: int, batches: int):
+    """Run the C harness on a list of (chunk_bytes, n_streams) cells; returns its JSON objects."""
+    exe = build_pipeline_timing()
+    cmd = [exe, direction, str(length), str(reps), str(batches)] + [f"{cb}:{ns}" for cb, ns in cells]
+    out = subprocess.run(cmd, capture_output=True, text=True, timeout=600)
+    if out.returncode != 0:
+        raise RuntimeError(f"pipeline_timing failed ({out.returncode}): {out.stderr[-500:]}")
+    return [json.loads(line) for line in out.stdout.splitlines() if line.startswith("{")]
+
+
+def traffic_from_profile():
+    """dram__bytes_read.sum + dram__bytes_write.sum of one launch of the headline kernel, from the committed ncu
+    summary (a line `dram_bytes_per_launch = <number>`); None when the file does not carry it."""
+    import re
+    path = os.path.join(ROOT, "profiles", "fr_crypt_kernel_decrypt_verify_256MiB_chunk4MiB.md")
+    try:
+        m = re.search(r"dram_bytes_per_launch\s*=\s*([0-9.eE+]+)", open(path).read())
+        return (float(m.group(1)), os.path.relpath(path, ROOT)) if m else (None, None)
+    except OSError:
+        return None, None
+
+
 def run_gpu(args):
     import numpy as np
     import torch
@@ -223,13 +260,14 @@ def run_gpu(args):
         raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback (use --impl reference for the oracle)")
     torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
     ranks = Ranks("nccl", "cuda")
-    rank, world, local, dist = ranks.rank, ranks.world, ranks.local, ranks.dist
+    rank, world, local = ranks.rank, ranks.world, ranks.local
     barrier, max_over_ranks = ranks.barrier, ranks.max_over_ranks
+    pk = peaks()
+    alu_peak = SMS * ROW_BYTES * pk["sm_max_mhz"] * 1e6 / WAVEFRONTS_PER_ROW_BEST / 1e9
 
     key, iv = synth.key_and_iv(4)
     K = LEN // CHUNK
     ctx = fastrack.Context(key, CHUNK)
-    ctx.reserve(LEN)
     stream = torch.cuda.current_stream()
     st = stream.cuda_stream
 
@@ -269,23 +307,28 @@ def run_gpu(args):
 
     sampler = ClockSampler(local) if rank == 0 else None
     windows = []
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
-    # ---- device-resident metric: exactly K steps, CUDA events on the launching stream, max over ranks
+    def timed_batch(fn, n):
+        """Exactly n calls between two events on the launching stream, a barrier and a synchronise on both sides;
+        returns milliseconds (this rank)."""
+        barrier()
+        w0 = time.time()
+        e0.record(stream)
+        for _ in range(n):
+            fn()
+        e1.record(stream)
+        barrier()
+        windows.append((w0, time.time()))
+        return e0.elapsed_time(e1)
+
+    # ---- device-resident metric: batches of exactly `steps` steps, CUDA events on the launching stream, max over ranks
     for _ in range(args.warmup):
         step()
-    barrier()
     launches0 = ctx.launches
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    w0 = time.time()
-    e0.record(stream)
-    for _ in range(args.steps):
-        step()
-    e1.record(stream)
-    barrier()
-    windows.append((w0, time.time()))
+    batch_ms = [max_over_ranks(timed_batch(step, args.steps)) for _ in range(args.batches)]
     gpu_launches = ctx.launches - launches0
-    ms_this_rank = e0.elapsed_time(e1)
-    ms_total = max_over_ranks(ms_this_rank)
+    ms_total = statistics.median(batch_ms)
     ms_per_step = ms_total / args.steps
     if not (args.kernel_only and args.kernel_pass in ("encrypt_tag", "ctr_crypt")):
         assert bool((d_ok == 1).all()), "verification failed inside the benchmark"
@@ -293,7 +336,7 @@ def run_gpu(args):
         assert bool((d_out == d_plain_src).all()), "decryption mismatch inside the benchmark"
     if args.kernel_only and args.kernel_pass == "encrypt_tag":
         assert bool((d_out == d_cipher).all()) and bool((d_tags2 == d_tags).all()), "encryption mismatch inside the benchmark"
-    value = ranks.aggregate_throughput(LEN * args.steps, ms_this_rank * 1e-3) / 1e9
+    value = world * LEN * args.steps / (ms_total * 1e-3) / 1e9
 
     if args.kernel_only:
         if sampler is not None:
@@ -306,59 +349,63 @@ def run_gpu(args):
         ranks.close()
         return
 
-    # ---- encrypt+tag (mirror path), same size, for the record
+    # ---- encrypt+tag (mirror path), same size
     enc_steps = max(3, min(args.steps, 50))
+
+    def enc_step():
+        ctx.encrypt_tag(iv, d_plain_src.data_ptr(), LEN, d_out.data_ptr(), d_tags.data_ptr(), st)
     for _ in range(3):
-        ctx.encrypt_tag(iv, d_plain_src.data_ptr(), LEN, d_out.data_ptr(), d_tags.data_ptr(), st)
-    barrier()
-    e0.record(stream)
-    for _ in range(enc_steps):
-        ctx.encrypt_tag(iv, d_plain_src.data_ptr(), LEN, d_out.data_ptr(), d_tags.data_ptr(), st)
-    e1.record(stream)
-    barrier()
-    enc_gbs = world * LEN / (max_over_ranks(e0.elapsed_time(e1)) / enc_steps * 1e-3) / 1e9
+        enc_step()
+    enc_ms = statistics.median(max_over_ranks(timed_batch(enc_step, enc_steps)) for _ in range(args.batches))
+    enc_gbs = world * LEN * enc_steps / (enc_ms * 1e-3) / 1e9
 
     # ---- end to end: pinned host ciphertext -> pipelined H2D + decrypt/verify -> verdicts back on the host
     e2e_steps = max(3, min(args.steps, 30))
     for _ in range(3):
         e2e_step()
-    barrier()
-    w0 = time.time()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        e2e_step()
-    torch.cuda.synchronize()
-    e2e_s = max_over_ranks(time.perf_counter() - t0)
-    windows.append((w0, time.time()))
+
+    def wall_batch(fn, n):
+        barrier()
+        w0 = time.time()
+        t0 = time.perf_counter()
+        for _ in range(n):
+            fn()
+        torch.cuda.synchronize()
+        dt = max_over_ranks(time.perf_counter() - t0)
+        windows.append((w0, time.time()))
+        return dt
+    e2e_batches = [wall_batch(e2e_step, e2e_steps) for _ in range(args.batches)]
+    e2e_s = statistics.median(e2e_batches)
     assert bool((h_ok == 1).all())
     e2e_gbs = world * LEN / (e2e_s / e2e_steps) / 1e9
 
     # ---- raw pinned cudaMemcpyAsync of the same bytes, same run (what the pipeline is compared with)
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
+    def raw_step():
         d_out.copy_(h_cipher, non_blocking=True)
         torch.cuda.current_stream().synchronize()
-    raw_s = max_over_ranks(time.perf_counter() - t0)
+    raw_s = statistics.median(wall_batch(raw_step, e2e_steps) for _ in range(args.batches))
     raw_gbs = world * LEN / (raw_s / e2e_steps) / 1e9
 
-    # ---- mirror pipeline: GPU encrypt+tag -> pinned host (device->host copies overlapped), for the record
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        ctx.pipelined_d2h(iv, d_plain_src.data_ptr(), LEN, d_out.data_ptr(), h_cipher.data_ptr(), h_tags.data_ptr(),
-                          args.streams)
-    d2h_gbs = world * LEN / (max_over_ranks(time.perf_counter() - t0) / e2e_steps) / 1e9
+    # ---- mirror pipeline: GPU encrypt+tag -> pinned host (device->host copies overlapped)
+    def d2h_step():
+        ctx.pipelined_d2h(iv, d_plain_src.data_ptr(), LEN, d_out.data_ptr(), h_cipher.data_ptr(), h_tags.data_ptr(), args.streams)
+    d2h_s = statistics.median(wall_batch(d2h_step, e2e_steps) for _ in range(args.batches))
+    d2h_gbs = world * LEN / (d2h_s / e2e_steps) / 1e9
+    ctx.close()
+    del d_plain_src, d_cipher, d_out, h_cipher, plain_h
+
+    # ---- the other configurations (rank 0, single GPU): paper-sized launches, chain sweep, pipelined transfers
+    extra = {"encrypt_tag_gbs": enc_gbs, "pipelined_d2h_encrypt_gbs": d2h_gbs}
+    if rank == 0 and world == 1 and not args.headline_only:
+        extra.update(other_configs(args, alu_peak, windows))
 
     if sampler is not None:
         sampler.stop()
     if rank == 0:
-        pk = peaks()
         clocks = sampler.summary(windows)
         per_gpu = value / world
-        alu_peak = SMS * ROW_BYTES * pk["sm_max_mhz"] * 1e6 / WAVEFRONTS_PER_ROW_BEST / 1e9
         hbm_payload_peak = pk["hbm_gbs"] / 2.0
-        traffic = DRAM_TRAFFIC_BYTES_PER_LAUNCH
+        traffic, traffic_source = traffic_from_profile()
         import oracle
         threads = oracle.host_threads()
         n_sample = max(1, min(64, threads))
@@ -372,12 +419,17 @@ def run_gpu(args):
             "config": {"workload": WORKLOAD, "len_bytes": LEN, "chunk_bytes": CHUNK, "chains": K,
                        "l2": "inputs larger than L2 (256 MiB in + 256 MiB out per step)",
                        "parallelism": "replicas only" if world > 1 else "single GPU", "pipeline_streams": args.streams},
+            "timing": {"batches": args.batches, "steps_per_batch": args.steps, "value_from": "median batch",
+                       "ms_per_step_min": min(batch_ms) / args.steps, "ms_per_step_max": max(batch_ms) / args.steps},
             "clocks": clocks,
             "e2e": {"value": e2e_gbs, "unit": UNIT, "h2d_bytes_per_step": LEN + 16 * K, "d2h_bytes_per_step": 4 * K,
-                    "steps": e2e_steps, "raw_pinned_h2d_gbs": raw_gbs, "fraction_of_raw_pcie": e2e_gbs / raw_gbs},
+                    "steps": e2e_steps, "batches": args.batches, "raw_pinned_h2d_gbs": raw_gbs,
+                    "fraction_of_raw_pcie": e2e_gbs / raw_gbs,
+                    "value_min": world * LEN / (max(e2e_batches) / e2e_steps) / 1e9,
+                    "value_max": world * LEN / (min(e2e_batches) / e2e_steps) / 1e9},
             "gpu_launches": gpu_launches,
             "roofline": {"bound": "alu", "achieved": per_gpu, "peak": alu_peak, "unit": "GB/s", "frac": per_gpu / alu_peak,
-                         "traffic": traffic,
+                         "traffic": traffic, "traffic_source": traffic_source,
                          "peak_source": f"shared-memory lookup rate: {SMS} SMs x 1 wavefront/clk x {pk['sm_max_mhz']:.0f} MHz x "
                                         f"{ROW_BYTES} B per {WAVEFRONTS_PER_ROW_BEST} wavefronts (payload GB/s)",
                          "hbm": {"achieved": 2 * per_gpu, "peak": pk["hbm_gbs"], "frac": 2 * per_gpu / pk["hbm_gbs"],
@@ -386,11 +438,95 @@ def run_gpu(args):
             "cpu_baseline": {"value": cpu_gbs, "unit": UNIT, "cores": threads, "kind": "oracle",
                              "sample": f"{n_sample} of the 64 chunks (4 MiB each), {threads} threads over chunks, {cpu_s:.1f} s",
                              "one_thread_value": cpu_one_gbs},
-            "extra": {"encrypt_tag_gbs": enc_gbs, "pipelined_d2h_encrypt_gbs": d2h_gbs},
+            "extra": extra,
         }
         print(json.dumps(line))
-    ctx.close()
     ranks.close()
+
+
+def other_configs(args, alu_peak, windows):
+    """Benchmark configurations beside the headline cell, for the `extra` object of the bench line.  Device-resident
+    cells: median of `batches` batches of back-to-back calls, CUDA events on the launching stream.  Pipelined cells:
+    the C harness under bench/ (wall clock around the blocking calls, raw copy in the same process)."""
+    import torch
+    from paper_2410_15240_b200 import fastrack, synth
+    key, iv = synth.key_and_iv(1)
+    stream = torch.cuda.current_stream()
+    st = stream.cuda_stream
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed(fn, n_bytes):
+        reps = max(5, min(100, int(1.5e9 // max(n_bytes, 1))))
+        for _ in range(3):
+            fn()
+        out = []
+        for _ in range(args.batches):
+            torch.cuda.synchronize()
+            w0 = time.time()
+            e0.record(stream)
+            for _ in range(reps):
+                fn()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            windows.append((w0, time.time()))
+            out.append(e0.elapsed_time(e1) / reps * 1e-3)
+        return out
+
+    def gbs(n, ts):
+        return {"gbs": n / statistics.median(ts) / 1e9, "gbs_min": n / max(ts) / 1e9, "gbs_max": n / min(ts) / 1e9,
+                "us": statistics.median(ts) * 1e6, "frac_of_roofline": n / statistics.median(ts) / 1e9 / alu_peak}
+
+    def device_cell(n, cb):
+        K = (n + cb - 1) // cb
+        with fastrack.Context(key, cb) as ctx:
+            d_p = torch.randint(0, 256, (n,), dtype=torch.uint8, device="cuda")
+            d_c, d_o = torch.empty_like(d_p), torch.empty_like(d_p)
+            d_t = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
+            d_ok = torch.zeros(K, dtype=torch.int32, device="cuda")
+            t_enc = timed(lambda: ctx.encrypt_tag(iv, d_p.data_ptr(), n, d_c.data_ptr(), d_t.data_ptr(), st), n)
+            t_dec = timed(lambda: ctx.decrypt_verify(iv, d_c.data_ptr(), n, d_t.data_ptr(), d_o.data_ptr(), d_ok.data_ptr(), st), n)
+            assert bool((d_ok == 1).all()) and bool((d_o == d_p).all())
+        return {"len": n, "chunk": cb, "K": K, "decrypt_verify": gbs(n, t_dec), "encrypt_tag": gbs(n, t_enc)}
+
+    def sample_batch_cell(sample_bytes, n_samples, chains):
+        cb = (sample_bytes // chains + 15) // 16 * 16
+        with fastrack.Context(key, cb) as ctx:
+            ctx.set_framing(chains)
+            n = sample_bytes * n_samples
+            K = n_samples * ((sample_bytes + cb - 1) // cb)
+            d_iv = torch.randint(0, 256, (12 * n_samples,), dtype=torch.uint8, device="cuda")
+            d_p = torch.randint(0, 256, (n,), dtype=torch.uint8, device="cuda")
+            d_c, d_o = torch.empty_like(d_p), torch.empty_like(d_p)
+            d_t = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
+            d_ok = torch.zeros(K, dtype=torch.int32, device="cuda")
+            ctx.encrypt_tag_samples(d_iv.data_ptr(), sample_bytes, n_samples, d_p.data_ptr(), d_c.data_ptr(), d_t.data_ptr(), st)
+            t_dec = timed(lambda: ctx.decrypt_verify_samples(d_iv.data_ptr(), sample_bytes, n_samples, d_c.data_ptr(),
+                                                             d_t.data_ptr(), d_o.data_ptr(), d_ok.data_ptr(), st), n)
+            assert bool((d_ok == 1).all()) and bool((d_o == d_p).all())
+        return {"sample_bytes": sample_bytes, "n_samples": n_samples, "chains_per_sample": chains, "chunk": cb, "len": n,
+                "decrypt_verify": gbs(n, t_dec)}
+
+    out = {"timing": f"median of {args.batches} batches of back-to-back calls per cell, min and max beside it"}
+    # paper-sized launches (Sections 5.1 / 5.2: batches of tens of MB), 4 MiB chunks, and a ResNet-style batch of
+    # 64 fp16 images cut into 16 chains each under per-image IVs
+    out["paper_sized"] = [device_cell(n, 4 << 20) for n in (4 << 20, 16 << 20, 64 << 20)]
+    out["sample_batch"] = sample_batch_cell(3 * 224 * 224 * 2, 64, 16)
+    # config 1: 64 MiB cut into K = 1 .. 1024 chains
+    out["config1_chain_sweep"] = [device_cell(64 << 20, (64 << 20) // k) for k in (1, 4, 16, 64, 256, 1024)]
+    # many chains at the headline size: 16 KiB chunks against 4 MiB chunks
+    out["chunk_16KiB"] = [device_cell(n, 16 << 10) for n in (64 << 20, 256 << 20)]
+    # config 3: 670 MB of bf16-sized state, device-resident, and the mirror pipeline
+    out["config3_device"] = device_cell(670_000_000, 4 << 20)
+    torch.cuda.empty_cache()
+    # config 2: the 77 MB fp16 image batch through fastrack_pipelined_h2d, 4 chunk sizes x 2-4 streams
+    w0 = time.time()
+    cells = [(cb, ns) for cb in (256 << 10, 1 << 20, 4 << 20, 8 << 20) for ns in (2, 3, 4)]
+    out["config2_pipelined_h2d"] = pipeline_timing("h2d", 77_070_336, cells, 10, args.batches)
+    out["config3_pipelined_d2h"] = pipeline_timing("d2h", 670_000_000, [(4 << 20, 2), (4 << 20, 4)], 3, args.batches)
+    out["small_transfers_h2d"] = [pipeline_timing("h2d", n, [(65536, 2)], 50, args.batches)[0]
+                                  for n in (256 << 10, 1 << 20, 4 << 20, 16 << 20)]
+    windows.append((w0, time.time()))
+    return out
 
 
 def run_sweep(args):
@@ -624,9 +760,12 @@ def run_peaks(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--streams", type=int, default=4)
+    ap.add_argument("--batches", type=int, default=5,
+                    help="every timed region is repeated this many times; the median is reported, min and max beside it")
+    ap.add_argument("--headline-only", action="store_true", help="skip the other configurations (the `extra` cells)")
     ap.add_argument("--impl", default="fastrack", choices=["fastrack", "reference"])
     ap.add_argument("--kernel-only", action="store_true",
                     help="time only the device-resident decrypt+verify loop (short run for profilers)")
