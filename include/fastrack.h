@@ -72,8 +72,8 @@ extern "C" {
 
 typedef struct fastrack_ctx fastrack_ctx;
 
-/* Context set-up (paper Section 2.3: the hash subkey H = E_K(0^128) "is used throughout the
- * authentication process"; Section 4.2: every chain uses the same H).
+/* Context set-up (paper Section 2.3: one hash subkey H = E_K(0^128) serves the whole authentication;
+ * Section 4.2: every chain uses the same H).
  * Copies the 32-byte AES-256 key (host pointer), expands it into the 15 round keys, derives H, and
  * builds on the current device the tables the kernels need, sized for `chunk_bytes`: the byte tables
  * of the fixed multiplier H^32 (and of H, for launches with many small chunks and for the sequential comparator) and the powers
@@ -95,8 +95,8 @@ FASTRACK_API size_t fastrack_num_chunks(const fastrack_ctx* ctx, size_t len);
  * fastrack_ctx_create; no later call of any kind allocates device memory for it.  Returns FASTRACK_OK. */
 FASTRACK_API int fastrack_ctx_reserve(fastrack_ctx* ctx, size_t max_len);
 
-/* Paper-faithful framing (Section 4.2: every chunk is "attached to one byte of additional authentication data
- * to indicate the chunk order"; Section 4.4: the serial number in the AAD defeats reordering).
+/* Paper-faithful framing (Section 4.2: one byte of additional authenticated data per chunk carries the chunk's
+ * serial number; Section 4.4: that serial number defeats reordering).
  * chains_per_sample = n in 1..256: the buffer is a sequence of samples of n chunks each, and chunk k
  * authenticates the single byte (k mod n) as AAD (so the length block carries an AAD length of 8 bits).
  * chains_per_sample = 0 (the default at creation): AAD empty, chunk order bound by the IV index only.
@@ -124,8 +124,8 @@ FASTRACK_API int fastrack_ctx_set_option(fastrack_ctx* ctx, int option, uint64_t
 /* CUDA error code (cudaError_t as int) of the last failing CUDA call made through ctx, else 0. */
 FASTRACK_API int fastrack_last_cuda_error(const fastrack_ctx* ctx);
 
-/* GPU-side authenticated decryption (paper Section 4.2: "decrypt and authenticate the received
- * data"; decryption kernel = AES-CTR, authentication = GMAC per chunk; here one fused pass).
+/* GPU-side authenticated decryption (paper Section 4.2: the GPU decrypts and authenticates what it
+ * received; decryption kernel = AES-CTR, authentication = GMAC per chunk; here one fused pass).
  *   iv_base  host, 12 bytes.
  *   d_cipher device, len bytes of ciphertext, chunks back to back.
  *   d_tags   device, 16*K bytes, tag of chunk k at byte 16*k.
@@ -216,8 +216,8 @@ FASTRACK_API int fastrack_verify(fastrack_ctx* ctx, const uint8_t iv_base[12], c
 
 /* ---- Sequential-chain comparator (paper Section 4.2, the baseline authentication kernel) ------------------
  * Same inputs, outputs and verdicts as fastrack_verify, computed the way the paper's starting point does it:
- * every chunk's GMAC chain is walked block by block by ONE thread ("the GMAC function will sequentially
- * evaluate m block multiplications"), so the only parallelism is across chunks and the time falls as 1/K when
+ * every chunk's GMAC chain is walked block by block by ONE thread (Section 4.2: the baseline evaluates the m
+ * block multiplications of a chain one after the other), so the only parallelism is across chunks and the time falls as 1/K when
  * a buffer is cut into K chunks (Section 5.3: 16 chains, up to 16x).  It exists to reproduce that curve next
  * to the parallel kernels; do not use it for throughput.  Asynchronous on `stream`; needs no scratch. */
 FASTRACK_API int fastrack_verify_sequential(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_cipher,
@@ -280,7 +280,9 @@ FASTRACK_API int fastrack_decrypt_verify_noalloc(fastrack_ctx* ctx, const uint8_
  *                   Otherwise its contents after the call are unspecified: a transfer too small to be cut (one
  *                   stage, up to about 3 MiB) is written to the host buffers by the kernel itself and skips it.
  *   h_cipher_pinned host, page-locked, len bytes out.
- *   h_tags          host, 16*K bytes out, pinned or pageable.
+ *   h_tags          host, 16*K bytes out, pinned or pageable.  Page-locked is the fast form: the tags of a stage then
+ *                   leave with that stage; tags bound for pageable memory are copied once, after the last stage
+ *                   (a device-to-host copy into pageable memory blocks the host, which would stall the pipeline).
  *   n_streams       1..8.
  * BLOCKING: returns when the ciphertext and the tags are complete in host memory. */
 FASTRACK_API int fastrack_pipelined_d2h(fastrack_ctx* ctx, const uint8_t iv_base[12], const void* d_plain, size_t len,

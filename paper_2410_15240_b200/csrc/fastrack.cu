@@ -272,7 +272,7 @@ __global__ void fr_pow_double_kernel(uint4* pow, uint32_t half, uint32_t n)
 }
 
 // Comparator, not the fast path: the authentication kernel in the shape the paper starts from (Section 4.2:
-// "the GMAC function will sequentially evaluate m block multiplications"; parallel only across chains).
+// the m block multiplications of a chain are evaluated one after the other; parallel only across chains).
 // One THREAD walks one chunk's whole chain, Y <- (Y xor X_i) * H, with the byte tables of H itself in shared
 // memory, then the length block, then E_K(J0) and the tag compare.  Time grows with the chain length, so it
 // falls as 1/K when a buffer is cut into K chunks -- the effect the paper's multi-chaining exploits.
@@ -515,6 +515,7 @@ extern "C" void fastrack_ctx_destroy(fastrack_ctx* ctx)
     if (ctx->d_gh_tab) { cudaMemset(ctx->d_gh_tab, 0, 65536); }
     if (ctx->d_gh1_tab) { cudaMemset(ctx->d_gh1_tab, 0, 65536); }
     if (ctx->d_pow) { cudaMemset(ctx->d_pow, 0, ctx->pow_entries * 16); }
+    if (ctx->d_tags_stage) { cudaMemset(ctx->d_tags_stage, 0, ctx->tags_stage_chunks * 32); }   // its second half held tag masks E_K(J0)
     cudaDeviceSynchronize();
     cudaFree(ctx->d_te0);
     cudaFree(ctx->d_gh_tab);
@@ -842,6 +843,7 @@ static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const vo
         size_t cap = ctx->tags_stage_chunks ? ctx->tags_stage_chunks : 1024;
         while (cap < need_slots) cap *= 2;
         FR_CUDA(ctx, cudaDeviceSynchronize());
+        if (ctx->d_tags_stage) cudaMemset(ctx->d_tags_stage, 0, ctx->tags_stage_chunks * 32);    // tag masks may be in there
         cudaFree(ctx->d_tags_stage);
         ctx->d_tags_stage = nullptr;
         ctx->tags_stage_chunks = 0;
@@ -963,6 +965,8 @@ static int pipelined_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], const vo
     FR_CUDA(ctx, cudaStreamSynchronize(tag_stream));
     if (d_pad) FR_CUDA(ctx, cudaStreamSynchronize(pad_stream));
     for (int i = 0; i < n_streams; i++) FR_CUDA(ctx, cudaStreamSynchronize(ctx->streams[i]));
+    if (d_pad) FR_CUDA(ctx, cudaMemsetAsync(d_mask, 0, 16 * K, tag_stream));   // the tag masks E_K(J0) are as sensitive as H: do not leave them behind
+    if (d_pad) FR_CUDA(ctx, cudaStreamSynchronize(tag_stream));
     if (ctx->trace_on) {
         ctx->trace_count = n_stages < FR_MAX_STAGES ? n_stages : FR_MAX_STAGES;
         for (size_t i = 0; i < ctx->trace_count; i++) {
@@ -1025,6 +1029,7 @@ static int pipelined_d2h_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], cons
         size_t cap = ctx->tags_stage_chunks ? ctx->tags_stage_chunks : 1024;
         while (cap < need_slots) cap *= 2;
         FR_CUDA(ctx, cudaDeviceSynchronize());
+        if (ctx->d_tags_stage) cudaMemset(ctx->d_tags_stage, 0, ctx->tags_stage_chunks * 32);    // tag masks may be in there
         cudaFree(ctx->d_tags_stage);
         ctx->d_tags_stage = nullptr;
         ctx->tags_stage_chunks = 0;
@@ -1072,6 +1077,15 @@ static int pipelined_d2h_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], cons
         FR_CUDA(ctx, se);
         return FASTRACK_OK;
     }
+    // Tags bound for page-locked memory leave with their stage.  A device-to-host copy into pageable memory blocks
+    // the host until it is done, which would keep the next stage's kernel from being queued under the current
+    // copy; such tags stay on the device until every stage is queued and leave in one copy at the end.
+    bool tags_pinned = false;
+    {
+        cudaPointerAttributes ta;
+        if (cudaPointerGetAttributes(&ta, h_tags) == cudaSuccess && ta.type == cudaMemoryTypeHost) tags_pinned = true;
+        (void)cudaGetLastError();
+    }
     bool waited[8] = {false, false, false, false, false, false, false, false};
     size_t off = 0;
     for (size_t i = 0; i < n_stages; i++) {
@@ -1095,8 +1109,8 @@ static int pipelined_d2h_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], cons
         if (rc == FASTRACK_OK) rc = launch_pass(ctx, FR_MODE_ENC, iv_base, k0, n, b, st);
         if (rc == FASTRACK_OK) {
             e = cudaMemcpyAsync((uint8_t*)h_cipher_pinned + off, (const uint8_t*)d_cipher + off, n, cudaMemcpyDeviceToHost, st);
-            if (e == cudaSuccess) e = cudaMemcpyAsync((uint8_t*)h_tags + 16 * k0, ctx->d_tags_stage + k0, 16 * k_here,
-                                                      cudaMemcpyDeviceToHost, st);
+            if (e == cudaSuccess && tags_pinned) e = cudaMemcpyAsync((uint8_t*)h_tags + 16 * k0, ctx->d_tags_stage + k0, 16 * k_here,
+                                                                     cudaMemcpyDeviceToHost, st);
             if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); rc = FASTRACK_ERR_CUDA; }
         }
         if (rc != FASTRACK_OK) {
@@ -1108,6 +1122,7 @@ static int pipelined_d2h_impl(fastrack_ctx* ctx, const uint8_t iv_base[12], cons
     }
     if (sample_bytes) FR_CUDA(ctx, cudaStreamSynchronize(iv_stream));
     for (int i = 0; i < n_streams; i++) FR_CUDA(ctx, cudaStreamSynchronize(ctx->streams[i]));
+    if (!tags_pinned) FR_CUDA(ctx, cudaMemcpy(h_tags, ctx->d_tags_stage, 16 * K, cudaMemcpyDeviceToHost));
     return FASTRACK_OK;
 }
 

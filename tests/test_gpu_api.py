@@ -151,3 +151,46 @@ def test_contexts_on_concurrent_streams_do_not_interfere():
     finally:
         for c in ctxs:
             c[0].close()
+
+
+def test_option_interface():
+    """Unknown options are refused; known ones are accepted at any time and never change results (the layout tests
+    cover the latter; here: a call after a change of layout on a live context is still exact)."""
+    key, iv = synth.key_and_iv(3)
+    cb, n = 4096, 4096 * 37 + 5
+    plain = synth.random_bytes(n, 3, salt=1)
+    c_ref, t_ref = oracle.mc_encrypt(key, iv, cb, plain, oracle.host_threads())
+    K = t_ref.shape[0]
+    with fastrack.Context(key, cb) as ctx:
+        assert fastrack.fastrack_ctx_set_option(ctx.handle, 0, 1) == fastrack.ERR_ARG
+        assert fastrack.fastrack_ctx_set_option(ctx.handle, 99, 1) == fastrack.ERR_ARG
+        d_p = torch.from_numpy(plain).cuda()
+        d_c = torch.empty_like(d_p)
+        d_t = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
+        for options in ({}, {fastrack.OPT_PACK_MAX_BLOCKS: 0}, {fastrack.OPT_ROW_SLOTS: 5}, {fastrack.OPT_PACK_MAX_BLOCKS: 4096, fastrack.OPT_PACK_RUN: 7},
+                        {fastrack.OPT_PACK_RUN: 0, fastrack.OPT_ROW_SLOTS: 0, fastrack.OPT_GENERIC_SMEM: 1, fastrack.OPT_NO_OVERLAP_LAUNCH: 1}):
+            for option, value in options.items():
+                ctx.set_option(option, value)
+            d_c.zero_(); d_t.zero_()
+            ctx.encrypt_tag(iv, d_p.data_ptr(), n, d_c.data_ptr(), d_t.data_ptr(), 0)
+            torch.cuda.synchronize()
+            assert np.array_equal(d_c.cpu().numpy(), c_ref) and np.array_equal(d_t.cpu().numpy().reshape(K, 16), t_ref)
+
+
+@pytest.mark.skipif(torch.cuda.device_count() < 2, reason="needs a second GPU to be the wrong current device")
+def test_calls_on_the_wrong_current_device_are_refused():
+    key, iv = synth.key_and_iv(3)
+    torch.cuda.set_device(0)
+    with fastrack.Context(key, 4096) as ctx:
+        buf = torch.zeros(8192, dtype=torch.uint8, device="cuda:0")
+        tags = torch.zeros(32, dtype=torch.uint8, device="cuda:0")
+        ok = torch.full((2,), 7, dtype=torch.int32, device="cuda:0")
+        torch.cuda.set_device(1)
+        try:
+            rc = fastrack.fastrack_decrypt_verify(ctx.handle, iv, buf.data_ptr(), 8192, tags.data_ptr(), buf.data_ptr(), ok.data_ptr(), 0)
+            assert rc == fastrack.ERR_ARG
+            assert fastrack.fastrack_ctr_crypt(ctx.handle, iv, buf.data_ptr(), 8192, buf.data_ptr(), 0) == fastrack.ERR_ARG
+        finally:
+            torch.cuda.set_device(0)
+        torch.cuda.synchronize()
+        assert bool((ok == 7).all())

@@ -53,11 +53,25 @@ def test_each_chunk_is_a_standalone_openssl_gcm_call(length, cb):
         assert c[k * cb:(k + 1) * cb].tobytes() + tags[k].tobytes() == ref
 
 
-def test_worked_example_structure():
-    """key 00..1f, iv_base 00..0b, P[i] = i, len 64, cb 32: chunk 1 is GCM under IV ..0a0c of P[32:]."""
+def test_worked_example_structure(golden):
+    """key 00..1f, iv_base 00..0b, P[i] = i, len 64, cb 32: chunk 1 is GCM under IV ..0a0c of P[32:].  The stored
+    values (tests/golden/multichain_worked_example.txt) are what SP 800-38D gives under the per-chunk IV rule; they
+    are compared with the oracle and, chunk by chunk, with OpenSSL."""
+    from cryptography.hazmat.primitives.ciphers.aead import AESGCM
+    g = golden("multichain_worked_example.txt")
     key, base = bytes(range(32)), bytes(range(12))
     p = bytes(range(64))
     c, tags = oracle.mc_encrypt(key, base, 32, p)
+    assert g["iv0"] == base and g["iv1"] == bytes(range(11)) + bytes([0x0C])
+    assert c[:32].tobytes() == g["c0"] and tags[0].tobytes() == g["t0"]
+    assert c[32:].tobytes() == g["c1"] and tags[1].tobytes() == g["t1"]
+    assert AESGCM(key).encrypt(g["iv0"], p[:32], None) == g["c0"] + g["t0"]
+    assert AESGCM(key).encrypt(g["iv1"], p[32:], None) == g["c1"] + g["t1"]
+    assert AESGCM(key).encrypt(g["iv1"], p[32:40], None) == g["tail8_c"] + g["tail8_t"]
+    c40g, t40g = oracle.mc_encrypt(key, base, 32, p[:40])
+    assert c40g[32:].tobytes() == g["tail8_c"] and t40g[1].tobytes() == g["tail8_t"]
+    h0 = oracle.hash_subkey(bytes(32))
+    assert oracle.gf128_mul(h0, h0) == g["h_zero_key_squared"]
     c1, t1 = oracle.gcm_encrypt(key, bytes(range(11)) + bytes([0x0C]), b"", p[32:])
     assert c[32:].tobytes() == c1 and tags[1].tobytes() == t1
     # the short-tail variant shares its first chunk and the prefix of chunk 1's keystream
