@@ -193,8 +193,8 @@ __global__ void __launch_bounds__(FR_THREADS, 1) fr_crypt_kernel(const __grid_co
     FR_STAMP_MAX(5); FR_STAMP_GTMAX(6);
 }
 
-// Packed rows (many short chains, see the device header): a warp takes pack_chunks whole chunks and walks their
-// slots 32 at a time; the per-chunk XOR of the lane terms is a segmented inclusive scan over the row (a lane adds
+// Packed rows (many short chains, see the device header): a warp takes a contiguous range of whole chunks and walks
+// their slots 32 at a time; the per-chunk XOR of the lane terms is a segmented inclusive scan over the row (a lane adds
 // the lane d below it only if that lane belongs to the same chunk), a chunk that continues into the next row hands
 // its running sum to that row's lane 0, and the lane holding a chunk's last slot finishes the tag.  No chunk is
 // shared between warps.  The shared-memory GHASH tables hold H here, not H^32.
@@ -206,8 +206,7 @@ __device__ __forceinline__ void fr_packed_body(const FrParams& P, const char* sm
     const FrPackGeom g = fr_pack_geom(P);
 
     for (uint32_t item = warp * gridDim.x + blockIdx.x; item < P.n_items; item += total_warps) {
-        const uint32_t kk0 = item * P.pack_chunks;
-        const uint32_t kk1 = (P.n_chunks - kk0 < P.pack_chunks) ? P.n_chunks : kk0 + P.pack_chunks;
+        const uint32_t kk0 = fr_pack_item_begin(P, item), kk1 = fr_pack_item_begin(P, item + 1u);
         const uint32_t slot_end = fr_pack_slot_begin(P, g, kk1);
         uint4 carry = make_uint4(0, 0, 0, 0);
         for (uint32_t base = fr_pack_slot_begin(P, g, kk0); base < slot_end; base += 32u) {
@@ -269,6 +268,27 @@ __global__ void fr_pow_double_kernel(uint4* pow, uint32_t half, uint32_t n)
     const uint32_t i = half + 1u + blockIdx.x * blockDim.x + threadIdx.x;
     const uint32_t last = (2u * half < n - 1u) ? 2u * half : n - 1u;
     if (i <= last) pow[i] = fr_gf128_mul(pow[i - half], pow[half]);
+}
+
+// Byte tables of H^e, in the layout of the shared-memory image (entry for byte position p and byte value v at
+// uint4 index v * 16 + p), from the table of powers: one block per byte position; eight threads multiply the unit
+// bytes 1 << b at that position by H^e, then thread v XORs the products its bits select.  The packed-row kernels
+// need the tables of H^lanes, which depends on the launch geometry; this runs only when that changes.
+__global__ void __launch_bounds__(256) fr_byte_tables_kernel(const uint4* __restrict__ pow, uint32_t e, uint4* __restrict__ out)
+{
+    __shared__ uint4 basis[8];
+    const uint32_t p = blockIdx.x, v = threadIdx.x;
+    if (v < 8u) {
+        uint32_t w[4] = {0, 0, 0, 0};
+        w[p >> 2] = (1u << v) << (8u * (p & 3u));
+        basis[v] = fr_gf128_mul(make_uint4(w[0], w[1], w[2], w[3]), pow[e]);
+    }
+    __syncthreads();
+    uint4 acc = make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (uint32_t b = 0; b < 8u; b++)
+        if (v & (1u << b)) acc = fr_xor4(acc, basis[b]);
+    out[v * 16u + p] = acc;
 }
 
 // Comparator, not the fast path: the authentication kernel in the shape the paper starts from (Section 4.2:
@@ -345,7 +365,9 @@ struct fastrack_ctx {
     uint8_t h[16];
     uint32_t* d_te0;
     uint4* d_gh_tab;           // byte tables of H^32
-    uint4* d_gh1_tab;          // byte tables of H (sequential-chain comparator only)
+    uint4* d_gh1_tab;          // byte tables of H (packed rows with one lane per chunk, sequential-chain comparator)
+    uint4* d_pack_tab[2];      // byte tables of H^lanes for the packed rows, per scratch bank (see launch_pass)
+    uint32_t pack_tab_lanes[2];   // which power each currently holds (0: none)
     uint4* d_pow;
     size_t pow_entries;
     uint32_t* d_timeouts;      // one word: how often a kernel's bulk copy of the H tables did not arrive in time (see fr_fill_smem)
@@ -457,6 +479,8 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
         if ((e = cudaMalloc(&ctx->d_te0, sizeof te0)) != cudaSuccess) break;
         if ((e = cudaMalloc(&ctx->d_gh_tab, 65536)) != cudaSuccess) break;
         if ((e = cudaMalloc(&ctx->d_gh1_tab, 65536)) != cudaSuccess) break;
+        if ((e = cudaMalloc(&ctx->d_pack_tab[0], 65536)) != cudaSuccess) break;
+        if ((e = cudaMalloc(&ctx->d_pack_tab[1], 65536)) != cudaSuccess) break;
         if ((e = cudaMalloc(&ctx->d_pow, ctx->pow_entries * 16)) != cudaSuccess) break;
         if ((e = cudaMalloc(&ctx->d_scratch, scratch_words(ctx) * sizeof(uint32_t))) != cudaSuccess) break;
         if ((e = cudaMemset(ctx->d_scratch, 0, scratch_words(ctx) * sizeof(uint32_t))) != cudaSuccess) break;
@@ -514,12 +538,16 @@ extern "C" void fastrack_ctx_destroy(fastrack_ctx* ctx)
     cudaDeviceSynchronize();
     if (ctx->d_gh_tab) { cudaMemset(ctx->d_gh_tab, 0, 65536); }
     if (ctx->d_gh1_tab) { cudaMemset(ctx->d_gh1_tab, 0, 65536); }
+    for (int i = 0; i < 2; i++)
+        if (ctx->d_pack_tab[i]) { cudaMemset(ctx->d_pack_tab[i], 0, 65536); }
     if (ctx->d_pow) { cudaMemset(ctx->d_pow, 0, ctx->pow_entries * 16); }
     if (ctx->d_tags_stage) { cudaMemset(ctx->d_tags_stage, 0, ctx->tags_stage_chunks * 32); }   // its second half held tag masks E_K(J0)
     cudaDeviceSynchronize();
     cudaFree(ctx->d_te0);
     cudaFree(ctx->d_gh_tab);
     cudaFree(ctx->d_gh1_tab);
+    cudaFree(ctx->d_pack_tab[0]);
+    cudaFree(ctx->d_pack_tab[1]);
     cudaFree(ctx->d_pow);
     cudaFree(ctx->d_scratch);
     cudaFree(ctx->d_timeouts);
@@ -648,7 +676,6 @@ static bool plan_packed(fastrack_ctx* ctx, int mode, size_t sample_bytes, size_t
     }
     if (!memo.plan.run) return false;
     P.pack_run = memo.plan.run;
-    P.pack_chunks = memo.plan.group;
     P.n_items = memo.plan.n_items;
     return true;
 }
@@ -708,11 +735,34 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
     P.ok = b.ok;
     P.te0 = ctx->d_te0;
     P.timeouts = ctx->d_timeouts;
-    P.gh_tab = packed ? ctx->d_gh1_tab : ctx->d_gh_tab;
+    P.gh_tab = ctx->d_gh_tab;
+    const size_t full_blocks = ((sample_bytes < ctx->chunk_bytes ? sample_bytes : ctx->chunk_bytes) + 15) / 16;
+    bool tables_rebuilt = false;
+    if (packed) {
+        // The packed rows fold with the fixed multiplier H^lanes (lanes = slots per chunk).  H and H^32 exist per
+        // context; any other power gets its byte tables built on the stream, in front of the kernel that needs
+        // them, and is kept until a launch asks for another one.  (Per scratch bank, so that a fastrack_verify on
+        // another stream does not pull the tables from under the pass it overlaps.)
+        const uint32_t lanes = (uint32_t)((full_blocks + P.pack_run) / P.pack_run);
+        if (lanes == 1u) {
+            P.gh_tab = ctx->d_gh1_tab;
+        } else if (lanes != FR_HORNER_STRIDE) {
+            if (ctx->pack_tab_lanes[b.bank] != lanes) {
+                ctx->pack_tab_lanes[b.bank] = 0;
+                fr_byte_tables_kernel<<<16, 256, 0, stream>>>(ctx->d_pow, lanes, ctx->d_pack_tab[b.bank]);
+                ctx->launches++;
+                FR_CUDA(ctx, cudaGetLastError());
+                // a pipelined call issues its stages on several streams: the others must not run ahead of this
+                if (b.window != 0) FR_CUDA(ctx, cudaStreamSynchronize(stream));
+                ctx->pack_tab_lanes[b.bank] = lanes;
+                tables_rebuilt = true;
+            }
+            P.gh_tab = ctx->d_pack_tab[b.bank];
+        }
+    }
     // One lane per chunk (run >= blocks + 1) has a kernel variant of its own that closes with two table steps and needs
     // no reduction across lanes.  It wins while the integer pipes are the busier ones (up to 3 blocks per chunk) or the
     // launch is short enough for the reduction's latency to show; beyond that the general product is the better closing.
-    const size_t full_blocks = ((sample_bytes < ctx->chunk_bytes ? sample_bytes : ctx->chunk_bytes) + 15) / 16;
     const bool whole = packed && P.pack_run > full_blocks &&
                        (full_blocks <= 3 || n_chunks <= 2 * (size_t)ctx->num_sms * FR_THREADS);
     P.pow = ctx->d_pow;
@@ -730,7 +780,7 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
     cfg.dynamicSmemBytes = FR_SMEM_LAUNCH_BYTES;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
-    if (!ctx->no_overlap_launch && !b.plain_launch) {
+    if (!ctx->no_overlap_launch && !b.plain_launch && !tables_rebuilt) {     // (the kernel reads its tables before it waits for its predecessor)
         // let this kernel's table build overlap the tail of the previous kernel in the stream (see the kernel)
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[0].val.programmaticStreamSerializationAllowed = 1;

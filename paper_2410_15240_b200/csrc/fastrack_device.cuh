@@ -79,7 +79,7 @@ struct FrParams {
     uint32_t n_slots;          // row kernels: warps that take work; slot j is warp j % warps_used of CTA j / warps_used
     uint32_t warps_used;       // row kernels: slots per CTA
     uint32_t n_chunks;         // chunks in this launch
-    uint32_t n_items;          // packed rows: work items
+    uint32_t n_items;          // packed rows: work items (warps that take work); item j covers chunks j * n_chunks / n_items .. (j + 1) * n_chunks / n_items - 1
     uint32_t generic_smem;     // 1: use the portable shared-memory addressing even where the absolute form would do
     uint32_t aad_mod;          // 0: no AAD; n: a chunk authenticates the one byte (its serial number mod n) as AAD
     uint64_t len;              // bytes in this launch
@@ -90,8 +90,8 @@ struct FrParams {
     uint32_t rows_full;        // rows of a full-size chunk
     uint32_t rows_last;        // rows of a sample's last chunk
     uint32_t chunks_per_sample;  // ceil(sample_bytes / chunk_bytes); only a sample's last chunk may be short
-    uint32_t pack_chunks;        // packed rows: chunks per work item; then n_items = ceil(n_chunks / pack_chunks)
-    uint32_t pack_run;           // packed rows: consecutive counters per slot (lane)
+    uint32_t pack_pad;
+    uint32_t pack_run;           // packed rows: most counters per slot (lane); a full chunk has ceil((blocks + 1) / pack_run) slots
     uint32_t pad2;
     const uint8_t* ivs;        // per-sample 12-byte IV bases (device), or null: one IV base for the whole launch
     const uint8_t* in;
@@ -641,38 +641,43 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
 // ---- Packed rows: many short chains -----------------------------------------------------------------------
 // The row layout above gives one warp 32 consecutive blocks of ONE chunk; a 16-byte chunk would keep 2 of its 32
 // lanes busy, and every chunk pays a closing product, a warp reduction and a ticket.  When a launch has many
-// chunks that are not large, it is laid out the other way round: a chunk's counters 1 .. nblk+1 (counter 1 = the
-// tag mask E_K(J0) and, under the serial-number framing, the AAD block; counter c >= 2 = data block c - 2) are cut
-// into runs of `pack_run` consecutive counters, one run = one SLOT = one lane.  A lane walks its run block by
-// block -- counter mode with the first two rounds shared as above, Horner's rule with the FIXED multiplier H
-// (byte tables of H in shared memory, same conflict-free lane rotation) -- and multiplies the result by the power
-// of H that aligns it to the end of the chunk.  Slots of a chunk are consecutive, a warp takes a run of whole chunks
-// and walks their slots 32 at a time; the per-chunk XOR of the lane terms is a segmented scan in the calling
-// kernel.  No chunk is shared between warps, so this path needs neither atomics nor scratch memory.  Lanes read
-// and write 16 bytes at a stride of 16 * pack_run bytes: short runs keep those accesses in few cache lines, long runs
-// amortise the closing product; the host picks the run length.
+// chunks that are not large, it is laid out the other way round.  A chunk's counters 1 .. nblk+1 (counter 1 = the
+// tag mask E_K(J0) and, under the serial-number framing, the AAD block; counter c >= 2 = data block c - 2) are
+// dealt to `lanes` = ceil((nblk + 1) / pack_run) SLOTS, one slot = one lane, round-robin: slot i takes counters
+// 1 + i, 1 + i + lanes, 1 + i + 2 * lanes, ...  (at most pack_run of them).  At every step the slots of a chunk
+// therefore touch 16 * lanes contiguous bytes, and a lane folds its blocks with Horner's rule and the FIXED
+// multiplier H^lanes (byte tables of that power in shared memory, same conflict-free lane rotation; built for the
+// launch by the host code), then multiplies by the power of H that aligns its last block to the end of the chunk.
+// Slots of a chunk are consecutive lanes, a warp takes a run of whole chunks and walks their slots 32 at a time;
+// the per-chunk XOR of the lane terms is a segmented scan in the calling kernel.  No chunk is shared between
+// warps, so this path needs neither atomics nor scratch memory.  Few lanes per chunk mean few closing products;
+// many lanes mean long contiguous pieces per memory request; lane counts that divide the number of counters
+// leave no lane idle.  The host picks.  (A sample's short last chunk gets the same number of slots as the
+// others, some of them empty.)
 struct FrPackGeom {
-    uint32_t run;               // counters per slot
-    uint32_t slots_full;        // slots of a full-size chunk
-    uint32_t slots_sample;      // slots of a whole sample
+    uint32_t lanes;             // slots of a chunk = stride of a slot's counters
 };
 
 __device__ __forceinline__ FrPackGeom fr_pack_geom(const FrParams& P)
 {
     const uint64_t first_len = P.sample_bytes < P.chunk_bytes ? P.sample_bytes : P.chunk_bytes;
-    const uint64_t last_len = P.sample_bytes - (uint64_t)(P.chunks_per_sample - 1u) * P.chunk_bytes;
     FrPackGeom g;
-    g.run = P.pack_run;
-    g.slots_full = ((uint32_t)((first_len + 15) >> 4) + g.run) / g.run;                  // ceil((nblk + 1) / run)
-    g.slots_sample = (P.chunks_per_sample - 1u) * g.slots_full + ((uint32_t)((last_len + 15) >> 4) + g.run) / g.run;
+    g.lanes = ((uint32_t)((first_len + 15) >> 4) + P.pack_run) / P.pack_run;         // ceil((nblk + 1) / run)
     return g;
 }
 
 // First slot of chunk kk (kk = n_chunks gives the total).
 __device__ __forceinline__ uint32_t fr_pack_slot_begin(const FrParams& P, const FrPackGeom& g, uint32_t kk)
 {
-    const uint32_t sample = kk / P.chunks_per_sample, k = kk - sample * P.chunks_per_sample;
-    return sample * g.slots_sample + k * g.slots_full;
+    (void)P;
+    return kk * g.lanes;
+}
+
+// Work item j of the packed rows: a contiguous range of whole chunks, all ranges equally long to within one chunk
+// (n_items <= n_chunks, so none is empty).
+__device__ __forceinline__ uint32_t fr_pack_item_begin(const FrParams& P, uint32_t j)      // j in 0 .. n_items
+{
+    return (uint32_t)((uint64_t)j * P.n_chunks / P.n_items);
 }
 
 struct FrSlot {
@@ -681,11 +686,11 @@ struct FrSlot {
     uint32_t last;      // index of the chunk's last slot
 };
 
-// One slot: encrypt or decrypt the blocks of its run (counter 1: produce the tag mask) and return the slot's
-// term of the tag, sum over its counters c of block_c * H^(nblk + 3 - c), plus E_K(J0) from counter 1.
-// XOR over a chunk's slots, plus the length term, is its tag.
-// WHOLE: every run is a whole chunk (one lane per chunk).  The run then always ends with the chunk's last block,
-// whose factor is H^2, so the closing product is two more table steps instead of the general product (the lookup
+// One slot: encrypt or decrypt its blocks (counter 1: produce the tag mask) and return the slot's term of the
+// tag, sum over its counters c of block_c * H^(nblk + 3 - c), plus E_K(J0) from counter 1.  XOR over a chunk's
+// slots, plus the length term, is its tag.
+// WHOLE: one lane per chunk.  The lane then always ends with the chunk's last block, whose factor is H^2, so the
+// closing product is two more table steps (the table is that of H) instead of the general product (the lookup
 // pipe has room for them where the integer pipes, busy with two ciphers per handful of bytes, do not), and the
 // value returned is the chunk's complete tag sum: the caller needs no reduction across lanes.
 template <int MODE, bool ABS, bool WHOLE>
@@ -696,30 +701,40 @@ __device__ __forceinline__ uint4 fr_packed_slot_lane(const FrParams& P, const ch
                   "packed rows exist for the fused passes and their two halves");
     constexpr bool DO_AES = MODE != FR_MODE_VERIFY;       // VERIFY still needs E_K(J0), counter 1
     constexpr bool DO_GHASH = MODE != FR_MODE_CTR;
-    const uint32_t sample = slot / g.slots_sample, t = slot - sample * g.slots_sample;
-    const uint32_t k = t / g.slots_full, i = t - k * g.slots_full;
-    const uint32_t kk = sample * P.chunks_per_sample + k;
+    const uint32_t kk = slot / g.lanes, i = slot - kk * g.lanes;
     const FrChunk ck = fr_chunk_info(P, kk);
     const uint32_t nblk = (uint32_t)((ck.len + 15) >> 4);
-    si.kk = kk; si.i = i; si.last = nblk / g.run;                        // ceil((nblk + 1) / run) - 1
-    const uint32_t c0 = i * g.run + 1u;                                  // the run's counters are c0 .. c1 - 1
-    uint32_t c1 = c0 + g.run;
-    if (c1 > nblk + 2u) c1 = nblk + 2u;
+    si.kk = kk; si.i = i; si.last = g.lanes - 1u;
+    // The slot's counters.  Data block j (counter j + 2) belongs to slot j mod lanes and is worked on in step
+    // 1 + j / lanes, so that in every step the slots of a chunk touch `lanes` consecutive blocks that start on a
+    // multiple of `lanes` blocks -- whole 32-byte sectors for even lane counts.  Counter 1 (tag mask and AAD block)
+    // is "block -1": it goes to the last slot, in a step 0 of its own in which the other slots idle, which keeps
+    // that slot's stride at `lanes` as well.
+    const uint32_t c_end = nblk + 2u;
+    const bool last_slot = (i + 1u == g.lanes);
+    const uint32_t steps = 1u + (nblk + g.lanes - 1u) / g.lanes;          // the same for every slot of the chunk
+    uint32_t c_last;                                                       // the slot's last counter
+    if (i + 2u < c_end) c_last = i + 2u + (c_end - 3u - i) / g.lanes * g.lanes;
+    else if (last_slot) c_last = 1u;
+    else return make_uint4(0, 0, 0, 0);                                    // an empty slot (a short last chunk)
     uint4 hpow = make_uint4(0, 0, 0, 0);
-    if (DO_GHASH && !WHOLE) hpow = P.pow[nblk + 4u - c1];                // for the run's last block, counter c1 - 1
+    if (DO_GHASH && !WHOLE) hpow = P.pow[nblk + 3u - c_last];
     const uint8_t* in = P.in + ck.off;
     uint8_t* out = P.out + ck.off;
     FrCtrChunk cc = {0, 0, 0, 0};
     FrCtrGroup cg = {0, 0, 0, 0};
-    if (DO_AES || c0 == 1u) {
-        cc = fr_ctr_chunk<ABS>(sm, L.lane4, P, ck.iv_w0, ck.iv_w1, fr_bswap(ck.iv_ctr));
-        cg = fr_ctr_group<ABS>(sm, L.lane4, P, cc, c0);
-    }
+    uint32_t group = 0xFFFFFFFFu;                                        // 256-counter group that cg belongs to
+    if (DO_AES || last_slot) cc = fr_ctr_chunk<ABS>(sm, L.lane4, P, ck.iv_w0, ck.iv_w1, fr_bswap(ck.iv_ctr));
     uint4 y = make_uint4(0, 0, 0, 0), extra = make_uint4(0, 0, 0, 0);
-    for (uint32_t c = c0; c < c1; c++) {
-        if (DO_AES && (c & 255u) == 0u && c != c0) cg = fr_ctr_group<ABS>(sm, L.lane4, P, cc, c);   // entered the next 256-counter group
+    for (uint32_t t = 0; t < steps; t++) {                               // every slot of the chunk walks the same steps, in step
+        const uint32_t c = t ? i + 2u + (t - 1u) * g.lanes : 1u;
+        if (t ? c >= c_end : !last_slot) continue;                         // idle: step 0 for all but the last slot, the last step past the end
+        const bool cipher = DO_AES ? (DO_GHASH || c != 1u) : (c == 1u);
         uint4 ks = make_uint4(0, 0, 0, 0);
-        if (DO_AES ? (DO_GHASH || c != 1u) : (c == 1u)) ks = fr_aes256_ctr_block<ABS>(sm, L.lane4, P, cc, cg, c);
+        if (cipher) {
+            if ((c >> 8) != group) { cg = fr_ctr_group<ABS>(sm, L.lane4, P, cc, c); group = c >> 8; }   // entered another 256-counter group
+            ks = fr_aes256_ctr_block<ABS>(sm, L.lane4, P, cc, cg, c);
+        }
         uint4 gblk;
         if (c == 1u) {
             extra = ks;                                                                      // E_K(J0)
@@ -738,10 +753,10 @@ __device__ __forceinline__ uint4 fr_packed_slot_lane(const FrParams& P, const ch
         }
         if (DO_GHASH) {
             y = fr_xor4(y, gblk);
-            // Horner step with the fixed multiplier H -- not after the run's last block (the closing product follows),
-            // and not at counter 1 without AAD, where y is still zero (when every lane of a warp starts its run
+            // Horner step with the fixed multiplier H^lanes -- not after the slot's last block (the closing product
+            // follows), and not at counter 1 without AAD, where y is still zero (when every lane of a warp starts
             // there -- one lane per small chunk -- the whole step is skipped)
-            if (c + 1u != c1 && (c != 1u || P.aad_mod)) y = fr_ghash_tabmul<ABS>(sm, L, y);
+            if (c != c_last && (c != 1u || P.aad_mod)) y = fr_ghash_tabmul<ABS>(sm, L, y);
         }
     }
     if (!DO_GHASH) return make_uint4(0, 0, 0, 0);

@@ -16,7 +16,6 @@
 #define FR_MAX_STAGES 96          // most stages a pipelined call is cut into
 #define FR_PLAN_ROW_BLOCKS 32     // blocks per row of the row kernels (one per lane)
 #define FR_PACK_MAX_BLOCKS 4096   // chunks of more blocks than this never take the packed-row kernels
-#define FR_PACK_MAX_ITEM_SLOTS 1024   // most runs (lanes' worth of work) in one packed work item
 
 struct FrPlanConfig {
     int num_sms;
@@ -41,9 +40,8 @@ struct FrRowPlan {
 };
 
 struct FrPackPlan {
-    uint32_t run;               // counters per lane; 0 = use the row kernels
-    uint32_t group;             // whole chunks per work item
-    uint32_t n_items;           // ceil(n_chunks / group)
+    uint32_t run;               // most counters per lane; 0 = use the row kernels.  A chunk has ceil(counters / run) lanes
+    uint32_t n_items;           // warps that take work; item j covers chunks j * n_chunks / n_items .. (j + 1) * n_chunks / n_items - 1
 };
 
 enum FrPassKind : int { FR_PASS_FUSED = 0, FR_PASS_CTR = 1, FR_PASS_VERIFY = 2 };
@@ -90,31 +88,29 @@ static inline FrRowPlan fr_plan_rows(const FrPlanConfig& cfg, size_t sample_byte
 // Cost constants of the two layouts for one kind of pass, in SM clocks.
 struct FrPackCosts {
     size_t row_clocks, seg_clocks, row_step_latency;      // row kernels: per row, per segment; latency of a row for a lone warp
-    size_t fixed, step_latency;                           // packed rows: per row of 32 runs; latency per counter for a lone warp
-    size_t step[14];                                      // packed rows: clocks per counter of a run, by run length (0 unused)
-    size_t step_long;                                     // ... for longer runs
+    size_t close, step, step_latency;                     // packed rows, per row of 32 lanes: the closing; one counter step; its latency for a lone warp
 };
 
 // Decides between the row kernels (`rows` is their plan) and the packed-row kernels, and in the latter case picks
-// the run length and the work-item size.  Both are judged by the same kind of estimate: the shared-memory work of
-// the busiest SM or the latency of the busiest warp, whichever is larger (plus a quarter of the other: between the
-// two regimes both show).  For the fused passes a row kernel costs about 285 clocks per row plus 400 per segment;
-// a packed row costs about 280 plus, per counter of its run, 258 clocks for runs up to 3 counters and more beyond (a
-// lane's 16-byte loads and stores are 16 * run bytes apart, so longer runs touch more cache lines per request; runs
-// whose byte stride is a power of two do worst: the lanes' pieces fall on the same few cache banks).  The two
-// halves of the fused pass have constants of their own.
+// how many lanes share a chunk and how many warps take work.  Both layouts are judged by the same kind of
+// estimate: the shared-memory work of the busiest SM or the latency of the busiest warp, whichever is larger
+// (plus a quarter of the other: between the two regimes both show).
+// Packed rows: a chunk of B blocks on L lanes takes S = 1 + ceil(B / L) steps (one for counter 1, in which only
+// one lane of the chunk works); a warp that holds n chunks walks ceil(n * L / 32) rows of S steps each plus one
+// closing per row.  Few lanes per chunk mean long runs and few closings, but coarse rows (a warp's last row is
+// partly empty) and short contiguous pieces per memory request (16 * L bytes: an odd number of blocks does not
+// fill whole 32-byte sectors, which costs extra cycles on the memory pipe that bounds the kernel); lane counts
+// that do not divide B leave lanes idle in the last step.  All of that is counted below; the constants are fitted
+// to measurements on B200.
 static inline FrPackPlan fr_plan_packed(const FrPlanConfig& cfg, int kind, size_t sample_bytes, size_t n_chunks,
                                         const FrRowPlan& rows)
 {
     static const FrPackCosts costs[3] = {
-        // fused passes: cipher + Horner step per counter, one general product per run
-        {285, 400, 1000, 280, 2250, {0, 258, 257, 256, 289, 264, 281, 330, 396, 302, 304, 304, 327, 305}, 335},
-        // counter mode only: no product, no reduction
-        {218, 100, 900, 30, 2000, {0, 227, 227, 227, 245, 227, 240, 270, 330, 250, 252, 252, 270, 255}, 260},
-        // verify only: no cipher (but counter 1), so the closing product weighs more and longer runs pay
-        {85, 400, 300, 465, 700, {0, 65, 65, 65, 80, 65, 75, 85, 120, 86, 88, 88, 100, 90}, 95},
+        {279, 400, 1000, 300, 279, 2250},     // fused passes: cipher + Horner step per counter, one general product per lane
+        {218, 100, 900, 30, 227, 2000},       // counter mode only: no product, no reduction
+        {85, 400, 300, 465, 65, 700},         // verify only: no cipher (but counter 1), so the closing weighs more
     };
-    const FrPackPlan rows_kernels = {0, 0, 0};
+    const FrPackPlan rows_kernels = {0, 0};
     if (!cfg.pack_max_blocks || n_chunks == 0) return rows_kernels;
     const FrPackCosts& C = costs[kind];
     const size_t first_len = sample_bytes < cfg.chunk_bytes ? sample_bytes : cfg.chunk_bytes;
@@ -131,39 +127,44 @@ static inline FrPackPlan fr_plan_packed(const FrPlanConfig& cfg, int kind, size_
     const size_t row_lat = rows_per_slot * C.row_step_latency + segs_per_slot * 4000;
     const size_t row_cost = row_thr > row_lat ? row_thr : row_lat;
 
-    size_t best_run = 0, best_group = 1, best_cost = ~(size_t)0;
-    const size_t cand[] = {1, 2, 3, 4, 5, 6, 9, 10, 11, 13, counters <= 64 ? counters : 5};
-    for (size_t run : cand) {
-        if (cfg.pack_run_override) run = cfg.pack_run_override;
-        if (run > counters) run = counters;
-        const size_t slots = (counters + run - 1) / run;
-        // slots and chunks are counted in 32 bits; a row may overshoot by 31, an item's first chunk index by its size
-        if (n_chunks * slots >= ((size_t)1 << 32) - 2 * FR_PACK_MAX_ITEM_SLOTS) continue;
-        const size_t per_row = C.fixed + run * (run < 14 ? C.step[run] : C.step_long);
-        const size_t row_latency = 2500 + run * C.step_latency;       // one warp alone on its SM partition
-        // a work item is `group` whole chunks.  Its last row is only partly filled, and an instruction costs the same
-        // with idle lanes; on the other hand a launch with fewer items than warps leaves warps idle.  Try a range of
-        // item sizes and count the rows each really takes.
-        const size_t sizes[] = {1, 2, 3, 4, 5, 6, 8, 10, 12, 16, 24, 32, 48, 64, 96, 128, 256, 512,
-                                32 / slots, 64 / slots, 128 / slots, 256 / slots, 512 / slots};
-        for (size_t group : sizes) {
-            if (cfg.pack_group_override) group = cfg.pack_group_override;
-            if (group < 1 || group * slots > FR_PACK_MAX_ITEM_SLOTS) continue;
-            if (group > n_chunks) group = n_chunks;
-            const size_t rows_per_item = (group * slots + 31) / 32;
-            const size_t items = (n_chunks + group - 1) / group;
-            const size_t thr = (items * rows_per_item + sms - 1) / sms * per_row;
-            const size_t lat = (items + warps - 1) / warps * rows_per_item * row_latency;
+    size_t best_run = 0, best_items = 1, best_cost = ~(size_t)0;
+    const size_t max_lanes = counters < 64 ? counters : 64;
+    for (size_t lanes = 1; lanes <= max_lanes + 1; lanes++) {
+        size_t run = lanes <= max_lanes ? (counters + lanes - 1) / lanes : 1;     // (last round: one counter per lane)
+        if (cfg.pack_run_override) run = cfg.pack_run_override < counters ? cfg.pack_run_override : counters;
+        const size_t l = (counters + run - 1) / run;                               // the lane count this run length gives
+        if (!cfg.pack_run_override && lanes <= max_lanes && l != lanes) continue;  // not reachable as ceil(counters / run)
+        const size_t steps = 1 + (counters - 1 + l - 1) / l;
+        // slots and chunks are counted in 32 bits; a row may overshoot by 31 slots
+        if (n_chunks * l >= ((size_t)1 << 32) - 64) continue;
+        // memory pipe: a chunk's lanes touch 16 * l contiguous bytes per step, starting on a multiple of that; per row of
+        // 32 lanes that is 32 / l such pieces against the 16 sectors of a dense request
+        const size_t row_sectors2 = (64 * ((l + 1) / 2) + l - 1) / l;                              // twice the sectors per row
+        const size_t extra = row_sectors2 > 32 ? (row_sectors2 - 32) * 5 / 4 : 0;                  // about 2.5 clocks per extra sector, load and store
+        const size_t per_row = C.close + steps * (C.step + extra);
+        const size_t row_latency = 2500 + steps * C.step_latency;       // one warp alone on its SM partition
+        // a work item is one warp's contiguous range of whole chunks, and every warp takes one (fewer warps with longer
+        // ranges would fill their last rows better, but measured slower)
+        for (size_t div = 1; div <= 1; div *= 2) {
+            size_t items = warps / div;
+            if (cfg.pack_group_override) items = (n_chunks + cfg.pack_group_override - 1) / cfg.pack_group_override;
+            if (items > n_chunks) items = n_chunks;
+            if (items < 1) items = 1;
+            const size_t most = (n_chunks + items - 1) / items;                    // chunks of the longest item
+            const size_t rows_most = (most * l + 31) / 32;
+            const size_t per_sm = (items + sms - 1) / sms;                          // warps of the busiest SM
+            const size_t thr = per_sm * rows_most * per_row;
+            const size_t lat = rows_most * row_latency;
             const size_t cost = thr > lat ? thr + lat / 4 : lat + thr / 4;
-            if (cost < best_cost) { best_cost = cost; best_run = run; best_group = group; }
+            if (cost < best_cost) { best_cost = cost; best_run = run; best_items = items; }
         }
+        if (cfg.pack_run_override) break;
     }
     if (!best_run) return rows_kernels;
     if (!cfg.pack_run_override && best_cost >= row_cost) return rows_kernels;
     FrPackPlan p;
     p.run = (uint32_t)best_run;
-    p.group = (uint32_t)best_group;
-    p.n_items = (uint32_t)((n_chunks + best_group - 1) / best_group);
+    p.n_items = (uint32_t)best_items;
     return p;
 }
 

@@ -62,7 +62,7 @@ struct Setup {
 };
 
 // The same derivation fastrack_ctx_create performs (host part) plus the power table and the shared-memory fill.
-void setup(Setup& S, const uint8_t key[32], size_t cb, int squarings = 5)   // byte tables of H^(2^squarings): H^32, or H for the packed rows
+void setup(Setup& S, const uint8_t key[32], size_t cb, uint32_t power = 32)   // byte tables of H^power: H^32 for the rows, H^lanes for the packed rows
 {
     memset(&S.P, 0, sizeof S.P);
     uint8_t sbox[256];
@@ -74,8 +74,9 @@ void setup(Setup& S, const uint8_t key[32], size_t cb, int squarings = 5)   // b
     expand_key(key, sbox, S.P.rk);
     const uint8_t zero[16] = {0};
     encrypt_block_host(S.P.rk, S.te0, sbox, zero, S.h);
-    Gf128 G = gf_load(S.h);
-    for (int i = 0; i < squarings; i++) G = gf_mul(G, G);
+    const Gf128 H = gf_load(S.h);
+    Gf128 G = H;
+    for (uint32_t i = 1; i < power; i++) G = gf_mul(G, H);
     S.gh_tab.assign(65536, 0);
     for (int p = 0; p < 16; p++) {
         Gf128 basis[8];
@@ -260,8 +261,8 @@ static void run_packed(Setup& S, const uint8_t* tags_in, uint8_t* tags_out, uint
     FrParams& P = S.P;
     const FrPackGeom g = fr_pack_geom(P);
     for (uint32_t item = 0; item < P.n_items; item++) {
-        const uint32_t kk0 = item * P.pack_chunks;
-        const uint32_t kk1 = (P.n_chunks - kk0 < P.pack_chunks) ? P.n_chunks : kk0 + P.pack_chunks;
+        const uint32_t kk0 = fr_pack_item_begin(P, item), kk1 = fr_pack_item_begin(P, item + 1u);
+        if (kk1 <= kk0 || kk1 > P.n_chunks) abort();                       // no empty item, nothing past the end
         const uint32_t slot_end = fr_pack_slot_begin(P, g, kk1);
         uint4 carry = {0, 0, 0, 0};
         for (uint32_t base = fr_pack_slot_begin(P, g, kk0); base < slot_end; base += 32u) {
@@ -299,13 +300,16 @@ static void run_packed(Setup& S, const uint8_t* tags_in, uint8_t* tags_out, uint
     }
 }
 
-// One packed-row pass (mode 0 = decrypt + verify, 1 = encrypt + tag, 2 = counter mode only, 3 = verify only): pack_run counters per slot, pack_chunks chunks per work item.
+// One packed-row pass (mode 0 = decrypt + verify, 1 = encrypt + tag, 2 = counter mode only, 3 = verify only): at most pack_run counters per slot, about pack_chunks chunks per work item.
 extern "C" int emu_packed(int mode, const uint8_t* key, const uint8_t* iv_base, size_t cb, const uint8_t* in, size_t len,
                           uint8_t* out, const uint8_t* tags_in, uint8_t* tags_out, uint32_t* ok, uint32_t pack_chunks,
                           uint32_t pack_run, uint32_t first_chunk, uint32_t aad_mod, size_t sample_bytes, const uint8_t* ivs)
 {
+    if (sample_bytes == 0) sample_bytes = len;
+    const uint32_t run_ = pack_run ? pack_run : 1;
+    const uint32_t lanes = (uint32_t)(((std::min(sample_bytes, cb) + 15) / 16 + run_) / run_);      // slots per chunk, as fr_pack_geom has it
     Setup S;
-    setup(S, key, cb, 0);
+    setup(S, key, cb, lanes);
     FrParams& P = S.P;
     auto be32 = [](const uint8_t* p) { return ((uint32_t)p[0] << 24) | ((uint32_t)p[1] << 16) | ((uint32_t)p[2] << 8) | p[3]; };
     auto le32 = [](const uint8_t* p) { return ((uint32_t)p[3] << 24) | ((uint32_t)p[2] << 16) | ((uint32_t)p[1] << 8) | p[0]; };
@@ -323,9 +327,8 @@ extern "C" int emu_packed(int mode, const uint8_t* key, const uint8_t* iv_base, 
     P.chunks_per_sample = (uint32_t)cps;
     P.ivs = ivs;
     P.n_chunks = (uint32_t)n_chunks;
-    P.pack_chunks = pack_chunks ? pack_chunks : 1;
     P.pack_run = pack_run ? pack_run : 1;
-    P.n_items = (uint32_t)((n_chunks + P.pack_chunks - 1) / P.pack_chunks);
+    P.n_items = (uint32_t)((n_chunks + (pack_chunks ? pack_chunks : 1) - 1) / (pack_chunks ? pack_chunks : 1));   // items of about pack_chunks chunks
     P.lenh_full = length_term(S, std::min(sample_bytes, cb), aad_mod);
     P.lenh_last = length_term(S, sample_bytes - (cps - 1) * cb, aad_mod);
     P.in = in;

@@ -13,7 +13,7 @@ static FrPlanConfig make(int num_sms, size_t chunk_bytes, uint32_t row_slots, ui
     return c;
 }
 
-// out[0..2] = grid, warps_used, n_slots of the row kernels; out[3..5] = run, group, n_items of the packed rows;
+// out[0..2] = grid, warps_used, n_slots of the row kernels; out[3..5] = run, lanes per chunk, n_items of the packed rows;
 // out[6..9] = rows_full, rows_last, rows_sample, total_rows
 void plan_launch(int num_sms, size_t chunk_bytes, uint32_t row_slots, uint32_t pack_max, uint32_t run, uint32_t group, int kind,
                  size_t sample_bytes, size_t n_chunks, uint64_t out[10])
@@ -22,7 +22,8 @@ void plan_launch(int num_sms, size_t chunk_bytes, uint32_t row_slots, uint32_t p
     const FrRowPlan r = fr_plan_rows(c, sample_bytes, n_chunks);
     const FrPackPlan p = fr_plan_packed(c, kind, sample_bytes, n_chunks, r);
     out[0] = r.grid; out[1] = r.warps_used; out[2] = r.n_slots;
-    out[3] = p.run; out[4] = p.group; out[5] = p.n_items;
+    const size_t first_len = sample_bytes < chunk_bytes ? sample_bytes : chunk_bytes;
+    out[3] = p.run; out[4] = p.run ? ((first_len + 15) / 16 + p.run) / p.run : 0; out[5] = p.n_items;
     out[6] = r.rows_full; out[7] = r.rows_last; out[8] = r.rows_sample; out[9] = r.total_rows;
 }
 
@@ -33,6 +34,5 @@ size_t plan_stages(size_t chunk_bytes, size_t stage_bytes, size_t len, size_t un
 }
 
 int plan_max_stages(void) { return FR_MAX_STAGES; }
-int plan_max_item_slots(void) { return FR_PACK_MAX_ITEM_SLOTS; }
 
 }

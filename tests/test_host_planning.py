@@ -49,16 +49,16 @@ def test_launch_plans_are_consistent(plan, kind):
             assert 1 <= n_slots <= min(total, WARPS) and 1 <= grid <= 148 and 1 <= wu <= 32
             assert (grid - 1) * wu < n_slots <= grid * wu, "every CTA of the grid holds at least one slot"
             assert n_slots * total < 1 << 63, "slot boundaries are computed in 64 bits"
-            # packed rows: whole chunks per item, bounded item size, everything within 32 bits
+            # packed rows: whole chunks per item, no empty item, everything within 32 bits
+            lanes = group
             if run:
                 counters = blocks + 1
                 assert 1 <= run <= counters and blocks <= 4096
-                slots = -(-counters // run)
-                assert 1 <= group <= n_chunks and group * slots <= 1024
-                assert p_items == -(-n_chunks // group)
-                assert n_chunks * slots < (1 << 32) - 2048
+                assert lanes == -(-counters // run)
+                assert 1 <= p_items <= min(n_chunks, WARPS)
+                assert n_chunks * lanes < (1 << 32) - 64
             else:
-                assert group == 0 and p_items == 0
+                assert lanes == 0 and p_items == 0
             # a few long chains stay with the row kernels
             if blocks > 31 and n_chunks * 8 < WARPS:
                 assert run == 0
@@ -73,7 +73,7 @@ def test_packed_rows_can_be_switched_off_and_forced(plan):
                 assert got[3] == min(run, cb // 16 + 1) or got[3] == 0          # 0: no admissible item size
                 forced = launch(plan, cb, cb * n_chunks, n_chunks, run=run, group=7)
                 if forced[3]:
-                    assert forced[4] == min(7, n_chunks)
+                    assert forced[5] == -(-n_chunks // 7)                 # items of about seven chunks
     assert launch(plan, 65552, 65552 * 100000, 100000)[3] == 0                 # 4097 blocks: above the packed limit
     assert launch(plan, 65536, 65536 * 100000, 100000, run=5)[3] == 5          # 4096 blocks: still admissible
 
