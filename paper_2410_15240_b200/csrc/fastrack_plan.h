@@ -54,9 +54,7 @@ static inline uint32_t fr_rows_of(size_t bytes)
 
 // Row-kernel geometry of a launch over n_chunks chunks of samples of `sample_bytes` bytes (a plain buffer is one
 // sample).  Every warp that takes work pays one closing GF(2^128) product per chunk it touches, at least one; a
-// warp's rows run one after the other.  So a launch of T rows on S SMs wants about sqrt(T / S) warps per SM: more
-// warps shorten the row sequence of each, fewer warps mean fewer closings -- up to the 32 a CTA has, from about
-// 64 MiB on.  (Fitted on B200: best rows per warp 3 / 4 / 6 / 9 / 13 at 1 / 2 / 4 / 8 / 16 MiB.)
+// warp's rows run one after the other.  (Fitted on B200; see the comment at the choice below.)
 static inline FrRowPlan fr_plan_rows(const FrPlanConfig& cfg, size_t sample_bytes, size_t n_chunks)
 {
     FrRowPlan p;
@@ -71,8 +69,16 @@ static inline FrRowPlan fr_plan_rows(const FrPlanConfig& cfg, size_t sample_byte
     if (cfg.row_slots_override) {
         slots = cfg.row_slots_override;
     } else {
-        const uint64_t per_sm = p.total_rows / sms;
-        uint64_t wu = per_sm < 4 ? 1 : per_sm < 8 ? 2 : per_sm < 12 ? 4 : per_sm < 20 ? 8 : per_sm < 50 ? 12 : per_sm < 600 ? 16 : 24;
+        // Small launches are bound by the latency of a warp's row sequence (a row takes a lone warp about as long as it
+        // takes sixteen warps to do one each), so they want at most two rows per warp; from four warps per SM on only
+        // whole numbers of warps per quarter of an SM (each quarter has its own scheduler).  Large launches are bound by
+        // the lookup pipe, which sixteen warps saturate; beyond that, more warps hide a little more latency.
+        const uint64_t per_sm = (p.total_rows + sms - 1) / sms;
+        uint64_t wu = per_sm < 600 ? 16 : 24;
+        if (per_sm <= 32) {
+            wu = (per_sm + 1) / 2;
+            if (wu > 4) wu = (wu + 3) / 4 * 4;
+        }
         if (wu > FR_WARPS) wu = FR_WARPS;
         slots = sms * wu;
     }
