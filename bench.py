@@ -716,6 +716,55 @@ def run_sweep(args):
             device_cell(4 ** e, cb, "config4")
 
 
+def run_layouts(args):
+    """The planner's choice against every forced layout of the packed rows: decrypt+verify GB/s per chunk size for
+    the row kernels alone, for the planner, and for every number of lanes per chunk (one JSON line per chunk size)."""
+    import torch
+    from paper_2410_15240_b200 import fastrack, synth
+    torch.cuda.set_device(0)
+    key, iv = synth.key_and_iv(1)
+    stream = torch.cuda.current_stream()
+    st = stream.cuda_stream
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for n in (16 << 20, 256 << 20):
+        p = torch.randint(0, 256, (n,), dtype=torch.uint8, device="cuda")
+        c, o = torch.empty_like(p), torch.empty_like(p)
+        for cb in (16, 64, 256, 1024, 4096, 16384):
+            K = n // cb
+            t = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
+            ok = torch.zeros(K, dtype=torch.int32, device="cuda")
+
+            def measure(options):
+                with fastrack.Context(key, cb, options) as ctx:
+                    ctx.encrypt_tag(iv, p.data_ptr(), n, c.data_ptr(), t.data_ptr(), st)
+
+                    def call():
+                        ctx.decrypt_verify(iv, c.data_ptr(), n, t.data_ptr(), o.data_ptr(), ok.data_ptr(), st)
+                    for _ in range(3):
+                        call()
+                    torch.cuda.synchronize()
+                    reps, best = max(5, min(100, int(2e9 // n))), float("inf")
+                    for _ in range(3):
+                        e0.record(stream)
+                        for _ in range(reps):
+                            call()
+                        e1.record(stream)
+                        torch.cuda.synchronize()
+                        best = min(best, e0.elapsed_time(e1) / reps)
+                    assert bool((ok == 1).all()) and bool((o == p).all())
+                return n / best / 1e6
+            counters = cb // 16 + 1
+            forced = {}
+            for lanes in (1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 12, 13, 16, 20, 24, 32, 41, 64, counters):
+                run = -(-counters // lanes)
+                if lanes <= counters and -(-counters // run) not in forced:
+                    forced[-(-counters // run)] = measure({fastrack.OPT_PACK_RUN: run})
+            rows_only, auto = measure({fastrack.OPT_PACK_MAX_BLOCKS: 0}), measure({})
+            best = max(max(forced.values()), rows_only)
+            print(json.dumps({"len": n, "chunk": cb, "rows_only_gbs": rows_only, "planner_gbs": auto, "best_forced_gbs": best,
+                              "planner_over_best": auto / best, "forced_gbs_by_lanes": forced}), flush=True)
+
+
 def run_trace(args):
     """Stage-level timelines of fastrack_pipelined_h2d (best of 20 traced calls), one JSON line per transfer."""
     import torch
@@ -772,6 +821,8 @@ def main():
     ap.add_argument("--sweep", action="store_true",
                     help="print throughput over the benchmark configurations instead of the one bench line")
     ap.add_argument("--trace", action="store_true", help="print stage-level timelines of the pipelined H2D call")
+    ap.add_argument("--layouts", action="store_true",
+                    help="small chunks: the planner's choice against the row kernels and every forced packed layout")
     ap.add_argument("--peaks", action="store_true", help="measure the unit rates the kernel roofline is derived from")
     ap.add_argument("--pass", dest="kernel_pass", default="decrypt_verify",
                     choices=["decrypt_verify", "encrypt_tag", "ctr_crypt", "verify"],
@@ -791,6 +842,8 @@ def main():
         run_peaks(args)
     elif args.trace:
         run_trace(args)
+    elif args.layouts:
+        run_layouts(args)
     elif args.sweep:
         run_sweep(args)
     elif args.impl == "reference":
