@@ -35,8 +35,8 @@
  *     come from a trusted source.
  *   - There is no CPU implementation behind these calls: without a usable CUDA device they fail.
  *   - chunk_bytes may be anything from 16 bytes to 1 GiB.  Two kernel layouts serve that range -- a warp per run
- *     of 32 consecutive blocks of a chunk, or, when a launch has many chunks that are not large, a lane per short
- *     run of one chunk's blocks -- and the library picks per launch; results do not depend on the choice.
+ *     of 32 consecutive blocks of a chunk, or, when a launch has many chunks that are not large, a few lanes per
+ *     chunk that take its blocks in turn -- and the library picks per launch; results do not depend on the choice.
  */
 #ifndef FASTRACK_H
 #define FASTRACK_H
@@ -250,10 +250,12 @@ FASTRACK_API int fastrack_pipelined_h2d_ahead(fastrack_ctx* ctx, const uint8_t i
  * deployment variant of the same operation.)
  * Who needs it: code that runs after start-up in a process whose device memory is fully owned by another
  * allocator or a fixed budget, or inside a serving loop where the device-wide synchronisation that comes with
- * a device allocation would stall every other stream.  fastrack_decrypt_verify grows its per-chunk scratch
- * with cudaMalloc the first time a call covers more chunks than any call before; this variant never does:
- * its per-chunk scratch is a fixed array inside the library image (320 KiB, held by every GPU that loads
- * the library until the process exits), and it calls no cudaMalloc, cudaFree or other allocating routine.
+ * a device allocation would stall every other stream.  The guarantee is part of this call's contract: it calls
+ * no cudaMalloc, cudaFree or other allocating routine, and the records in which the CTAs of a launch combine
+ * their pieces of a chunk are a fixed array inside the library image (32 KiB, held by every GPU that loads the
+ * library until the process exits) rather than memory of the context.  (fastrack_decrypt_verify keeps its
+ * records in the context; they have a fixed size and are allocated by fastrack_ctx_create, but that call's
+ * contract does not promise it.)
  * Arguments, outputs, alignment and overlap rules, and asynchrony on `stream` are exactly those of
  * fastrack_decrypt_verify, and the results are bit-identical to it.  Differences:
  *   - at most FASTRACK_NOALLOC_MAX_CHUNKS chunks per call; more returns FASTRACK_ERR_LIMIT and does nothing;
