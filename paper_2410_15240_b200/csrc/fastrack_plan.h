@@ -95,6 +95,8 @@ static inline FrRowPlan fr_plan_rows(const FrPlanConfig& cfg, size_t sample_byte
 struct FrPackCosts {
     size_t row_clocks, seg_clocks, row_step_latency;      // row kernels: per row, per segment; latency of a row for a lone warp
     size_t close, step, step_latency;                     // packed rows, per row of 32 lanes: the closing; one counter step; its latency for a lone warp
+    size_t row_fixed, pack_fixed;                         // per launch, beyond what scales with the work: rows (closing products of all
+                                                          // warps at once, the hand-over between CTAs), packed rows
 };
 
 // Decides between the row kernels (`rows` is their plan) and the packed-row kernels, and in the latter case picks
@@ -112,9 +114,9 @@ static inline FrPackPlan fr_plan_packed(const FrPlanConfig& cfg, int kind, size_
                                         const FrRowPlan& rows)
 {
     static const FrPackCosts costs[3] = {
-        {279, 400, 1000, 300, 279, 2250},     // fused passes: cipher + Horner step per counter, one general product per lane
-        {218, 100, 900, 30, 227, 2000},       // counter mode only: no product, no reduction
-        {85, 400, 300, 465, 65, 700},         // verify only: no cipher (but counter 1), so the closing weighs more
+        {279, 400, 1000, 300, 279, 2250, 10800, 4900},     // fused passes: cipher + Horner step per counter, one general product per lane
+        {218, 100, 900, 30, 227, 2000, 0, 0},              // counter mode only: no product, no reduction
+        {85, 400, 300, 465, 65, 700, 0, 0},                // verify only: no cipher (but counter 1), so the closing weighs more
     };
     const FrPackPlan rows_kernels = {0, 0};
     if (!cfg.pack_max_blocks || n_chunks == 0) return rows_kernels;
@@ -123,7 +125,7 @@ static inline FrPackPlan fr_plan_packed(const FrPlanConfig& cfg, int kind, size_
     const size_t counters = (first_len + 15) / 16 + 1;
     if (counters - 1 > cfg.pack_max_blocks) return rows_kernels;
     const size_t sms = (size_t)cfg.num_sms, warps = sms * FR_WARPS;
-    if (!cfg.pack_run_override && counters > 32 && n_chunks * 8 < warps) return rows_kernels;   // a few long chains: rows, no search needed
+    if (!cfg.pack_run_override && counters > 32 && n_chunks * 16 < warps) return rows_kernels;  // a few long chains: rows, no search needed
 
     // row kernels: every slot closes one segment per chunk it touches
     const size_t pieces = (size_t)rows.n_slots + n_chunks;
@@ -131,7 +133,7 @@ static inline FrPackPlan fr_plan_packed(const FrPlanConfig& cfg, int kind, size_
     const size_t segs_per_slot = (pieces + rows.n_slots - 1) / rows.n_slots;
     const size_t row_thr = (size_t)((rows.total_rows + sms - 1) / sms) * C.row_clocks + (pieces + sms - 1) / sms * C.seg_clocks;
     const size_t row_lat = rows_per_slot * C.row_step_latency + segs_per_slot * 4000;
-    const size_t row_cost = row_thr > row_lat ? row_thr : row_lat;
+    const size_t row_cost = (row_thr > row_lat ? row_thr : row_lat) + C.row_fixed;
 
     size_t best_run = 0, best_items = 1, best_cost = ~(size_t)0;
     const size_t max_lanes = counters < 64 ? counters : 64;
@@ -161,7 +163,7 @@ static inline FrPackPlan fr_plan_packed(const FrPlanConfig& cfg, int kind, size_
             const size_t per_sm = (items + sms - 1) / sms;                          // warps of the busiest SM
             const size_t thr = per_sm * rows_most * per_row;
             const size_t lat = rows_most * row_latency;
-            const size_t cost = thr > lat ? thr + lat / 4 : lat + thr / 4;
+            const size_t cost = (thr > lat ? thr + lat / 4 : lat + thr / 4) + C.pack_fixed;
             if (cost < best_cost) { best_cost = cost; best_run = run; best_items = items; }
         }
         if (cfg.pack_run_override) break;
