@@ -117,7 +117,10 @@ enum {
     FASTRACK_OPT_DIRECT_SMALL = 5,      /* 0: single-stage pipelined transfers use the copy engine too (default 1) */
     FASTRACK_OPT_PACK_MAX_BLOCKS = 6,   /* packed layout only for chunks of at most this many blocks (0 = never; default and cap 4096) */
     FASTRACK_OPT_PACK_RUN = 7,          /* packed layout with this many counters per lane wherever it applies (0 = automatic) */
-    FASTRACK_OPT_PACK_GROUP = 8         /* packed layout: whole chunks per work item (0 = automatic) */
+    FASTRACK_OPT_PACK_GROUP = 8,        /* packed layout: whole chunks per work item (0 = automatic) */
+    FASTRACK_OPT_FOLD_TAIL = 9          /* row layout, fused passes: a chunk's last row of one or two blocks is worked on apart from
+                                           its rows: 0 = where it pays (default), 1 = never, 2 = wherever a chunk ends that way;
+                                           any other value: FASTRACK_ERR_ARG */
 };
 FASTRACK_API int fastrack_ctx_set_option(fastrack_ctx* ctx, int option, uint64_t value);
 

@@ -78,7 +78,7 @@ __device__ __forceinline__ void fr_await_tables(const char* sm, const uint4* gh_
     if (!done) atomicAdd(timeouts, 1u);
 }
 
-template <int MODE, bool ABS>
+template <int MODE, bool ABS, bool FOLD>
 __device__ __forceinline__ void fr_crypt_body(const FrParams& P, char* sm, FrLane L)
 {
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
@@ -92,11 +92,32 @@ __device__ __forceinline__ void fr_crypt_body(const FrParams& P, char* sm, FrLan
     uint64_t g = fr_slot_begin(P, slot);
     const uint64_t end = fr_slot_begin(P, slot + 1u);
     bool await_tables = true;                            // the H tables may still be on their way into shared memory (per thread)
+    uint4* const pre_results = (uint4*)(sm + FR_SM_PRE) + warp * FR_PRE_CHUNKS;
+    uint32_t pre_first = 0, pre_count = 0;               // FOLD: the chunks whose prework results the warp holds
     while (g < end) {                                    // one segment per chunk that the warp's range touches
         const FrRowPos pos = fr_locate_row(P, g);
         uint32_t take = pos.rows_k - pos.r;
         if (take > end - g) take = (uint32_t)(end - g);
-        uint4 z = fr_process_segment_lane<MODE, ABS>(P, sm, L, lane, pos.kk, pos.r, pos.r + take, await_tables);
+        if constexpr (FOLD) {
+            // Folded tails: the warp in whose range a chunk begins also makes that chunk's tag mask and works on the
+            // one or two blocks behind its last row, for up to ten chunks of its range in one pass (see fr_prework_lane).
+            if (pos.r == 0u && pos.kk - pre_first >= pre_count) {
+                bool j0_lane;
+                uint4 t = fr_prework_lane<MODE, ABS>(P, sm, L, lane, pos.kk, end, j0_lane);
+                t.x ^= __shfl_down_sync(0xFFFFFFFFu, t.x, 1) ^ __shfl_down_sync(0xFFFFFFFFu, t.x, 2);
+                t.y ^= __shfl_down_sync(0xFFFFFFFFu, t.y, 1) ^ __shfl_down_sync(0xFFFFFFFFu, t.y, 2);
+                t.z ^= __shfl_down_sync(0xFFFFFFFFu, t.z, 1) ^ __shfl_down_sync(0xFFFFFFFFu, t.z, 2);
+                t.w ^= __shfl_down_sync(0xFFFFFFFFu, t.w, 1) ^ __shfl_down_sync(0xFFFFFFFFu, t.w, 2);
+                if (j0_lane) pre_results[lane / 3u] = t;
+                pre_first = pos.kk;
+                pre_count = __popc(__ballot_sync(0xFFFFFFFFu, j0_lane));
+                __syncwarp();
+            }
+        }
+        uint4 z = fr_process_segment_lane<MODE, ABS, FOLD>(P, sm, L, lane, pos.kk, pos.r, pos.r + take, await_tables);
+        if constexpr (FOLD) {
+            if (pos.r == 0u && lane == 1u) z = fr_xor4(z, pre_results[pos.kk - pre_first]);
+        }
         const uint64_t g0 = g - pos.r;                   // the chunk's first row in the row space
         g += take;
         if (MODE != FR_MODE_CTR && MODE != FR_MODE_PADGEN) {                // the other passes authenticate
@@ -167,7 +188,7 @@ __device__ __forceinline__ void fr_crypt_body(const FrParams& P, char* sm, FrLan
 
 // Fused pass: keystream, XOR, per-segment GHASH partial, per-chunk tag.  Every warp that takes work walks one
 // contiguous range of the launch's rows (see fr_slot_begin in the device header).
-template <int MODE>
+template <int MODE, bool FOLD = false>
 __global__ void __launch_bounds__(FR_THREADS, 1) fr_crypt_kernel(const __grid_constant__ FrParams P)
 {
     extern __shared__ __align__(256) char sm[];
@@ -190,8 +211,8 @@ __global__ void __launch_bounds__(FR_THREADS, 1) fr_crypt_kernel(const __grid_co
     L.lane4 |= after_barrier;
     L.qe |= after_barrier;
     L.qo |= after_barrier;
-    if ((uint32_t)__cvta_generic_to_shared(sm) == FR_SMEM_ABS_BASE && !P.generic_smem) fr_crypt_body<MODE, true>(P, sm, L);
-    else fr_crypt_body<MODE, false>(P, sm, L);
+    if ((uint32_t)__cvta_generic_to_shared(sm) == FR_SMEM_ABS_BASE && !P.generic_smem) fr_crypt_body<MODE, true, FOLD>(P, sm, L);
+    else fr_crypt_body<MODE, false, FOLD>(P, sm, L);
     FR_STAMP_MAX(5); FR_STAMP_GTMAX(6);
 }
 
@@ -504,6 +525,8 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
         if ((e = cudaGetLastError()) != cudaSuccess) break;
         if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_DEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
         if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_ENC>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_DEC, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
+        if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_ENC, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
         if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_CTR>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
         if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_VERIFY>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
         if ((e = cudaFuncSetAttribute(fr_crypt_kernel<FR_MODE_PADGEN>, cudaFuncAttributeMaxDynamicSharedMemorySize, FR_SMEM_LAUNCH_BYTES)) != cudaSuccess) break;
@@ -590,6 +613,7 @@ extern "C" int fastrack_ctx_set_option(fastrack_ctx* ctx, int option, uint64_t v
         case FASTRACK_OPT_PACK_MAX_BLOCKS:   ctx->plan.pack_max_blocks = (uint32_t)(value > FR_PACK_MAX_BLOCKS ? FR_PACK_MAX_BLOCKS : value); break;
         case FASTRACK_OPT_PACK_RUN:          ctx->plan.pack_run_override = (uint32_t)(value > 0xFFFFFFFFull ? 0xFFFFFFFFull : value); break;
         case FASTRACK_OPT_PACK_GROUP:        ctx->plan.pack_group_override = (uint32_t)(value > 0xFFFFFFFFull ? 0xFFFFFFFFull : value); break;
+        case FASTRACK_OPT_FOLD_TAIL:         if (value > 2) return FASTRACK_ERR_ARG; ctx->plan.fold_tail_mode = (uint32_t)value; break;
         default: return FASTRACK_ERR_ARG;
     }
     return FASTRACK_OK;
@@ -645,9 +669,10 @@ static uint4 length_term(const fastrack_ctx* ctx, uint64_t bytes)
 }
 
 // Fills the geometry of a launch into P: the row kernels' plan (fastrack_plan.h) and the per-sample layout.
-static FrRowPlan plan_rows(const fastrack_ctx* ctx, size_t sample_bytes, size_t n_chunks, FrParams& P)
+static FrRowPlan plan_rows(const fastrack_ctx* ctx, int mode, size_t sample_bytes, size_t n_chunks, FrParams& P)
 {
-    const FrRowPlan rows = fr_plan_rows(ctx->plan, sample_bytes, n_chunks);
+    const FrRowPlan rows = fr_plan_rows(ctx->plan, sample_bytes, n_chunks, mode == FR_MODE_DEC || mode == FR_MODE_ENC);
+    P.fold_tail = rows.fold_tail;
     P.n_slots = rows.n_slots;
     P.warps_used = rows.warps_used;
     P.rows_full = rows.rows_full;
@@ -723,7 +748,7 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
     const size_t n_chunks = (len / sample_bytes) * cps;            // len is a whole number of samples
     P.n_chunks = (uint32_t)n_chunks;
 
-    const FrRowPlan rows = plan_rows(ctx, sample_bytes, n_chunks, P);
+    const FrRowPlan rows = plan_rows(ctx, mode, sample_bytes, n_chunks, P);
     // Many short chains: one run of counters per lane (see fr_packed_body) when that is predicted to be faster.
     const bool packed = !b.rows_only && (mode == FR_MODE_DEC || mode == FR_MODE_ENC || mode == FR_MODE_CTR || mode == FR_MODE_VERIFY) &&
                         plan_packed(ctx, mode, sample_bytes, n_chunks, rows, P);
@@ -793,10 +818,12 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
     switch (mode) {
         case FR_MODE_DEC:    le = packed ? (whole ? cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_DEC, true>, P)
                                                   : cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_DEC, false>, P))
-                                         : cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_DEC>, P); break;
+                                         : P.fold_tail ? cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_DEC, true>, P)
+                                                       : cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_DEC>, P); break;
         case FR_MODE_ENC:    le = packed ? (whole ? cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_ENC, true>, P)
                                                   : cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_ENC, false>, P))
-                                         : cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_ENC>, P); break;
+                                         : P.fold_tail ? cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_ENC, true>, P)
+                                                       : cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_ENC>, P); break;
         case FR_MODE_CTR:    le = packed ? (whole ? cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_CTR, true>, P)
                                                   : cudaLaunchKernelEx(&cfg, fr_packed_kernel<FR_MODE_CTR, false>, P))
                                          : cudaLaunchKernelEx(&cfg, fr_crypt_kernel<FR_MODE_CTR>, P); break;

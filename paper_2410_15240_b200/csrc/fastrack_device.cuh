@@ -35,7 +35,8 @@
 #define FR_SMEM_BYTES 196608u // the three tables
 #define FR_SM_COMB 196608u    // row kernels: 33 records of 8 words in which the warps of a CTA combine their pieces of a chunk
 #define FR_SM_MBAR (FR_SM_COMB + 33u * 32u)   // arrival barrier of the bulk copy that brings in the H-power byte tables
-#define FR_SMEM_LAUNCH_BYTES (FR_SMEM_BYTES + 2048u)   // dynamic shared memory of a launch: the tables and the records
+#define FR_SM_PRE (FR_SM_COMB + 2048u)   // row kernels with folded tails: per warp, the results of its last prework pass (FR_PRE_CHUNKS x 16 bytes)
+#define FR_SMEM_LAUNCH_BYTES (FR_SMEM_BYTES + 2048u + 32u * 10u * 16u)   // dynamic shared memory of a launch: the tables, the records, the prework results
 
 // What one pass does.  DEC / ENC are the fused passes.  CTR and VERIFY split them (paper Section 4.3, eager
 // evaluation: plaintext first, authentication later).  PADGEN / PADDEC split the keystream from the XOR
@@ -92,7 +93,7 @@ struct FrParams {
     uint32_t chunks_per_sample;  // ceil(sample_bytes / chunk_bytes); only a sample's last chunk may be short
     uint32_t pack_pad;
     uint32_t pack_run;           // packed rows: most counters per slot (lane); a full chunk has ceil((blocks + 1) / pack_run) slots
-    uint32_t pad2;
+    uint32_t fold_tail;          // row kernels: 1 = a chunk's last one or two counters are not a row of their own (see fr_prework_lane)
     const uint8_t* ivs;        // per-sample 12-byte IV bases (device), or null: one IV base for the whole launch
     const uint8_t* in;
     uint8_t* out;
@@ -446,7 +447,17 @@ __device__ __forceinline__ FrChunk fr_chunk_info(const FrParams& P, uint32_t kk)
 // Rows are aligned to the COUNTER, not to the block index: row r of a chunk holds counters 32r .. 32r+31,
 // lane = counter mod 32.  Data block j uses counter j + 2, so row 0 carries 30 data blocks; its lane 1
 // (counter 1) produces E_K(J0), the tag mask, as a by-product and lane 0 idles.
-__device__ __forceinline__ uint32_t fr_chunk_rows(uint32_t nblk) { return (nblk + 2u + FR_ROW_BLOCKS - 1) / FR_ROW_BLOCKS; }
+//
+// Folded tails (fold_tail, decided per launch by the host): a chunk of a whole number of rows' worth of blocks --
+// every power-of-two chunk size -- ends, because of that offset of two, in a row that holds one or two counters
+// and costs as much as a full one (3 % of a 16 KiB chunk).  With fold_tail such a chunk has one row less; its last
+// one or two blocks, and E_K(J0) of every chunk, are worked on by fr_prework_lane, ten chunks per pass.
+__device__ __forceinline__ uint32_t fr_chunk_rows(uint32_t nblk, uint32_t fold_tail)
+{
+    uint32_t rows = (nblk + 2u + FR_ROW_BLOCKS - 1) / FR_ROW_BLOCKS;
+    if (fold_tail && nblk >= 31u && ((nblk + 2u) & 31u) - 1u < 2u) rows--;
+    return rows;
+}
 
 // Work distribution of the row kernels.  The rows of all chunks of a launch, one chunk after the other, form
 // one row space of total_rows rows; it is cut into n_slots contiguous, equally long (to within one row) ranges and
@@ -542,11 +553,12 @@ __device__ __forceinline__ uint4 fr_mask_bytes(uint4 v, uint32_t n)
 #ifndef FR_AWAIT_TABLES
 #define FR_AWAIT_TABLES(sm, P) do { } while (0)
 #endif
-template <int MODE, bool ABS>
+template <int MODE, bool ABS, bool FOLD = false>
 __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, const char* sm, const FrLane& L,
                                                          uint32_t lane, uint32_t kk, uint32_t row0, uint32_t row1,
                                                          bool& await_tables)
 {
+    static_assert(!FOLD || MODE == FR_MODE_DEC || MODE == FR_MODE_ENC, "tails are folded in the fused passes only");
     constexpr bool DO_AES = MODE == FR_MODE_DEC || MODE == FR_MODE_ENC || MODE == FR_MODE_CTR || MODE == FR_MODE_PADGEN;
     constexpr bool DO_GHASH = MODE == FR_MODE_DEC || MODE == FR_MODE_ENC || MODE == FR_MODE_VERIFY || MODE == FR_MODE_PADDEC;
     constexpr bool DO_LOAD = MODE != FR_MODE_PADGEN;
@@ -612,6 +624,8 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
         } else if (ctr == 1u && MODE != FR_MODE_CTR) {
             if (MODE == FR_MODE_PADDEC) {
                 extra = P.mask[kk];
+            } else if (FOLD) {
+                // E_K(J0) comes out of the prework pass together with the folded tail's terms; the caller adds them
             } else {
                 extra = fr_aes256_ctr_block<ABS>(sm, L.lane4, P, cc, cg, 1u);         // E_K(J0)
                 if (MODE == FR_MODE_PADGEN) P.mask[kk] = extra;
@@ -630,12 +644,58 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
     return fr_xor4(fr_gf128_mul(pend, hpow), extra);
 }
 
-template <int MODE, bool ABS>
+template <int MODE, bool ABS, bool FOLD = false>
 __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, const char* sm, const FrLane& L,
                                                          uint32_t lane, uint32_t kk, uint32_t row0, uint32_t row1)
 {
     bool tables_are_there = false;
-    return fr_process_segment_lane<MODE, ABS>(P, sm, L, lane, kk, row0, row1, tables_are_there);
+    return fr_process_segment_lane<MODE, ABS, FOLD>(P, sm, L, lane, kk, row0, row1, tables_are_there);
+}
+
+// Folded tails: what the rows of a chunk leave out.  One pass of a warp serves up to FR_PRE_CHUNKS consecutive
+// chunks, three lanes each: lane 3m of the pass makes E_K(J0) of chunk kk_first + m (counter 1), lanes 3m + 1 and
+// 3m + 2 take the one or two counters behind the chunk's last row (none if the chunk's tail is not folded) --
+// cipher, XOR, store, and the block's term of the tag, block * H^(nblk + 3 - counter), by the general product.
+// The XOR of the three lanes' results takes the place of the E_K(J0) that lane 1 of row 0 produces otherwise: the
+// warp that owns row 0 of the chunk adds it to the result of that segment.  Only chunks whose
+// first row lies before row `row_end` of the row space (the end of the calling warp's range) take part; the
+// function returns zero for every other lane.  Needs the AES tables only.
+#define FR_PRE_CHUNKS 10u
+
+__device__ __forceinline__ uint64_t fr_chunk_first_row(const FrParams& P, uint32_t kk)
+{
+    const uint32_t sample = kk / P.chunks_per_sample, k = kk - sample * P.chunks_per_sample;
+    return (uint64_t)sample * P.rows_sample + (uint64_t)k * P.rows_full;
+}
+
+template <int MODE, bool ABS>
+__device__ __forceinline__ uint4 fr_prework_lane(const FrParams& P, const char* sm, const FrLane& L, uint32_t lane,
+                                                 uint32_t kk_first, uint64_t row_end, bool& j0_lane)
+{
+    static_assert(MODE == FR_MODE_DEC || MODE == FR_MODE_ENC, "tails are folded in the fused passes only");
+    const uint32_t m = lane / 3u, role = lane - 3u * m, kk = kk_first + m;
+    j0_lane = false;
+    if (m >= FR_PRE_CHUNKS || kk >= P.n_chunks || fr_chunk_first_row(P, kk) >= row_end) return make_uint4(0, 0, 0, 0);
+    const FrChunk ck = fr_chunk_info(P, kk);
+    const uint32_t nblk = (uint32_t)((ck.len + 15) >> 4);
+    const uint32_t rows_k = ck.last_of_sample ? P.rows_last : P.rows_full;
+    const uint32_t ctr = role == 0u ? 1u : rows_k * FR_ROW_BLOCKS + role - 1u;
+    j0_lane = role == 0u;
+    if (role != 0u && ctr > nblk + 1u) return make_uint4(0, 0, 0, 0);      // the rows cover the chunk up to its last counter
+    const FrCtrChunk cc = fr_ctr_chunk<ABS>(sm, L.lane4, P, ck.iv_w0, ck.iv_w1, fr_bswap(ck.iv_ctr));
+    const FrCtrGroup cg = fr_ctr_group<ABS>(sm, L.lane4, P, cc, ctr);
+    const uint4 ks = fr_aes256_ctr_block<ABS>(sm, L.lane4, P, cc, cg, ctr);
+    if (role == 0u) return ks;
+    const uint64_t boff = (uint64_t)(ctr - 2u) << 4;
+    const bool full = ck.len - boff >= 16;
+    const uint32_t nvalid = full ? 16u : (uint32_t)(ck.len - boff);
+    const uint8_t* in = P.in + ck.off + boff;
+    uint8_t* out = P.out + ck.off + boff;
+    const uint4 x = full ? *(const uint4*)in : fr_load_partial(in, nvalid);
+    const uint4 o = fr_xor4(x, ks);
+    if (full) *(uint4*)out = o; else fr_store_partial(out, o, nvalid);
+    const uint4 g = (MODE == FR_MODE_ENC) ? (full ? o : fr_mask_bytes(o, nvalid)) : x;
+    return fr_gf128_mul(g, P.pow[nblk + 3u - ctr]);
 }
 
 // ---- Packed rows: many short chains -----------------------------------------------------------------------

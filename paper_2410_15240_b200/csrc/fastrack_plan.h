@@ -25,6 +25,7 @@ struct FrPlanConfig {
     uint32_t pack_run_override;     // 0 = automatic; else packed rows with this run length wherever they apply (tests)
     uint32_t pack_group_override;   // 0 = automatic; else this many chunks per packed work item (tests)
     size_t stage_bytes_override;    // 0 = automatic; else the stage size of pipelined transfers (experiments)
+    uint32_t fold_tail_mode;        // row kernels, fused passes: 0 = fold the tails of chunks where it pays, 1 = never, 2 = wherever a chunk has one (tests)
 };
 
 // How the row kernels spread a launch over warps: the rows of all chunks, one chunk after the other, are cut into
@@ -37,6 +38,7 @@ struct FrRowPlan {
     uint32_t rows_last;         // rows of a sample's last chunk
     uint64_t rows_sample;       // rows of a sample
     uint64_t total_rows;
+    uint32_t fold_tail;         // 1: the row counts above are those of folded tails (see fr_rows_of)
 };
 
 struct FrPackPlan {
@@ -46,45 +48,71 @@ struct FrPackPlan {
 
 enum FrPassKind : int { FR_PASS_FUSED = 0, FR_PASS_CTR = 1, FR_PASS_VERIFY = 2 };
 
-// Rows of a chunk of `bytes` bytes: rows are aligned to the counter and block j sits at counter j + 2.
-static inline uint32_t fr_rows_of(size_t bytes)
+// Rows of a chunk of `bytes` bytes: rows are aligned to the counter and block j sits at counter j + 2, so a chunk of
+// a whole number of rows' worth of blocks (or one block less) ends in a row of two counters (or one).  With `fold`
+// that row does not exist: the kernel works on those counters in a pass that it makes anyway for the tag masks of
+// up to ten chunks at a time (fr_prework_lane in the device header).
+static inline bool fr_tail_folds(size_t bytes)
 {
-    return (uint32_t)(((bytes + 15) / 16 + 2 + FR_PLAN_ROW_BLOCKS - 1) / FR_PLAN_ROW_BLOCKS);
+    const size_t blocks = (bytes + 15) / 16, in_last_row = (blocks + 2) % FR_PLAN_ROW_BLOCKS;
+    return blocks >= 31 && (in_last_row == 1 || in_last_row == 2);
+}
+
+static inline uint32_t fr_rows_of(size_t bytes, bool fold)
+{
+    const uint32_t rows = (uint32_t)(((bytes + 15) / 16 + 2 + FR_PLAN_ROW_BLOCKS - 1) / FR_PLAN_ROW_BLOCKS);
+    return fold && fr_tail_folds(bytes) ? rows - 1 : rows;
 }
 
 // Row-kernel geometry of a launch over n_chunks chunks of samples of `sample_bytes` bytes (a plain buffer is one
 // sample).  Every warp that takes work pays one closing GF(2^128) product per chunk it touches, at least one; a
 // warp's rows run one after the other.  (Fitted on B200; see the comment at the choice below.)
-static inline FrRowPlan fr_plan_rows(const FrPlanConfig& cfg, size_t sample_bytes, size_t n_chunks)
+// may_fold: the pass is one that can fold tails (decrypt + verify, encrypt + tag); whether it does is decided here.
+static inline FrRowPlan fr_plan_rows(const FrPlanConfig& cfg, size_t sample_bytes, size_t n_chunks, bool may_fold = false)
 {
     FrRowPlan p;
     const size_t cps = (sample_bytes + cfg.chunk_bytes - 1) / cfg.chunk_bytes;
     const size_t first_len = sample_bytes < cfg.chunk_bytes ? sample_bytes : cfg.chunk_bytes;
-    p.rows_full = fr_rows_of(first_len);
-    p.rows_last = fr_rows_of(sample_bytes - (cps - 1) * cfg.chunk_bytes);
-    p.rows_sample = (uint64_t)(cps - 1) * p.rows_full + p.rows_last;
-    p.total_rows = (uint64_t)(n_chunks / cps) * p.rows_sample;
+    const size_t last_len = sample_bytes - (cps - 1) * cfg.chunk_bytes;
     const uint64_t sms = (uint64_t)cfg.num_sms, cap = sms * FR_WARPS;
-    uint64_t slots;
-    if (cfg.row_slots_override) {
-        slots = cfg.row_slots_override;
-    } else {
-        // Small launches are bound by the latency of a warp's row sequence (a row takes a lone warp about as long as it
-        // takes sixteen warps to do one each), so they want at most two rows per warp; from four warps per SM on only
-        // whole numbers of warps per quarter of an SM (each quarter has its own scheduler).  Large launches are bound by
-        // the lookup pipe, which sixteen warps saturate; beyond that, more warps hide a little more latency.
-        const uint64_t per_sm = (p.total_rows + sms - 1) / sms;
-        uint64_t wu = per_sm < 600 ? 16 : 24;
-        if (per_sm <= 32) {
-            wu = (per_sm + 1) / 2;
-            if (wu > 4) wu = (wu + 3) / 4 * 4;
+    auto geometry = [&](bool fold) {
+        p.fold_tail = fold ? 1u : 0u;
+        p.rows_full = fr_rows_of(first_len, fold);
+        p.rows_last = fr_rows_of(last_len, fold);
+        p.rows_sample = (uint64_t)(cps - 1) * p.rows_full + p.rows_last;
+        p.total_rows = (uint64_t)(n_chunks / cps) * p.rows_sample;
+    };
+    auto slots_for = [&](uint64_t total_rows) {
+        uint64_t slots;
+        if (cfg.row_slots_override) {
+            slots = cfg.row_slots_override;
+        } else {
+            // Small launches are bound by the latency of a warp's row sequence (a row takes a lone warp about as long as it
+            // takes sixteen warps to do one each), so they want at most two rows per warp; from four warps per SM on only
+            // whole numbers of warps per quarter of an SM (each quarter has its own scheduler).  Large launches are bound by
+            // the lookup pipe, which sixteen warps saturate; beyond that, more warps hide a little more latency.
+            const uint64_t per_sm = (total_rows + sms - 1) / sms;
+            uint64_t wu = per_sm < 600 ? 16 : 24;
+            if (per_sm <= 32) {
+                wu = (per_sm + 1) / 2;
+                if (wu > 4) wu = (wu + 3) / 4 * 4;
+            }
+            if (wu > FR_WARPS) wu = FR_WARPS;
+            slots = sms * wu;
         }
-        if (wu > FR_WARPS) wu = FR_WARPS;
-        slots = sms * wu;
-    }
-    if (slots > cap) slots = cap;
-    if (slots > p.total_rows) slots = p.total_rows;
-    if (slots < 1) slots = 1;
+        if (slots > cap) slots = cap;
+        if (slots > total_rows) slots = total_rows;
+        if (slots < 1) slots = 1;
+        return slots;
+    };
+    geometry(false);
+    // Folding pays where a warp's range holds a chunk start or several, so that the extra pass serves them all (measured
+    // with 16 KiB chunks: 3.5 % at seven chunks per warp, 1.5 % at 1.7; 0.5 % with 64 KiB chunks at 1.2), and loses
+    // where chunks are spread over several warps and most warps would make the pass for one chunk (17 % at 0.4).
+    if (may_fold && cfg.fold_tail_mode != 1 && (fr_tail_folds(first_len) || fr_tail_folds(last_len)) &&
+        (cfg.fold_tail_mode == 2 || n_chunks >= slots_for(p.total_rows)))
+        geometry(true);
+    const uint64_t slots = slots_for(p.total_rows);
     p.n_slots = (uint32_t)slots;
     p.warps_used = (uint32_t)((slots + sms - 1) / sms);
     p.grid = (uint32_t)((slots + p.warps_used - 1) / p.warps_used);
@@ -131,7 +159,11 @@ static inline FrPackPlan fr_plan_packed(const FrPlanConfig& cfg, int kind, size_
     const size_t pieces = (size_t)rows.n_slots + n_chunks;
     const size_t rows_per_slot = (size_t)((rows.total_rows + rows.n_slots - 1) / rows.n_slots);
     const size_t segs_per_slot = (pieces + rows.n_slots - 1) / rows.n_slots;
-    const size_t row_thr = (size_t)((rows.total_rows + sms - 1) / sms) * C.row_clocks + (pieces + sms - 1) / sms * C.seg_clocks;
+    // (folded tails: one more pass of a cipher block and a product per ten chunk starts, at least one per warp that sees a start)
+    size_t pre_passes = rows.fold_tail ? n_chunks / 10 + rows.n_slots : 0;
+    if (pre_passes > n_chunks) pre_passes = n_chunks;
+    const size_t row_thr = (size_t)((rows.total_rows + sms - 1) / sms) * C.row_clocks + (pieces + sms - 1) / sms * C.seg_clocks +
+                           (pre_passes + sms - 1) / sms * (C.step + C.close);
     const size_t row_lat = rows_per_slot * C.row_step_latency + segs_per_slot * 4000;
     const size_t row_cost = (row_thr > row_lat ? row_thr : row_lat) + C.row_fixed;
 

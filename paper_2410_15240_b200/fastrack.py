@@ -20,7 +20,7 @@ MAX_CHUNK_BYTES = 1 << 30
 
 # fastrack_ctx_set_option: test and tuning controls (the library reads no environment variable)
 OPT_ROW_SLOTS, OPT_GENERIC_SMEM, OPT_NO_OVERLAP_LAUNCH, OPT_STAGE_BYTES = 1, 2, 3, 4
-OPT_DIRECT_SMALL, OPT_PACK_MAX_BLOCKS, OPT_PACK_RUN, OPT_PACK_GROUP = 5, 6, 7, 8
+OPT_DIRECT_SMALL, OPT_PACK_MAX_BLOCKS, OPT_PACK_RUN, OPT_PACK_GROUP, OPT_FOLD_TAIL = 5, 6, 7, 8, 9
 
 EXPORTS = ("fastrack_ctx_create", "fastrack_ctx_destroy", "fastrack_num_chunks", "fastrack_ctx_reserve", "fastrack_ctx_set_option",
            "fastrack_last_cuda_error", "fastrack_decrypt_verify", "fastrack_encrypt_tag",

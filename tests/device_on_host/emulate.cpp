@@ -123,7 +123,7 @@ uint4 length_term(const Setup& S, uint64_t bytes, uint32_t aad_mod)
 // the XOR of the pieces of a chunk done in a plain array instead of the shared-memory and global records.  What the
 // kernel derives from fr_chunk_share -- how many warps of the CTA and how many CTAs meet on a chunk, and in which
 // record -- is checked here against what the walk really does.  Returns 0, or a code that says which check failed.
-template <int MODE>
+template <int MODE, bool FOLD = false>
 int run_pass(Setup& S, std::vector<uint4>& acc)
 {
     const FrParams& P = S.P;
@@ -137,15 +137,39 @@ int run_pass(Setup& S, std::vector<uint4>& acc)
         const uint64_t end = fr_slot_begin(P, slot + 1u);
         if (end <= g) return 11;                                                     // no empty range
         if (fr_slot_of_row(P, g) != slot || fr_slot_of_row(P, end - 1) != slot) return 12;
+        uint4 pre_results[FR_PRE_CHUNKS];                                            // folded tails, as fr_crypt_body keeps them
+        uint32_t pre_first = 0, pre_count = 0;
         while (g < end) {
             const FrRowPos pos = fr_locate_row(P, g);
             if (pos.kk >= P.n_chunks || pos.r >= pos.rows_k) return 13;
             uint32_t take = pos.rows_k - pos.r;
             if (take > end - g) take = (uint32_t)(end - g);
+            bool add_pre = false;
+            if constexpr (FOLD) {
+                if (pos.r == 0u) {
+                    if (pos.kk - pre_first >= pre_count) {
+                        uint4 t[34];
+                        bool j0_lane[32];
+                        for (uint32_t lane = 0; lane < 32; lane++)
+                            t[lane] = fr_prework_lane<MODE, false>(P, S.sm.data(), fr_make_lane(lane), lane, pos.kk, end, j0_lane[lane]);
+                        t[32] = t[33] = uint4{0, 0, 0, 0};
+                        pre_count = 0;
+                        for (uint32_t lane = 0; lane < 32; lane++) {
+                            if (!j0_lane[lane]) continue;
+                            if (lane % 3u != 0u || lane / 3u != pre_count) return 21;        // the chunks of a pass are consecutive, three lanes each
+                            pre_results[pre_count++] = fr_xor4(t[lane], fr_xor4(t[lane + 1], t[lane + 2]));
+                        }
+                        pre_first = pos.kk;
+                        if (pre_count == 0) return 22;                                       // the chunk that asked is always served
+                    }
+                    add_pre = true;
+                }
+            }
             for (uint32_t lane = 0; lane < 32; lane++) {                             // the warp, one lane after the other
                 const FrLane L = fr_make_lane(lane);
-                acc[pos.kk] = fr_xor4(acc[pos.kk], fr_process_segment_lane<MODE, false>(P, S.sm.data(), L, lane, pos.kk, pos.r, pos.r + take));
+                acc[pos.kk] = fr_xor4(acc[pos.kk], fr_process_segment_lane<MODE, false, FOLD>(P, S.sm.data(), L, lane, pos.kk, pos.r, pos.r + take));
             }
+            if (add_pre) acc[pos.kk] = fr_xor4(acc[pos.kk], pre_results[pos.kk - pre_first]);
             pieces_of[pos.kk]++;
             rows_done[pos.kk] += take;
             if (take != pos.rows_k) partial[pos.kk].push_back(Piece{slot, g - pos.r, pos.rows_k});
@@ -189,7 +213,7 @@ int run_pass(Setup& S, std::vector<uint4>& acc)
 extern "C" int emu_pass(int mode, const uint8_t* key, const uint8_t* iv_base, size_t cb, const uint8_t* in, size_t len,
                         uint8_t* out, const uint8_t* pad, uint8_t* mask, const uint8_t* tags_in, uint8_t* tags_out,
                         uint32_t* ok, uint32_t rows_per_slot, uint32_t num_sms, uint32_t first_chunk, uint32_t aad_mod,
-                        size_t sample_bytes, const uint8_t* ivs)
+                        size_t sample_bytes, const uint8_t* ivs, uint32_t fold_mode)
 {
     Setup S;
     setup(S, key, cb);
@@ -215,11 +239,14 @@ extern "C" int emu_pass(int mode, const uint8_t* key, const uint8_t* iv_base, si
     memset(&cfg, 0, sizeof cfg);
     cfg.num_sms = (int)(num_sms ? num_sms : 148);
     cfg.chunk_bytes = cb;
-    FrRowPlan rows = fr_plan_rows(cfg, sample_bytes, n_chunks);
+    cfg.fold_tail_mode = fold_mode;                                              // as FASTRACK_OPT_FOLD_TAIL
+    const bool may_fold = mode == FR_MODE_DEC || mode == FR_MODE_ENC;
+    FrRowPlan rows = fr_plan_rows(cfg, sample_bytes, n_chunks, may_fold);
     if (rows_per_slot) {
         cfg.row_slots_override = (uint32_t)((rows.total_rows + rows_per_slot - 1) / rows_per_slot);
-        rows = fr_plan_rows(cfg, sample_bytes, n_chunks);
+        rows = fr_plan_rows(cfg, sample_bytes, n_chunks, may_fold);
     }
+    P.fold_tail = rows.fold_tail;
     P.n_slots = rows.n_slots;
     P.warps_used = rows.warps_used;
     P.rows_full = rows.rows_full;
@@ -236,8 +263,8 @@ extern "C" int emu_pass(int mode, const uint8_t* key, const uint8_t* iv_base, si
     std::vector<uint4> acc(n_chunks, uint4{0, 0, 0, 0});
     int rc;
     switch (mode) {
-        case FR_MODE_DEC: rc = run_pass<FR_MODE_DEC>(S, acc); break;
-        case FR_MODE_ENC: rc = run_pass<FR_MODE_ENC>(S, acc); break;
+        case FR_MODE_DEC: rc = P.fold_tail ? run_pass<FR_MODE_DEC, true>(S, acc) : run_pass<FR_MODE_DEC>(S, acc); break;
+        case FR_MODE_ENC: rc = P.fold_tail ? run_pass<FR_MODE_ENC, true>(S, acc) : run_pass<FR_MODE_ENC>(S, acc); break;
         case FR_MODE_CTR: return run_pass<FR_MODE_CTR>(S, acc);
         case FR_MODE_VERIFY: rc = run_pass<FR_MODE_VERIFY>(S, acc); break;
         case FR_MODE_PADGEN: return run_pass<FR_MODE_PADGEN>(S, acc);
@@ -401,8 +428,9 @@ static int run_case(size_t cb, size_t len, uint32_t seg, uint32_t first, uint32_
         for (size_t i = 0; i < 16 * K; i++) { mask[i] = (uint8_t)(lcg(s) >> 24); tin[i] = (uint8_t)(lcg(s) >> 24); tout[i] = 0; }
         for (size_t i = 0; i < K; i++) ok[i] = 9;
         if (ivs) for (size_t i = 0; i < 12 * n_samples; i++) ivs[i] = (uint8_t)(lcg(s) >> 24);
-        bad |= emu_pass(mode, key, iv, cb, in, len, out, pad, mask, tin, tout, ok, seg, 2 + seg % 3, first, aad, sample_bytes, ivs);
-        bad |= emu_pass(mode, key, iv, cb, in, len, out, pad, mask, tin, tout, ok, 0, 148, first, aad, sample_bytes, ivs);
+        bad |= emu_pass(mode, key, iv, cb, in, len, out, pad, mask, tin, tout, ok, seg, 2 + seg % 3, first, aad, sample_bytes, ivs, 2);   // tails folded wherever a chunk has one
+        bad |= emu_pass(mode, key, iv, cb, in, len, out, pad, mask, tin, tout, ok, seg, 2 + seg % 3, first, aad, sample_bytes, ivs, 1);   // and never
+        bad |= emu_pass(mode, key, iv, cb, in, len, out, pad, mask, tin, tout, ok, 0, 148, first, aad, sample_bytes, ivs, 0);
         if (mode <= FR_MODE_VERIFY)                     // the packed-row form of the same pass, seg doubling as group size and run length
             for (uint32_t run : {1u, seg + 1u, 40u})
                 bad |= emu_packed(mode, key, iv, cb, in, len, out, tin, tout, ok, seg * 3 - 2, run, first, aad, sample_bytes, ivs);

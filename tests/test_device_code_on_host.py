@@ -21,7 +21,7 @@ def emu(tmp_path_factory):
                            os.path.join(ROOT, "tests", "device_on_host", "emulate.cpp")])
     lib = ctypes.CDLL(str(so))
     V, Z, U = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_uint32
-    lib.emu_pass.argtypes = [ctypes.c_int, V, V, Z, V, Z, V, V, V, V, V, V, U, U, U, U, Z, V]
+    lib.emu_pass.argtypes = [ctypes.c_int, V, V, Z, V, Z, V, V, V, V, V, V, U, U, U, U, Z, V, U]
     lib.emu_pass.restype = ctypes.c_int
     for name in ("emu_gf128_mul_device", "emu_gf128_mul_keysetup"):
         getattr(lib, name).argtypes = [ctypes.c_char_p] * 3
@@ -31,8 +31,8 @@ def emu(tmp_path_factory):
     return lib
 
 
-def run(lib, mode, key, iv, cb, data, n, pad=None, mask=None, tags=None, seg=8, first=0, aad=0, sample_bytes=0, ivs=None, sms=3):
-    """seg = rows per warp (0: the planner's own choice) on an emulated GPU of `sms` SMs: few SMs, so that chunks are
+def run(lib, mode, key, iv, cb, data, n, pad=None, mask=None, tags=None, seg=8, first=0, aad=0, sample_bytes=0, ivs=None, sms=3, fold=0):
+    """fold = the tail-folding option (0 automatic, 1 never, 2 wherever a chunk allows); seg = rows per warp (0: the planner's own choice) on an emulated GPU of `sms` SMs: few SMs, so that chunks are
     shared between warps of one CTA and between CTAs even in small cases."""
     K = (n + cb - 1) // cb if not sample_bytes else (n // sample_bytes) * ((sample_bytes + cb - 1) // cb)
     k = np.frombuffer(key, np.uint8).copy()
@@ -48,7 +48,7 @@ def run(lib, mode, key, iv, cb, data, n, pad=None, mask=None, tags=None, seg=8, 
         out[:n] = src                                   # the pass does not store; keep the guard check meaningful
     rc = lib.emu_pass(mode, k.ctypes.data, v.ctypes.data, cb, src.ctypes.data, n, out.ctypes.data, pad_a.ctypes.data,
                       mask_a.ctypes.data, tin.ctypes.data, tout.ctypes.data, ok.ctypes.data, seg, sms, first, aad, sample_bytes,
-                      ivs.ctypes.data if ivs is not None else None)
+                      ivs.ctypes.data if ivs is not None else None, fold)
     assert rc == 0, f"emulation reports inconsistency {rc}"
     assert (out[n:] == 0xA5).all()
     return out[:n], tout, ok, mask_a
@@ -121,6 +121,43 @@ def test_fused_and_split_passes_match_oracle(emu, n, cb, seg, aad):
     pad, _, _, mask = run(emu, PADGEN, key, iv, cb, None, n, seg=seg, aad=aad)
     assert np.array_equal(pad, oracle.mc_encrypt(key, iv, cb, np.zeros(n, np.uint8), 4)[0])
     out, _, ok, _ = run(emu, PADDEC, key, iv, cb, bad_c, n, pad=pad, mask=mask, tags=bad_t, seg=seg, aad=aad)
+    assert np.array_equal(out, p_ref) and np.array_equal(ok, ok_ref)
+
+
+FOLD_SHAPES = [  # n, chunk bytes, rows per warp (0: planner), emulated SMs
+    (512 * 40, 512, 8, 3),                  # 32 blocks: two counters behind the last row; 40 chunks, several passes of ten per warp
+    (512 * 40 - 5, 512, 1, 3),              # the folded block is the buffer's partial last block
+    (496 * 25, 496, 3, 2),                  # 31 blocks: one counter behind the last row, one row per chunk
+    (1008 * 9 + 16 * 31, 1008, 2, 3),       # 63 blocks; the short last chunk (31 blocks) folds too
+    (1024 * 30 + 400, 1024, 5, 3),          # the short last chunk (25 blocks) does not fold
+    (16384 * 12 - 1, 16384, 8, 3),          # 1024 blocks (the benchmark's small chunk), chunks shared between warps
+    (16384 * 12, 16384, 40, 2),             # a warp holds whole chunks and pieces
+    (65536 * 3 + 4096, 65536, 0, 3),        # planner's own slots
+    (2 * 1048576 + 512, 1048576, 0, 4),     # 2049 rows: folded only when forced
+]
+
+
+@pytest.mark.parametrize("n,cb,seg,sms", FOLD_SHAPES)
+@pytest.mark.parametrize("aad", [0, 7])
+@pytest.mark.parametrize("fold", [0, 1, 2])
+def test_folded_tails_match_oracle(emu, n, cb, seg, sms, aad, fold):
+    """Chunks that end in a row of one or two counters: with the tail folded (the kernel's prework pass takes those
+    counters and every tag mask, ten chunks at a time) and without, the same bytes, tags and verdicts as the oracle."""
+    rng = np.random.default_rng(n + cb + aad)
+    key, iv = rng.bytes(32), rng.bytes(8) + bytes([0xFF, 0xFF, 0xFF, 0xFD])
+    p = np.frombuffer(rng.bytes(n), np.uint8)
+    c_ref, t_ref = oracle.mc_encrypt_framed(key, iv, cb, aad, p, 4) if aad else oracle.mc_encrypt(key, iv, cb, p, 4)
+    K = t_ref.shape[0]
+    c, t, _, _ = run(emu, ENC, key, iv, cb, p, n, seg=seg, aad=aad, sms=sms, fold=fold)
+    assert np.array_equal(c, c_ref) and np.array_equal(t, t_ref)
+    bad_c, bad_t = c_ref.copy(), t_ref.copy()
+    bad_c[min(n - 1, cb - 3)] ^= 0x40                    # inside the folded tail of chunk 0 (its last block)
+    if K > 2:
+        bad_t[K - 2, 15] ^= 1
+    p_ref, ok_ref = (oracle.mc_decrypt_framed(key, iv, cb, aad, bad_c, bad_t, 4) if aad else
+                     oracle.mc_decrypt(key, iv, cb, bad_c, bad_t, 4))
+    assert ok_ref[0] == 0 and ok_ref.sum() == K - (2 if K > 2 else 1)
+    out, _, ok, _ = run(emu, DEC, key, iv, cb, bad_c, n, tags=bad_t, seg=seg, aad=aad, sms=sms, fold=fold)
     assert np.array_equal(out, p_ref) and np.array_equal(ok, ok_ref)
 
 

@@ -164,10 +164,11 @@ def test_option_interface():
     with fastrack.Context(key, cb) as ctx:
         assert fastrack.fastrack_ctx_set_option(ctx.handle, 0, 1) == fastrack.ERR_ARG
         assert fastrack.fastrack_ctx_set_option(ctx.handle, 99, 1) == fastrack.ERR_ARG
+        assert fastrack.fastrack_ctx_set_option(ctx.handle, fastrack.OPT_FOLD_TAIL, 3) == fastrack.ERR_ARG      # 0, 1 or 2
         d_p = torch.from_numpy(plain).cuda()
         d_c = torch.empty_like(d_p)
         d_t = torch.empty(16 * K, dtype=torch.uint8, device="cuda")
-        for options in ({}, {fastrack.OPT_PACK_MAX_BLOCKS: 0}, {fastrack.OPT_ROW_SLOTS: 5}, {fastrack.OPT_PACK_MAX_BLOCKS: 4096, fastrack.OPT_PACK_RUN: 7},
+        for options in ({}, {fastrack.OPT_PACK_MAX_BLOCKS: 0}, {fastrack.OPT_ROW_SLOTS: 5}, {fastrack.OPT_FOLD_TAIL: 2}, {fastrack.OPT_FOLD_TAIL: 1}, {fastrack.OPT_PACK_MAX_BLOCKS: 4096, fastrack.OPT_PACK_RUN: 7},
                         {fastrack.OPT_PACK_RUN: 0, fastrack.OPT_ROW_SLOTS: 0, fastrack.OPT_GENERIC_SMEM: 1, fastrack.OPT_NO_OVERLAP_LAUNCH: 1}):
             for option, value in options.items():
                 ctx.set_option(option, value)

@@ -23,6 +23,9 @@ FAMILIES = {      # kernel layouts forced through fastrack_ctx_set_option
     "general": {fastrack.OPT_PACK_MAX_BLOCKS: 0},                                  # row kernels only
     "general-every-warp": {fastrack.OPT_PACK_MAX_BLOCKS: 0, fastrack.OPT_ROW_SLOTS: 148 * 32},   # ... rows spread as thinly as they go
     "general-37-warps": {fastrack.OPT_PACK_MAX_BLOCKS: 0, fastrack.OPT_ROW_SLOTS: 37},   # ... chunks shared between warps and CTAs
+    "general-folded": {fastrack.OPT_PACK_MAX_BLOCKS: 0, fastrack.OPT_FOLD_TAIL: 2},  # ... a chunk's last row of one or two blocks folded away wherever there is one
+    "general-folded-37-warps": {fastrack.OPT_PACK_MAX_BLOCKS: 0, fastrack.OPT_FOLD_TAIL: 2, fastrack.OPT_ROW_SLOTS: 37},
+    "general-unfolded": {fastrack.OPT_PACK_MAX_BLOCKS: 0, fastrack.OPT_FOLD_TAIL: 1},  # ... and nowhere
     "auto": {},                                                                   # the planner decides
     "run1": {fastrack.OPT_PACK_RUN: 1},                                           # packed rows, one counter per lane
     "run5": {fastrack.OPT_PACK_RUN: 5},                                           # packed rows, five counters per lane

@@ -18,15 +18,15 @@ def plan(tmp_path_factory):
                            os.path.join(ROOT, "tests", "host_logic", "plan_check.cpp")])
     lib = ctypes.CDLL(str(so))
     Z, U = ctypes.c_size_t, ctypes.c_uint32
-    lib.plan_launch.argtypes = [ctypes.c_int, Z, U, U, U, U, ctypes.c_int, Z, Z, ctypes.c_void_p]
+    lib.plan_launch.argtypes = [ctypes.c_int, Z, U, U, U, U, ctypes.c_int, Z, Z, U, ctypes.c_void_p]
     lib.plan_stages.argtypes = [Z, Z, Z, Z, ctypes.c_void_p]
     lib.plan_stages.restype = Z
     return lib
 
 
-def launch(lib, cb, sample_bytes, n_chunks, kind=0, row_slots=0, pack_max=4096, run=0, group=0, sms=148, geometry=False):
-    out = np.zeros(10, np.uint64)
-    lib.plan_launch(sms, cb, row_slots, pack_max, run, group, kind, sample_bytes, n_chunks, out.ctypes.data)
+def launch(lib, cb, sample_bytes, n_chunks, kind=0, row_slots=0, pack_max=4096, run=0, group=0, sms=148, geometry=False, fold=0):
+    out = np.zeros(11, np.uint64)
+    lib.plan_launch(sms, cb, row_slots, pack_max, run, group, kind, sample_bytes, n_chunks, fold, out.ctypes.data)
     return [int(x) for x in (out if geometry else out[:6])]
 
 
@@ -42,10 +42,16 @@ def test_launch_plans_are_consistent(plan, kind):
         for n_chunks in COUNTS:
             if cb * n_chunks > 1 << 42:
                 continue
-            grid, wu, n_slots, run, group, p_items, rows_full, rows_last, rows_sample, total = launch(
+            grid, wu, n_slots, run, group, p_items, rows_full, rows_last, rows_sample, total, fold = launch(
                 plan, cb, cb * n_chunks, n_chunks, kind, geometry=True)
+            # folded tails: only the fused passes, only chunks that end in a row of one or two counters, only where a
+            # warp's range holds a chunk start or more
+            foldable = kind == 0 and blocks >= 31 and (blocks + 2) % 32 in (1, 2)
+            assert fold in ((0, 1) if foldable else (0,))
+            if foldable:
+                assert fold == (1 if n_chunks >= launch(plan, cb, cb * n_chunks, n_chunks, kind, fold=1)[2] else 0)
             # row kernels: the slots cover the row space without an empty range, on at most one CTA per SM
-            assert rows_full == rows and rows_last == rows and rows_sample == rows * n_chunks == total
+            assert rows_full == rows - fold and rows_last == rows - fold and rows_sample == (rows - fold) * n_chunks == total
             assert 1 <= n_slots <= min(total, WARPS) and 1 <= grid <= 148 and 1 <= wu <= 32
             assert (grid - 1) * wu < n_slots <= grid * wu, "every CTA of the grid holds at least one slot"
             assert n_slots * total < 1 << 63, "slot boundaries are computed in 64 bits"
@@ -95,13 +101,42 @@ def test_small_chunks_in_large_numbers_take_the_packed_rows(plan):
     assert launch(plan, 2048, 4 << 20, 2048)[3] >= 1
 
 
+def test_folded_tails_follow_the_option_and_the_shape(plan):
+    """A chunk whose last row would hold one or two counters has one row less when its tail is folded; by itself the
+    planner folds where there are at least as many chunks as warps at work; the option switches that off or forces it; a sample's
+    short last chunk is judged by its own length."""
+    for cb, rows in ((512, 2), (16384, 33), (65536, 129), (496, 2), (1 << 20, 2049)):
+        for n_chunks in (100, 16384, 1 << 20):
+            auto, never, always = (launch(plan, cb, cb * n_chunks, n_chunks, geometry=True, fold=f, pack_max=0) for f in (0, 1, 2))
+            assert never[6] == rows and never[10] == 0
+            assert always[6] == rows - 1 and always[10] == 1
+            assert auto[6:] == (always[6:] if n_chunks >= never[2] else never[6:])
+    assert launch(plan, 16384, 256 << 20, 16384, geometry=True)[10] == 1        # the benchmark's 256 MiB of 16 KiB chunks: folded
+    assert launch(plan, 16384, 64 << 20, 4096, geometry=True)[10] == 1          # 64 MiB: 1.7 chunks per warp
+    assert launch(plan, 16384, 16 << 20, 1024, geometry=True)[10] == 0          # 16 MiB of them: a chunk spans two warps
+    assert launch(plan, 4 << 20, 256 << 20, 64, geometry=True)[10] == 0         # the headline shape: never
+    for cb in (48, 480, 528, 16400):                       # no tail of one or two counters: nothing to fold, whatever the option says
+        assert launch(plan, cb, cb * 100, 100, geometry=True, fold=2)[10] == 0
+    # samples of 3 chunks of 1 KiB and a last one of 496 bytes (31 blocks: folds) / of 400 bytes (25 blocks: does not)
+    got = launch(plan, 1024, 3 * 1024 + 496, 4 * 50, geometry=True, pack_max=0, fold=2)
+    assert got[10] == 1 and got[6] == 2 and got[7] == 1 and got[8] == 7 and got[9] == 7 * 50
+    got = launch(plan, 1024, 3 * 1024 + 400, 4 * 50, geometry=True, pack_max=0, fold=2)
+    assert got[10] == 1 and got[6] == 2 and got[7] == 1
+    got = launch(plan, 1040, 3 * 1040 + 496, 4 * 50, geometry=True, pack_max=0, fold=2)      # only the last chunk folds
+    assert got[10] == 1 and got[6] == 3 and got[7] == 1
+    for kind in (1, 2):                                    # the other passes never fold
+        assert launch(plan, 16384, 16384 * 100, 100, kind=kind, geometry=True, fold=2)[10] == 0
+
+
 def test_sample_batches_plan_on_the_sample_geometry(plan):
     # samples shorter than a chunk: the chunk that exists is the sample
     got = launch(plan, 4096, 400, 262144, geometry=True)
     assert got[3] >= 1 and got[6] == got[7] == 1 and got[9] == 262144
     # samples of several chunks: three full ones and a 16-byte one
-    got = launch(plan, 1024, 3 * 1024 + 16, 4 * 50000, geometry=True)
+    got = launch(plan, 1024, 3 * 1024 + 16, 4 * 50000, geometry=True, fold=1)
     assert got[6] == 3 and got[7] == 1 and got[8] == 10 and got[9] == 10 * 50000
+    got = launch(plan, 1024, 3 * 1024 + 16, 4 * 50000, geometry=True)              # the 1 KiB chunks' tails folded
+    assert got[10] == 1 and got[6] == 2 and got[7] == 1 and got[8] == 7 and got[9] == 7 * 50000
 
 
 def test_row_slots_follow_the_size_of_the_launch(plan):
