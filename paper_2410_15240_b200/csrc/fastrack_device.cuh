@@ -265,6 +265,31 @@ __device__ __forceinline__ uint4 fr_aes256_rounds(const char* sm, uint32_t lane4
     return make_uint4(o[0], o[1], o[2], o[3]);
 }
 
+// The same rounds as a loop that is not unrolled: a tenth of the code for a block that is computed rarely (what
+// such code costs is its footprint in the instruction cache of the warps that are in the row loop meanwhile).
+template <bool ABS>
+__device__ __forceinline__ uint4 fr_aes256_rounds_compact(const char* sm, uint32_t lane4, const FrParams& P, int first,
+                                                          uint32_t s0, uint32_t s1, uint32_t s2, uint32_t s3)
+{
+#pragma unroll 1
+    for (int r = first; r < 14; r++) {
+        uint32_t t0 = FR_TE0(s0, 0) ^ FR_TE1(s1, 1) ^ FR_TE2(s2, 2) ^ FR_TE3(s3, 3) ^ P.rk[4 * r + 0];
+        uint32_t t1 = FR_TE0(s1, 0) ^ FR_TE1(s2, 1) ^ FR_TE2(s3, 2) ^ FR_TE3(s0, 3) ^ P.rk[4 * r + 1];
+        uint32_t t2 = FR_TE0(s2, 0) ^ FR_TE1(s3, 1) ^ FR_TE2(s0, 2) ^ FR_TE3(s1, 3) ^ P.rk[4 * r + 2];
+        uint32_t t3 = FR_TE0(s3, 0) ^ FR_TE1(s0, 1) ^ FR_TE2(s1, 2) ^ FR_TE3(s2, 3) ^ P.rk[4 * r + 3];
+        s0 = t0; s1 = t1; s2 = t2; s3 = t3;
+    }
+    return fr_aes256_rounds<ABS, 14>(sm, lane4, P, s0, s1, s2, s3);      // the last round only
+}
+
+// E_K(IV || BE32(ctr)) from the IV words, without the shared first rounds and in compact code.
+template <bool ABS>
+__device__ __forceinline__ uint4 fr_aes256_block_compact(const char* sm, uint32_t lane4, const FrParams& P, uint32_t ivw0,
+                                                         uint32_t ivw1, uint32_t ivw2, uint32_t ctr)
+{
+    return fr_aes256_rounds_compact<ABS>(sm, lane4, P, 1, ivw0 ^ P.rk[0], ivw1 ^ P.rk[1], ivw2 ^ P.rk[2], fr_bswap(ctr) ^ P.rk[3]);
+}
+
 // Counter-mode sharing of the first two rounds.  In the counter block IV_k || BE32(ctr) only byte 15
 // changes from block to block, byte 14 every 256 blocks, bytes 12-13 hardly ever.  After round 1 three
 // of the four columns depend only on ctr >> 8, and in round 2 every output column takes exactly one
@@ -403,6 +428,12 @@ __device__ __forceinline__ uint4 fr_gf128_mul(uint4 x, uint4 y)
     const uint32_t z1 = p[1] ^ f[1], z2 = p[2] ^ f[2], z3 = p[3] ^ f[3];
     return make_uint4(fr_bswap(__brev(z0)), fr_bswap(__brev(z1)), fr_bswap(__brev(z2)), fr_bswap(__brev(z3)));
 }
+
+// The same product as a function that is called, for kernels that use it in more than one place.
+#ifndef FR_NOINLINE
+#define FR_NOINLINE __noinline__
+#endif
+__device__ FR_NOINLINE uint4 fr_gf128_mul_called(uint4 x, uint4 y) { return fr_gf128_mul(x, y); }
 
 // Where chunk kk of the launch lives and what it is keyed with.  The launch is a sequence of equal samples
 // (a plain buffer is one sample); inside a sample the chunks are chunk_bytes long except possibly the last.
@@ -641,7 +672,7 @@ __device__ __forceinline__ uint4 fr_process_segment_lane(const FrParams& P, cons
     FR_STAMP_MIN(3); FR_STAMP_MAX(4);
     if (!DO_GHASH) return make_uint4(0, 0, 0, 0);
     if (c_last == 0u) return extra;
-    return fr_xor4(fr_gf128_mul(pend, hpow), extra);
+    return fr_xor4(FOLD ? fr_gf128_mul_called(pend, hpow) : fr_gf128_mul(pend, hpow), extra);
 }
 
 template <int MODE, bool ABS, bool FOLD = false>
@@ -682,9 +713,7 @@ __device__ __forceinline__ uint4 fr_prework_lane(const FrParams& P, const char* 
     const uint32_t ctr = role == 0u ? 1u : rows_k * FR_ROW_BLOCKS + role - 1u;
     j0_lane = role == 0u;
     if (role != 0u && ctr > nblk + 1u) return make_uint4(0, 0, 0, 0);      // the rows cover the chunk up to its last counter
-    const FrCtrChunk cc = fr_ctr_chunk<ABS>(sm, L.lane4, P, ck.iv_w0, ck.iv_w1, fr_bswap(ck.iv_ctr));
-    const FrCtrGroup cg = fr_ctr_group<ABS>(sm, L.lane4, P, cc, ctr);
-    const uint4 ks = fr_aes256_ctr_block<ABS>(sm, L.lane4, P, cc, cg, ctr);
+    const uint4 ks = fr_aes256_block_compact<ABS>(sm, L.lane4, P, ck.iv_w0, ck.iv_w1, fr_bswap(ck.iv_ctr), ctr);
     if (role == 0u) return ks;
     const uint64_t boff = (uint64_t)(ctr - 2u) << 4;
     const bool full = ck.len - boff >= 16;
@@ -695,7 +724,7 @@ __device__ __forceinline__ uint4 fr_prework_lane(const FrParams& P, const char* 
     const uint4 o = fr_xor4(x, ks);
     if (full) *(uint4*)out = o; else fr_store_partial(out, o, nvalid);
     const uint4 g = (MODE == FR_MODE_ENC) ? (full ? o : fr_mask_bytes(o, nvalid)) : x;
-    return fr_gf128_mul(g, P.pow[nblk + 3u - ctr]);
+    return fr_gf128_mul_called(g, P.pow[nblk + 3u - ctr]);
 }
 
 // ---- Packed rows: many short chains -----------------------------------------------------------------------

@@ -106,11 +106,14 @@ static inline FrRowPlan fr_plan_rows(const FrPlanConfig& cfg, size_t sample_byte
         return slots;
     };
     geometry(false);
-    // Folding pays where a warp's range holds a chunk start or several, so that the extra pass serves them all (measured
-    // with 16 KiB chunks: 3.5 % at seven chunks per warp, 1.5 % at 1.7; 0.5 % with 64 KiB chunks at 1.2), and loses
-    // where chunks are spread over several warps and most warps would make the pass for one chunk (17 % at 0.4).
+    // Folding pays where a warp's range holds a chunk start or several, so that the extra pass serves them all: measured
+    // at 4.6 chunks per warp 4 % with 16 KiB chunks, 8 % with 8 KiB, 15 % with 4 KiB (more than the row saved, since
+    // row 0 of a chunk then no longer runs the cipher a second time for the tag mask), still 1 to 2 % at one chunk per
+    // warp.  Below that most warps would make a pass for a single chunk: a gain of under 1 % down to half a chunk per
+    // warp where 24 warps per SM hide the pass, a loss of 1 to 3 % with 16.
+    const uint64_t plain_slots = slots_for(p.total_rows);
     if (may_fold && cfg.fold_tail_mode != 1 && (fr_tail_folds(first_len) || fr_tail_folds(last_len)) &&
-        (cfg.fold_tail_mode == 2 || n_chunks >= slots_for(p.total_rows)))
+        (cfg.fold_tail_mode == 2 || n_chunks >= plain_slots || (plain_slots >= sms * 24 && 2 * n_chunks >= plain_slots)))
         geometry(true);
     const uint64_t slots = slots_for(p.total_rows);
     p.n_slots = (uint32_t)slots;
@@ -125,6 +128,8 @@ struct FrPackCosts {
     size_t close, step, step_latency;                     // packed rows, per row of 32 lanes: the closing; one counter step; its latency for a lone warp
     size_t row_fixed, pack_fixed;                         // per launch, beyond what scales with the work: rows (closing products of all
                                                           // warps at once, the hand-over between CTAs), packed rows
+    size_t seg_folded;                                    // row kernels with folded tails, per segment (row 0 no longer runs the cipher
+                                                          // a second time for the tag mask; that comes from the prework passes)
 };
 
 // Decides between the row kernels (`rows` is their plan) and the packed-row kernels, and in the latter case picks
@@ -142,9 +147,9 @@ static inline FrPackPlan fr_plan_packed(const FrPlanConfig& cfg, int kind, size_
                                         const FrRowPlan& rows)
 {
     static const FrPackCosts costs[3] = {
-        {279, 400, 1000, 300, 279, 2250, 10800, 4900},     // fused passes: cipher + Horner step per counter, one general product per lane
-        {218, 100, 900, 30, 227, 2000, 0, 0},              // counter mode only: no product, no reduction
-        {85, 400, 300, 465, 65, 700, 0, 0},                // verify only: no cipher (but counter 1), so the closing weighs more
+        {279, 400, 1000, 300, 279, 2250, 10800, 4900, 260},     // fused passes: cipher + Horner step per counter, one general product per lane
+        {218, 100, 900, 30, 227, 2000, 0, 0, 0},              // counter mode only: no product, no reduction
+        {85, 400, 300, 465, 65, 700, 0, 0, 0},                // verify only: no cipher (but counter 1), so the closing weighs more
     };
     const FrPackPlan rows_kernels = {0, 0};
     if (!cfg.pack_max_blocks || n_chunks == 0) return rows_kernels;
@@ -162,7 +167,8 @@ static inline FrPackPlan fr_plan_packed(const FrPlanConfig& cfg, int kind, size_
     // (folded tails: one more pass of a cipher block and a product per ten chunk starts, at least one per warp that sees a start)
     size_t pre_passes = rows.fold_tail ? n_chunks / 10 + rows.n_slots : 0;
     if (pre_passes > n_chunks) pre_passes = n_chunks;
-    const size_t row_thr = (size_t)((rows.total_rows + sms - 1) / sms) * C.row_clocks + (pieces + sms - 1) / sms * C.seg_clocks +
+    const size_t row_thr = (size_t)((rows.total_rows + sms - 1) / sms) * C.row_clocks +
+                           (pieces + sms - 1) / sms * (rows.fold_tail ? C.seg_folded : C.seg_clocks) +
                            (pre_passes + sms - 1) / sms * (C.step + C.close);
     const size_t row_lat = rows_per_slot * C.row_step_latency + segs_per_slot * 4000;
     const size_t row_cost = (row_thr > row_lat ? row_thr : row_lat) + C.row_fixed;

@@ -19,6 +19,7 @@
 // ---- what the device header needs from CUDA, as plain C++ ----
 #define __device__
 #define __forceinline__ inline
+#define FR_NOINLINE inline
 struct uint4 { uint32_t x, y, z, w; };
 static inline uint4 make_uint4(uint32_t a, uint32_t b, uint32_t c, uint32_t d) { return uint4{a, b, c, d}; }
 
