@@ -4,7 +4,9 @@
 // values, lane = counter mod 32, and the block at counter c is data block c - 2 of the chunk (GCM keeps
 // counter 1 for the tag mask), so a row is 512 contiguous bytes and global loads and stores are 128-bit and
 // coalesced.  Counter 1 of row 0 is a spare lane: it yields E_K(J0), and with the serial-number framing it
-// also absorbs the one-byte AAD block.
+// also absorbs the one-byte AAD block.  (In the variant with folded tails that lane idles as far as the cipher
+// goes: the tag masks, and the one or two counters that would make up a chunk's last row, are worked on in a
+// pass of their own for ten chunks at a time -- see fr_chunk_rows and fr_prework_lane.)
 //
 // AES (paper Section 2.3, "The AES block cipher": AES in counter mode, every block independent):
 //   four round tables Te0..Te3 live in shared memory, each entry replicated 32 times so that lane l
