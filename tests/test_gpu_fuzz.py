@@ -31,8 +31,12 @@ def _shapes(seed, count):
         yield n, cb, int(rng.choice([0, 0, 1, 4, 16, 256])), bool(rng.integers(0, 2)), int(rng.integers(0, 1 << 30))
 
 
+LAYOUTS = {"planner": {}, "rows-folded-tails": {fastrack.OPT_PACK_MAX_BLOCKS: 0, fastrack.OPT_FOLD_TAIL: 2}}
+
+
+@pytest.mark.parametrize("layout", list(LAYOUTS))
 @pytest.mark.parametrize("seed", [1, 2, 3, 4])
-def test_random_shapes_all_entry_points(seed):
+def test_random_shapes_all_entry_points(seed, layout):
     key, iv = synth.key_and_iv(seed)
     for n, cb, chains, in_place, salt in _shapes(seed, 30):
         plain = synth.random_bytes(n, seed, salt=salt)
@@ -42,7 +46,7 @@ def test_random_shapes_all_entry_points(seed):
             c, t = oracle.mc_encrypt(key, iv, cb, plain, NT)
         K = t.shape[0]
         what = f"n={n} cb={cb} chains={chains} in_place={in_place}"
-        with fastrack.Context(key, cb) as ctx:
+        with fastrack.Context(key, cb, LAYOUTS[layout]) as ctx:
             ctx.set_framing(chains)
             st = torch.cuda.current_stream().cuda_stream
             # encrypt
@@ -114,6 +118,12 @@ def test_portable_shared_addressing_path():
     is exercised on hardware where the fast form applies."""
     _every_pass_on([(1, 16, 0), (70001, 4096, 0), ((1 << 20) + 33, 65536, 16), ((5 << 20) + 7, 1 << 20, 0)],
                    {fastrack.OPT_GENERIC_SMEM: 1})
+
+
+def test_portable_shared_addressing_path_folded_tails():
+    """The same fallback in the row kernels' variant with folded tails."""
+    _every_pass_on([(512 * 50 + 9, 512, 0), (16384 * 21 - 3, 16384, 4), ((1 << 20) + 33, 65536, 16)],
+                   {fastrack.OPT_GENERIC_SMEM: 1, fastrack.OPT_PACK_MAX_BLOCKS: 0, fastrack.OPT_FOLD_TAIL: 2})
 
 
 def test_portable_shared_addressing_path_packed_rows():
