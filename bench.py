@@ -515,6 +515,9 @@ def other_configs(args, alu_peak, windows):
     out["config1_chain_sweep"] = [device_cell(64 << 20, (64 << 20) // k) for k in (1, 4, 16, 64, 256, 1024)]
     # many chains at the headline size: 16 KiB chunks against 4 MiB chunks
     out["chunk_16KiB"] = [device_cell(n, 16 << 10) for n in (64 << 20, 256 << 20)]
+    # chunks below the benchmark's range at the headline size (samples of tens to thousands of bytes): the planner picks the
+    # packed rows for the small ones and the row kernels with folded tails from 4 KiB up
+    out["small_chunks_256MiB"] = [device_cell(256 << 20, cb) for cb in (64, 256, 1024, 4096)]
     # config 3: 670 MB of bf16-sized state, device-resident, and the mirror pipeline
     out["config3_device"] = device_cell(670_000_000, 4 << 20)
     torch.cuda.empty_cache()
