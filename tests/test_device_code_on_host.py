@@ -173,8 +173,10 @@ def test_a_stage_that_starts_at_a_later_chunk(emu):
 
 
 @pytest.mark.parametrize("sample_bytes,cb,n_samples,aad,seg", [(64, 16, 3, 0, 8), (1024, 1024, 5, 0, 2), (1040, 1024, 4, 16, 8),
-                                                              (3 * 4096 + 160, 4096, 6, 4, 4), (301056, 65536, 2, 16, 8)])
-def test_batch_of_samples_each_under_its_own_iv(emu, sample_bytes, cb, n_samples, aad, seg):
+                                                              (3 * 4096 + 160, 4096, 6, 4, 4), (301056, 65536, 2, 16, 8),
+                                                              (2 * 1024 + 496, 1024, 23, 5, 3), (1040 + 512, 1040, 9, 0, 1)])
+@pytest.mark.parametrize("fold", [1, 2])
+def test_batch_of_samples_each_under_its_own_iv(emu, sample_bytes, cb, n_samples, aad, seg, fold):
     """Paper Section 4.2: every sample is its own multi-chain message; a batch is many of them in one launch."""
     rng = np.random.default_rng(sample_bytes + n_samples)
     key = rng.bytes(32)
@@ -189,11 +191,11 @@ def test_batch_of_samples_each_under_its_own_iv(emu, sample_bytes, cb, n_samples
         cs.append(c1)
         ts.append(t1)
     c_ref, t_ref = np.concatenate(cs), np.concatenate(ts)
-    c, t, _, _ = run(emu, ENC, key, bytes(12), cb, p, n, seg=seg, aad=aad, sample_bytes=sample_bytes, ivs=ivs)
+    c, t, _, _ = run(emu, ENC, key, bytes(12), cb, p, n, seg=seg, aad=aad, sample_bytes=sample_bytes, ivs=ivs, fold=fold)
     assert np.array_equal(c, c_ref) and np.array_equal(t, t_ref)
     bad_t = t_ref.copy()
     bad_t[len(bad_t) // 2, 0] ^= 1
-    out, _, ok, _ = run(emu, DEC, key, bytes(12), cb, c_ref, n, tags=bad_t, seg=seg, aad=aad, sample_bytes=sample_bytes, ivs=ivs)
+    out, _, ok, _ = run(emu, DEC, key, bytes(12), cb, c_ref, n, tags=bad_t, seg=seg, aad=aad, sample_bytes=sample_bytes, ivs=ivs, fold=fold)
     exp = np.ones(len(bad_t), np.uint32)
     exp[len(bad_t) // 2] = 0
     assert np.array_equal(out, p) and np.array_equal(ok, exp)

@@ -129,6 +129,32 @@ def test_folded_tails_follow_the_option_and_the_shape(plan):
         assert launch(plan, 16384, 16384 * 100, 100, kind=kind, geometry=True, fold=2)[10] == 0
 
 
+def test_row_geometry_of_random_sample_shapes(plan):
+    """Whatever the folding: a sample's last chunk never has more rows than a full one (the kernel locates a row by
+    dividing by the rows of a full chunk), the rows add up, and no warp's range is empty."""
+    rng = np.random.default_rng(9)
+    for _ in range(3000):
+        cb = 16 * int(rng.integers(1, 5000))
+        cps = int(rng.integers(1, 6))
+        last = 16 * int(rng.integers(1, cb // 16 + 1)) - int(rng.integers(0, 16))
+        sample = (cps - 1) * cb + last
+        n_samples = int(rng.choice([1, 2, 7, 300, 100000]))
+        for fold in (0, 1, 2):
+            grid, wu, n_slots, _, _, _, rows_full, rows_last, rows_sample, total, folded = launch(
+                plan, cb, sample, cps * n_samples, geometry=True, fold=fold, pack_max=0)
+            assert 1 <= rows_last <= rows_full
+            assert rows_sample == (cps - 1) * rows_full + rows_last and total == rows_sample * n_samples
+            assert 1 <= n_slots <= total and (grid - 1) * wu < n_slots <= grid * wu
+            blocks_full, blocks_last = -(-min(cb, sample) // 16), -(-last // 16)
+            for blocks, rows in ((blocks_full, rows_full), (blocks_last, rows_last)):
+                plain = (blocks + 2 + 31) // 32
+                folds = folded and blocks >= 31 and (blocks + 2) % 32 in (1, 2)
+                assert rows == plain - (1 if folds else 0)
+                assert 32 * rows >= blocks + 2 - (2 if folds else 0) > 32 * (rows - 1)      # the rows cover every counter that is theirs
+            if fold == 1:
+                assert not folded
+
+
 def test_sample_batches_plan_on_the_sample_geometry(plan):
     # samples shorter than a chunk: the chunk that exists is the sample
     got = launch(plan, 4096, 400, 262144, geometry=True)
