@@ -20,14 +20,13 @@ using namespace fr_host;
 
 // ------------------------------------------------------------------------------------ kernels ----
 
-// Te0 (AES S-box folded with MixColumns; the same for every key).  Written once per device by fastrack_ctx_create.
-// (Tried instead: the 256 words as immediates in the code of the warp that stores them -- slower, 2.0 against
-// 1.4 us for the fill, because then every warp runs code of its own and the instruction fetch becomes the cost.)
-__constant__ uint32_t fr_te0_const[256];
+// (Te0 reaches the kernels as a parameter, FrParams::te0c.  Tried instead: the 256 words as immediates in the code of
+// the warp that stores them -- slower, 2.0 against 1.4 us for the fill, because then every warp runs code of its own
+// and the instruction fetch becomes the cost; a __constant__ array -- a cold miss per isolated launch.)
 
 // Fills shared memory at the start of a kernel, up to but not including the barrier that publishes it.
 //   AES rows: every thread replicates eight entries of Te0 (and its byte rotations) across the 32 banks; the
-//     entries come from constant memory with a warp-uniform index.
+//     entries come from the kernel parameters (constant bank) with a warp-uniform index.
 //   H-power byte tables (64 KiB, per context): two bulk asynchronous copies, global -> shared, issued by thread 0
 //     before anything else and signalled on an mbarrier.  Nobody waits for them here: every lane starts with a
 //     cipher block, which needs the AES rows only, and waits in front of its first table multiply
@@ -35,7 +34,7 @@ __constant__ uint32_t fr_te0_const[256];
 //     (Passes that do not authenticate have no use for them and start no copy: a CTA must not exit with a copy
 //     into its shared memory still in flight, and only the table multiply waits for it.)
 template <uint32_t NTHREADS, bool WITH_H_TABLES>
-__device__ __forceinline__ void fr_fill_smem(char* sm, const uint4* __restrict__ gh_tab)
+__device__ __forceinline__ void fr_fill_smem(char* sm, const uint4* __restrict__ gh_tab, const FrParams& P)
 {
     const uint32_t tid = threadIdx.x;
     if (WITH_H_TABLES && tid == 0) {
@@ -54,7 +53,7 @@ __device__ __forceinline__ void fr_fill_smem(char* sm, const uint4* __restrict__
 #pragma unroll
     for (uint32_t n = 0; n < N_AES; n++) {
         const uint32_t i = tid + n * NTHREADS, q = i & 7u, t = (i >> 3) & 3u, v = i >> 5;
-        const uint32_t e = fr_te0_const[v];
+        const uint32_t e = P.te0c[v];
         const uint32_t w = __funnelshift_l(e, e, 8u * t);                 // Te1..Te3 are Te0 rotated left by 1..3 bytes
         const uint32_t off = ((t >> 1) ? FR_SM_T23 : FR_SM_T01) + v * 256u + (t & 1u) * 128u + q * 16u;
         *(uint4*)(sm + off) = make_uint4(w, w, w, w);
@@ -193,7 +192,7 @@ __global__ void __launch_bounds__(FR_THREADS, 1) fr_crypt_kernel(const __grid_co
 {
     extern __shared__ __align__(256) char sm[];
     FR_STAMP_GT(0); FR_STAMP_SET(7);
-    fr_fill_smem<FR_THREADS, MODE != FR_MODE_CTR && MODE != FR_MODE_PADGEN>(sm, P.gh_tab);
+    fr_fill_smem<FR_THREADS, MODE != FR_MODE_CTR && MODE != FR_MODE_PADGEN>(sm, P.gh_tab, P);
     FR_STAMP_SET(1);
     // Programmatic dependent launch: the table build above touches only per-context constants, so it may run
     // while the previous kernel in the stream is still finishing; everything below waits until that kernel has
@@ -270,7 +269,7 @@ template <int MODE, bool WHOLE>
 __global__ void __launch_bounds__(FR_THREADS, 1) fr_packed_kernel(const __grid_constant__ FrParams P)
 {
     extern __shared__ __align__(256) char sm[];
-    fr_fill_smem<FR_THREADS, MODE != FR_MODE_CTR>(sm, P.gh_tab);
+    fr_fill_smem<FR_THREADS, MODE != FR_MODE_CTR>(sm, P.gh_tab, P);
     asm volatile("griddepcontrol.wait;" ::: "memory");           // as in fr_crypt_kernel
     asm volatile("griddepcontrol.launch_dependents;");
     __syncthreads();
@@ -387,6 +386,7 @@ struct fastrack_ctx {
     uint32_t rk[60];
     uint8_t h[16];
     uint32_t* d_te0;
+    uint32_t te0_host[256];    // Te0, copied into every launch's parameters
     uint4* d_gh_tab;           // byte tables of H^32
     uint4* d_gh1_tab;          // byte tables of H (packed rows with one lane per chunk, sequential-chain comparator)
     uint4* d_pack_tab[2];      // byte tables of H^lanes for the packed rows, per scratch bank (see launch_pass)
@@ -474,6 +474,7 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
     expand_key(key, sbox, ctx->rk);
     uint8_t zero[16] = {0};
     encrypt_block_host(ctx->rk, te0, sbox, zero, ctx->h);
+    memcpy(ctx->te0_host, te0, sizeof te0);
 
     Gf128 H = gf_load(ctx->h), G = H;
     for (int i = 0; i < 5; i++) G = gf_mul(G, G);           // H^32
@@ -508,7 +509,6 @@ extern "C" int fastrack_ctx_create(const uint8_t key[32], size_t chunk_bytes, fa
         if ((e = cudaMalloc(&ctx->d_scratch, scratch_words(ctx) * sizeof(uint32_t))) != cudaSuccess) break;
         if ((e = cudaMemset(ctx->d_scratch, 0, scratch_words(ctx) * sizeof(uint32_t))) != cudaSuccess) break;
         if ((e = cudaMemcpy(ctx->d_te0, te0, sizeof te0, cudaMemcpyHostToDevice)) != cudaSuccess) break;
-        if ((e = cudaMemcpyToSymbol(fr_te0_const, te0, sizeof te0)) != cudaSuccess) break;       // key-independent: every context writes the same words
         if ((e = cudaMalloc(&ctx->d_timeouts, 256)) != cudaSuccess) break;
         if ((e = cudaMemset(ctx->d_timeouts, 0, 256)) != cudaSuccess) break;
         if ((e = cudaMemcpy(ctx->d_gh_tab, tab, 65536, cudaMemcpyHostToDevice)) != cudaSuccess) break;
@@ -732,6 +732,7 @@ static int launch_pass(fastrack_ctx* ctx, int mode, const uint8_t iv_base[12], s
     FrParams P;
     memset(&P, 0, sizeof P);
     memcpy(P.rk, ctx->rk, sizeof P.rk);
+    memcpy(P.te0c, ctx->te0_host, sizeof P.te0c);
     if (iv_base) {
         P.iv_w0 = load_le32(iv_base);
         P.iv_w1 = load_le32(iv_base + 4);
@@ -1317,6 +1318,7 @@ extern "C" int fastrack_verify_sequential(fastrack_ctx* ctx, const uint8_t iv_ba
     FrParams P;
     memset(&P, 0, sizeof P);
     memcpy(P.rk, ctx->rk, sizeof P.rk);
+    memcpy(P.te0c, ctx->te0_host, sizeof P.te0c);
     P.iv_w0 = load_le32(iv_base);
     P.iv_w1 = load_le32(iv_base + 4);
     P.iv_ctr = load_be32(iv_base + 8);

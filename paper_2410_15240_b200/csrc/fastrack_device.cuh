@@ -111,6 +111,9 @@ struct FrParams {
     uint4* mask;               // E_K(J0) per chunk: written by FR_MODE_PADGEN, read by FR_MODE_PADDEC
     uint4 lenh_full;           // (BE64(0) || BE64(8 * chunk_bytes)) * H: the length block's term of a full chunk
     uint4 lenh_last;           // the same for the launch's last chunk (differs when that chunk is short)
+    uint32_t te0c[256];        // Te0 (the AES S-box folded with MixColumns; the same for every key): read at kernel entry to fill shared
+                               // memory.  As a parameter it is in the constant bank when the kernel starts (a __constant__ array
+                               // costs an isolated launch a cold miss, 0.25 us)
 };
 
 // Byte permute, PTX prmt.b32 in generic mode: result byte i = byte (sel nibble i & 7) of {a (0..3), b (4..7)};
