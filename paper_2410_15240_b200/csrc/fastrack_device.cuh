@@ -381,18 +381,24 @@ __device__ __forceinline__ uint32_t fr_to_natural(uint32_t le_word)     // bit i
 }
 
 // 32 x 32 -> 64 carry-less product from 16 integer multiplies (see above).
+// Phase products whose phase sums differ by four may be ADDED instead of XORed (the multiply-add does that for
+// nothing): their 4-bit fields line up one field apart, field s of the lower against field s - 1 of the higher, and
+// the counts of two such fields are at most min(s + 1, 15 - s) + min(s, 16 - s) <= 15, so the sum still fits its
+// field and its low bit is still the GF(2) sum.  (Two products of the same phase sum can both count 8 in the middle
+// field; those must be XORed.)
 __device__ __forceinline__ uint64_t fr_clmul32(uint32_t a, uint32_t b)
 {
     uint32_t as[4], bs[4];
 #pragma unroll
     for (int k = 0; k < 4; k++) { as[k] = a & (0x11111111u << k); bs[k] = b & (0x11111111u << k); }
-    uint64_t z[4] = {0, 0, 0, 0};
-#pragma unroll
-    for (int i = 0; i < 4; i++)
-#pragma unroll
-        for (int j = 0; j < 4; j++) z[(i + j) & 3] ^= (uint64_t)as[i] * (uint64_t)bs[j];
-    return (z[0] & 0x1111111111111111ull) | (z[1] & 0x2222222222222222ull) | (z[2] & 0x4444444444444444ull) |
-           (z[3] & 0x8888888888888888ull);
+#define FR_MUL(i, j) ((uint64_t)as[i] * (uint64_t)bs[j])
+    const uint64_t z0 = (FR_MUL(0, 0) + FR_MUL(1, 3)) ^ FR_MUL(2, 2) ^ FR_MUL(3, 1);
+    const uint64_t z1 = (FR_MUL(0, 1) + FR_MUL(2, 3)) ^ (FR_MUL(1, 0) + FR_MUL(3, 2));
+    const uint64_t z2 = (FR_MUL(0, 2) + FR_MUL(3, 3)) ^ FR_MUL(1, 1) ^ FR_MUL(2, 0);
+    const uint64_t z3 = FR_MUL(0, 3) ^ FR_MUL(1, 2) ^ FR_MUL(2, 1) ^ FR_MUL(3, 0);
+#undef FR_MUL
+    return (z0 & 0x1111111111111111ull) | (z1 & 0x2222222222222222ull) | (z2 & 0x4444444444444444ull) |
+           (z3 & 0x8888888888888888ull);
 }
 
 // 64 x 64 -> 128 by Karatsuba: three 32 x 32 products.
